@@ -1,0 +1,178 @@
+/*
+ * libchimera — GPU-resident late-interaction (MaxSim) retrieval over centroid + residual codes, for NVIDIA B200
+ * (sm_100a).  C ABI: plain pointers and sizes, no C++ or framework types.
+ *
+ * Pipeline run by every search call, all on the device, on the caller's stream, with no host round trip between
+ * stages (paper: Algorithm 1 skeleton "generate -> refine -> score -> top-k"; Definition 1 for every score):
+ *   stage 1  score table      S[c,i] = <q_i, centroid_c> for all query tokens x all centroids, in exact Q.24
+ *                             fixed point (Definition 1's inner product; integer so that later discrete choices do
+ *                             not depend on summation order)
+ *   stage 2  candidates       per query token the nprobe best centroids; union of their posting lists; the set of
+ *                             documents owning at least one such token (Sec. 3.2 step 1, sets L_q and S)
+ *   stage 3  pruning          CI(d) = sum_i max_{t in d} S[cid_t, i] (Chamfer aggregation rule of Sec. 4.2 applied
+ *                             to centroid scores); keep the n_prune candidates with the largest CI
+ *   stage 4  residual scores  score(d) = sum_i max_{t in d} <q_i, centroid_{cid_t} + residual(code_t)>
+ *                             (Definition 1 on the decoded tokens)
+ *   stage 5  top-k            the k best scores, best first (Definition 2, Eq. 1)
+ * Ties are always broken towards the smaller id.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global-memory addresses valid on the index's device; "host" pointers are ordinary
+ *     process memory.  The caller owns every buffer it passes and keeps it alive until the work enqueued on the
+ *     stream has finished.  The library owns only what chimera_build_index allocates inside the index.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Every function returns a chimera_status; chimera_last_error() gives a text for the calling thread's last
+ *     failure.  No function throws, traps the device, or leaves a kernel waiting on anything.
+ *   - Search calls only enqueue work (they are asynchronous to the host) unless stated otherwise.
+ */
+#ifndef CHIMERA_H
+#define CHIMERA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CHIMERA_OK = 0,
+    CHIMERA_INVALID_ARG = 1,        /* bad pointer, size or parameter; nothing was enqueued */
+    CHIMERA_CUDA_ERROR = 2,         /* a CUDA runtime call failed; text in chimera_last_error() */
+    CHIMERA_WORKSPACE_TOO_SMALL = 3,
+    CHIMERA_CAPACITY_OVERFLOW = 4,  /* a query produced more candidates than max_candidates (reported by status) */
+    CHIMERA_TIMEOUT = 5,            /* a bounded device-side wait gave up (reported by status) */
+    CHIMERA_UNSUPPORTED = 6         /* dim, nbits or a size outside the supported set */
+} chimera_status;
+
+#define CHIMERA_MAX_NPROBE 64       /* nprobe per query token */
+#define CHIMERA_MAX_QLEN 128        /* tokens per query */
+#define CHIMERA_MAX_NPRUNE 16384    /* n_prune */
+#define CHIMERA_MAX_K 16384         /* k */
+
+typedef struct chimera_index chimera_index; /* opaque */
+
+/* Index-time description.  Residual codes are uniform `nbits`-bit bucket indices per dimension over
+ * [res_lo, res_hi): value u decodes to res_lo + (u + 0.5) * (res_hi - res_lo) / 2^nbits.  Packing is little-endian
+ * within a byte: 2-bit codes put dimension 4g+t in bits [2t, 2t+1] of byte g; 1-bit codes put dimension 8g+t in bit
+ * t of byte g. */
+typedef struct {
+    int32_t dim;         /* multiple of 32, <= 128 (96 and 128 are the tuned cases) */
+    int32_t nbits;       /* 1 or 2 */
+    float res_lo;        /* e.g. -0.25f */
+    float res_hi;        /* e.g. +0.25f */
+    int64_t n_centroids; /* K >= 1 */
+    int64_t n_docs;      /* N >= 1 */
+    int64_t n_tokens;    /* T = sum of doclens */
+} chimera_index_desc;
+
+/* Library version as major*10000 + minor*100 + patch. */
+int chimera_version(void);
+
+/* Text of the calling thread's most recent failure ("" if none).  The pointer stays valid until that thread's next
+ * failing call. */
+const char *chimera_last_error(void);
+
+/* Build the device-resident index (offline step; Sec. 3.1: centroids, posting lists, per-token codes).
+ *   desc       host pointer.
+ *   centroids  device, [K, dim] float32 row-major, unit-norm rows (every |element| <= 1).  Copied (as fixed-point
+ *              digits); may be freed after the call returns.
+ *   cids       device, [T] int32 in [0, K), document-major (document 0's tokens first).  REFERENCED, not copied:
+ *              must outlive the index.
+ *   codes      device, [T, dim*nbits/8] uint8, document-major.  REFERENCED, not copied: must outlive the index.
+ *   doclens    device, [N] int32, each >= 1, summing to T.  Copied (as prefix sums).
+ *   stream     work is enqueued on it and the call synchronises it before returning.
+ *   out        host pointer receiving the handle.
+ * Allocates (cudaMalloc) prefix sums, centroid digits and an inverted file: for each centroid the unique ids of the
+ * documents owning a token assigned to it, in unspecified order.
+ * Errors: INVALID_ARG (null pointer, sizes < 1, a cid outside [0,K), a doclen < 1, lengths not summing to T),
+ * UNSUPPORTED (dim / nbits), CUDA_ERROR.  On error nothing stays allocated and *out is NULL. */
+int chimera_build_index(const chimera_index_desc *desc, const float *centroids, const int32_t *cids,
+                        const uint8_t *codes, const int32_t *doclens, void *stream, chimera_index **out);
+
+/* Free everything the index owns (not the referenced cids / codes).  NULL is accepted. */
+int chimera_destroy_index(chimera_index *index);
+
+/* Bytes of device workspace a search call with these parameters needs.  max_candidates bounds the candidate list of
+ * one query (0 = n_docs, which can never overflow).  out: host pointer.
+ * Errors: INVALID_ARG / UNSUPPORTED for parameters outside: 1 <= q_len <= CHIMERA_MAX_QLEN,
+ * 1 <= nprobe <= min(K, CHIMERA_MAX_NPROBE), 1 <= n_prune <= CHIMERA_MAX_NPRUNE, 1 <= k <= CHIMERA_MAX_K,
+ * n_queries >= 1. */
+int chimera_workspace_bytes(const chimera_index *index, int32_t n_queries, int32_t q_len, int32_t nprobe,
+                            int32_t n_prune, int32_t k, int64_t max_candidates, size_t *out);
+
+/* Stages 1-5 for a batch of queries (Algorithm 1 with the stage list at the top of this file).
+ *   queries     device, [n_queries, q_len, dim] float32, unit-norm rows (the library does not normalise).
+ *   workspace   device, 256-byte aligned, at least chimera_workspace_bytes(...) bytes; contents are scratch.  Two
+ *               calls that may overlap on the device need distinct workspaces.
+ *   out_ids     device, [n_queries, k] int32: best first; -1 where fewer than k documents survive.
+ *   out_scores  device, [n_queries, k] float32: -inf beside every -1.
+ * Results do not depend on n_queries (a batch equals the same queries run one by one).
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL (nothing enqueued), CUDA_ERROR (launch failure). */
+int chimera_search(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                   int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                   size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores);
+
+/* The same search with HOST query and result buffers: copies the queries to the device (into the workspace), runs
+ * chimera_search, copies ids and scores back and synchronises the stream before returning.  Pinned host memory makes
+ * the copies asynchronous to each other but is not required.  The workspace must be
+ * chimera_workspace_bytes(...) bytes as for chimera_search (the staging areas are included in that figure). */
+int chimera_search_host(const chimera_index *index, const float *queries_host, int32_t n_queries, int32_t q_len,
+                        int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                        size_t workspace_bytes, void *stream, int32_t *out_ids_host, float *out_scores_host);
+
+/* Intermediate results ("taps") of a search: caller-owned device buffers, each optional (NULL = skip).
+ * They are copies of what the stages hand to each other, never a different computation. */
+typedef struct {
+    int32_t *score_table; /* [n_queries, K, q_len]  Q.24 fixed-point <q_i, c>, centroid-major                  */
+    int32_t *probes;      /* [n_queries, q_len, nprobe] best first (score desc, id asc)                         */
+    int32_t *cand;        /* [n_queries, max_candidates] ascending document ids; entries past n_cand undefined  */
+    int32_t *n_cand;      /* [n_queries]                                                                        */
+    int32_t *ci;          /* [n_queries, max_candidates] centroid-interaction score of cand[...] (Q.24 sum)     */
+    int32_t *pruned;      /* [n_queries, n_prune] ascending document ids, -1 padded                             */
+    int32_t *n_pruned;    /* [n_queries]                                                                        */
+    float *score4;        /* [n_queries, n_prune] stage-4 score of pruned[...], -inf beside -1                  */
+} chimera_taps;
+
+/* chimera_search that also copies the intermediates out (same kernels, same order).  taps: host pointer to a struct
+ * of device pointers; max_candidates = 0 means n_docs here as well. */
+int chimera_search_tapped(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                          int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                          size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
+                          const chimera_taps *taps);
+
+/* Run only stages first_stage..last_stage (1..5, first <= last).  Results of the stages before first_stage are read
+ * from `inout`, which must then hold: first_stage 2, 3 or 4: score_table; first_stage 3: also cand and n_cand;
+ * first_stage 4 or 5: pruned and n_pruned; first_stage 5: also score4.  Results of the stages that ran are written
+ * to the other non-NULL members of `inout`.  out_ids / out_scores may be NULL unless last_stage is 5.  For tests that feed one stage with
+ * another implementation's output. */
+int chimera_run_stages(const chimera_index *index, int32_t first_stage, int32_t last_stage, const float *queries,
+                       int32_t n_queries, int32_t q_len, int32_t nprobe, int32_t n_prune, int32_t k,
+                       int64_t max_candidates, void *workspace, size_t workspace_bytes, void *stream,
+                       const chimera_taps *inout, int32_t *out_ids, float *out_scores);
+
+/* Device-side status of the last search that used this workspace: synchronises the stream, then writes CHIMERA_OK,
+ * CHIMERA_CAPACITY_OVERFLOW (some query had more than max_candidates candidates; its results are computed on the
+ * first max_candidates of them and are not the specified output), CHIMERA_INVALID_ARG (a query element outside
+ * [-1, 1]) or CHIMERA_TIMEOUT to *status (host pointer). */
+int chimera_workspace_status(const void *workspace, void *stream, int32_t *status);
+
+/* Sizes held by an index (host pointers, each optional). */
+int chimera_index_info(const chimera_index *index, chimera_index_desc *desc, int64_t *posting_entries,
+                       int32_t *max_doclen);
+
+/* Per-stage device timing.  After chimera_profile_enable(1) every search records CUDA events around its stages on
+ * the search's stream; chimera_profile_read synchronises those events and returns, per stage slot, the summed
+ * milliseconds and the number of kernels launched since the last read, then resets both.  Slots:
+ * 0 score table, 1 probes, 2 candidate gather, 3 centroid interaction, 4 top-n_prune selection, 5 residual scores,
+ * 6 top-k, 7 copies/clears.  ms and launches: host arrays of CHIMERA_PROFILE_SLOTS entries.  At most
+ * CHIMERA_PROFILE_MAX_CALLS searches are kept between reads (later ones are not timed).  Not thread-safe. */
+#define CHIMERA_PROFILE_SLOTS 8
+#define CHIMERA_PROFILE_MAX_CALLS 256
+int chimera_profile_enable(int32_t on);
+int chimera_profile_read(float *ms, int64_t *launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHIMERA_H */

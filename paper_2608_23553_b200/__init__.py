@@ -1,0 +1,7 @@
+"""B200-native (sm_100a) late-interaction retrieval: thin Python binding over libchimera's C ABI.
+
+Every step of a search runs in the CUDA library; this package only marshals arguments (torch tensors supply device
+memory and the stream).  There is no CPU fallback: importing the binding without the built library fails loudly.
+"""
+from .binding import (ChimeraError, Index, Taps, lib, library_path, profile_enable, profile_read,  # noqa: F401
+                      PROFILE_SLOTS)

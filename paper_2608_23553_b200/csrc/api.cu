@@ -1,0 +1,433 @@
+// C ABI of libchimera: argument checks, workspace layout, stage sequencing, taps, status and profiling.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace chimera {
+
+// ------------------------------------------------------------------------------------------------ errors ---------
+static thread_local char g_err[512] = "";
+
+int fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+// ------------------------------------------------------------------------------------------------ profiling ------
+constexpr int PROF_MARKS = 12;
+struct ProfCall {
+    cudaEvent_t ev[PROF_MARKS];
+    int slot[PROF_MARKS];     // slot[i] = stage that ran between ev[i-1] and ev[i]
+    int n = 0;
+    bool created = false;
+};
+static bool g_prof_on = false;
+static ProfCall g_calls[CHIMERA_PROFILE_MAX_CALLS];
+static int g_n_calls = 0;
+static int64_t g_launches[CHIMERA_PROFILE_SLOTS] = {0};
+static ProfCall *g_cur = nullptr;
+
+void count_launch(int slot, int n) { g_launches[slot] += n; }
+
+static void prof_begin(cudaStream_t st)
+{
+    g_cur = nullptr;
+    if (!g_prof_on || g_n_calls >= CHIMERA_PROFILE_MAX_CALLS) return;
+    ProfCall *c = &g_calls[g_n_calls];
+    if (!c->created) {
+        for (int i = 0; i < PROF_MARKS; ++i)
+            if (cudaEventCreate(&c->ev[i]) != cudaSuccess) return;
+        c->created = true;
+    }
+    c->n = 0;
+    if (cudaEventRecord(c->ev[0], st) != cudaSuccess) return;
+    c->slot[0] = -1;
+    c->n = 1;
+    g_cur = c;
+    ++g_n_calls;
+}
+static void prof_mark(int slot, cudaStream_t st)
+{
+    if (!g_cur || g_cur->n >= PROF_MARKS) return;
+    if (cudaEventRecord(g_cur->ev[g_cur->n], st) != cudaSuccess) return;
+    g_cur->slot[g_cur->n] = slot;
+    ++g_cur->n;
+}
+
+// ------------------------------------------------------------------------------------------------ layout ---------
+static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+Layout make_layout(const Index &ix, const Params &p)
+{
+    Layout L;
+    memset(&L, 0, sizeof(L));
+    // probe stage: enough blocks to fill the device at small batch, at most 64 per query, at least ~512 rows each
+    int64_t blocks = (2LL * ix.sm_count + p.B - 1) / p.B;
+    int64_t by_rows = (ix.K + 511) / 512;
+    if (blocks > by_rows) blocks = by_rows;
+    if (blocks > 64) blocks = 64;
+    if (blocks < 1) blocks = 1;
+    L.probe_blocks = (int32_t)blocks;
+    L.n_part = L.probe_blocks * PROBE_WARPS;
+    L.words = (ix.N + 31) / 32;
+    L.n_chunks = (int32_t)((L.words + BITMAP_CHUNK_WORDS - 1) / BITMAP_CHUNK_WORDS);
+
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+    const size_t B = (size_t)p.B, nq = (size_t)p.nq;
+    L.status = take(64 * sizeof(uint32_t));
+    L.q_stage = take(B * nq * ix.D * sizeof(float));
+    L.out_ids = take(B * p.k * sizeof(int32_t));
+    L.out_scores = take(B * p.k * sizeof(float));
+    L.qdig = take(3 * B * nq * ix.D);
+    L.table = take(B * (size_t)ix.K * nq * sizeof(int32_t));
+    L.part = take(B * L.n_part * p.P * nq * sizeof(unsigned long long));
+    L.probes = take(B * nq * p.P * sizeof(int32_t));
+    L.bitmap = take(B * (size_t)L.words * sizeof(uint32_t));
+    L.chunk_cnt = take(B * (size_t)(L.n_chunks + 1) * sizeof(int32_t));
+    L.cand = take(B * (size_t)p.maxc * sizeof(int32_t));
+    L.n_cand = take(B * sizeof(int32_t));
+    L.ci = take(B * (size_t)p.maxc * sizeof(int32_t));
+    L.pruned = take(B * p.n_prune * sizeof(int32_t));
+    L.n_pruned = take(B * sizeof(int32_t));
+    L.score4 = take(B * p.n_prune * sizeof(float));
+    L.total = o;
+    return L;
+}
+
+static int check_params(const Index *ix, int32_t B, int32_t nq, int32_t P, int32_t n_prune, int32_t k,
+                        int64_t max_candidates, Params *out)
+{
+    if (!ix) return fail(CHIMERA_INVALID_ARG, "index is NULL");
+    if (B < 1 || B > 65535) return fail(CHIMERA_INVALID_ARG, "n_queries must be in [1, 65535], got %d", B);
+    if (nq < 1 || nq > CHIMERA_MAX_QLEN) return fail(CHIMERA_INVALID_ARG, "q_len must be in [1, %d], got %d", CHIMERA_MAX_QLEN, nq);
+    if (P < 1 || P > CHIMERA_MAX_NPROBE || P > ix->K)
+        return fail(CHIMERA_INVALID_ARG, "nprobe must be in [1, min(n_centroids, %d)], got %d", CHIMERA_MAX_NPROBE, P);
+    if (n_prune < 1 || n_prune > CHIMERA_MAX_NPRUNE)
+        return fail(CHIMERA_INVALID_ARG, "n_prune must be in [1, %d], got %d", CHIMERA_MAX_NPRUNE, n_prune);
+    if (k < 1 || k > CHIMERA_MAX_K) return fail(CHIMERA_INVALID_ARG, "k must be in [1, %d], got %d", CHIMERA_MAX_K, k);
+    if (max_candidates < 0) return fail(CHIMERA_INVALID_ARG, "max_candidates must be >= 0");
+    out->B = B; out->nq = nq; out->P = P; out->n_prune = n_prune; out->k = k;
+    out->maxc = (max_candidates == 0 || max_candidates > ix->N) ? ix->N : max_candidates;
+    return CHIMERA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ pipeline -------
+static int copy_d2d(void *dst, const void *src, size_t bytes, cudaStream_t st)
+{
+    if (bytes == 0) return CHIMERA_OK;
+    CHIMERA_CUDA(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st));
+    return CHIMERA_OK;
+}
+
+static int run(const Index &ix, const Params &p, int first, int last, const float *queries, void *workspace,
+               size_t workspace_bytes, cudaStream_t st, const chimera_taps *taps, int32_t *out_ids, float *out_scores)
+{
+    if (!workspace || ((uintptr_t)workspace & 255)) return fail(CHIMERA_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
+    const Layout L = make_layout(ix, p);
+    if (workspace_bytes < L.total)
+        return fail(CHIMERA_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
+    if ((first <= 1 || (first <= 4 && last >= 4)) && !queries) return fail(CHIMERA_INVALID_ARG, "queries is NULL");
+    if (last >= 5 && (!out_ids || !out_scores)) return fail(CHIMERA_INVALID_ARG, "out_ids / out_scores is NULL");
+
+    char *ws = (char *)workspace;
+    uint32_t *status = (uint32_t *)(ws + L.status);
+    int8_t *qdig = (int8_t *)(ws + L.qdig);
+    int32_t *table = (int32_t *)(ws + L.table);
+    unsigned long long *part = (unsigned long long *)(ws + L.part);
+    int32_t *probes = (int32_t *)(ws + L.probes);
+    uint32_t *bitmap = (uint32_t *)(ws + L.bitmap);
+    int32_t *chunk_cnt = (int32_t *)(ws + L.chunk_cnt);
+    int32_t *cand = (int32_t *)(ws + L.cand);
+    int32_t *n_cand = (int32_t *)(ws + L.n_cand);
+    int32_t *ci = (int32_t *)(ws + L.ci);
+    int32_t *pruned = (int32_t *)(ws + L.pruned);
+    int32_t *n_pruned = (int32_t *)(ws + L.n_pruned);
+    float *score4 = (float *)(ws + L.score4);
+
+    const size_t B = (size_t)p.B;
+    const size_t table_bytes = B * (size_t)ix.K * p.nq * sizeof(int32_t);
+    const size_t cand_bytes = B * (size_t)p.maxc * sizeof(int32_t);
+    const size_t pruned_bytes = B * p.n_prune * sizeof(int32_t);
+    int rc;
+
+    prof_begin(st);
+    CHIMERA_CUDA(cudaMemsetAsync(status, 0, 64 * sizeof(uint32_t), st));
+
+    // results of the stages that do not run come from the caller
+    if (first > 1) {
+        if (!taps) return fail(CHIMERA_INVALID_ARG, "taps are required when first_stage > 1");
+        if (first <= 4) {       // stages 2-4 read the score table
+            if (!taps->score_table) return fail(CHIMERA_INVALID_ARG, "taps->score_table is required");
+            if ((rc = copy_d2d(table, taps->score_table, table_bytes, st))) return rc;
+        }
+        if (first == 3) {
+            if (!taps->cand || !taps->n_cand) return fail(CHIMERA_INVALID_ARG, "taps->cand / n_cand are required");
+            if ((rc = copy_d2d(cand, taps->cand, cand_bytes, st))) return rc;
+            if ((rc = copy_d2d(n_cand, taps->n_cand, B * sizeof(int32_t), st))) return rc;
+        }
+        if (first >= 4) {
+            if (!taps->pruned || !taps->n_pruned) return fail(CHIMERA_INVALID_ARG, "taps->pruned / n_pruned are required");
+            if ((rc = copy_d2d(pruned, taps->pruned, pruned_bytes, st))) return rc;
+            if ((rc = copy_d2d(n_pruned, taps->n_pruned, B * sizeof(int32_t), st))) return rc;
+        }
+        if (first == 5) {
+            if (!taps->score4) return fail(CHIMERA_INVALID_ARG, "taps->score4 is required");
+            if ((rc = copy_d2d(score4, taps->score4, B * p.n_prune * sizeof(float), st))) return rc;
+        }
+    }
+    prof_mark(SLOT_MISC, st);
+
+    if (first <= 1 && last >= 1) {
+        if ((rc = launch_score_table(ix, p, queries, qdig, table, status, st))) return rc;
+        prof_mark(SLOT_G1, st);
+    }
+    if (first <= 2 && last >= 2) {
+        if ((rc = launch_probes(ix, p, L, table, part, probes, st))) return rc;
+        prof_mark(SLOT_PROBE, st);
+        if ((rc = launch_gather(ix, p, L, probes, bitmap, chunk_cnt, cand, n_cand, status, st))) return rc;
+        prof_mark(SLOT_GATHER, st);
+    }
+    if (first <= 3 && last >= 3) {
+        if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, st))) return rc;
+        prof_mark(SLOT_CI, st);
+        if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
+        prof_mark(SLOT_SELECT, st);
+    }
+    if (first <= 4 && last >= 4) {
+        if ((rc = launch_residual_scores(ix, p, queries, table, pruned, score4, st))) return rc;
+        prof_mark(SLOT_G4, st);
+    }
+    if (last >= 5) {
+        if ((rc = launch_topk(ix, p, pruned, score4, out_ids, out_scores, st))) return rc;
+        prof_mark(SLOT_TOPK, st);
+    }
+
+    if (taps) {
+        if (taps->score_table && first <= 1 && last >= 1 && (rc = copy_d2d(taps->score_table, table, table_bytes, st))) return rc;
+        if (first <= 2 && last >= 2) {
+            if (taps->probes && (rc = copy_d2d(taps->probes, probes, B * p.nq * p.P * sizeof(int32_t), st))) return rc;
+            if (taps->cand && (rc = copy_d2d(taps->cand, cand, cand_bytes, st))) return rc;
+            if (taps->n_cand && (rc = copy_d2d(taps->n_cand, n_cand, B * sizeof(int32_t), st))) return rc;
+        }
+        if (first <= 3 && last >= 3) {
+            if (taps->ci && (rc = copy_d2d(taps->ci, ci, cand_bytes, st))) return rc;
+            if (taps->pruned && (rc = copy_d2d(taps->pruned, pruned, pruned_bytes, st))) return rc;
+            if (taps->n_pruned && (rc = copy_d2d(taps->n_pruned, n_pruned, B * sizeof(int32_t), st))) return rc;
+        }
+        if (first <= 4 && last >= 4 && taps->score4 &&
+            (rc = copy_d2d(taps->score4, score4, B * p.n_prune * sizeof(float), st)))
+            return rc;
+        prof_mark(SLOT_MISC, st);
+    }
+    return CHIMERA_OK;
+}
+
+}  // namespace chimera
+
+using namespace chimera;
+
+// ================================================================================================ C ABI ==========
+extern "C" {
+
+int chimera_version(void) { return 100; }
+
+const char *chimera_last_error(void) { return g_err; }
+
+int chimera_build_index(const chimera_index_desc *desc, const float *centroids, const int32_t *cids,
+                        const uint8_t *codes, const int32_t *doclens, void *stream, chimera_index **out)
+{
+    if (out) *out = nullptr;
+    if (!desc || !centroids || !cids || !codes || !doclens || !out) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if (desc->n_centroids < 1 || desc->n_docs < 1 || desc->n_tokens < 1)
+        return fail(CHIMERA_INVALID_ARG, "n_centroids, n_docs and n_tokens must be >= 1");
+    if (desc->n_centroids > 0x7fffffffLL || desc->n_docs > 0x7fffffffLL)
+        return fail(CHIMERA_UNSUPPORTED, "n_centroids and n_docs must fit int32");
+    if (desc->dim < 32 || desc->dim > 128 || desc->dim % 32) return fail(CHIMERA_UNSUPPORTED, "dim must be 32, 64, 96 or 128, got %d", desc->dim);
+    if (desc->nbits != 1 && desc->nbits != 2) return fail(CHIMERA_UNSUPPORTED, "nbits must be 1 or 2, got %d", desc->nbits);
+    if (!(desc->res_hi > desc->res_lo)) return fail(CHIMERA_INVALID_ARG, "res_hi must exceed res_lo");
+    if (((uintptr_t)cids & 3) || ((uintptr_t)codes & 15) || ((uintptr_t)centroids & 15))
+        return fail(CHIMERA_INVALID_ARG, "centroids and codes must be 16-byte aligned");
+
+    Index *ix = new (std::nothrow) Index();
+    if (!ix) return fail(CHIMERA_CUDA_ERROR, "out of host memory");
+    cudaError_t e = cudaGetDevice(&ix->device);
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, ix->device);
+    if (e != cudaSuccess) {
+        delete ix;
+        return fail(CHIMERA_CUDA_ERROR, "no usable CUDA device: %s", cudaGetErrorString(e));
+    }
+    if (prop.major != 10) {
+        delete ix;
+        return fail(CHIMERA_UNSUPPORTED, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+    }
+    ix->sm_count = prop.multiProcessorCount;
+    ix->D = desc->dim;
+    ix->nbits = desc->nbits;
+    ix->CB = desc->dim * desc->nbits / 8;
+    ix->K = desc->n_centroids;
+    ix->N = desc->n_docs;
+    ix->T = desc->n_tokens;
+    ix->res_lo = desc->res_lo;
+    ix->res_hi = desc->res_hi;
+    ix->cids = cids;
+    ix->codes = codes;
+    int rc = build_index_device(*ix, centroids, doclens, (cudaStream_t)stream);
+    if (rc) {
+        chimera_destroy_index(reinterpret_cast<chimera_index *>(ix));
+        return rc;
+    }
+    *out = reinterpret_cast<chimera_index *>(ix);
+    return CHIMERA_OK;
+}
+
+int chimera_destroy_index(chimera_index *index)
+{
+    Index *ix = reinterpret_cast<Index *>(index);
+    if (!ix) return CHIMERA_OK;
+    cudaFree(ix->doc_off);
+    cudaFree(ix->cdig);
+    cudaFree(ix->ivf_off);
+    cudaFree(ix->ivf_doc);
+    delete ix;
+    return CHIMERA_OK;
+}
+
+int chimera_index_info(const chimera_index *index, chimera_index_desc *desc, int64_t *posting_entries,
+                       int32_t *max_doclen)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    if (!ix) return fail(CHIMERA_INVALID_ARG, "index is NULL");
+    if (desc) {
+        desc->dim = ix->D; desc->nbits = ix->nbits; desc->res_lo = ix->res_lo; desc->res_hi = ix->res_hi;
+        desc->n_centroids = ix->K; desc->n_docs = ix->N; desc->n_tokens = ix->T;
+    }
+    if (posting_entries) *posting_entries = ix->ivf_len;
+    if (max_doclen) *max_doclen = ix->max_doclen;
+    return CHIMERA_OK;
+}
+
+int chimera_workspace_bytes(const chimera_index *index, int32_t n_queries, int32_t q_len, int32_t nprobe,
+                            int32_t n_prune, int32_t k, int64_t max_candidates, size_t *out)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc) return rc;
+    if (!out) return fail(CHIMERA_INVALID_ARG, "out is NULL");
+    *out = make_layout(*ix, p).total;
+    return CHIMERA_OK;
+}
+
+int chimera_search_tapped(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                          int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                          size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
+                          const chimera_taps *taps)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc) return rc;
+    return run(*ix, p, 1, 5, queries, workspace, workspace_bytes, (cudaStream_t)stream, taps, out_ids, out_scores);
+}
+
+int chimera_search(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                   int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                   size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores)
+{
+    return chimera_search_tapped(index, queries, n_queries, q_len, nprobe, n_prune, k, max_candidates, workspace,
+                                 workspace_bytes, stream, out_ids, out_scores, nullptr);
+}
+
+int chimera_search_host(const chimera_index *index, const float *queries_host, int32_t n_queries, int32_t q_len,
+                        int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                        size_t workspace_bytes, void *stream, int32_t *out_ids_host, float *out_scores_host)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc) return rc;
+    if (!queries_host || !out_ids_host || !out_scores_host) return fail(CHIMERA_INVALID_ARG, "NULL host buffer");
+    if (!workspace || ((uintptr_t)workspace & 255)) return fail(CHIMERA_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
+    const Layout L = make_layout(*ix, p);
+    if (workspace_bytes < L.total)
+        return fail(CHIMERA_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = (char *)workspace;
+    float *dq = (float *)(ws + L.q_stage);
+    int32_t *dids = (int32_t *)(ws + L.out_ids);
+    float *dsc = (float *)(ws + L.out_scores);
+    const size_t qbytes = (size_t)p.B * p.nq * ix->D * sizeof(float);
+    CHIMERA_CUDA(cudaMemcpyAsync(dq, queries_host, qbytes, cudaMemcpyHostToDevice, st));
+    rc = run(*ix, p, 1, 5, dq, workspace, workspace_bytes, st, nullptr, dids, dsc);
+    if (rc) return rc;
+    CHIMERA_CUDA(cudaMemcpyAsync(out_ids_host, dids, (size_t)p.B * p.k * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CHIMERA_CUDA(cudaMemcpyAsync(out_scores_host, dsc, (size_t)p.B * p.k * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CHIMERA_CUDA(cudaStreamSynchronize(st));
+    return CHIMERA_OK;
+}
+
+int chimera_run_stages(const chimera_index *index, int32_t first_stage, int32_t last_stage, const float *queries,
+                       int32_t n_queries, int32_t q_len, int32_t nprobe, int32_t n_prune, int32_t k,
+                       int64_t max_candidates, void *workspace, size_t workspace_bytes, void *stream,
+                       const chimera_taps *inout, int32_t *out_ids, float *out_scores)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc) return rc;
+    if (first_stage < 1 || last_stage > 5 || first_stage > last_stage)
+        return fail(CHIMERA_INVALID_ARG, "stages must satisfy 1 <= first <= last <= 5");
+    return run(*ix, p, first_stage, last_stage, queries, workspace, workspace_bytes, (cudaStream_t)stream, inout,
+               out_ids, out_scores);
+}
+
+int chimera_workspace_status(const void *workspace, void *stream, int32_t *status)
+{
+    if (!workspace || !status) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    uint32_t bits = 0;
+    CHIMERA_CUDA(cudaMemcpyAsync(&bits, workspace, sizeof(bits), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CHIMERA_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    if (bits & ST_TIMEOUT) *status = CHIMERA_TIMEOUT;
+    else if (bits & ST_BAD_QUERY) *status = CHIMERA_INVALID_ARG;
+    else if (bits & ST_OVERFLOW) *status = CHIMERA_CAPACITY_OVERFLOW;
+    else *status = CHIMERA_OK;
+    return CHIMERA_OK;
+}
+
+int chimera_profile_enable(int32_t on)
+{
+    g_prof_on = on != 0;
+    return CHIMERA_OK;
+}
+
+int chimera_profile_read(float *ms, int64_t *launches)
+{
+    if (!ms || !launches) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    for (int s = 0; s < CHIMERA_PROFILE_SLOTS; ++s) { ms[s] = 0.f; launches[s] = g_launches[s]; g_launches[s] = 0; }
+    for (int c = 0; c < g_n_calls; ++c) {
+        ProfCall &pc = g_calls[c];
+        if (pc.n < 2) continue;
+        CHIMERA_CUDA(cudaEventSynchronize(pc.ev[pc.n - 1]));
+        for (int i = 1; i < pc.n; ++i) {
+            float t = 0.f;
+            CHIMERA_CUDA(cudaEventElapsedTime(&t, pc.ev[i - 1], pc.ev[i]));
+            if (pc.slot[i] >= 0 && pc.slot[i] < CHIMERA_PROFILE_SLOTS) ms[pc.slot[i]] += t;
+        }
+        pc.n = 0;
+    }
+    g_n_calls = 0;
+    g_cur = nullptr;
+    return CHIMERA_OK;
+}
+
+}  // extern "C"

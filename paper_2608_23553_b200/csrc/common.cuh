@@ -1,0 +1,142 @@
+// Shared declarations of libchimera's translation units (host side + small device helpers).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "chimera.h"
+
+namespace chimera {
+
+// ---------------------------------------------------------------------------------------------------------------
+// Index: everything resident on the device between searches.
+// ---------------------------------------------------------------------------------------------------------------
+struct Index {
+    int device = 0;
+    int sm_count = 0;
+    int D = 0, nbits = 0, CB = 0;     // dim, residual bits per dim, code bytes per token
+    int64_t K = 0, N = 0, T = 0;
+    float res_lo = 0.f, res_hi = 0.f;
+    const int32_t *cids = nullptr;    // [T]        borrowed
+    const uint8_t *codes = nullptr;   // [T, CB]    borrowed
+    int64_t *doc_off = nullptr;       // [N+1]      owned: first token of each document
+    int8_t *cdig = nullptr;           // [3][K][D]  owned: balanced base-256 digits of rint(c * 2^22)
+    int64_t *ivf_off = nullptr;       // [K+1]      owned
+    int32_t *ivf_doc = nullptr;       // [ivf_len]  owned: unique document ids per centroid, unordered
+    int64_t ivf_len = 0;
+    int32_t max_doclen = 0;
+};
+
+// Device status bits kept in the first word of a workspace.
+enum : uint32_t { ST_OVERFLOW = 1u, ST_BAD_QUERY = 2u, ST_TIMEOUT = 4u };
+
+// ---------------------------------------------------------------------------------------------------------------
+// Workspace layout (all offsets 256-byte aligned).
+// ---------------------------------------------------------------------------------------------------------------
+struct Params {
+    int32_t B, nq, P, n_prune, k;
+    int64_t maxc;                     // candidate capacity per query
+};
+
+struct Layout {
+    size_t status;        // uint32[64]
+    size_t q_stage;       // float  [B, nq, D]        (host-entry staging of the queries)
+    size_t out_ids;       // int32  [B, k]            (host-entry staging)
+    size_t out_scores;    // float  [B, k]
+    size_t qdig;          // int8   [3][B*nq][D]
+    size_t table;         // int32  [B][K][nq]
+    size_t part;          // uint64 [B][n_part][P][nq] partial top-P keys
+    size_t probes;        // int32  [B][nq][P]
+    size_t bitmap;        // uint32 [B][words]
+    size_t chunk_cnt;     // int32  [B][n_chunks + 1]
+    size_t cand;          // int32  [B][maxc]
+    size_t n_cand;        // int32  [B]
+    size_t ci;            // int32  [B][maxc]
+    size_t pruned;        // int32  [B][n_prune]
+    size_t n_pruned;      // int32  [B]
+    size_t score4;        // float  [B][n_prune]
+    size_t total;
+    // derived sizes
+    int32_t n_part;       // partial lists per query in the probe stage
+    int32_t probe_blocks; // blocks per query in the probe stage
+    int64_t words;        // bitmap words per query
+    int32_t n_chunks;     // bitmap chunks per query
+};
+
+constexpr int PROBE_WARPS = 8;          // warps per block in the probe stage (each keeps its own partial list)
+constexpr int BITMAP_CHUNK_WORDS = 1024; // bitmap words per compaction block
+
+Layout make_layout(const Index &ix, const Params &p);
+
+// ---------------------------------------------------------------------------------------------------------------
+// Error text (thread local) and helpers.
+// ---------------------------------------------------------------------------------------------------------------
+int fail(int code, const char *fmt, ...);
+#define CHIMERA_CUDA(call)                                                                      \
+    do {                                                                                        \
+        cudaError_t e__ = (call);                                                               \
+        if (e__ != cudaSuccess)                                                                 \
+            return ::chimera::fail(CHIMERA_CUDA_ERROR, "%s: %s", #call, cudaGetErrorString(e__)); \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------------------------
+// Profiling hooks (api.cu).
+// ---------------------------------------------------------------------------------------------------------------
+enum Slot { SLOT_G1 = 0, SLOT_PROBE, SLOT_GATHER, SLOT_CI, SLOT_SELECT, SLOT_G4, SLOT_TOPK, SLOT_MISC };
+void count_launch(int slot, int n = 1);
+
+// ---------------------------------------------------------------------------------------------------------------
+// Stage launchers (one per .cu file).  Each only enqueues kernels on `st` and returns a chimera_status.
+// ---------------------------------------------------------------------------------------------------------------
+int build_index_device(Index &ix, const float *centroids, const int32_t *doclens, cudaStream_t st);
+// rows x D float32 in [-1, 1] -> three int8 digit planes [3][rows][D]; out-of-range elements set ST_BAD_QUERY.
+int launch_digits(const float *x, int64_t rows, int D, int8_t *dig, uint32_t *status, cudaStream_t st);
+
+int launch_score_table(const Index &ix, const Params &p, const float *queries, int8_t *qdig, int32_t *table,
+                       uint32_t *status, cudaStream_t st);
+int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32_t *table, unsigned long long *part,
+                  int32_t *probes, cudaStream_t st);
+int launch_gather(const Index &ix, const Params &p, const Layout &L, const int32_t *probes, uint32_t *bitmap,
+                  int32_t *chunk_cnt, int32_t *cand, int32_t *n_cand, uint32_t *status, cudaStream_t st);
+int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
+                                const int32_t *n_cand, int32_t *ci, cudaStream_t st);
+int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
+                  int32_t *pruned, int32_t *n_pruned, cudaStream_t st);
+int launch_residual_scores(const Index &ix, const Params &p, const float *queries, const int32_t *table,
+                           const int32_t *pruned, float *score4, cudaStream_t st);
+int launch_topk(const Index &ix, const Params &p, const int32_t *pruned, const float *score4, int32_t *out_ids,
+                float *out_scores, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------------------
+// Device helpers.
+// ---------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int warp_sum(int v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_max(unsigned long long v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long w = __shfl_xor_sync(0xffffffffu, v, o);
+        v = w > v ? w : v;
+    }
+    return v;
+}
+
+// Order-preserving key of (score desc, id asc): a larger key is a better entry.
+__device__ __forceinline__ unsigned long long key_int(int32_t score, int32_t id)
+{
+    return ((unsigned long long)((uint32_t)score ^ 0x80000000u) << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
+}
+__device__ __forceinline__ int32_t key_id(unsigned long long key) { return (int32_t)(0xFFFFFFFFu - (uint32_t)key); }
+
+}  // namespace chimera
