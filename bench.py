@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Benchmark of the GPU-resident retrieval path (stages 1-5 behind chimera_search).
+
+A step is one chimera_search call over one batch of synthetic queries on the Mid corpus (500k documents, ~60M
+tokens, 65,536 centroids, 2-bit residual codes; nprobe 4, n_prune 1024, k 10).  `value` is queries per second at
+batch 256 with the queries already on the device; `e2e` is the same through chimera_search_host with pinned host
+buffers (host->device and device->host copies inside the timed region); `qps_batch1` follows the paper's protocol of
+one synchronised query at a time.  The path does not shard: with --gpus N every rank runs an independent replica.
+
+`--impl reference` times the CPU oracle (as it stands, one thread) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from synth import CONFIGS, make_corpus, make_queries  # noqa: E402
+
+METRIC = "QPS at batch 256 (Mid corpus, nprobe 4, n_prune 1024, k 10)"
+UNIT = "queries/s"
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_workload(cfg, device):
+    t0 = time.time()
+    corp = make_corpus(cfg, device=device)
+    q = make_queries(cfg, device=device)
+    torch.cuda.synchronize() if device.type == "cuda" else None
+    return corp, q, time.time() - t0
+
+
+def oracle_index(corp, cfg):
+    import oracle
+    return oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+
+
+def time_oracle(oix, q_np, cfg, budget_s, min_q, max_q):
+    """Runs the oracle pipeline on queries 0.. until the time budget is used; returns (queries, seconds)."""
+    import oracle
+    n, t0 = 0, time.perf_counter()
+    while n < max_q and (n < min_q or time.perf_counter() - t0 < budget_s):
+        oracle.pipeline(q_np[n % q_np.shape[0]], oix, cfg.nprobe, cfg.n_prune, cfg.k)
+        n += 1
+    return n, time.perf_counter() - t0
+
+
+def run_reference(args, cfg, rank, world):
+    """The CPU oracle as the reference arm: rank 0 only; a step is one query (a bounded sample of a batch)."""
+    if rank != 0:
+        return
+    device = torch.device("cuda:0") if torch.cuda.is_available() else torch.device("cpu")
+    corp, q, _ = build_workload(cfg, device)
+    oix = oracle_index(corp, cfg)
+    q_np = q.cpu().numpy()
+    del corp
+    import oracle
+    for s in range(args.warmup):
+        oracle.pipeline(q_np[s % len(q_np)], oix, cfg.nprobe, cfg.n_prune, cfg.k)
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        oracle.pipeline(q_np[(args.warmup + s) % len(q_np)], oix, cfg.nprobe, cfg.n_prune, cfg.k)
+    dt = time.perf_counter() - t0
+    qps = args.steps / dt
+    sample = "1 query per step (of the %d-query batch), %d steps, single thread" % (args.batch, args.steps)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64+f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": 1, "sample": sample},
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="mid")
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--batch1-queries", type=int, default=200)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    cfg = CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+
+    import paper_2608_23553_b200 as pkg
+    pkg.lib()                                    # fails loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    corp, q, gen_s = build_workload(cfg, device)
+    t0 = time.time()
+    index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    build_s = time.time() - t0
+    B, nq, P, n_prune, k = args.batch, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
+
+    # batches cycle through the config's query set
+    n_batches = max(1, min(args.steps + args.warmup, (q.shape[0] + B - 1) // B + 1))
+    idx = (torch.arange(n_batches * B, device=device) % q.shape[0]).view(n_batches, B)
+    batches = q[idx].contiguous()                                   # [n_batches, B, nq, D] on the device
+    host_batches = batches.cpu().pin_memory()
+    out = (torch.empty(B, k, dtype=torch.int32, device=device), torch.empty(B, k, dtype=torch.float32, device=device))
+    host_out = (torch.empty(B, k, dtype=torch.int32).pin_memory(), torch.empty(B, k, dtype=torch.float32).pin_memory())
+
+    # algorithmic work per batch (outside the timed region): candidate documents and their tokens, from the taps
+    doclens64 = corp.doclens.to(torch.int64)
+    work = []
+    for bi in range(n_batches):
+        taps = index.alloc_taps(B, nq, P, n_prune, table=False)
+        index.search(batches[bi], P, n_prune, k, taps=taps)
+        assert index.status() == 0
+        mask = torch.arange(index.N, device=device)[None, :] < taps.n_cand[:, None].to(torch.int64)
+        toks = (doclens64[taps.cand.to(torch.int64).clamp_(0, index.N - 1)] * mask).sum()
+        pr = taps.pruned.to(torch.int64)
+        toks4 = (doclens64[pr.clamp(min=0)] * (pr >= 0)).sum()
+        work.append({"cand": int(taps.n_cand.sum()), "cand_tokens": int(toks), "pruned_tokens": int(toks4)})
+        del taps, mask
+    torch.cuda.empty_cache()
+
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps ------------------------------------
+    for s in range(args.warmup):
+        index.search(batches[s % n_batches], P, n_prune, k, out=out)
+    barrier()
+    pkg.profile_enable(True)
+    pkg.profile_read()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(args.steps):
+        index.search(batches[(args.warmup + s) % n_batches], P, n_prune, k, out=out)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    stage_ms, launches = pkg.profile_read()
+    pkg.profile_enable(False)
+    t = torch.tensor([ms_total], device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    qps = world * B * args.steps / (ms_total / 1e3)
+
+    # ---- end to end through the host entry point: pinned host queries in, host ids/scores out -------------------
+    for s in range(2):
+        index.search_host(host_batches[s % n_batches], P, n_prune, k, out=host_out)
+    barrier()
+    w0 = time.perf_counter()
+    for s in range(args.steps):
+        index.search_host(host_batches[(args.warmup + s) % n_batches], P, n_prune, k, out=host_out)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - w0
+    t = torch.tensor([e2e_s], device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_qps = world * B * args.steps / float(t.item())
+    h2d = B * nq * cfg.dim * 4
+    d2h = B * k * 8
+
+    # ---- batch 1: one synchronised query at a time (the paper's protocol: latency = 1 / QPS) --------------------
+    n1 = min(args.batch1_queries, q.shape[0])
+    out1 = (torch.empty(1, k, dtype=torch.int32, device=device), torch.empty(1, k, dtype=torch.float32, device=device))
+    for i in range(5):
+        index.search(q[i:i + 1], P, n_prune, k, out=out1)
+    torch.cuda.synchronize()
+    lat = []
+    for i in range(n1):
+        a = time.perf_counter()
+        index.search(q[i:i + 1], P, n_prune, k, out=out1)
+        torch.cuda.synchronize()
+        lat.append(time.perf_counter() - a)
+    lat = np.array(lat)
+    host_q1 = q[:n1].cpu().pin_memory()
+    hout1 = (torch.empty(1, k, dtype=torch.int32).pin_memory(), torch.empty(1, k, dtype=torch.float32).pin_memory())
+    w0 = time.perf_counter()
+    for i in range(n1):
+        index.search_host(host_q1[i:i + 1], P, n_prune, k, out=hout1)
+    e2e1_qps = n1 / (time.perf_counter() - w0)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the centroid-interaction scan) ----------------------------------------
+    peak, peak_kind = measured_peaks()
+    used = [work[(args.warmup + s) % n_batches] for s in range(args.steps)]
+    mean = lambda key: float(np.mean([u[key] for u in used]))       # noqa: E731
+    n_prof = min(args.steps, 256)                                    # the library times at most 256 calls per read
+    ci_ms = stage_ms["centroid_interaction"] / n_prof
+    # algorithmic bytes of one launch: centroid ids of every candidate token (4 B) + per candidate document its id
+    # (4 B) and two offsets (16 B) + the CI written (4 B)
+    ci_bytes = 4.0 * mean("cand_tokens") + 24.0 * mean("cand")
+    ci_gbs = ci_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0
+    l2_bytes = mean("cand_tokens") * nq * 4.0
+    g4_ms = stage_ms["residual_scores"] / n_prof
+    g4_bytes = mean("pruned_tokens") * (4.0 + cfg.code_bytes)
+    stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
+    roofline = {
+        "kernel": "ci_kernel (stage 3 centroid-interaction scan)", "bound": "hbm",
+        "achieved": ci_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+        "frac": ci_gbs / peak, "traffic": None, "ms_per_launch": ci_ms, "algorithmic_bytes_per_launch": ci_bytes,
+        "binding_roof": {"bound": "l2_gather", "bytes_per_launch": l2_bytes,
+                         "achieved_gbs": l2_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0},
+        "stage_ms_per_step": stages,
+        "stage4": {"ms_per_launch": g4_ms, "code_gbs": g4_bytes / (g4_ms * 1e-3) / 1e9 if g4_ms > 0 else 0.0,
+                   "tflops": 2.0 * mean("pruned_tokens") * nq * cfg.dim / (g4_ms * 1e-3) / 1e12 if g4_ms > 0 else 0.0},
+    }
+
+    result = {
+        "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32 fixed point (stages 1-3) + f32 (stage 4)", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": B, "n_docs": cfg.n_docs, "n_tokens": corp.n_tokens,
+                   "n_centroids": cfg.n_centroids, "dim": cfg.dim, "nbits": cfg.nbits, "q_len": nq, "nprobe": P,
+                   "n_prune": n_prune, "k": k, "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (2.2 GB index, 2.1 GB score table per batch); no flush",
+                   "gen_s": round(gen_s, 1), "index_build_s": round(build_s, 2)},
+        "qps_batch1": float(1.0 / lat.mean()),
+        "latency_ms_batch1": {"mean": float(lat.mean() * 1e3), "p50": float(np.percentile(lat, 50) * 1e3),
+                              "p95": float(np.percentile(lat, 95) * 1e3), "p99": float(np.percentile(lat, 99) * 1e3)},
+        "e2e": {"value": e2e_qps, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "batch1_value": e2e1_qps},
+        "gpu_launches": int(sum(launches.values())),
+        "clocks": clocks,
+        "roofline": roofline,
+    }
+
+    if world == 1 and not args.no_cpu_baseline:
+        oix = oracle_index(corp, cfg)
+        n, secs = time_oracle(oix, q.cpu().numpy(), cfg, budget_s=12.0, min_q=3, max_q=16)
+        result["cpu_baseline"] = {"value": n / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                  "sample": "first %d queries of the workload, all stages, %.1f s" % (n, secs)}
+    print(json.dumps(result))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
