@@ -72,6 +72,68 @@ ci_kernel(const int32_t *__restrict__ table, int64_t K, int nq, const int32_t *_
     }
 }
 
+// Wide variant for q_len = 4 * LPR (LPR = 8, 16 or 32 lanes per table row): every lane loads 16 bytes (four query
+// tokens) of a row, so one load instruction of the warp covers 32 / LPR document tokens.  Lane group g = lane / LPR
+// takes tokens g, g + TPL, g + 2 TPL, ... of each 32-token slab; the group maxima are merged with shuffles at the end.
+template <int LPR>
+__global__ void __launch_bounds__(CI_THREADS)
+ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__restrict__ cand,
+               const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
+               const int64_t *__restrict__ doc_off, int32_t *__restrict__ ci)
+{
+    constexpr int NQ = 4 * LPR;
+    constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
+    constexpr int UNROLL = 4;
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const int grp = lane / LPR, sub = lane % LPR;
+    const int n = n_cand[b];
+    const int4 *tb = reinterpret_cast<const int4 *>(table + (int64_t)b * K * NQ) + sub;
+    const int32_t *cb = cand + (int64_t)b * maxc;
+    int32_t *out = ci + (int64_t)b * maxc;
+    const int warps_per_query = gridDim.x * CI_WARPS;
+    for (int j = blockIdx.x * CI_WARPS + (threadIdx.x >> 5); j < n; j += warps_per_query) {
+        const int64_t d = cb[j];
+        const int64_t t0 = doc_off[d], t1 = doc_off[d + 1];
+        int4 m = make_int4(INT_MIN, INT_MIN, INT_MIN, INT_MIN);
+        for (int64_t base = t0; base < t1; base += 32) {
+            const int cnt = (int)((t1 - base) < 32 ? (t1 - base) : 32);
+            // lanes past the end repeat the last token: a duplicate cannot change a maximum
+            const int32_t cidv = cids[base + (lane < cnt ? lane : cnt - 1)];
+            for (int s = 0; s * TPL < cnt; s += UNROLL) {
+                int4 v[UNROLL];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    int src = (s + u) * TPL + grp;
+                    src = src < 32 ? src : 31;    // lane 31 holds a valid (possibly repeated) token
+                    const int32_t c = __shfl_sync(0xffffffffu, cidv, src);
+                    v[u] = __ldg(tb + (int64_t)c * LPR);
+                }
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    m.x = max(m.x, v[u].x);
+                    m.y = max(m.y, v[u].y);
+                    m.z = max(m.z, v[u].z);
+                    m.w = max(m.w, v[u].w);
+                }
+            }
+        }
+        // merge the TPL lane groups (same columns, different tokens)
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+            m.x = max(m.x, __shfl_xor_sync(0xffffffffu, m.x, o));
+            m.y = max(m.y, __shfl_xor_sync(0xffffffffu, m.y, o));
+            m.z = max(m.z, __shfl_xor_sync(0xffffffffu, m.z, o));
+            m.w = max(m.w, __shfl_xor_sync(0xffffffffu, m.w, o));
+        }
+        // sum over the NQ columns: four per lane, LPR lanes
+        int sum = m.x + m.y + m.z + m.w;
+#pragma unroll
+        for (int o = LPR >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) out[j] = sum;
+    }
+}
+
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
                                 const int32_t *n_cand, int32_t *ci, cudaStream_t st)
 {
@@ -81,7 +143,13 @@ int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t 
     if (gx < 1) gx = 1;
     dim3 grid(gx, (unsigned)p.B);
     const int nqw = (p.nq + 31) / 32;
-    if (nqw == 1)
+    if (p.nq == 32)
+        ci_wide_kernel<8><<<grid, CI_THREADS, 0, st>>>(table, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
+    else if (p.nq == 64)
+        ci_wide_kernel<16><<<grid, CI_THREADS, 0, st>>>(table, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
+    else if (p.nq == 128)
+        ci_wide_kernel<32><<<grid, CI_THREADS, 0, st>>>(table, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
+    else if (nqw == 1)
         ci_kernel<1><<<grid, CI_THREADS, 0, st>>>(table, ix.K, p.nq, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
     else if (nqw == 2)
         ci_kernel<2><<<grid, CI_THREADS, 0, st>>>(table, ix.K, p.nq, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
