@@ -87,7 +87,7 @@ Layout make_layout(const Index &ix, const Params &p)
     L.q_stage = take(B * nq * ix.D * sizeof(float));
     L.out_ids = take(B * p.k * sizeof(int32_t));
     L.out_scores = take(B * p.k * sizeof(float));
-    L.qdig = take(3 * B * nq * ix.D);
+    L.qdig = take(3 * B * nq * 128);
     L.table = take(B * (size_t)ix.K * nq * sizeof(int32_t));
     L.part = take(B * L.n_part * p.P * nq * sizeof(unsigned long long));
     L.probes = take(B * nq * p.P * sizeof(int32_t));

@@ -20,7 +20,7 @@ struct Index {
     const int32_t *cids = nullptr;    // [T]        borrowed
     const uint8_t *codes = nullptr;   // [T, CB]    borrowed
     int64_t *doc_off = nullptr;       // [N+1]      owned: first token of each document
-    int8_t *cdig = nullptr;           // [3][K][D]  owned: balanced base-256 digits of rint(c * 2^22)
+    int8_t *cdig = nullptr;           // [3][K][128] owned: balanced base-256 digits of rint(c * 2^22), zero padded
     int64_t *ivf_off = nullptr;       // [K+1]      owned
     int32_t *ivf_doc = nullptr;       // [ivf_len]  owned: unique document ids per centroid, unordered
     int64_t ivf_len = 0;
@@ -43,7 +43,7 @@ struct Layout {
     size_t q_stage;       // float  [B, nq, D]        (host-entry staging of the queries)
     size_t out_ids;       // int32  [B, k]            (host-entry staging)
     size_t out_scores;    // float  [B, k]
-    size_t qdig;          // int8   [3][B*nq][D]
+    size_t qdig;          // int8   [3][B*nq][128]
     size_t table;         // int32  [B][K][nq]
     size_t part;          // uint64 [B][n_part][P][nq] partial top-P keys
     size_t probes;        // int32  [B][nq][P]
@@ -89,7 +89,8 @@ void count_launch(int slot, int n = 1);
 // Stage launchers (one per .cu file).  Each only enqueues kernels on `st` and returns a chimera_status.
 // ---------------------------------------------------------------------------------------------------------------
 int build_index_device(Index &ix, const float *centroids, const int32_t *doclens, cudaStream_t st);
-// rows x D float32 in [-1, 1] -> three int8 digit planes [3][rows][D]; out-of-range elements set ST_BAD_QUERY.
+// rows x D float32 in [-1, 1] -> three int8 digit planes [3][rows][128] (zero padded); out-of-range elements set
+// ST_BAD_QUERY.
 int launch_digits(const float *x, int64_t rows, int D, int8_t *dig, uint32_t *status, cudaStream_t st);
 
 int launch_score_table(const Index &ix, const Params &p, const float *queries, int8_t *qdig, int32_t *table,

@@ -6,60 +6,275 @@
 // Products of equal weight a+b share an accumulator (five accumulators, each |.| < 2^23); the epilogue recombines
 // them with shifts in int64 and rounds.
 //
-// This file: digit split of the queries + the contraction on CUDA cores with dp4a (exact int32 accumulation).
+// The contraction runs on the 5th-generation tensor cores: tcgen05.mma kind::i8 (int8 operands, int32 accumulators in
+// tensor memory), M = 128 centroids x N = 48 query tokens x K = 32 dimensions per instruction.  Both operands are
+// K-major digit planes with a 128-byte row pitch (dimensions beyond D are zero), brought into 128-byte-swizzled shared
+// memory by TMA (plain per-CTA cp.async.bulk.tensor loads, no multicast).  One CTA owns a tile of 128 centroids (its
+// three digit planes stay in shared memory) and walks over tiles of 48 query-token rows, double-buffering the query
+// planes.  The five accumulators take 240 of the 256 tensor-memory columns a CTA allocates, so two CTAs share an SM and
+// one's epilogue overlaps the other's MMAs.  Every wait on an mbarrier is bounded; a wait that gives up sets the
+// workspace's TIMEOUT status bit and the CTA frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace chimera {
 
-constexpr int G1_CT = 64;        // centroids per block
-constexpr int G1_THREADS = 256;
+constexpr int G1_M = 128;            // centroids per tile (MMA M)
+constexpr int G1_N = 48;             // query-token rows per tile (MMA N)
+constexpr int G1_ROW_BYTES = 128;    // digit-plane row pitch = padded dimension count
+constexpr int G1_THREADS = 128;
+constexpr int G1_TMEM_COLS = 256;
+constexpr uint32_t G1_A_PLANE = G1_M * G1_ROW_BYTES;      // 16 KB
+constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;      // 6 KB
+constexpr uint32_t G1_SMEM = 3 * G1_A_PLANE + 2 * 3 * G1_B_PLANE + 1024 /* alignment slack */ + 64 /* barriers */;
+constexpr long long G1_WAIT_CYCLES = 2000000000LL;         // ~1 s at 2 GHz
 
-// grid (ceil(K / G1_CT), B).  smem: query digits transposed [3][D/4][nq] and centroid digits [3][G1_CT][D/4].
-__global__ void __launch_bounds__(G1_THREADS)
-score_table_dp4a(const int8_t *__restrict__ qdig, const int8_t *__restrict__ cdig, int64_t K, int D, int nq,
-                 int64_t q_rows_total, int32_t *__restrict__ table)
+// ------------------------------------------------------------------------------------------------ PTX wrappers ---
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    extern __shared__ int smem_i[];
-    const int G = D >> 2;                       // 4-dim groups
-    int *qs = smem_i;                           // [3][G][nq]
-    int *cs = smem_i + 3 * G * nq;              // [3][G1_CT][G]
-    const int b = blockIdx.y;
-    const int64_t c0 = (int64_t)blockIdx.x * G1_CT;
-    const int n_c = (int)((K - c0) < G1_CT ? (K - c0) : G1_CT);
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity to complete.  false = gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.b32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (clock64() - t0 > G1_WAIT_CYCLES) return false;
+    }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+// Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
+{
+    return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
+        "[%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
 
-    const int *q32 = reinterpret_cast<const int *>(qdig);
-    const int *c32 = reinterpret_cast<const int *>(cdig);
-    for (int e = threadIdx.x; e < 3 * nq * G; e += G1_THREADS) {
-        int p = e / (nq * G), r = e % (nq * G), i = r / G, g = r % G;
-        qs[(p * G + g) * nq + i] = q32[((int64_t)p * q_rows_total + (int64_t)b * nq + i) * G + g];
+__device__ __forceinline__ int32_t combine_digits(int32_t a0, int32_t a1, int32_t a2, int32_t a3, int32_t a4)
+{
+    long long T = (long long)a0 + (long long)a1 * 256LL + (long long)a2 * 65536LL + (long long)a3 * 16777216LL +
+                  (long long)a4 * 4294967296LL;
+    return (int32_t)((T + (1LL << 19)) >> 20);
+}
+
+// grid (ceil(K / 128), n_splits).  Each CTA: centroid tile blockIdx.x, query-row tiles [blockIdx.y * tiles_per_split, ...).
+__global__ void __launch_bounds__(G1_THREADS)
+score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_q, int64_t K,
+                 int nq, int64_t q_rows, int k_steps, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
+                 uint32_t *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sA = base;                                  // 3 planes x 16 KB
+    const uint32_t sB = base + 3 * G1_A_PLANE;                 // 2 stages x 3 planes x 6 KB
+    const uint32_t bars = sB + 2 * 3 * G1_B_PLANE;             // full_a, full_b[2], mma_done
+    const uint32_t bar_a = bars, bar_b0 = bars + 8, bar_mma = bars + 24;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t c0 = (int64_t)blockIdx.x * G1_M;
+    const int t_begin = blockIdx.y * tiles_per_split;
+    int t_end = t_begin + tiles_per_split;
+    if (t_end > n_tiles) t_end = n_tiles;
+
+    if (tid == 0) {
+        mbar_init(bar_a, 1);
+        mbar_init(bar_b0, 1);
+        mbar_init(bar_b0 + 8, 1);
+        mbar_init(bar_mma, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int e = threadIdx.x; e < 3 * n_c * G; e += G1_THREADS) {
-        int p = e / (n_c * G), r = e % (n_c * G), c = r / G, g = r % G;
-        cs[(p * G1_CT + c) * G + g] = c32[((int64_t)p * K + c0 + c) * G + g];
+    if (warp == 0) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                     "r"(G1_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s_tmem_base;
 
-    int32_t *out = table + ((int64_t)b * K + c0) * nq;
-    for (int o = threadIdx.x; o < n_c * nq; o += G1_THREADS) {
-        const int c = o / nq, i = o % nq;
-        int a0 = 0, a1 = 0, a2 = 0, a3 = 0, a4 = 0;
-        for (int g = 0; g < G; ++g) {
-            int q0 = qs[(0 * G + g) * nq + i], q1 = qs[(1 * G + g) * nq + i], q2 = qs[(2 * G + g) * nq + i];
-            int x0 = cs[(0 * G1_CT + c) * G + g], x1 = cs[(1 * G1_CT + c) * G + g], x2 = cs[(2 * G1_CT + c) * G + g];
-            a0 = __dp4a(q0, x0, a0);
-            a1 = __dp4a(q0, x1, a1);
-            a1 = __dp4a(q1, x0, a1);
-            a2 = __dp4a(q0, x2, a2);
-            a2 = __dp4a(q1, x1, a2);
-            a2 = __dp4a(q2, x0, a2);
-            a3 = __dp4a(q1, x2, a3);
-            a3 = __dp4a(q2, x1, a3);
-            a4 = __dp4a(q2, x2, a4);
-        }
-        long long T = (long long)a0 + (long long)a1 * 256LL + (long long)a2 * 65536LL + (long long)a3 * 16777216LL +
-                      (long long)a4 * 4294967296LL;
-        out[o] = (int32_t)((T + (1LL << 19)) >> 20);
+    // instruction descriptor: D = S32, A and B signed 8-bit, both K-major, N = 48, M = 128
+    constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(G1_N >> 3) << 17) |
+                               ((uint32_t)(G1_M >> 4) << 24);
+
+    if (tid == 0 && t_begin < t_end) {
+        mbar_expect_tx(bar_a, 3 * G1_A_PLANE);
+        for (int p = 0; p < 3; ++p) tma_load_3d(sA + p * G1_A_PLANE, &map_c, 0, (int)c0, p, bar_a);
+        mbar_expect_tx(bar_b0, 3 * G1_B_PLANE);
+        for (int p = 0; p < 3; ++p) tma_load_3d(sB + p * G1_B_PLANE, &map_q, 0, t_begin * G1_N, p, bar_b0);
     }
+
+    for (int t = t_begin; t < t_end; ++t) {
+        const int it = t - t_begin, stage = it & 1;
+        if (tid == 0) {
+            bool ok = true;
+            if (t + 1 < t_end) {           // the other stage was released by the previous tile's completed MMAs
+                const uint32_t nb = bar_b0 + 8 * (stage ^ 1);
+                mbar_expect_tx(nb, 3 * G1_B_PLANE);
+                for (int p = 0; p < 3; ++p)
+                    tma_load_3d(sB + ((stage ^ 1) * 3 + p) * G1_B_PLANE, &map_q, 0, (t + 1) * G1_N, p, nb);
+            }
+            if (it == 0) ok = mbar_wait(bar_a, 0);
+            if (ok) ok = mbar_wait(bar_b0 + 8 * stage, (it >> 1) & 1);
+            if (ok) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int w = 0; w < 5; ++w) {              // accumulator = digit weight a + b
+                    bool first = true;
+                    for (int a = 0; a < 3; ++a) {          // query digit
+                        const int bdig = w - a;            // centroid digit
+                        if (bdig < 0 || bdig > 2) continue;
+                        const uint64_t da = umma_desc(sA + bdig * G1_A_PLANE);
+                        const uint64_t db = umma_desc(sB + (stage * 3 + a) * G1_B_PLANE);
+                        for (int k = 0; k < k_steps; ++k) {
+                            umma_i8(tmem + w * G1_N, da + 2 * k, db + 2 * k, IDESC, first ? 0u : 1u);
+                            first = false;
+                        }
+                    }
+                }
+                umma_commit(bar_mma);
+            } else {
+                s_abort = 1;
+                atomicOr(status, ST_TIMEOUT);
+            }
+        }
+        __syncwarp();
+        // everybody waits for the accumulators (bounded), then drains them
+        const bool ok = mbar_wait(bar_mma, it & 1);
+        if (!__syncthreads_and(ok && !*(volatile int *)&s_abort)) {      // uniform decision for the whole CTA
+            if (tid == 0) atomicOr(status, ST_TIMEOUT);
+            break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        __syncwarp();
+        const int64_t c = c0 + warp * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+        for (int chunk = 0; chunk < G1_N / 16; ++chunk) {
+            int32_t acc[5][16];
+#pragma unroll
+            for (int w = 0; w < 5; ++w) tmem_ld16(lane_addr + w * G1_N + chunk * 16, acc[w]);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            int32_t out[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) out[e] = combine_digits(acc[0][e], acc[1][e], acc[2][e], acc[3][e], acc[4][e]);
+            const int64_t r0 = (int64_t)t * G1_N + chunk * 16;       // first query-token row of this chunk
+            if (c < K) {
+                if ((nq & 3) == 0) {
+#pragma unroll
+                    for (int e = 0; e < 16; e += 4) {
+                        const int64_t r = r0 + e;
+                        if (r < q_rows) {                             // q_rows is a multiple of 4 here
+                            const int64_t b = r / nq, i = r % nq;
+                            *reinterpret_cast<int4 *>(table + (b * K + c) * nq + i) =
+                                make_int4(out[e], out[e + 1], out[e + 2], out[e + 3]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int64_t r = r0 + e;
+                        if (r < q_rows) {
+                            const int64_t b = r / nq, i = r % nq;
+                            table[(b * K + c) * nq + i] = out[e];
+                        }
+                    }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();                   // accumulators drained before the next tile overwrites them
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(G1_TMEM_COLS) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side ------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// Digit planes [3][rows][128] int8 as a 3-D tensor (128 bytes, rows, 3 planes); box = (128, box_rows, 1); rows past
+// the end read as zeros.
+int make_plane_map(CUtensorMap *map, const int8_t *planes, int64_t rows, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(CHIMERA_CUDA_ERROR, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[3] = {(cuuint64_t)G1_ROW_BYTES, (cuuint64_t)rows, 3};
+    cuuint64_t strides[2] = {(cuuint64_t)G1_ROW_BYTES, (cuuint64_t)rows * G1_ROW_BYTES};
+    cuuint32_t box[3] = {(cuuint32_t)G1_ROW_BYTES, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, (void *)planes, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(CHIMERA_CUDA_ERROR, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return CHIMERA_OK;
 }
 
 int launch_score_table(const Index &ix, const Params &p, const float *queries, int8_t *qdig, int32_t *table,
@@ -68,15 +283,26 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     const int64_t rows = (int64_t)p.B * p.nq;
     int rc = launch_digits(queries, rows, ix.D, qdig, status, st);
     if (rc) return rc;
-    count_launch(SLOT_G1);
-    const int G = ix.D / 4;
-    size_t smem = sizeof(int) * (size_t)(3 * G * p.nq + 3 * G1_CT * G);
-    if (smem > 48 * 1024)
-        CHIMERA_CUDA(cudaFuncSetAttribute(score_table_dp4a, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    dim3 grid((unsigned)((ix.K + G1_CT - 1) / G1_CT), (unsigned)p.B);
-    score_table_dp4a<<<grid, G1_THREADS, smem, st>>>(qdig, ix.cdig, ix.K, ix.D, p.nq, rows, table);
+    CUtensorMap map_c, map_q;
+    if ((rc = make_plane_map(&map_c, ix.cdig, ix.K, G1_M))) return rc;
+    if ((rc = make_plane_map(&map_q, qdig, rows, G1_N))) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G1_SMEM));
+        attr_set = true;
+    }
+    const int c_tiles = (int)((ix.K + G1_M - 1) / G1_M);
+    const int n_tiles = (int)((rows + G1_N - 1) / G1_N);
+    // about eight waves of two CTAs per SM, so the last wave is mostly full
+    int splits = (16 * ix.sm_count + c_tiles - 1) / c_tiles;
+    if (splits > n_tiles) splits = n_tiles;
+    if (splits < 1) splits = 1;
+    const int tiles_per_split = (n_tiles + splits - 1) / splits;
+    dim3 grid((unsigned)c_tiles, (unsigned)((n_tiles + tiles_per_split - 1) / tiles_per_split));
+    score_table_umma<<<grid, G1_THREADS, G1_SMEM, st>>>(map_c, map_q, ix.K, p.nq, rows, ix.D / 32, n_tiles,
+                                                        tiles_per_split, table, status);
     CHIMERA_CUDA(cudaGetLastError());
-    count_launch(SLOT_G1);
+    count_launch(SLOT_G1, 2);
     return CHIMERA_OK;
 }
 

@@ -109,24 +109,32 @@ static int exclusive_scan(const int32_t *in, int64_t n, int64_t *out, int64_t *t
 
 // ------------------------------------------------------------------------------------------------ digit planes ---
 // X = rint(x * 2^22) split into balanced base-256 digits X = d0 + 256 d1 + 65536 d2, d0, d1 in [-128, 127],
-// |d2| <= 64.  Plane p of row r, dimension d sits at dig[(p * rows + r) * D + d].
+// |d2| <= 64.  Planes have a fixed row pitch of DIGIT_PITCH (128) bytes, dimensions >= D are zero:
+// plane p of row r, dimension d sits at dig[(p * rows + r) * 128 + d].
+constexpr int DIGIT_PITCH = 128;
+
 __global__ void digits_kernel(const float *__restrict__ x, int64_t rows, int D, int8_t *__restrict__ dig,
                               uint32_t *status)
 {
-    int64_t n = rows * D;
-    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t n = rows * DIGIT_PITCH;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    float v = x[i];
-    if (!(fabsf(v) <= 1.0f)) {
-        if (status) atomicOr(status, ST_BAD_QUERY);
-        v = fminf(fmaxf(v, -1.0f), 1.0f);
-        if (v != v) v = 0.f;
+    const int64_t r = i / DIGIT_PITCH;
+    const int d = (int)(i % DIGIT_PITCH);
+    int d0 = 0, d1 = 0, d2 = 0;
+    if (d < D) {
+        float v = x[r * D + d];
+        if (!(fabsf(v) <= 1.0f)) {
+            if (status) atomicOr(status, ST_BAD_QUERY);
+            v = fminf(fmaxf(v, -1.0f), 1.0f);
+            if (v != v) v = 0.f;
+        }
+        const int X = __float2int_rn(v * 4194304.0f);
+        d0 = ((X + 128) & 255) - 128;
+        const int X1 = (X - d0) >> 8;
+        d1 = ((X1 + 128) & 255) - 128;
+        d2 = (X1 - d1) >> 8;
     }
-    int X = __float2int_rn(v * 4194304.0f);
-    int d0 = ((X + 128) & 255) - 128;
-    int X1 = (X - d0) >> 8;
-    int d1 = ((X1 + 128) & 255) - 128;
-    int d2 = (X1 - d1) >> 8;
     dig[i] = (int8_t)d0;
     dig[n + i] = (int8_t)d1;
     dig[2 * n + i] = (int8_t)d2;
@@ -134,7 +142,7 @@ __global__ void digits_kernel(const float *__restrict__ x, int64_t rows, int D, 
 
 int launch_digits(const float *x, int64_t rows, int D, int8_t *dig, uint32_t *status, cudaStream_t st)
 {
-    int64_t n = rows * D;
+    const int64_t n = rows * DIGIT_PITCH;
     digits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(x, rows, D, dig, status);
     CHIMERA_CUDA(cudaGetLastError());
     return CHIMERA_OK;
@@ -215,14 +223,10 @@ int build_index_device(Index &ix, const float *centroids, const int32_t *doclens
     ix.max_doclen = h_flags[1];
 
     // centroid digit planes
-    BUILD_CUDA(cudaMalloc(&ix.cdig, (size_t)3 * ix.K * ix.D));
+    BUILD_CUDA(cudaMalloc(&ix.cdig, (size_t)3 * ix.K * DIGIT_PITCH));
     BUILD_CUDA(cudaMemsetAsync(flags, 0, sizeof(int32_t), st));
-    {
-        int64_t n = ix.K * ix.D;
-        digits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(centroids, ix.K, ix.D, ix.cdig,
-                                                                   (uint32_t *)flags);
-        BUILD_CUDA(cudaGetLastError());
-    }
+    rc = launch_digits(centroids, ix.K, ix.D, ix.cdig, (uint32_t *)flags, st);
+    if (rc) { cleanup(); return rc; }
 
     // inverted file
     BUILD_CUDA(cudaMemsetAsync(count, 0, sizeof(int32_t) * ix.K, st));
