@@ -172,6 +172,32 @@ int chimera_index_info(const chimera_index *index, chimera_index_desc *desc, int
 int chimera_profile_enable(int32_t on);
 int chimera_profile_read(float *ms, int64_t *launches);
 
+/* Top-nprobe centroids per query token WITHOUT any device allocation and without a workspace (the paper has no
+ * counterpart: this is a packaging variant of stage 2a for callers that cannot allocate).
+ *
+ * Who needs it: callers that may not call cudaMalloc (or any allocating routine) at query time -- serving loops that
+ * fix all memory at start-up, or processes where another component owns the device memory pool.  The stage's scratch
+ * (partial top-nprobe lists) lives in a 4 MiB array built into the library image; every GPU that loads the library
+ * holds those 4 MiB until the process exits.
+ *
+ *   score_table  device, [n_queries, n_centroids, q_len] int32, centroid-major (stage 1's output layout).
+ *   out_probes   device, [n_queries, q_len, nprobe] int32, best first (score descending, centroid id ascending):
+ *                identical to the probes of chimera_search / chimera_run_stages for the same table.
+ *   stream       cudaStream_t as void*; the two kernels are enqueued on it, the call does not synchronise.
+ *
+ * Limits: n_queries * lists * nprobe * q_len * 8 bytes must fit the 4 MiB array, where lists = 8 * min(64,
+ * ceil(2 * SM count / n_queries), ceil(n_centroids / 512)); e.g. one query of 32 tokens with nprobe 4 against 65,536
+ * centroids needs 512 KiB, a batch of 8 such queries 2.3 MiB.  Larger calls return CHIMERA_WORKSPACE_TOO_SMALL and
+ * enqueue nothing (use chimera_search with a workspace).  Other argument limits are those of chimera_search.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device current)
+ * and caches it; make that first call before starting any stream capture.  The call itself allocates and frees
+ * nothing.  All calls share the one array per device and it keeps the previous call's contents: the kernels overwrite
+ * every entry they later read, so no clearing is needed, but two calls whose kernels may overlap on the same device
+ * (different streams, or concurrent host threads) race on it -- serialise them. */
+int chimera_probes_static(const int32_t *score_table, int64_t n_centroids, int32_t n_queries, int32_t q_len,
+                          int32_t nprobe, void *stream, int32_t *out_probes);
+
 #ifdef __cplusplus
 }
 #endif

@@ -239,3 +239,20 @@ class Index:
         st = ctypes.c_int32()
         _check(lib().chimera_workspace_status(_ptr(self._ws), _stream(), ctypes.byref(st)))
         return st.value
+
+
+def probes_static(score_table: torch.Tensor, nprobe: int) -> torch.Tensor:
+    """Top-nprobe centroids per query token through chimera_probes_static: no workspace and no device allocation
+    inside the library (its scratch is a fixed 4 MiB array in the library image).  For callers that must not allocate
+    at query time; sizes beyond the built-in array raise ChimeraError(WORKSPACE_TOO_SMALL).
+
+    score_table: [B, K, q_len] int32 CUDA tensor (centroid-major).  Returns probes [B, q_len, nprobe] int32.
+    The output tensor is allocated here by torch, outside the library; pass `out=` style buffers through the C ABI
+    directly if even that must be avoided."""
+    assert score_table.is_cuda and score_table.dtype == torch.int32 and score_table.is_contiguous()
+    B, K, q_len = score_table.shape
+    out = torch.empty(B, q_len, nprobe, dtype=torch.int32, device=score_table.device)
+    with torch.cuda.device(score_table.device):
+        _check(lib().chimera_probes_static(_ptr(score_table), ctypes.c_int64(K), ctypes.c_int32(B),
+                                           ctypes.c_int32(q_len), ctypes.c_int32(nprobe), _stream(), _ptr(out)))
+    return out

@@ -112,4 +112,80 @@ int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32
     return CHIMERA_OK;
 }
 
+// =====================================================================================================================
+// Allocation-free variant of the probe stage.
+//
+// Some callers cannot allocate device memory at all: latency-critical serving loops that size everything at start-up
+// and forbid allocator calls afterwards (an allocation can synchronise the device or fail late), and processes in
+// which another component owns the device memory pool, so that a cudaMalloc from here would fail or take memory that
+// was promised elsewhere.  For them this entry point runs the same two kernels as the probe stage but keeps the partial
+// lists (the stage's only scratch) in a fixed array that is part of the library image: nothing is allocated or freed
+// and no workspace is passed.
+//
+// The array below lives on every GPU that loads the library, from load until the process exits.  All calls share it
+// and it keeps the last call's contents.
+// =====================================================================================================================
+constexpr size_t STATIC_PROBE_SCRATCH_BYTES = 4u << 20;     // 4 MiB
+static __device__ __align__(256) unsigned long long g_probe_scratch[STATIC_PROBE_SCRATCH_BYTES / 8];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+// Device address of g_probe_scratch on each device (0 = not looked up yet).  In host code the symbol's name is only a
+// handle for the runtime, not a device address: it must be translated with cudaGetSymbolAddress, with the device in
+// question current, before a kernel can be given it.
+static unsigned long long *g_probe_scratch_ptr[STATIC_MAX_DEVICES] = {nullptr};
+
 }  // namespace chimera
+
+extern "C" int chimera_probes_static(const int32_t *score_table, int64_t n_centroids, int32_t n_queries, int32_t q_len,
+                                     int32_t nprobe, void *stream, int32_t *out_probes)
+{
+    using namespace chimera;
+    if (!score_table || !out_probes) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if (n_centroids < 1 || n_centroids > 0x7fffffffLL) return fail(CHIMERA_INVALID_ARG, "n_centroids out of range");
+    if (n_queries < 1 || n_queries > 65535) return fail(CHIMERA_INVALID_ARG, "n_queries must be in [1, 65535]");
+    if (q_len < 1 || q_len > CHIMERA_MAX_QLEN) return fail(CHIMERA_INVALID_ARG, "q_len must be in [1, %d]", CHIMERA_MAX_QLEN);
+    if (nprobe < 1 || nprobe > CHIMERA_MAX_NPROBE || nprobe > n_centroids)
+        return fail(CHIMERA_INVALID_ARG, "nprobe must be in [1, min(n_centroids, %d)]", CHIMERA_MAX_NPROBE);
+
+    int dev = 0, sm_count = 0;
+    CHIMERA_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return fail(CHIMERA_UNSUPPORTED, "device ordinal %d is not supported", dev);
+    CHIMERA_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    if (!g_probe_scratch_ptr[dev]) {          // first call on this device (it is the current one)
+        void *p = nullptr;
+        CHIMERA_CUDA(cudaGetSymbolAddress(&p, g_probe_scratch));
+        g_probe_scratch_ptr[dev] = static_cast<unsigned long long *>(p);
+    }
+    unsigned long long *part = g_probe_scratch_ptr[dev];
+
+    // same slicing rule as the workspace-based stage: fill the device at small batch, at least ~512 rows per block
+    int64_t blocks = (2LL * sm_count + n_queries - 1) / n_queries;
+    const int64_t by_rows = (n_centroids + 511) / 512;
+    if (blocks > by_rows) blocks = by_rows;
+    if (blocks > 64) blocks = 64;
+    if (blocks < 1) blocks = 1;
+    const int n_part = (int)blocks * PROBE_WARPS;
+    const size_t need = sizeof(unsigned long long) * (size_t)n_queries * n_part * nprobe * q_len;
+    if (need > STATIC_PROBE_SCRATCH_BYTES)
+        return fail(CHIMERA_WORKSPACE_TOO_SMALL,
+                    "this call needs %zu bytes of probe scratch; the built-in array holds %zu (use chimera_search with "
+                    "a workspace for larger problems)", need, (size_t)STATIC_PROBE_SCRATCH_BYTES);
+
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t smem = sizeof(unsigned long long) * (size_t)nprobe * PROBE_THREADS;
+    if (smem > 48 * 1024) {
+        CHIMERA_CUDA(cudaFuncSetAttribute(probe_partial, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CHIMERA_CUDA(cudaFuncSetAttribute(probe_final, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
+    const int rows_per_block = (int)((n_centroids + blocks - 1) / blocks);
+    const unsigned col_groups = (unsigned)((q_len + 31) / 32);
+    // probe_partial writes every entry probe_final reads (all n_part lists x nprobe keys x q_len columns), so nothing
+    // of the previous call's contents survives into this call's result and nothing needs clearing.
+    probe_partial<<<dim3((unsigned)blocks, (unsigned)n_queries, col_groups), PROBE_THREADS, smem, st>>>(
+        score_table, n_centroids, q_len, nprobe, rows_per_block, n_part, part);
+    CHIMERA_CUDA(cudaGetLastError());
+    probe_final<<<dim3(1, (unsigned)n_queries, col_groups), PROBE_THREADS, smem, st>>>(part, q_len, nprobe, n_part,
+                                                                                        out_probes);
+    CHIMERA_CUDA(cudaGetLastError());
+    return CHIMERA_OK;
+}
