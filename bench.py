@@ -197,14 +197,15 @@ def main():
     doclens64 = corp.doclens.to(torch.int64)
     work = []
     for bi in range(n_batches):
-        taps = index.alloc_taps(B, nq, P, n_prune, table=False)
+        taps = index.alloc_taps(B, nq, P, n_prune, table=False, ci=False)
         index.search(batches[bi], P, n_prune, k, taps=taps)
         assert index.status() == 0
         mask = torch.arange(index.N, device=device)[None, :] < taps.n_cand[:, None].to(torch.int64)
         toks = (doclens64[taps.cand.to(torch.int64).clamp_(0, index.N - 1)] * mask).sum()
         pr = taps.pruned.to(torch.int64)
         toks4 = (doclens64[pr.clamp(min=0)] * (pr >= 0)).sum()
-        work.append({"cand": int(taps.n_cand.sum()), "cand_tokens": int(toks), "pruned_tokens": int(toks4)})
+        work.append({"cand": int(taps.n_cand.sum()), "cand_tokens": int(toks), "pruned_tokens": int(toks4),
+                     "contenders": int(taps.n_contenders.sum())})
         del taps, mask
     torch.cuda.empty_cache()
 
@@ -256,11 +257,15 @@ def main():
         index.search(q[i:i + 1], P, n_prune, k, out=out1)
     torch.cuda.synchronize()
     lat = []
+    pkg.profile_enable(True)
+    pkg.profile_read()
     for i in range(n1):
         a = time.perf_counter()
         index.search(q[i:i + 1], P, n_prune, k, out=out1)
         torch.cuda.synchronize()
         lat.append(time.perf_counter() - a)
+    stage_ms1, _ = pkg.profile_read()
+    pkg.profile_enable(False)
     lat = np.array(lat)
     host_q1 = q[:n1].cpu().pin_memory()
     hout1 = (torch.empty(1, k, dtype=torch.int32).pin_memory(), torch.empty(1, k, dtype=torch.float32).pin_memory())
@@ -284,7 +289,10 @@ def main():
     # (4 B) and two offsets (16 B) + the CI written (4 B)
     ci_bytes = 4.0 * mean("cand_tokens") + 24.0 * mean("cand")
     ci_gbs = ci_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0
-    l2_bytes = mean("cand_tokens") * nq * 4.0
+    # L2 gathers: one q_len-byte row of the 8-bit table per candidate token (bound phase) + one 4*q_len-byte row of
+    # the exact table per contender token (contender tokens estimated with the candidates' mean length)
+    cont_frac = mean("contenders") / max(mean("cand"), 1.0)
+    l2_bytes = mean("cand_tokens") * nq * (1.0 + 4.0 * cont_frac)
     g4_ms = stage_ms["residual_scores"] / n_prof
     g4_bytes = mean("pruned_tokens") * (4.0 + cfg.code_bytes)
     stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
@@ -292,6 +300,7 @@ def main():
         "kernel": "ci_kernel (stage 3 centroid-interaction scan)", "bound": "hbm",
         "achieved": ci_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
         "frac": ci_gbs / peak, "traffic": None, "ms_per_launch": ci_ms, "algorithmic_bytes_per_launch": ci_bytes,
+        "contender_fraction": cont_frac,
         "binding_roof": {"bound": "l2_gather", "bytes_per_launch": l2_bytes,
                          "achieved_gbs": l2_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0},
         "stage_ms_per_step": stages,
@@ -309,6 +318,7 @@ def main():
                    "l2": "inputs larger than L2 (2.2 GB index, 2.1 GB score table per batch); no flush",
                    "gen_s": round(gen_s, 1), "index_build_s": round(build_s, 2)},
         "qps_batch1": float(1.0 / lat.mean()),
+        "stage_ms_batch1": {name: round(v / min(n1, 256), 4) for name, v in stage_ms1.items()},
         "latency_ms_batch1": {"mean": float(lat.mean() * 1e3), "p50": float(np.percentile(lat, 50) * 1e3),
                               "p95": float(np.percentile(lat, 95) * 1e3), "p99": float(np.percentile(lat, 99) * 1e3)},
         "e2e": {"value": e2e_qps, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -46,7 +46,7 @@ typedef enum {
 } chimera_status;
 
 #define CHIMERA_MAX_NPROBE 64       /* nprobe per query token */
-#define CHIMERA_MAX_QLEN 128        /* tokens per query */
+#define CHIMERA_MAX_QLEN 127        /* tokens per query (keeps sum_i max S[., i] inside int32) */
 #define CHIMERA_MAX_NPRUNE 16384    /* n_prune */
 #define CHIMERA_MAX_K 16384         /* k */
 
@@ -128,10 +128,14 @@ typedef struct {
     int32_t *probes;      /* [n_queries, q_len, nprobe] best first (score desc, id asc)                         */
     int32_t *cand;        /* [n_queries, max_candidates] ascending document ids; entries past n_cand undefined  */
     int32_t *n_cand;      /* [n_queries]                                                                        */
-    int32_t *ci;          /* [n_queries, max_candidates] centroid-interaction score of cand[...] (Q.24 sum)     */
+    int32_t *ci;          /* [n_queries, max_candidates] exact centroid-interaction score of cand[...] (Q.24
+                             sum); the search itself needs it only for documents that can reach the top n_prune,
+                             so asking for this tap runs the exact kernel over every candidate as well          */
     int32_t *pruned;      /* [n_queries, n_prune] ascending document ids, -1 padded                             */
     int32_t *n_pruned;    /* [n_queries]                                                                        */
     float *score4;        /* [n_queries, n_prune] stage-4 score of pruned[...], -inf beside -1                  */
+    int32_t *n_contenders;/* [n_queries] documents whose CI upper bound reached the pruning threshold and got an
+                             exact CI (q_len 32 or 64); n_cand for other q_len                                  */
 } chimera_taps;
 
 /* chimera_search that also copies the intermediates out (same kernels, same order).  taps: host pointer to a struct

@@ -38,7 +38,7 @@ class _Desc(ctypes.Structure):
 
 class _Taps(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
-                ("score_table", "probes", "cand", "n_cand", "ci", "pruned", "n_pruned", "score4")]
+                ("score_table", "probes", "cand", "n_cand", "ci", "pruned", "n_pruned", "score4", "n_contenders")]
 
 
 def library_path() -> str:
@@ -82,6 +82,7 @@ class Taps:
     pruned: Optional[torch.Tensor] = None        # [B, n_prune] int32
     n_pruned: Optional[torch.Tensor] = None      # [B] int32
     score4: Optional[torch.Tensor] = None        # [B, n_prune] float32
+    n_contenders: Optional[torch.Tensor] = None  # [B] int32
 
     def _c(self) -> _Taps:
         c = _Taps()
@@ -165,14 +166,15 @@ class Index:
     def _maxc(self, max_candidates):
         return self.N if (max_candidates == 0 or max_candidates > self.N) else max_candidates
 
-    def alloc_taps(self, B, q_len, nprobe, n_prune, max_candidates=0, table=True) -> Taps:
+    def alloc_taps(self, B, q_len, nprobe, n_prune, max_candidates=0, table=True, ci=True) -> Taps:
         dev, i32 = self.device, torch.int32
         mc = self._maxc(max_candidates)
         return Taps(
             score_table=torch.empty(B, self.K, q_len, dtype=i32, device=dev) if table else None,
             probes=torch.empty(B, q_len, nprobe, dtype=i32, device=dev),
             cand=torch.empty(B, mc, dtype=i32, device=dev), n_cand=torch.empty(B, dtype=i32, device=dev),
-            ci=torch.empty(B, mc, dtype=i32, device=dev),
+            ci=torch.empty(B, mc, dtype=i32, device=dev) if ci else None,
+            n_contenders=torch.empty(B, dtype=i32, device=dev),
             pruned=torch.empty(B, n_prune, dtype=i32, device=dev), n_pruned=torch.empty(B, dtype=i32, device=dev),
             score4=torch.empty(B, n_prune, dtype=torch.float32, device=dev))
 

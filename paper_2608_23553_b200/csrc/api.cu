@@ -22,7 +22,7 @@ int fail(int code, const char *fmt, ...)
 }
 
 // ------------------------------------------------------------------------------------------------ profiling ------
-constexpr int PROF_MARKS = 12;
+constexpr int PROF_MARKS = 16;
 struct ProfCall {
     cudaEvent_t ev[PROF_MARKS];
     int slot[PROF_MARKS];     // slot[i] = stage that ran between ev[i-1] and ev[i]
@@ -89,6 +89,7 @@ Layout make_layout(const Index &ix, const Params &p)
     L.out_scores = take(B * p.k * sizeof(float));
     L.qdig = take(3 * B * nq * 128);
     L.table = take(B * (size_t)ix.K * nq * sizeof(int32_t));
+    L.table8 = take(coarse_supported(p.nq) ? B * (size_t)ix.K * nq : 0);
     L.part = take(B * L.n_part * p.P * nq * sizeof(unsigned long long));
     L.probes = take(B * nq * p.P * sizeof(int32_t));
     L.bitmap = take(B * (size_t)L.words * sizeof(uint32_t));
@@ -96,6 +97,11 @@ Layout make_layout(const Index &ix, const Params &p)
     L.cand = take(B * (size_t)p.maxc * sizeof(int32_t));
     L.n_cand = take(B * sizeof(int32_t));
     L.ci = take(B * (size_t)p.maxc * sizeof(int32_t));
+    const size_t two_phase = coarse_supported(p.nq) ? B * (size_t)p.maxc * sizeof(int32_t) : 0;
+    L.lo = take(two_phase);
+    L.hi = take(two_phase);
+    L.cont = take(two_phase);
+    L.n_cont = take(B * sizeof(int32_t));
     L.pruned = take(B * p.n_prune * sizeof(int32_t));
     L.n_pruned = take(B * sizeof(int32_t));
     L.score4 = take(B * p.n_prune * sizeof(float));
@@ -149,6 +155,12 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int32_t *cand = (int32_t *)(ws + L.cand);
     int32_t *n_cand = (int32_t *)(ws + L.n_cand);
     int32_t *ci = (int32_t *)(ws + L.ci);
+    const bool two_phase = coarse_supported(p.nq);
+    uint8_t *table8 = two_phase ? (uint8_t *)(ws + L.table8) : nullptr;
+    int32_t *lo = (int32_t *)(ws + L.lo);
+    int32_t *hi = (int32_t *)(ws + L.hi);
+    int32_t *cont = (int32_t *)(ws + L.cont);
+    int32_t *n_cont = (int32_t *)(ws + L.n_cont);
     int32_t *pruned = (int32_t *)(ws + L.pruned);
     int32_t *n_pruned = (int32_t *)(ws + L.n_pruned);
     float *score4 = (float *)(ws + L.score4);
@@ -187,7 +199,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     prof_mark(SLOT_MISC, st);
 
     if (first <= 1 && last >= 1) {
-        if ((rc = launch_score_table(ix, p, queries, qdig, table, status, st))) return rc;
+        if ((rc = launch_score_table(ix, p, queries, qdig, table, table8, status, st))) return rc;
         prof_mark(SLOT_G1, st);
     }
     if (first <= 2 && last >= 2) {
@@ -197,10 +209,26 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
         prof_mark(SLOT_GATHER, st);
     }
     if (first <= 3 && last >= 3) {
-        if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, st))) return rc;
-        prof_mark(SLOT_CI, st);
-        if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
-        prof_mark(SLOT_SELECT, st);
+        if (two_phase) {
+            if (first > 1) {                       // the table came from the caller: derive its coarse copy
+                if ((rc = launch_coarse_table(ix, p, table, table8, st))) return rc;
+                prof_mark(SLOT_MISC, st);
+            }
+            // bounds for every candidate, contenders for the top n_prune, exact CI and selection among those
+            if ((rc = launch_coarse_bounds(ix, p, table8, cand, n_cand, lo, hi, st))) return rc;
+            prof_mark(SLOT_CI, st);
+            if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, st))) return rc;
+            prof_mark(SLOT_SELECT, st);
+            if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, 2 * ix.sm_count, st))) return rc;
+            prof_mark(SLOT_CI, st);
+            if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, st))) return rc;
+            prof_mark(SLOT_SELECT, st);
+        } else {
+            if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, 0, st))) return rc;
+            prof_mark(SLOT_CI, st);
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
+            prof_mark(SLOT_SELECT, st);
+        }
     }
     if (first <= 4 && last >= 4) {
         if ((rc = launch_residual_scores(ix, p, queries, table, pruned, score4, st))) return rc;
@@ -219,7 +247,15 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if (taps->n_cand && (rc = copy_d2d(taps->n_cand, n_cand, B * sizeof(int32_t), st))) return rc;
         }
         if (first <= 3 && last >= 3) {
-            if (taps->ci && (rc = copy_d2d(taps->ci, ci, cand_bytes, st))) return rc;
+            if (taps->ci) {
+                if (two_phase) {                   // the search only needed exact CI for the contenders: the tap asks
+                                                   // for every candidate, so the exact kernel runs over all of them
+                    if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, taps->ci, 0, st))) return rc;
+                } else if ((rc = copy_d2d(taps->ci, ci, cand_bytes, st))) return rc;
+            }
+            if (taps->n_contenders &&
+                (rc = copy_d2d(taps->n_contenders, two_phase ? n_cont : n_cand, B * sizeof(int32_t), st)))
+                return rc;
             if (taps->pruned && (rc = copy_d2d(taps->pruned, pruned, pruned_bytes, st))) return rc;
             if (taps->n_pruned && (rc = copy_d2d(taps->n_pruned, n_pruned, B * sizeof(int32_t), st))) return rc;
         }

@@ -45,13 +45,18 @@ struct Layout {
     size_t out_scores;    // float  [B, k]
     size_t qdig;          // int8   [3][B*nq][128]
     size_t table;         // int32  [B][K][nq]
+    size_t table8;        // uint8  [B][K][nq]        coarse copy: min((S + 2^24 + 64) >> 17, 255)
     size_t part;          // uint64 [B][n_part][P][nq] partial top-P keys
     size_t probes;        // int32  [B][nq][P]
     size_t bitmap;        // uint32 [B][words]
     size_t chunk_cnt;     // int32  [B][n_chunks + 1]
     size_t cand;          // int32  [B][maxc]
     size_t n_cand;        // int32  [B]
-    size_t ci;            // int32  [B][maxc]
+    size_t ci;            // int32  [B][maxc]         exact CI of the contenders (of every candidate: generic q_len / tap)
+    size_t lo;            // int32  [B][maxc]         lower bound on CI of every candidate
+    size_t hi;            // int32  [B][maxc]         upper bound
+    size_t cont;          // int32  [B][maxc]         contender ids, ascending
+    size_t n_cont;        // int32  [B]
     size_t pruned;        // int32  [B][n_prune]
     size_t n_pruned;      // int32  [B]
     size_t score4;        // float  [B][n_prune]
@@ -93,14 +98,21 @@ int build_index_device(Index &ix, const float *centroids, const int32_t *doclens
 // ST_BAD_QUERY.
 int launch_digits(const float *x, int64_t rows, int D, int8_t *dig, uint32_t *status, cudaStream_t st);
 
+// table8 may be NULL (no coarse copy wanted).
 int launch_score_table(const Index &ix, const Params &p, const float *queries, int8_t *qdig, int32_t *table,
-                       uint32_t *status, cudaStream_t st);
+                       uint8_t *table8, uint32_t *status, cudaStream_t st);
 int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32_t *table, unsigned long long *part,
                   int32_t *probes, cudaStream_t st);
 int launch_gather(const Index &ix, const Params &p, const Layout &L, const int32_t *probes, uint32_t *bitmap,
                   int32_t *chunk_cnt, int32_t *cand, int32_t *n_cand, uint32_t *status, cudaStream_t st);
+bool coarse_supported(int nq);
+int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st);
+int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
+                         const int32_t *n_cand, int32_t *lo, int32_t *hi, cudaStream_t st);
+int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
+                      const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st);
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
-                                const int32_t *n_cand, int32_t *ci, cudaStream_t st);
+                                const int32_t *n_cand, int32_t *ci, int blocks_cap, cudaStream_t st);
 int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
                   int32_t *pruned, int32_t *n_pruned, cudaStream_t st);
 int launch_residual_scores(const Index &ix, const Params &p, const float *queries, const int32_t *table,

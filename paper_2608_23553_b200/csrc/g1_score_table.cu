@@ -106,7 +106,7 @@ __device__ __forceinline__ int32_t combine_digits(int32_t a0, int32_t a1, int32_
 __global__ void __launch_bounds__(G1_THREADS)
 score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_q, int64_t K,
                  int nq, int64_t q_rows, int k_steps, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
-                 uint32_t *status)
+                 uint8_t *__restrict__ table8, uint32_t *status)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t s_tmem_base;
@@ -207,6 +207,24 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
 #pragma unroll
             for (int e = 0; e < 16; ++e) out[e] = combine_digits(acc[0][e], acc[1][e], acc[2][e], acc[3][e], acc[4][e]);
             const int64_t r0 = (int64_t)t * G1_N + chunk * 16;       // first query-token row of this chunk
+            if (table8 != nullptr && c < K && r0 < q_rows) {
+                // coarse copy for the bound phase of stage 3: min((S + 2^24 + 64) >> 17, 255); q_len is a multiple of
+                // 16 here, so the 16 rows of a chunk belong to one query and the store is 16-byte aligned
+                uint32_t w[4];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    uint32_t pack = 0;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        int v = (out[4 * g + e] + (1 << 24) + 64) >> 17;
+                        v = v > 255 ? 255 : v;
+                        pack |= (uint32_t)v << (8 * e);
+                    }
+                    w[g] = pack;
+                }
+                const int64_t b = r0 / nq, i = r0 % nq;
+                *reinterpret_cast<uint4 *>(table8 + (b * K + c) * nq + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
             if (c < K) {
                 if ((nq & 3) == 0) {
 #pragma unroll
@@ -278,7 +296,7 @@ int make_plane_map(CUtensorMap *map, const int8_t *planes, int64_t rows, int box
 }
 
 int launch_score_table(const Index &ix, const Params &p, const float *queries, int8_t *qdig, int32_t *table,
-                       uint32_t *status, cudaStream_t st)
+                       uint8_t *table8, uint32_t *status, cudaStream_t st)
 {
     const int64_t rows = (int64_t)p.B * p.nq;
     int rc = launch_digits(queries, rows, ix.D, qdig, status, st);
@@ -300,7 +318,7 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
     dim3 grid((unsigned)c_tiles, (unsigned)((n_tiles + tiles_per_split - 1) / tiles_per_split));
     score_table_umma<<<grid, G1_THREADS, G1_SMEM, st>>>(map_c, map_q, ix.K, p.nq, rows, ix.D / 32, n_tiles,
-                                                        tiles_per_split, table, status);
+                                                        tiles_per_split, table, table8, status);
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_G1, 2);
     return CHIMERA_OK;

@@ -4,6 +4,10 @@
 //                                                tokens -- applied to the centroid scores; integers, order-free)
 //   keep the n_prune candidates with the largest CI, ties towards the smaller document id.
 //
+// Two phases when q_len is 32, 64 or 128: cheap bounds lo(d) <= CI(d) <= hi(d) for every candidate from an 8-bit
+// copy of the table (ci_coarse_kernel), the documents whose hi reaches the n_prune-th largest lo (contender_kernel),
+// then exact CI and exact selection among those only.  Other q_len: exact CI for every candidate.
+//
 // ci_kernel: one warp per candidate document.  The document's centroid ids are streamed with coalesced 128-byte
 // loads (lane = token), each is broadcast with a shuffle, and the warp gathers the table row S[cid, :] with
 // lane = query token (one 128-byte line for 32 query tokens), keeping a running maximum per lane.
@@ -11,6 +15,7 @@
 // select_kernel: one block per query.  Radix select (11 + 11 + 10 bits) of the n_prune-th largest CI, then an
 // ordered compaction of the candidate list (which is ascending in id), so equal scores are resolved towards smaller
 // ids and the survivors come out ascending.
+#include <cuda_fp16.h>
 #include <limits.h>
 
 #include "common.cuh"
@@ -72,7 +77,7 @@ ci_kernel(const int32_t *__restrict__ table, int64_t K, int nq, const int32_t *_
     }
 }
 
-// Wide variant for q_len = 4 * LPR (LPR = 8, 16 or 32 lanes per table row): every lane loads 16 bytes (four query
+// Wide variant for q_len = 4 * LPR (LPR = 8 or 16 lanes per table row): every lane loads 16 bytes (four query
 // tokens) of a row, so one load instruction of the warp covers 32 / LPR document tokens.  Lane group g = lane / LPR
 // takes tokens g, g + TPL, g + 2 TPL, ... of each 32-token slab; the group maxima are merged with shuffles at the end.
 template <int LPR>
@@ -134,11 +139,162 @@ ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__re
     }
 }
 
-int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
-                                const int32_t *n_cand, int32_t *ci, cudaStream_t st)
+// ------------------------------------------------------------------------------------------------ coarse bounds --
+// Bounds on CI from the 8-bit table U8[c, i] = min((S[c, i] + 2^24 + 64) >> 17, 255) (stage 1 writes it next to the
+// exact table; S + 2^24 + 64 > 0 always).  The map is monotone, so with m_i = max_t U8[cid_t, i]
+//     lo(d) = sum_i (2^17 m_i - 2^24 - 64)  <=  CI(d)  <=  lo(d) + nq (2^17 - 1) + 2^18 #{i : m_i = 255} = hi(d)
+// (the last term covers the saturated top bucket).  A row of U8 is q_len bytes -- one 32-byte sector for 32 query
+// tokens instead of four -- and a lane's 16-byte load covers 16 query tokens, so one warp load covers 32 / LPR tokens
+// (LPR = q_len / 16 lanes per row).  Bytes are widened to fp16 with one byte-permute per pair (0x64xx = 1024 + x,
+// exact) so that the running maxima use the native packed-half max.
+__device__ __forceinline__ uint32_t hmax2_bits(uint32_t a, uint32_t b)
+{
+    __half2 r = __hmax2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b));
+    return *reinterpret_cast<uint32_t *>(&r);
+}
+__device__ __forceinline__ void coarse_accumulate(uint32_t (&m)[8], const int4 &v)
+{
+    const uint32_t w[4] = {(uint32_t)v.x, (uint32_t)v.y, (uint32_t)v.z, (uint32_t)v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        m[2 * k] = hmax2_bits(m[2 * k], __byte_perm(w[k], 0x64646464u, 0x4140));         // bytes 0, 1
+        m[2 * k + 1] = hmax2_bits(m[2 * k + 1], __byte_perm(w[k], 0x64646464u, 0x4342)); // bytes 2, 3
+    }
+}
+
+template <int LPR>
+__global__ void __launch_bounds__(CI_THREADS)
+ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *__restrict__ cand,
+                 const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
+                 const int64_t *__restrict__ doc_off, int32_t *__restrict__ lo, int32_t *__restrict__ hi)
+{
+    constexpr int NQ = 16 * LPR;
+    constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
+    constexpr int STEPS = 32 / TPL;               // loads per 32-token slab (= LPR)
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const int grp = lane / LPR, sub = lane % LPR;
+    const int n = n_cand[b];
+    const int4 *tb = reinterpret_cast<const int4 *>(table8 + (int64_t)b * K * NQ) + sub;
+    const int32_t *cb = cand + (int64_t)b * maxc;
+    const int warps_per_query = gridDim.x * CI_WARPS;
+    for (int j = blockIdx.x * CI_WARPS + (threadIdx.x >> 5); j < n; j += warps_per_query) {
+        const int64_t d = cb[j];
+        const int64_t t0 = doc_off[d], t1 = doc_off[d + 1];
+        uint32_t m[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) m[r] = 0x64006400u;       // 1024 + 0 in both halves
+        for (int64_t base = t0; base < t1; base += 64) {
+            // two 32-token slabs per iteration; lanes past the end repeat the last token (harmless for a maximum)
+            const int64_t last = t1 - 1;
+            const int64_t i0 = base + lane, i1 = base + 32 + lane;
+            const int32_t cid0 = cids[i0 < last ? i0 : last];
+            const int32_t cid1 = cids[i1 < last ? i1 : last];
+            const bool second = base + 32 < t1;
+            int4 v[2 * STEPS];
+#pragma unroll
+            for (int s = 0; s < STEPS; ++s) {
+                const int32_t c = __shfl_sync(0xffffffffu, cid0, s * TPL + grp);
+                v[s] = __ldg(tb + (int64_t)c * LPR);
+            }
+            if (second) {
+#pragma unroll
+                for (int s = 0; s < STEPS; ++s) {
+                    const int32_t c = __shfl_sync(0xffffffffu, cid1, s * TPL + grp);
+                    v[STEPS + s] = __ldg(tb + (int64_t)c * LPR);
+                }
+            }
+#pragma unroll
+            for (int s = 0; s < STEPS; ++s) coarse_accumulate(m, v[s]);
+            if (second) {
+#pragma unroll
+                for (int s = 0; s < STEPS; ++s) coarse_accumulate(m, v[STEPS + s]);
+            }
+        }
+        // Merge the lane groups (same columns, different tokens).  While a lane still holds several registers each
+        // exchange keeps one half of them and hands the other half to the partner, so the data halves per step;
+        // the remaining steps exchange the last register whole (those lanes end up with duplicates).
+        int nreg = 8;
+        uint32_t dup_mask = 0;
+#pragma unroll
+        for (int o = 16; o >= LPR; o >>= 1) {
+            if (nreg > 1) {
+                const int half = nreg >> 1;
+                const bool up = (lane & o) != 0;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if (r < half) {
+                        const uint32_t send = up ? m[r] : m[r + half];
+                        const uint32_t keep = up ? m[r + half] : m[r];
+                        m[r] = hmax2_bits(keep, __shfl_xor_sync(0xffffffffu, send, o));
+                    }
+                }
+                nreg = half;
+            } else {
+                m[0] = hmax2_bits(m[0], __shfl_xor_sync(0xffffffffu, m[0], o));
+                dup_mask |= (uint32_t)o;
+            }
+        }
+        // every lane now holds the maxima of two columns; sum over columns (skipping duplicate lanes)
+        const float2 f = __half22float2(*reinterpret_cast<__half2 *>(&m[0]));
+        int sum = 0, sat = 0;
+        if ((lane & dup_mask) == 0) {
+            sum = (int)(f.x + f.y) - 2048;                      // two halves of 1024 + u, exact
+            sat = (f.x >= 1279.0f) + (f.y >= 1279.0f);
+        }
+        sum = warp_sum(sum);
+        sat = warp_sum(sat);
+        if (lane == 0) {
+            const int l = (sum - 128 * NQ) * (1 << 17) - 64 * NQ;
+            lo[(int64_t)b * maxc + j] = l;
+            hi[(int64_t)b * maxc + j] = l + NQ * ((1 << 17) - 1) + sat * (1 << 18);
+        }
+    }
+}
+
+bool coarse_supported(int nq) { return nq == 32 || nq == 64; }
+
+int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
+                         const int32_t *n_cand, int32_t *lo, int32_t *hi, cudaStream_t st)
 {
     int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
     int64_t cap = (int64_t)ix.sm_count * 8;
+    unsigned gx = (unsigned)(want < cap ? want : cap);
+    if (gx < 1) gx = 1;
+    dim3 grid(gx, (unsigned)p.B);
+    if (p.nq == 32)
+        ci_coarse_kernel<2><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, lo, hi);
+    else
+        ci_coarse_kernel<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, lo, hi);
+    CHIMERA_CUDA(cudaGetLastError());
+    count_launch(SLOT_CI);
+    return CHIMERA_OK;
+}
+
+// table [rows] int32 -> table8 [rows] uint8 (only needed when stage 1 did not run in this call).
+__global__ void coarse_table_kernel(const int32_t *__restrict__ table, int64_t n, uint8_t *__restrict__ table8)
+{
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) {
+        int v = (table[i] + (1 << 24) + 64) >> 17;
+        table8[i] = (uint8_t)(v > 255 ? 255 : v);
+    }
+}
+int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st)
+{
+    const int64_t n = (int64_t)p.B * ix.K * p.nq;
+    coarse_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(table, n, table8);
+    CHIMERA_CUDA(cudaGetLastError());
+    count_launch(SLOT_MISC);
+    return CHIMERA_OK;
+}
+
+// Exact CI of a list of documents.  blocks_cap bounds the blocks per query (0 = default).
+int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
+                                const int32_t *n_cand, int32_t *ci, int blocks_cap, cudaStream_t st)
+{
+    int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
+    int64_t cap = blocks_cap > 0 ? blocks_cap : (int64_t)ix.sm_count * 8;
     unsigned gx = (unsigned)(want < cap ? want : cap);
     if (gx < 1) gx = 1;
     dim3 grid(gx, (unsigned)p.B);
@@ -147,8 +303,6 @@ int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t 
         ci_wide_kernel<8><<<grid, CI_THREADS, 0, st>>>(table, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
     else if (p.nq == 64)
         ci_wide_kernel<16><<<grid, CI_THREADS, 0, st>>>(table, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
-    else if (p.nq == 128)
-        ci_wide_kernel<32><<<grid, CI_THREADS, 0, st>>>(table, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
     else if (nqw == 1)
         ci_kernel<1><<<grid, CI_THREADS, 0, st>>>(table, ix.K, p.nq, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
     else if (nqw == 2)
@@ -188,7 +342,51 @@ __device__ __forceinline__ int sel_block_scan(int v, int *total, int *warp_part 
     return before + incl - v;
 }
 
-// grid (B).  pruned[b][0..n_prune) ascending ids, -1 padded; n_pruned[b].
+// Radix select (11 + 11 + 10 bits, most significant first) of the `want`-th largest value of sb[0..n) in the order of
+// u = value ^ 0x80000000.  Needs n >= want >= 1.  Returns that value's u; *need_eq = how many entries equal to it
+// belong to the top `want` (the rest of the top `want` are strictly greater).  Whole block, uniform.
+__device__ __forceinline__ uint32_t radix_select(const int32_t *__restrict__ sb, int n, int want_in, int *hist,
+                                                 int *warp_part, uint32_t *s_prefix, int *s_want, int *need_eq)
+{
+    if (threadIdx.x == 0) { *s_prefix = 0u; *s_want = want_in; }
+    const int shifts[3] = {21, 10, 0};
+    const int widths[3] = {11, 11, 10};
+    uint32_t known_mask = 0u;
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = shifts[pass], bins = 1 << widths[pass];
+        for (int i = threadIdx.x; i < 2048; i += SEL_THREADS) hist[i] = 0;
+        __syncthreads();
+        const uint32_t prefix = *s_prefix;
+        const int want = *s_want;
+        for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
+            uint32_t u = (uint32_t)sb[j] ^ 0x80000000u;
+            if ((u & known_mask) == prefix) atomicAdd(&hist[(u >> shift) & (bins - 1)], 1);
+        }
+        __syncthreads();
+        // descending bins: thread t owns bins (bins-1-2t) and (bins-2-2t)
+        int hi_bin = bins - 1 - 2 * (int)threadIdx.x, lo_bin = hi_bin - 1;
+        int h_hi = hi_bin >= 0 ? hist[hi_bin] : 0;
+        int h_lo = lo_bin >= 0 ? hist[lo_bin] : 0;
+        int total;
+        int before = sel_block_scan(h_hi + h_lo, &total, warp_part);
+        // the wanted rank falls in the first bin whose cumulative count reaches `want`
+        if (before < want && want <= before + h_hi + h_lo) {
+            if (want <= before + h_hi) {
+                *s_prefix = prefix | ((uint32_t)hi_bin << shift);
+                *s_want = want - before;
+            } else {
+                *s_prefix = prefix | ((uint32_t)lo_bin << shift);
+                *s_want = want - before - h_hi;
+            }
+        }
+        known_mask |= (uint32_t)(bins - 1) << shift;
+        __syncthreads();
+    }
+    *need_eq = *s_want;
+    return *s_prefix;
+}
+
+// grid (B).  pruned[b][0..n_prune) ascending ids, -1 padded; n_pruned[b].  
 __global__ void __launch_bounds__(SEL_THREADS)
 select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, const int32_t *__restrict__ ci,
               int64_t maxc, int n_prune, int32_t *__restrict__ pruned, int32_t *__restrict__ n_pruned)
@@ -208,44 +406,8 @@ select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_ca
         if (threadIdx.x == 0) n_pruned[b] = n;
         return;
     }
-
-    // Radix select on u = ci ^ 0x80000000 (unsigned order = signed order), most significant digit first.
-    if (threadIdx.x == 0) { s_prefix = 0u; s_want = n_prune; }
-    const int shifts[3] = {21, 10, 0};
-    const int widths[3] = {11, 11, 10};
-    uint32_t known_mask = 0u;
-    for (int pass = 0; pass < 3; ++pass) {
-        const int shift = shifts[pass], bins = 1 << widths[pass];
-        for (int i = threadIdx.x; i < 2048; i += SEL_THREADS) hist[i] = 0;
-        __syncthreads();
-        const uint32_t prefix = s_prefix;
-        const int want = s_want;
-        for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
-            uint32_t u = (uint32_t)sb[j] ^ 0x80000000u;
-            if ((u & known_mask) == prefix) atomicAdd(&hist[(u >> shift) & (bins - 1)], 1);
-        }
-        __syncthreads();
-        // descending bins: thread t owns bins (bins-1-2t) and (bins-2-2t)
-        int hi_bin = bins - 1 - 2 * (int)threadIdx.x, lo_bin = hi_bin - 1;
-        int h_hi = hi_bin >= 0 ? hist[hi_bin] : 0;
-        int h_lo = lo_bin >= 0 ? hist[lo_bin] : 0;
-        int total;
-        int before = sel_block_scan(h_hi + h_lo, &total, warp_part);
-        // the wanted rank falls in the first bin whose cumulative count reaches `want`
-        if (before < want && want <= before + h_hi + h_lo) {
-            if (want <= before + h_hi) {
-                s_prefix = prefix | ((uint32_t)hi_bin << shift);
-                s_want = want - before;
-            } else {
-                s_prefix = prefix | ((uint32_t)lo_bin << shift);
-                s_want = want - before - h_hi;
-            }
-        }
-        known_mask |= (uint32_t)(bins - 1) << shift;
-        __syncthreads();
-    }
-    const uint32_t thr = s_prefix;       // the n_prune-th largest value
-    const int need_eq = s_want;          // how many entries equal to it are kept (the first ones in id order)
+    int need_eq;
+    const uint32_t thr = radix_select(sb, n, n_prune, hist, warp_part, &s_prefix, &s_want, &need_eq);
 
     // Ordered compaction: keep u > thr, and the first need_eq entries with u == thr.
     int run_gt = 0, run_eq = 0;
@@ -263,6 +425,52 @@ select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_ca
         run_eq += total & 0xffff;
     }
     if (threadIdx.x == 0) n_pruned[b] = n_prune;
+}
+
+// grid (B).  Contenders for the top n_prune: with tau = the n_prune-th largest lower bound, every document of the
+// true top n_prune has hi >= CI >= (n_prune-th largest CI) >= tau.  Writes their ids (ascending) and their number.
+__global__ void __launch_bounds__(SEL_THREADS)
+contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, const int32_t *__restrict__ lo,
+                 const int32_t *__restrict__ hi, int64_t maxc, int n_prune, int32_t *__restrict__ cont,
+                 int32_t *__restrict__ n_cont)
+{
+    __shared__ int hist[2048];
+    __shared__ int warp_part[32];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_want;
+    const int b = blockIdx.x;
+    const int n = n_cand[b];
+    const int32_t *cb = cand + (int64_t)b * maxc;
+    const int32_t *hb = hi + (int64_t)b * maxc;
+    int32_t *out = cont + (int64_t)b * maxc;
+    if (n <= n_prune) {
+        for (int j = threadIdx.x; j < n; j += SEL_THREADS) out[j] = cb[j];
+        if (threadIdx.x == 0) n_cont[b] = n;
+        return;
+    }
+    int need_eq;
+    const uint32_t thr = radix_select(lo + (int64_t)b * maxc, n, n_prune, hist, warp_part, &s_prefix, &s_want, &need_eq);
+    const int32_t tau = (int32_t)(thr ^ 0x80000000u);
+    int run = 0;
+    for (int base = 0; base < n; base += SEL_THREADS) {
+        int j = base + threadIdx.x;
+        int keep = (j < n && hb[j] >= tau) ? 1 : 0;
+        int total;
+        int before = sel_block_scan(keep, &total, warp_part);
+        if (keep) out[run + before] = cb[j];
+        run += total;
+    }
+    if (threadIdx.x == 0) n_cont[b] = run;
+}
+
+int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
+                      const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st)
+{
+    (void)ix;
+    contender_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, lo, hi, p.maxc, p.n_prune, cont, n_cont);
+    CHIMERA_CUDA(cudaGetLastError());
+    count_launch(SLOT_SELECT);
+    return CHIMERA_OK;
 }
 
 int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
