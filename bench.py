@@ -27,8 +27,28 @@ import torch  # noqa: E402
 
 from synth import CONFIGS, make_corpus, make_queries  # noqa: E402
 
-METRIC = "QPS at batch 256 (Mid corpus, nprobe 4, n_prune 1024, k 10)"
 UNIT = "queries/s"
+
+
+def metric_name(cfg, batch):
+    return "QPS at batch %d (%s corpus, nprobe %d, n_prune %d, k %d)" % (batch, cfg.name.capitalize(), cfg.nprobe,
+                                                                         cfg.n_prune, cfg.k)
+
+
+def candidate_capacity(index, q, nq, P, n_prune, k):
+    """max_candidates for a workload: all documents for small corpora, else 1.25x the largest candidate count seen on
+    a few probe queries (bounds the workspace on corpora with millions of documents)."""
+    if index.N <= 1_000_000:
+        return 0
+    nb = min(8, q.shape[0])
+    taps = index.alloc_taps(nb, nq, P, n_prune, table=False, ci=False)
+    index.search(q[:nb].contiguous(), P, n_prune, k, taps=taps)
+    assert index.status() == 0
+    worst = int(taps.n_cand.max())
+    del taps
+    index._ws = None
+    torch.cuda.empty_cache()
+    return min(index.N, (int(worst * 1.25) + 1023) // 1024 * 1024)
 
 
 def measured_peaks():
@@ -133,13 +153,75 @@ def run_reference(args, cfg, rank, world):
     qps = args.steps / dt
     sample = "1 query per step (of the %d-query batch), %d steps, single thread" % (args.batch, args.steps)
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": metric_name(cfg, args.batch), "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64+f64", "data": "synthetic",
         "config": {"workload": cfg.name, "batch": 1, "sample": sample},
         "cpu_baseline": {"value": qps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
+
+
+def exhaustive_truth(index, q, cfg, k_max, chunk=16384):
+    """Ground truth for Recall@k: the stage-4 score (residual-decode MaxSim) of EVERY document for each query, through
+    the library's stage-isolated entry point in chunks of `chunk` documents, then the k_max best per query.  The
+    stage-4 kernel is itself parity-tested against the CPU oracle; here it only replaces candidate generation and
+    pruning by "all documents"."""
+    dev = q.device
+    B, nq = q.shape[0], cfg.q_len
+    taps = index.alloc_taps(B, nq, cfg.nprobe, chunk, max_candidates=1024, table=True, ci=False)
+    index.run_stages(1, 1, q, B, nq, cfg.nprobe, chunk, 1, taps, max_candidates=1024)
+    scores = torch.empty(B, index.N, dtype=torch.float32, device=dev)
+    taps.n_pruned = torch.full((B,), chunk, dtype=torch.int32, device=dev)
+    for d0 in range(0, index.N, chunk):
+        ids = torch.arange(d0, d0 + chunk, device=dev, dtype=torch.int32)
+        ids[ids >= index.N] = -1
+        taps.pruned = ids[None, :].expand(B, chunk).contiguous()
+        index.run_stages(4, 4, q, B, nq, cfg.nprobe, chunk, 1, taps, max_candidates=1024)
+        n = min(chunk, index.N - d0)
+        scores[:, d0:d0 + n] = taps.score4[:, :n]
+    top = torch.topk(scores, k_max, dim=1)
+    del scores, taps
+    index._ws = None
+    torch.cuda.empty_cache()
+    return top.indices.to(torch.int32), top.values
+
+
+def run_sweep(args, cfg, pkg, index, corp, q):
+    """QPS (batch `--batch`) and Recall@k (Def. 3, against exhaustive MaxSim over the decoded corpus, on the first
+    `--sweep-queries` queries) for nprobe x n_prune x k.  Prints one JSON line per point."""
+    dev = q.device
+    B, nq = args.batch, cfg.q_len
+    nrec = min(args.sweep_queries, q.shape[0])
+    qrec = q[:nrec].contiguous()
+    t0 = time.time()
+    truth_ids, _ = exhaustive_truth(index, qrec, cfg, 1000)
+    truth_s = time.time() - t0
+    n_batches = max(1, min(3, q.shape[0] // B))
+    batches = q[:n_batches * B].view(n_batches, B, nq, cfg.dim).contiguous()
+    print(json.dumps({"sweep": cfg.name, "batch": B, "recall_queries": nrec, "ground_truth": "library stage 4 over "
+                      "every document (chunks of 16384), top-1000 per query", "ground_truth_s": round(truth_s, 1)}))
+    for P in (1, 2, 4, 8, 16, 32):
+        if P > index.K:
+            continue
+        maxc = candidate_capacity(index, q, nq, P, 256, 10)
+        for n_prune in (256, 1024, 4096, 16384):
+            for k in (10, 100, 1000):
+                out = (torch.empty(B, k, dtype=torch.int32, device=dev), torch.empty(B, k, dtype=torch.float32, device=dev))
+                index.search(batches[0], P, n_prune, k, max_candidates=maxc, out=out)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for s in range(args.steps):
+                    index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / args.steps
+                assert index.status() == 0
+                ids, _ = index.search(qrec, P, n_prune, k, max_candidates=maxc)
+                hits = (ids[:, :, None] == truth_ids[:, None, :k]).any(dim=2).sum(dim=1).float()
+                print(json.dumps({"nprobe": P, "n_prune": n_prune, "k": k, "qps": B / (ms * 1e-3),
+                                  "ms_per_step": ms, "recall": float((hits / k).mean()), "max_candidates": maxc}))
 
 
 def main():
@@ -149,13 +231,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="mid")
-    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--batch", type=int, default=0, help="queries per call (default 256; 64 for the long-document configs)")
+    ap.add_argument("--sweep", action="store_true", help="QPS vs recall over nprobe x n_prune x k (see run_sweep)")
+    ap.add_argument("--sweep-queries", type=int, default=200)
     ap.add_argument("--batch1-queries", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     cfg = CONFIGS[args.config]
+    if args.batch <= 0:
+        args.batch = 64 if cfg.name.startswith("long") else 256
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -184,6 +270,11 @@ def main():
     index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
     build_s = time.time() - t0
     B, nq, P, n_prune, k = args.batch, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args, cfg, pkg, index, corp, q)
+        return
+    maxc = candidate_capacity(index, q, nq, P, n_prune, k)
 
     # batches cycle through the config's query set
     n_batches = max(1, min(args.steps + args.warmup, (q.shape[0] + B - 1) // B + 1))
@@ -197,10 +288,10 @@ def main():
     doclens64 = corp.doclens.to(torch.int64)
     work = []
     for bi in range(n_batches):
-        taps = index.alloc_taps(B, nq, P, n_prune, table=False, ci=False)
-        index.search(batches[bi], P, n_prune, k, taps=taps)
+        taps = index.alloc_taps(B, nq, P, n_prune, max_candidates=maxc, table=False, ci=False)
+        index.search(batches[bi], P, n_prune, k, max_candidates=maxc, taps=taps)
         assert index.status() == 0
-        mask = torch.arange(index.N, device=device)[None, :] < taps.n_cand[:, None].to(torch.int64)
+        mask = torch.arange(taps.cand.shape[1], device=device)[None, :] < taps.n_cand[:, None].to(torch.int64)
         toks = (doclens64[taps.cand.to(torch.int64).clamp_(0, index.N - 1)] * mask).sum()
         pr = taps.pruned.to(torch.int64)
         toks4 = (doclens64[pr.clamp(min=0)] * (pr >= 0)).sum()
@@ -211,7 +302,7 @@ def main():
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps ------------------------------------
     for s in range(args.warmup):
-        index.search(batches[s % n_batches], P, n_prune, k, out=out)
+        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out)
     barrier()
     pkg.profile_enable(True)
     pkg.profile_read()
@@ -220,7 +311,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for s in range(args.steps):
-        index.search(batches[(args.warmup + s) % n_batches], P, n_prune, k, out=out)
+        index.search(batches[(args.warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc, out=out)
     e1.record()
     barrier()
     clocks = sampler.stop()
@@ -236,11 +327,12 @@ def main():
 
     # ---- end to end through the host entry point: pinned host queries in, host ids/scores out -------------------
     for s in range(2):
-        index.search_host(host_batches[s % n_batches], P, n_prune, k, out=host_out)
+        index.search_host(host_batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=host_out)
     barrier()
     w0 = time.perf_counter()
     for s in range(args.steps):
-        index.search_host(host_batches[(args.warmup + s) % n_batches], P, n_prune, k, out=host_out)
+        index.search_host(host_batches[(args.warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc,
+                          out=host_out)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - w0
     t = torch.tensor([e2e_s], device=device)
@@ -254,14 +346,14 @@ def main():
     n1 = min(args.batch1_queries, q.shape[0])
     out1 = (torch.empty(1, k, dtype=torch.int32, device=device), torch.empty(1, k, dtype=torch.float32, device=device))
     for i in range(5):
-        index.search(q[i:i + 1], P, n_prune, k, out=out1)
+        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1)
     torch.cuda.synchronize()
     lat = []
     pkg.profile_enable(True)
     pkg.profile_read()
     for i in range(n1):
         a = time.perf_counter()
-        index.search(q[i:i + 1], P, n_prune, k, out=out1)
+        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1)
         torch.cuda.synchronize()
         lat.append(time.perf_counter() - a)
     stage_ms1, _ = pkg.profile_read()
@@ -271,7 +363,7 @@ def main():
     hout1 = (torch.empty(1, k, dtype=torch.int32).pin_memory(), torch.empty(1, k, dtype=torch.float32).pin_memory())
     w0 = time.perf_counter()
     for i in range(n1):
-        index.search_host(host_q1[i:i + 1], P, n_prune, k, out=hout1)
+        index.search_host(host_q1[i:i + 1], P, n_prune, k, max_candidates=maxc, out=hout1)
     e2e1_qps = n1 / (time.perf_counter() - w0)
 
     if rank != 0:
@@ -309,13 +401,15 @@ def main():
     }
 
     result = {
-        "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": metric_name(cfg, B), "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32 fixed point (stages 1-3) + f32 (stage 4)", "data": "synthetic",
         "config": {"workload": cfg.name, "batch": B, "n_docs": cfg.n_docs, "n_tokens": corp.n_tokens,
                    "n_centroids": cfg.n_centroids, "dim": cfg.dim, "nbits": cfg.nbits, "q_len": nq, "nprobe": P,
                    "n_prune": n_prune, "k": k, "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": "inputs larger than L2 (2.2 GB index, 2.1 GB score table per batch); no flush",
+                   "max_candidates": maxc if maxc else cfg.n_docs,
+                   "l2": "inputs larger than L2 (index %.1f GB, score table %.1f GB per batch); no flush"
+                         % ((corp.cids.numel() * 4 + corp.codes.numel()) / 1e9, B * cfg.n_centroids * nq * 4 / 1e9),
                    "gen_s": round(gen_s, 1), "index_build_s": round(build_s, 2)},
         "qps_batch1": float(1.0 / lat.mean()),
         "stage_ms_batch1": {name: round(v / min(n1, 256), 4) for name, v in stage_ms1.items()},

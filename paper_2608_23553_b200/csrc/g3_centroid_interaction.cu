@@ -171,6 +171,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
     constexpr int NQ = 16 * LPR;
     constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
     constexpr int STEPS = 32 / TPL;               // loads per 32-token slab (= LPR)
+    constexpr int SLABS = 2;                      // 32-token slabs per iteration (more costs occupancy and loses)
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int grp = lane / LPR, sub = lane % LPR;
@@ -184,31 +185,33 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
         uint32_t m[8];
 #pragma unroll
         for (int r = 0; r < 8; ++r) m[r] = 0x64006400u;       // 1024 + 0 in both halves
-        for (int64_t base = t0; base < t1; base += 64) {
-            // two 32-token slabs per iteration; lanes past the end repeat the last token (harmless for a maximum)
+        for (int64_t base = t0; base < t1; base += 32 * SLABS) {
+            // up to SLABS 32-token slabs per iteration, all their row loads in flight together; lanes past the end
+            // repeat the last token (harmless for a maximum)
             const int64_t last = t1 - 1;
-            const int64_t i0 = base + lane, i1 = base + 32 + lane;
-            const int32_t cid0 = cids[i0 < last ? i0 : last];
-            const int32_t cid1 = cids[i1 < last ? i1 : last];
-            const bool second = base + 32 < t1;
-            int4 v[2 * STEPS];
+            int32_t cid[SLABS];
 #pragma unroll
-            for (int s = 0; s < STEPS; ++s) {
-                const int32_t c = __shfl_sync(0xffffffffu, cid0, s * TPL + grp);
-                v[s] = __ldg(tb + (int64_t)c * LPR);
+            for (int k = 0; k < SLABS; ++k) {
+                const int64_t i = base + 32 * k + lane;
+                cid[k] = cids[i < last ? i : last];
             }
-            if (second) {
+            int4 v[SLABS * STEPS];
 #pragma unroll
-                for (int s = 0; s < STEPS; ++s) {
-                    const int32_t c = __shfl_sync(0xffffffffu, cid1, s * TPL + grp);
-                    v[STEPS + s] = __ldg(tb + (int64_t)c * LPR);
+            for (int k = 0; k < SLABS; ++k) {
+                if (k == 0 || base + 32 * k < t1) {
+#pragma unroll
+                    for (int s = 0; s < STEPS; ++s) {
+                        const int32_t c = __shfl_sync(0xffffffffu, cid[k], s * TPL + grp);
+                        v[k * STEPS + s] = __ldg(tb + (int64_t)c * LPR);
+                    }
                 }
             }
 #pragma unroll
-            for (int s = 0; s < STEPS; ++s) coarse_accumulate(m, v[s]);
-            if (second) {
+            for (int k = 0; k < SLABS; ++k) {
+                if (k == 0 || base + 32 * k < t1) {
 #pragma unroll
-                for (int s = 0; s < STEPS; ++s) coarse_accumulate(m, v[STEPS + s]);
+                    for (int s = 0; s < STEPS; ++s) coarse_accumulate(m, v[k * STEPS + s]);
+                }
             }
         }
         // Merge the lane groups (same columns, different tokens).  While a lane still holds several registers each

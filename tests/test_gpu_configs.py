@@ -1,0 +1,82 @@
+"""Parity on the other workload shapes: the long-document precision variants (512-token documents, 64-token queries,
+dim 96/128, 1/2 residual bits) at reduced document count, and the passage-corpus-shaped Large corpus (8.8M documents,
+~600M tokens, 262,144 centroids) at full size with sampled queries."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from parity import check_query, taps_to_numpy
+
+pytestmark = pytest.mark.gpu
+
+
+def _properties(tn, ids_np, sc_np, b, cfg, N, k):
+    n = int(tn["n_cand"][b])
+    cand = tn["cand"][b, :n]
+    assert np.all(np.diff(cand) > 0) and cand[0] >= 0 and cand[-1] < N
+    m = int(tn["n_pruned"][b])
+    pruned = tn["pruned"][b, :m]
+    assert m == min(cfg.n_prune, n) and np.all(np.diff(pruned) > 0) and np.all(np.isin(pruned, cand))
+    valid = ids_np[b] >= 0
+    assert np.all(np.isin(ids_np[b][valid], pruned)) and np.all(np.diff(sc_np[b][valid]) <= 0)
+    best = np.lexsort((pruned, -tn["score4"][b, :m].astype(np.float64)))[:k]
+    assert np.array_equal(pruned[best], ids_np[b][:len(best)])
+
+
+@pytest.mark.parametrize("name", ["long_d128_b2", "long_d128_b1", "long_d96_b2", "long_d96_b1"])
+def test_long_document_variants_reduced(name):
+    import paper_2608_23553_b200 as pkg
+    from synth import CONFIGS, make_corpus, make_queries
+    cfg = CONFIGS[name].replace(n_docs=4000, n_prune=256, n_queries=4)
+    dev = torch.device("cuda:0")
+    corp = make_corpus(cfg, device=dev)
+    q = make_queries(cfg, device=dev)
+    gix = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    B = q.shape[0]
+    taps = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, cfg.n_prune)
+    ids, sc = gix.search(q, cfg.nprobe, cfg.n_prune, cfg.k, taps=taps)
+    assert gix.status() == 0
+    tn = taps_to_numpy(taps)
+    ids_np, sc_np, q_np = ids.cpu().numpy(), sc.cpu().numpy(), q.cpu().numpy()
+    for b in (0, B - 1):
+        res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
+        assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune) == 0
+    for b in range(B):
+        _properties(tn, ids_np, sc_np, b, cfg, oix.N, cfg.k)
+
+
+def test_large_corpus_full_size_sampled_queries():
+    import psutil
+    import paper_2608_23553_b200 as pkg
+    from synth import CONFIGS, make_corpus, make_queries
+    if psutil.virtual_memory().available < 48e9:
+        pytest.skip("needs ~25 GB of host memory for the oracle's copy of the corpus")
+    free, _ = torch.cuda.mem_get_info()
+    if free < 90e9:
+        pytest.skip("needs ~60 GB of device memory")
+    cfg = CONFIGS["large"]
+    dev = torch.device("cuda:0")
+    corp = make_corpus(cfg, device=dev)
+    assert abs(corp.doclens.float().mean().item() - 68.0) < 0.3 and 5.9e8 < corp.n_tokens < 6.1e8
+    q = make_queries(cfg, 256, device=dev)
+    gix = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    B, maxc = 256, 512 * 1024
+    taps = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, cfg.n_prune, max_candidates=maxc, table=False)
+    ids, sc = gix.search(q, cfg.nprobe, cfg.n_prune, cfg.k, max_candidates=maxc, taps=taps)
+    assert gix.status() == 0
+    tn = taps_to_numpy(taps)
+    ids_np, sc_np, q_np = ids.cpu().numpy(), sc.cpu().numpy(), q.cpu().numpy()
+    for b in range(B):
+        _properties(tn, ids_np, sc_np, b, cfg, cfg.n_docs, cfg.k)
+    # stage 1 for one query, on its own
+    t1 = gix.alloc_taps(1, cfg.q_len, cfg.nprobe, cfg.n_prune, max_candidates=1024, table=True)
+    gix.run_stages(1, 1, q[77:78].contiguous(), 1, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k, t1, max_candidates=1024)
+    table77 = t1.score_table[0].cpu().numpy()
+    oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    for b in (77, 255):
+        res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
+        if b == 77:
+            assert np.array_equal(table77, res.S)
+        assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) == 0
