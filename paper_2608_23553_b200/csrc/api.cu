@@ -231,7 +231,15 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
         }
     }
     if (first <= 4 && last >= 4) {
-        if ((rc = launch_residual_scores(ix, p, queries, table, pruned, score4, st))) return rc;
+        if (residual_umma_supported(p.nq)) {
+            if (first > 1) {                       // stage 1 did not run in this call: build the query digit planes
+                if ((rc = launch_digits(queries, (int64_t)p.B * p.nq, ix.D, qdig, status, st))) return rc;
+                count_launch(SLOT_G4);
+            }
+            if ((rc = launch_residual_scores_umma(ix, p, queries, qdig, table, pruned, score4, status, st))) return rc;
+        } else if ((rc = launch_residual_scores(ix, p, queries, table, pruned, score4, st))) {
+            return rc;
+        }
         prof_mark(SLOT_G4, st);
     }
     if (last >= 5) {

@@ -117,6 +117,11 @@ int launch_select(const Index &ix, const Params &p, const int32_t *cand, const i
                   int32_t *pruned, int32_t *n_pruned, cudaStream_t st);
 int launch_residual_scores(const Index &ix, const Params &p, const float *queries, const int32_t *table,
                            const int32_t *pruned, float *score4, cudaStream_t st);
+// Tensor-core variant of stage 4 for q_len <= 64; qdig = the query digit planes of stage 1.
+bool residual_umma_supported(int nq);
+int launch_residual_scores_umma(const Index &ix, const Params &p, const float *queries, const int8_t *qdig,
+                                const int32_t *table, const int32_t *pruned, float *score4, uint32_t *status,
+                                cudaStream_t st);
 int launch_topk(const Index &ix, const Params &p, const int32_t *pruned, const float *score4, int32_t *out_ids,
                 float *out_scores, cudaStream_t st);
 

@@ -1,0 +1,332 @@
+// Stage 4 on the tensor cores (q_len <= 64): residual-decode MaxSim of the surviving documents (Definition 1 on the
+// decoded tokens),
+//   score(d) = sum_i max_{t in d} <q_i, c_{cid_t} + r^(code_t)>
+//            = sum_i [ max_t ( S[cid_t, i] + delta * sum_x q_i[x] u_t[x] ) + (lo + delta/2) * sum_x q_i[x] ].
+// The code contraction sum_x q_i[x] u_t[x] is a dense [tokens x D] x [D x q_len] product with tiny integer entries on
+// one side, so it runs as an exact integer MMA: the bucket indices u (0..3) are int8, the query is the same three
+// int8 digit planes of rint(q * 2^22) that stage 1 built, and tcgen05.mma kind::i8 gives sum_x u digit_a exactly in
+// int32; the three planes are recombined in fp32 (relative error 2^-24).
+//
+// A CTA owns one query and a run of its surviving documents, whose tokens form one stream cut into tiles of 128
+// (MMA M).  Per tile: every thread expands the packed code of one token through a 256-entry byte table into a 128-byte
+// int8 row and stores it, 128-byte swizzled, into the A tile; one thread issues D/32 MMAs (N = 3 * padded q_len: the
+// three digit planes side by side, loaded once per CTA by TMA); the accumulators come back with tcgen05.ld, get the
+// centroid term from the stage-1 table, and go to shared memory, where each warp folds its 32 tokens into per-document
+// maxima.  Tensor memory: 128 or 256 columns per CTA, so several CTAs share an SM and overlap each other's phases.
+// All mbarrier waits are bounded.
+#include <math.h>
+
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace chimera {
+
+constexpr int G4U_THREADS = 128;
+constexpr int G4U_TOK = 128;             // tokens per tile (MMA M)
+constexpr int G4U_MAX_DOCS = 32;         // documents per CTA, at most
+
+__device__ __forceinline__ uint32_t f_order(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float f_unorder(uint32_t o)
+{
+    return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
+}
+
+template <int NQP, int NBITS>
+__global__ void __launch_bounds__(G4U_THREADS)
+residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__restrict__ queries,
+                     const int32_t *__restrict__ table, int64_t K, int nq, int D, int CW, float delta, float kappa,
+                     const int32_t *__restrict__ pruned, int n_prune, int docs_per_cta,
+                     const int32_t *__restrict__ cids, const uint32_t *__restrict__ codes,
+                     const int64_t *__restrict__ doc_off, float *__restrict__ score4, uint32_t *status)
+{
+    constexpr int N = 3 * NQP;                               // MMA N: three digit planes side by side
+    constexpr uint32_t TMEM_COLS = N <= 128 ? 128 : 256;
+    constexpr uint32_t A_BYTES = G4U_TOK * 128;              // 16 KB
+    constexpr uint32_t B_BYTES = N * 128;
+    constexpr int VP = NQP + 1;                              // pitch of the value rows (floats)
+    constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) |
+                               ((uint32_t)(G4U_TOK >> 4) << 24);
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    __shared__ int s_off[G4U_MAX_DOCS + 1];                  // stream offset of each document
+    __shared__ long long s_t0[G4U_MAX_DOCS];                 // first global token of each document
+    __shared__ int s_rowdoc[G4U_TOK];                        // local document of each tile row (-1 = past the end)
+    __shared__ float s_sumq[NQP];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to the aligned area
+    const uint32_t sA = base, sB = base + A_BYTES;
+    float *vals = reinterpret_cast<float *>(gen + A_BYTES + B_BYTES);                       // [128][VP]
+    uint32_t *docmax = reinterpret_cast<uint32_t *>(vals + G4U_TOK * VP);                  // [MAX_DOCS][NQP]
+    uint32_t *lut = docmax + G4U_MAX_DOCS * NQP;                                           // 256 or 512 words
+    const uint32_t bars = smem_u32(lut + (NBITS == 2 ? 256 : 512));
+    const uint32_t bar_b = (bars + 7u) & ~7u, bar_mma = bar_b + 8;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.y;
+    const int j0 = blockIdx.x * docs_per_cta;
+    int nd = n_prune - j0;
+    if (nd > docs_per_cta) nd = docs_per_cta;
+
+    if (tid == 0) {
+        mbar_init(bar_b, 1);
+        mbar_init(bar_mma, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // stream offsets of this CTA's documents (padding slots have id -1 and no tokens)
+        int run = 0;
+        for (int dl = 0; dl < nd; ++dl) {
+            const int32_t d = pruned[(int64_t)b * n_prune + j0 + dl];
+            s_off[dl] = run;
+            if (d >= 0) {
+                const long long t0 = doc_off[d];
+                s_t0[dl] = t0;
+                run += (int)(doc_off[d + 1] - t0);
+            } else {
+                s_t0[dl] = 0;
+            }
+        }
+        s_off[nd] = run;
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(&s_tmem_base, TMEM_COLS);
+    }
+    // byte -> int8 bucket indices
+    if (NBITS == 2) {
+        for (int v = tid; v < 256; v += G4U_THREADS)
+            lut[v] = (uint32_t)(v & 3) | ((uint32_t)((v >> 2) & 3) << 8) | ((uint32_t)((v >> 4) & 3) << 16) |
+                     ((uint32_t)((v >> 6) & 3) << 24);
+    } else {
+        for (int v = tid; v < 256; v += G4U_THREADS) {
+            lut[2 * v] = (uint32_t)(v & 1) | ((uint32_t)((v >> 1) & 1) << 8) | ((uint32_t)((v >> 2) & 1) << 16) |
+                         ((uint32_t)((v >> 3) & 1) << 24);
+            lut[2 * v + 1] = (uint32_t)((v >> 4) & 1) | ((uint32_t)((v >> 5) & 1) << 8) |
+                             ((uint32_t)((v >> 6) & 1) << 16) | ((uint32_t)((v >> 7) & 1) << 24);
+        }
+    }
+    for (int e = tid; e < G4U_MAX_DOCS * NQP; e += G4U_THREADS) docmax[e] = 0u;     // below every real value
+    // sum_x q_i[x] per query token (warp per row, coalesced)
+    for (int i = warp; i < NQP; i += G4U_THREADS / 32) {
+        float s = 0.f;
+        if (i < nq)
+            for (int x = lane; x < D; x += 32) s += queries[((int64_t)b * nq + i) * D + x];
+        s = warp_sum(s);
+        if (lane == 0) s_sumq[i] = s;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+    const int total = s_off[nd];
+    const int n_tiles = (total + G4U_TOK - 1) / G4U_TOK;
+
+    if (tid == 0) {          // the query's three digit planes, side by side: rows [p * NQP, (p + 1) * NQP)
+        mbar_expect_tx(bar_b, B_BYTES);
+        for (int p = 0; p < 3; ++p) tma_load_3d(sB + p * NQP * 128, &map_q, 0, b * nq, p, bar_b);
+    }
+
+    const int32_t *tb = table + (int64_t)b * K * nq;
+    const bool vec_rows = (nq & 3) == 0;
+    const int k_steps = D >> 5;
+    const float code_scale = delta * (1.0f / 4194304.0f);    // delta * 2^-22
+    bool alive = true;
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        // ---- expand this thread's token into row `tid` of the A tile -------------------------------------------
+        const int s = tile * G4U_TOK + tid;
+        int32_t cid = -1;
+        int dl = -1;
+        if (s < total) {
+            dl = 0;
+            while (dl + 1 < nd && s_off[dl + 1] <= s) ++dl;
+            const long long t = s_t0[dl] + (s - s_off[dl]);
+            cid = cids[t];
+            const uint32_t *cw = codes + t * CW;
+            const uint32_t row = sA + ((uint32_t)(tid >> 3) << 10) + ((uint32_t)(tid & 7) << 7);
+            const uint32_t sw = (uint32_t)(tid & 7);
+            for (int w = 0; w < CW; ++w) {
+                const uint32_t word = __ldg(cw + w);
+                if (NBITS == 2) {
+                    const uint32_t c0 = lut[word & 255u], c1 = lut[(word >> 8) & 255u], c2 = lut[(word >> 16) & 255u],
+                                   c3 = lut[word >> 24];
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)w ^ sw) << 4)),
+                                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                                 : "memory");
+                } else {
+                    const uint32_t b0 = word & 255u, b1 = (word >> 8) & 255u, b2 = (word >> 16) & 255u, b3 = word >> 24;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)(2 * w) ^ sw) << 4)),
+                                 "r"(lut[2 * b0]), "r"(lut[2 * b0 + 1]), "r"(lut[2 * b1]), "r"(lut[2 * b1 + 1])
+                                 : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)(2 * w + 1) ^ sw) << 4)),
+                                 "r"(lut[2 * b2]), "r"(lut[2 * b2 + 1]), "r"(lut[2 * b3]), "r"(lut[2 * b3 + 1])
+                                 : "memory");
+                }
+            }
+        }
+        s_rowdoc[tid] = dl;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // rows visible to the tensor core's reads
+        tc_fence_before();
+        __syncthreads();
+
+        // ---- one thread issues the MMAs --------------------------------------------------------------------------
+        if (tid == 0) {
+            bool ok = true;
+            if (tile == 0) ok = mbar_wait(bar_b, 0);
+            if (ok) {
+                tc_fence_after();
+                const uint64_t da = umma_desc(sA), db = umma_desc(sB);
+                for (int k = 0; k < k_steps; ++k) umma_i8(tmem, da + 2 * k, db + 2 * k, IDESC, k > 0 ? 1u : 0u);
+                umma_commit(bar_mma);
+            } else {
+                s_abort = 1;
+            }
+        }
+        __syncwarp();
+        const bool ok = mbar_wait(bar_mma, tile & 1);
+        if (!__syncthreads_and(ok && !*(volatile int *)&s_abort)) {
+            if (tid == 0) atomicOr(status, ST_TIMEOUT);
+            alive = false;
+            break;
+        }
+        tc_fence_after();
+        __syncwarp();
+
+        // ---- accumulators -> values of this thread's token for every query token -----------------------------------
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        float *vrow = vals + tid * VP;
+#pragma unroll 1
+        for (int ch = 0; ch < NQP / 16; ++ch) {
+            int32_t a0[16], a1[16], a2[16];
+            tmem_ld16(lane_addr + 0 * NQP + ch * 16, a0);
+            tmem_ld16(lane_addr + 1 * NQP + ch * 16, a1);
+            tmem_ld16(lane_addr + 2 * NQP + ch * 16, a2);
+            tmem_ld_wait();
+            if (cid >= 0) {
+                const int32_t *srow = tb + (int64_t)cid * nq + ch * 16;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    int4 sv;
+                    const int col = ch * 16 + 4 * g;
+                    if (vec_rows && col + 3 < nq) {
+                        sv = __ldg(reinterpret_cast<const int4 *>(srow + 4 * g));
+                    } else {
+                        sv.x = col + 0 < nq ? __ldg(srow + 4 * g + 0) : 0;
+                        sv.y = col + 1 < nq ? __ldg(srow + 4 * g + 1) : 0;
+                        sv.z = col + 2 < nq ? __ldg(srow + 4 * g + 2) : 0;
+                        sv.w = col + 3 < nq ? __ldg(srow + 4 * g + 3) : 0;
+                    }
+                    const int32_t se[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int o = 4 * g + e;
+                        const float T = (float)a0[o] + 256.0f * (float)a1[o] + 65536.0f * (float)a2[o];
+                        vrow[col + e] = fmaf(code_scale, T, (float)se[e] * (1.0f / 16777216.0f));
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+
+        // ---- fold this warp's 32 tokens into the per-document maxima (lane = query token) -------------------------
+        {
+            int cur = -1;
+            float m0 = 0.f, m1 = 0.f;
+            for (int rr = 0; rr < 32; ++rr) {
+                const int r = warp * 32 + rr;
+                const int d2 = s_rowdoc[r];
+                if (d2 < 0) break;
+                const float v0 = vals[r * VP + lane];
+                const float v1 = NQP > 32 ? vals[r * VP + 32 + lane] : 0.f;
+                if (d2 != cur) {
+                    if (cur >= 0) {
+                        atomicMax(&docmax[cur * NQP + lane], f_order(m0));
+                        if (NQP > 32) atomicMax(&docmax[cur * NQP + 32 + lane], f_order(m1));
+                    }
+                    cur = d2;
+                    m0 = v0;
+                    m1 = v1;
+                } else {
+                    m0 = fmaxf(m0, v0);
+                    m1 = fmaxf(m1, v1);
+                }
+            }
+            if (cur >= 0) {
+                atomicMax(&docmax[cur * NQP + lane], f_order(m0));
+                if (NQP > 32) atomicMax(&docmax[cur * NQP + 32 + lane], f_order(m1));
+            }
+        }
+    }
+
+    if (n_tiles == 0 && tid == 0) mbar_wait(bar_b, 0);       // never leave with the TMA load in flight
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- per document: add the per-query-token constant, sum over query tokens ----------------------------------------
+    if (alive) {
+        for (int dl = warp; dl < nd; dl += G4U_THREADS / 32) {
+            const int32_t d = pruned[(int64_t)b * n_prune + j0 + dl];
+            float v = 0.f;
+            if (d >= 0) {
+                if (lane < nq) v = f_unorder(docmax[dl * NQP + lane]) + kappa * s_sumq[lane];
+                if (NQP > 32 && 32 + lane < nq) v += f_unorder(docmax[dl * NQP + 32 + lane]) + kappa * s_sumq[32 + lane];
+            }
+            v = warp_sum(v);
+            if (lane == 0) score4[(int64_t)b * n_prune + j0 + dl] = d >= 0 ? v : -INFINITY;
+        }
+    }
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
+}
+
+template <int NQP, int NBITS>
+static int launch_g4_umma(const Index &ix, const Params &p, const float *queries, const int8_t *qdig,
+                          const int32_t *table, const int32_t *pruned, float *score4, uint32_t *status, cudaStream_t st)
+{
+    constexpr int N = 3 * NQP;
+    const float delta = (ix.res_hi - ix.res_lo) / (float)(1 << ix.nbits);
+    const float kappa = ix.res_lo + 0.5f * delta;
+    CUtensorMap map_q;
+    int rc = make_plane_map(&map_q, qdig, (int64_t)p.B * p.nq, NQP);
+    if (rc) return rc;
+    const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 + sizeof(float) * G4U_TOK * (NQP + 1) +
+                        sizeof(uint32_t) * G4U_MAX_DOCS * NQP + sizeof(uint32_t) * (NBITS == 2 ? 256 : 512) + 32;
+    auto kern = residual_maxsim_umma<NQP, NBITS>;
+    CHIMERA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // documents per CTA: about four CTAs per SM in total, between 4 and 32 documents each
+    int64_t dpc = ((int64_t)p.n_prune * p.B + 4LL * ix.sm_count - 1) / (4LL * ix.sm_count);
+    if (dpc < 4) dpc = 4;
+    if (dpc > G4U_MAX_DOCS) dpc = G4U_MAX_DOCS;
+    if (dpc > p.n_prune) dpc = p.n_prune;
+    dim3 grid((unsigned)((p.n_prune + dpc - 1) / dpc), (unsigned)p.B);
+    kern<<<grid, G4U_THREADS, smem, st>>>(map_q, queries, table, ix.K, p.nq, ix.D, ix.CB / 4, delta, kappa, pruned,
+                                          p.n_prune, (int)dpc, ix.cids, reinterpret_cast<const uint32_t *>(ix.codes),
+                                          ix.doc_off, score4, status);
+    CHIMERA_CUDA(cudaGetLastError());
+    count_launch(SLOT_G4);
+    return CHIMERA_OK;
+}
+
+bool residual_umma_supported(int nq) { return nq <= 64; }
+
+int launch_residual_scores_umma(const Index &ix, const Params &p, const float *queries, const int8_t *qdig,
+                                const int32_t *table, const int32_t *pruned, float *score4, uint32_t *status,
+                                cudaStream_t st)
+{
+    if (ix.nbits == 2) {
+        if (p.nq <= 32) return launch_g4_umma<32, 2>(ix, p, queries, qdig, table, pruned, score4, status, st);
+        return launch_g4_umma<64, 2>(ix, p, queries, qdig, table, pruned, score4, status, st);
+    }
+    if (p.nq <= 32) return launch_g4_umma<32, 1>(ix, p, queries, qdig, table, pruned, score4, status, st);
+    return launch_g4_umma<64, 1>(ix, p, queries, qdig, table, pruned, score4, status, st);
+}
+
+}  // namespace chimera
