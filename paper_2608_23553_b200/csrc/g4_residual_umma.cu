@@ -56,7 +56,6 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     __shared__ int s_abort;
     __shared__ int s_off[G4U_MAX_DOCS + 1];                  // stream offset of each document
     __shared__ long long s_t0[G4U_MAX_DOCS];                 // first global token of each document
-    __shared__ int s_rowdoc[G4U_TOK];                        // local document of each tile row (-1 = past the end)
     __shared__ float s_sumq[NQP];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to the aligned area
@@ -136,40 +135,66 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     const int k_steps = D >> 5;
     const float code_scale = delta * (1.0f / 4194304.0f);    // delta * 2^-22
     bool alive = true;
+    constexpr int MAXCW = 8;                                  // 32 code bytes per token at most
 
-    for (int tile = 0; tile < n_tiles; ++tile) {
-        // ---- expand this thread's token into row `tid` of the A tile -------------------------------------------
+    // Token of stream position s (this thread's row of a tile): local document, centroid id, packed code words.
+    int dl_hint = 0;
+    auto fetch = [&](int tile, int &dl, int32_t &cid, uint32_t (&cw)[MAXCW]) {
         const int s = tile * G4U_TOK + tid;
-        int32_t cid = -1;
-        int dl = -1;
+        dl = -1;
+        cid = -1;
         if (s < total) {
-            dl = 0;
-            while (dl + 1 < nd && s_off[dl + 1] <= s) ++dl;
+            while (dl_hint + 1 < nd && s_off[dl_hint + 1] <= s) ++dl_hint;    // positions only move forward
+            dl = dl_hint;
             const long long t = s_t0[dl] + (s - s_off[dl]);
             cid = cids[t];
-            const uint32_t *cw = codes + t * CW;
+            const uint32_t *src = codes + t * CW;
+#pragma unroll
+            for (int w = 0; w < MAXCW; ++w)
+                if (w < CW) cw[w] = __ldg(src + w);
+        }
+    };
+
+    int dl, dl_next = -1;
+    int32_t cid, cid_next = -1;
+    uint32_t cw[MAXCW], cw_next[MAXCW];
+    if (n_tiles > 0) fetch(0, dl_next, cid_next, cw_next);
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        dl = dl_next;
+        cid = cid_next;
+#pragma unroll
+        for (int w = 0; w < MAXCW; ++w) cw[w] = cw_next[w];
+
+        // ---- expand this thread's token into row `tid` of the A tile -------------------------------------------
+        if (dl >= 0) {
             const uint32_t row = sA + ((uint32_t)(tid >> 3) << 10) + ((uint32_t)(tid & 7) << 7);
             const uint32_t sw = (uint32_t)(tid & 7);
-            for (int w = 0; w < CW; ++w) {
-                const uint32_t word = __ldg(cw + w);
-                if (NBITS == 2) {
-                    const uint32_t c0 = lut[word & 255u], c1 = lut[(word >> 8) & 255u], c2 = lut[(word >> 16) & 255u],
-                                   c3 = lut[word >> 24];
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)w ^ sw) << 4)),
-                                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                                 : "memory");
-                } else {
-                    const uint32_t b0 = word & 255u, b1 = (word >> 8) & 255u, b2 = (word >> 16) & 255u, b3 = word >> 24;
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)(2 * w) ^ sw) << 4)),
-                                 "r"(lut[2 * b0]), "r"(lut[2 * b0 + 1]), "r"(lut[2 * b1]), "r"(lut[2 * b1 + 1])
-                                 : "memory");
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)(2 * w + 1) ^ sw) << 4)),
-                                 "r"(lut[2 * b2]), "r"(lut[2 * b2 + 1]), "r"(lut[2 * b3]), "r"(lut[2 * b3 + 1])
-                                 : "memory");
+#pragma unroll
+            for (int w = 0; w < MAXCW; ++w) {
+                if (w < CW) {
+                    const uint32_t word = cw[w];
+                    if (NBITS == 2) {
+                        const uint32_t c0 = lut[word & 255u], c1 = lut[(word >> 8) & 255u],
+                                       c2 = lut[(word >> 16) & 255u], c3 = lut[word >> 24];
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)w ^ sw) << 4)),
+                                     "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                                     : "memory");
+                    } else {
+                        const uint32_t b0 = word & 255u, b1 = (word >> 8) & 255u, b2 = (word >> 16) & 255u,
+                                       b3 = word >> 24;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(
+                                         row + (((uint32_t)(2 * w) ^ sw) << 4)),
+                                     "r"(lut[2 * b0]), "r"(lut[2 * b0 + 1]), "r"(lut[2 * b1]), "r"(lut[2 * b1 + 1])
+                                     : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(
+                                         row + (((uint32_t)(2 * w + 1) ^ sw) << 4)),
+                                     "r"(lut[2 * b2]), "r"(lut[2 * b2 + 1]), "r"(lut[2 * b3]), "r"(lut[2 * b3 + 1])
+                                     : "memory");
+                    }
                 }
             }
         }
-        s_rowdoc[tid] = dl;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // rows visible to the tensor core's reads
         tc_fence_before();
         __syncthreads();
@@ -188,6 +213,26 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             }
         }
         __syncwarp();
+
+        // ---- while the tensor core works: this token's row of the score table, and the next tile's token -----------
+        int4 sv[NQP / 4];
+        if (cid >= 0) {
+            const int32_t *srow = tb + (int64_t)cid * nq;
+#pragma unroll
+            for (int g = 0; g < NQP / 4; ++g) {
+                const int col = 4 * g;
+                if (vec_rows && col + 3 < nq) {
+                    sv[g] = __ldg(reinterpret_cast<const int4 *>(srow + col));
+                } else {
+                    sv[g].x = col + 0 < nq ? __ldg(srow + col + 0) : 0;
+                    sv[g].y = col + 1 < nq ? __ldg(srow + col + 1) : 0;
+                    sv[g].z = col + 2 < nq ? __ldg(srow + col + 2) : 0;
+                    sv[g].w = col + 3 < nq ? __ldg(srow + col + 3) : 0;
+                }
+            }
+        }
+        if (tile + 1 < n_tiles) fetch(tile + 1, dl_next, cid_next, cw_next);
+
         const bool ok = mbar_wait(bar_mma, tile & 1);
         if (!__syncthreads_and(ok && !*(volatile int *)&s_abort)) {
             if (tid == 0) atomicOr(status, ST_TIMEOUT);
@@ -200,7 +245,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         // ---- accumulators -> values of this thread's token for every query token -----------------------------------
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
         float *vrow = vals + tid * VP;
-#pragma unroll 1
+#pragma unroll
         for (int ch = 0; ch < NQP / 16; ++ch) {
             int32_t a0[16], a1[16], a2[16];
             tmem_ld16(lane_addr + 0 * NQP + ch * 16, a0);
@@ -208,25 +253,16 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             tmem_ld16(lane_addr + 2 * NQP + ch * 16, a2);
             tmem_ld_wait();
             if (cid >= 0) {
-                const int32_t *srow = tb + (int64_t)cid * nq + ch * 16;
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
-                    int4 sv;
-                    const int col = ch * 16 + 4 * g;
-                    if (vec_rows && col + 3 < nq) {
-                        sv = __ldg(reinterpret_cast<const int4 *>(srow + 4 * g));
-                    } else {
-                        sv.x = col + 0 < nq ? __ldg(srow + 4 * g + 0) : 0;
-                        sv.y = col + 1 < nq ? __ldg(srow + 4 * g + 1) : 0;
-                        sv.z = col + 2 < nq ? __ldg(srow + 4 * g + 2) : 0;
-                        sv.w = col + 3 < nq ? __ldg(srow + 4 * g + 3) : 0;
-                    }
-                    const int32_t se[4] = {sv.x, sv.y, sv.z, sv.w};
+                    const int4 q4 = sv[ch * 4 + g];
+                    const int32_t se[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int o = 4 * g + e;
-                        const float T = (float)a0[o] + 256.0f * (float)a1[o] + 65536.0f * (float)a2[o];
-                        vrow[col + e] = fmaf(code_scale, T, (float)se[e] * (1.0f / 16777216.0f));
+                        // |sum_x u_x Xq_x| <= 3 * 2^22 * |q|_1 < 2^31: the plane recombination fits int32
+                        const int32_t T = a0[o] + a1[o] * 256 + a2[o] * 65536;
+                        vrow[ch * 16 + o] = fmaf(code_scale, (float)T, (float)se[e] * (1.0f / 16777216.0f));
                     }
                 }
             }
@@ -236,30 +272,24 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
 
         // ---- fold this warp's 32 tokens into the per-document maxima (lane = query token) -------------------------
         {
-            int cur = -1;
-            float m0 = 0.f, m1 = 0.f;
-            for (int rr = 0; rr < 32; ++rr) {
-                const int r = warp * 32 + rr;
-                const int d2 = s_rowdoc[r];
-                if (d2 < 0) break;
-                const float v0 = vals[r * VP + lane];
-                const float v1 = NQP > 32 ? vals[r * VP + 32 + lane] : 0.f;
-                if (d2 != cur) {
-                    if (cur >= 0) {
-                        atomicMax(&docmax[cur * NQP + lane], f_order(m0));
-                        if (NQP > 32) atomicMax(&docmax[cur * NQP + 32 + lane], f_order(m1));
-                    }
-                    cur = d2;
-                    m0 = v0;
-                    m1 = v1;
-                } else {
-                    m0 = fmaxf(m0, v0);
-                    m1 = fmaxf(m1, v1);
+            const int prev = __shfl_up_sync(0xffffffffu, dl, 1);
+            const uint32_t valid = __ballot_sync(0xffffffffu, dl >= 0);
+            uint32_t starts = __ballot_sync(0xffffffffu, dl >= 0 && (lane == 0 || dl != prev));
+            const int n_rows = __popc(valid);                 // valid rows are a prefix of the warp's rows
+            while (starts) {
+                const int a = __ffs(starts) - 1;
+                starts &= starts - 1;
+                const int e = starts ? __ffs(starts) - 1 : n_rows;
+                const int doc = __shfl_sync(0xffffffffu, dl, a);
+                const float *vp = vals + (warp * 32 + a) * VP + lane;
+                float m0 = vp[0], m1 = NQP > 32 ? vp[32] : 0.f;
+                for (int r = a + 1; r < e; ++r) {
+                    vp += VP;
+                    m0 = fmaxf(m0, vp[0]);
+                    if (NQP > 32) m1 = fmaxf(m1, vp[32]);
                 }
-            }
-            if (cur >= 0) {
-                atomicMax(&docmax[cur * NQP + lane], f_order(m0));
-                if (NQP > 32) atomicMax(&docmax[cur * NQP + 32 + lane], f_order(m1));
+                atomicMax(&docmax[doc * NQP + lane], f_order(m0));
+                if (NQP > 32) atomicMax(&docmax[doc * NQP + 32 + lane], f_order(m1));
             }
         }
     }
