@@ -189,9 +189,9 @@ int chimera_profile_read(float *ms, int64_t *launches);
  *                identical to the probes of chimera_search / chimera_run_stages for the same table.
  *   stream       cudaStream_t as void*; the two kernels are enqueued on it, the call does not synchronise.
  *
- * Limits: n_queries * lists * nprobe * q_len * 8 bytes must fit the 4 MiB array, where lists = 8 * min(64,
- * ceil(2 * SM count / n_queries), ceil(n_centroids / 512)); e.g. one query of 32 tokens with nprobe 4 against 65,536
- * centroids needs 512 KiB, a batch of 8 such queries 2.3 MiB.  Larger calls return CHIMERA_WORKSPACE_TOO_SMALL and
+ * Limits: n_queries * lists * nprobe * q_len * 8 bytes must fit the 4 MiB array, where lists = min(512,
+ * ceil(4 * SM count / n_queries), ceil(n_centroids / 256)); e.g. one query of 32 tokens with nprobe 4 against 65,536
+ * centroids needs 256 KiB, a batch of 64 such queries 640 KiB.  Larger calls return CHIMERA_WORKSPACE_TOO_SMALL and
  * enqueue nothing (use chimera_search with a workspace).  Other argument limits are those of chimera_search.
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device current)

@@ -69,14 +69,15 @@ Layout make_layout(const Index &ix, const Params &p)
 {
     Layout L;
     memset(&L, 0, sizeof(L));
-    // probe stage: enough blocks to fill the device at small batch, at most 64 per query, at least ~512 rows each
-    int64_t blocks = (2LL * ix.sm_count + p.B - 1) / p.B;
-    int64_t by_rows = (ix.K + 511) / 512;
+    // probe stage: about four blocks per SM over the whole batch, at most 512 per query, at least ~256 rows each;
+    // every block leaves one partial list per query token
+    int64_t blocks = (4LL * ix.sm_count + p.B - 1) / p.B;
+    int64_t by_rows = (ix.K + 255) / 256;
     if (blocks > by_rows) blocks = by_rows;
-    if (blocks > 64) blocks = 64;
+    if (blocks > 512) blocks = 512;
     if (blocks < 1) blocks = 1;
     L.probe_blocks = (int32_t)blocks;
-    L.n_part = L.probe_blocks * PROBE_WARPS;
+    L.n_part = L.probe_blocks;
     L.words = (ix.N + 31) / 32;
     L.n_chunks = (int32_t)((L.words + BITMAP_CHUNK_WORDS - 1) / BITMAP_CHUNK_WORDS);
 

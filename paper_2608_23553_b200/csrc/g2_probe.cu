@@ -25,7 +25,7 @@ __device__ __forceinline__ void list_insert(unsigned long long *list, int P, uns
     list[j * PROBE_THREADS] = key;
 }
 
-// grid (probe_blocks, B, ceil(nq / 32)).  part: [B][n_part][P][nq], n_part = probe_blocks * PROBE_WARPS.
+// grid (probe_blocks, B, ceil(nq / 32)).  part: [B][n_part][P][nq], n_part = probe_blocks (one list per block).
 __global__ void __launch_bounds__(PROBE_THREADS)
 probe_partial(const int32_t *__restrict__ table, int64_t K, int nq, int P, int rows_per_block, int n_part,
               unsigned long long *__restrict__ part)
@@ -52,7 +52,19 @@ probe_partial(const int32_t *__restrict__ table, int64_t K, int nq, int P, int r
             list_insert(mine, P, key_int(s3, (int32_t)(r + 3 * PROBE_WARPS)));
         }
         for (; r < r1; r += PROBE_WARPS) list_insert(mine, P, key_int(tb[r * nq], (int32_t)r));
-        unsigned long long *dst = part + (((int64_t)b * n_part + (int64_t)blockIdx.x * PROBE_WARPS + warp) * P) * nq + col;
+    }
+    // fold the block's eight lists into warp 0's, then write one list per block and column
+    __syncthreads();
+    if (warp == 0 && col < nq) {
+        for (int w = 1; w < PROBE_WARPS; ++w) {
+            const unsigned long long *src = lists + w * 32 + lane;
+            for (int j = 0; j < P; ++j) {
+                unsigned long long key = src[j * PROBE_THREADS];
+                if (key <= mine[(P - 1) * PROBE_THREADS]) break;
+                list_insert(mine, P, key);
+            }
+        }
+        unsigned long long *dst = part + (((int64_t)b * n_part + blockIdx.x) * P) * nq + col;
         for (int j = 0; j < P; ++j) dst[(int64_t)j * nq] = mine[j * PROBE_THREADS];
     }
 }
@@ -158,13 +170,14 @@ extern "C" int chimera_probes_static(const int32_t *score_table, int64_t n_centr
     }
     unsigned long long *part = g_probe_scratch_ptr[dev];
 
-    // same slicing rule as the workspace-based stage: fill the device at small batch, at least ~512 rows per block
-    int64_t blocks = (2LL * sm_count + n_queries - 1) / n_queries;
-    const int64_t by_rows = (n_centroids + 511) / 512;
+    // same slicing rule as the workspace-based stage: about four blocks per SM over the batch, at most 512 per query,
+    // at least ~256 rows per block; one partial list per block
+    int64_t blocks = (4LL * sm_count + n_queries - 1) / n_queries;
+    const int64_t by_rows = (n_centroids + 255) / 256;
     if (blocks > by_rows) blocks = by_rows;
-    if (blocks > 64) blocks = 64;
+    if (blocks > 512) blocks = 512;
     if (blocks < 1) blocks = 1;
-    const int n_part = (int)blocks * PROBE_WARPS;
+    const int n_part = (int)blocks;
     const size_t need = sizeof(unsigned long long) * (size_t)n_queries * n_part * nprobe * q_len;
     if (need > STATIC_PROBE_SCRATCH_BYTES)
         return fail(CHIMERA_WORKSPACE_TOO_SMALL,

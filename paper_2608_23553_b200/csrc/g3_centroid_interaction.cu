@@ -361,9 +361,19 @@ __device__ __forceinline__ uint32_t radix_select(const int32_t *__restrict__ sb,
         __syncthreads();
         const uint32_t prefix = *s_prefix;
         const int want = *s_want;
-        for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
-            uint32_t u = (uint32_t)sb[j] ^ 0x80000000u;
-            if ((u & known_mask) == prefix) atomicAdd(&hist[(u >> shift) & (bins - 1)], 1);
+        // eight independent loads per thread before their histogram updates (the loop is latency-bound otherwise)
+        for (int base = 0; base < n; base += 8 * SEL_THREADS) {
+            uint32_t u[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int j = base + e * SEL_THREADS + threadIdx.x;
+                u[e] = j < n ? ((uint32_t)sb[j] ^ 0x80000000u) : 0u;
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int j = base + e * SEL_THREADS + threadIdx.x;
+                if (j < n && (u[e] & known_mask) == prefix) atomicAdd(&hist[(u[e] >> shift) & (bins - 1)], 1);
+            }
         }
         __syncthreads();
         // descending bins: thread t owns bins (bins-1-2t) and (bins-2-2t)
@@ -412,18 +422,37 @@ select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_ca
     int need_eq;
     const uint32_t thr = radix_select(sb, n, n_prune, hist, warp_part, &s_prefix, &s_want, &need_eq);
 
-    // Ordered compaction: keep u > thr, and the first need_eq entries with u == thr.
+    // Ordered compaction: keep u > thr, and the first need_eq entries with u == thr.  Each thread owns four
+    // consecutive entries per round, so one block scan covers 4096 entries.
     int run_gt = 0, run_eq = 0;
-    for (int base = 0; base < n; base += SEL_THREADS) {
-        int j = base + threadIdx.x;
-        uint32_t u = j < n ? ((uint32_t)sb[j] ^ 0x80000000u) : 0u;
-        int gt = (j < n && u > thr) ? 1 : 0;
-        int eq = (j < n && u == thr) ? 1 : 0;
+    for (int base = 0; base < n; base += 4 * SEL_THREADS) {
+        const int j0 = base + 4 * threadIdx.x;
+        uint32_t u[4];
+        int32_t id[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = j0 + e;
+            u[e] = j < n ? ((uint32_t)sb[j] ^ 0x80000000u) : 0u;
+            id[e] = j < n ? cb[j] : 0;
+        }
+        int gt = 0, eq = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            gt += (j0 + e < n && u[e] > thr) ? 1 : 0;
+            eq += (j0 + e < n && u[e] == thr) ? 1 : 0;
+        }
         int total;
-        int before = sel_block_scan((gt << 16) | eq, &total, warp_part);   // <= 1024 per field
+        const int before = sel_block_scan((gt << 16) | eq, &total, warp_part);   // <= 4096 per field
         int gt_before = run_gt + (before >> 16), eq_before = run_eq + (before & 0xffff);
-        bool keep = gt || (eq && eq_before < need_eq);
-        if (keep) out[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = cb[j];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (j0 + e >= n) break;
+            const bool is_gt = u[e] > thr, is_eq = u[e] == thr;
+            if (is_gt || (is_eq && eq_before < need_eq))
+                out[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = id[e];
+            gt_before += is_gt ? 1 : 0;
+            eq_before += is_eq ? 1 : 0;
+        }
         run_gt += total >> 16;
         run_eq += total & 0xffff;
     }
@@ -455,12 +484,23 @@ contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n
     const uint32_t thr = radix_select(lo + (int64_t)b * maxc, n, n_prune, hist, warp_part, &s_prefix, &s_want, &need_eq);
     const int32_t tau = (int32_t)(thr ^ 0x80000000u);
     int run = 0;
-    for (int base = 0; base < n; base += SEL_THREADS) {
-        int j = base + threadIdx.x;
-        int keep = (j < n && hb[j] >= tau) ? 1 : 0;
+    for (int base = 0; base < n; base += 4 * SEL_THREADS) {
+        const int j0 = base + 4 * threadIdx.x;
+        int32_t h[4], id[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = j0 + e;
+            h[e] = j < n ? hb[j] : INT_MIN;
+            id[e] = j < n ? cb[j] : 0;
+        }
+        int keep = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) keep += (j0 + e < n && h[e] >= tau) ? 1 : 0;
         int total;
-        int before = sel_block_scan(keep, &total, warp_part);
-        if (keep) out[run + before] = cb[j];
+        int pos = run + sel_block_scan(keep, &total, warp_part);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (j0 + e < n && h[e] >= tau) out[pos++] = id[e];
         run += total;
     }
     if (threadIdx.x == 0) n_cont[b] = run;

@@ -45,7 +45,7 @@ def test_static_probes_match_workspace_probes_on_two_calls_in_a_row():
 
 def test_static_probes_reject_sizes_beyond_the_built_in_array():
     import paper_2608_23553_b200 as pkg
-    # 64 queries x (8 lists x 5 blocks) x nprobe 64 x q_len 120 x 8 B is far beyond 4 MiB
+    # 64 queries x 10 lists x nprobe 64 x q_len 120 x 8 B is far beyond 4 MiB
     table = torch.zeros(64, 4096, 120, dtype=torch.int32, device="cuda:0")
     with pytest.raises(pkg.ChimeraError) as e:
         pkg.probes_static(table, 64)
