@@ -60,6 +60,18 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
+def ncu_traffic(cfg, batch):
+    """DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture, or None.  The capture
+    (profiles/ncu_ci_coarse_mid.md) was taken on the Mid corpus at batch 8; traffic is proportional to the number of
+    queries (every query has its own table and candidate list), so it is scaled by batch / 8."""
+    if cfg.name == "mid" and NCU_CI_COARSE_MID_B8_BYTES:
+        return NCU_CI_COARSE_MID_B8_BYTES * batch / 8.0
+    return None
+
+
+NCU_CI_COARSE_MID_B8_BYTES = 467.2e6    # dram__bytes_read.sum + dram__bytes_write.sum of one launch at batch 8
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -371,33 +383,38 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel (the centroid-interaction scan) ----------------------------------------
+    # ---- roofline of the dominant kernel: the stage-3 bound scan over every candidate token (ci_coarse_kernel) -------
     peak, peak_kind = measured_peaks()
     used = [work[(args.warmup + s) % n_batches] for s in range(args.steps)]
     mean = lambda key: float(np.mean([u[key] for u in used]))       # noqa: E731
     n_prof = min(args.steps, 256)                                    # the library times at most 256 calls per read
     ci_ms = stage_ms["centroid_interaction"] / n_prof
-    # algorithmic bytes of one launch: centroid ids of every candidate token (4 B) + per candidate document its id
-    # (4 B) and two offsets (16 B) + the CI written (4 B)
-    ci_bytes = 4.0 * mean("cand_tokens") + 24.0 * mean("cand")
+    # algorithmic HBM bytes of one launch: the centroid id of every candidate token (4 B) + per candidate document
+    # its id (4 B), two token offsets (16 B) and the two bounds written (8 B)
+    ci_bytes = 4.0 * mean("cand_tokens") + 28.0 * mean("cand")
     ci_gbs = ci_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0
-    # L2 gathers: one q_len-byte row of the 8-bit table per candidate token (bound phase) + one 4*q_len-byte row of
-    # the exact table per contender token (contender tokens estimated with the candidates' mean length)
+    # what binds it: one table-row lookup per candidate token; a lookup is one distinct 128-byte line for the SM's
+    # load pipe, which retires one line per cycle, so the roof is SMs x SM clock row lookups per second
+    rows = mean("cand_tokens")
+    lookup_roof = 148 * 1.965e9
     cont_frac = mean("contenders") / max(mean("cand"), 1.0)
-    l2_bytes = mean("cand_tokens") * nq * (1.0 + 4.0 * cont_frac)
     g4_ms = stage_ms["residual_scores"] / n_prof
     g4_bytes = mean("pruned_tokens") * (4.0 + cfg.code_bytes)
     stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
     roofline = {
-        "kernel": "ci_kernel (stage 3 centroid-interaction scan)", "bound": "hbm",
+        "kernel": "ci_coarse_kernel (stage 3 bound scan over every candidate token)", "bound": "hbm",
         "achieved": ci_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-        "frac": ci_gbs / peak, "traffic": None, "ms_per_launch": ci_ms, "algorithmic_bytes_per_launch": ci_bytes,
-        "contender_fraction": cont_frac,
-        "binding_roof": {"bound": "l2_gather", "bytes_per_launch": l2_bytes,
-                         "achieved_gbs": l2_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0},
+        "frac": ci_gbs / peak, "traffic": ncu_traffic(cfg, B), "ms_per_launch": ci_ms,
+        "algorithmic_bytes_per_launch": ci_bytes, "contender_fraction": cont_frac,
+        "binding_roof": {"bound": "table-row lookups (one 128-byte line per SM cycle)", "lookups_per_launch": rows,
+                         "achieved_glookups_s": rows / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0,
+                         "peak_glookups_s": lookup_roof / 1e9,
+                         "frac": rows / (ci_ms * 1e-3) / lookup_roof if ci_ms > 0 else 0.0,
+                         "l2_bytes_per_launch": rows * nq},
         "stage_ms_per_step": stages,
-        "stage4": {"ms_per_launch": g4_ms, "code_gbs": g4_bytes / (g4_ms * 1e-3) / 1e9 if g4_ms > 0 else 0.0,
-                   "tflops": 2.0 * mean("pruned_tokens") * nq * cfg.dim / (g4_ms * 1e-3) / 1e12 if g4_ms > 0 else 0.0},
+        "stage4": {"kernel": "residual_maxsim_umma (tcgen05 kind::i8)", "ms_per_launch": g4_ms,
+                   "code_gbs": g4_bytes / (g4_ms * 1e-3) / 1e9 if g4_ms > 0 else 0.0,
+                   "int8_tops": 2.0 * 3.0 * mean("pruned_tokens") * nq * cfg.dim / (g4_ms * 1e-3) / 1e12 if g4_ms > 0 else 0.0},
     }
 
     result = {

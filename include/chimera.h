@@ -168,10 +168,11 @@ int chimera_index_info(const chimera_index *index, chimera_index_desc *desc, int
 /* Per-stage device timing.  After chimera_profile_enable(1) every search records CUDA events around its stages on
  * the search's stream; chimera_profile_read synchronises those events and returns, per stage slot, the summed
  * milliseconds and the number of kernels launched since the last read, then resets both.  Slots:
- * 0 score table, 1 probes, 2 candidate gather, 3 centroid interaction, 4 top-n_prune selection, 5 residual scores,
- * 6 top-k, 7 copies/clears.  ms and launches: host arrays of CHIMERA_PROFILE_SLOTS entries.  At most
+ * 0 score table, 1 probes, 2 candidate gather, 3 centroid-interaction bounds over every candidate (or the exact scan
+ * when q_len is not 32/64), 4 selections (contenders, top n_prune), 5 residual scores, 6 top-k, 7 copies/clears,
+ * 8 exact centroid interaction of the contenders.  ms and launches: host arrays of CHIMERA_PROFILE_SLOTS entries.  At most
  * CHIMERA_PROFILE_MAX_CALLS searches are kept between reads (later ones are not timed).  Not thread-safe. */
-#define CHIMERA_PROFILE_SLOTS 8
+#define CHIMERA_PROFILE_SLOTS 9
 #define CHIMERA_PROFILE_MAX_CALLS 256
 int chimera_profile_enable(int32_t on);
 int chimera_profile_read(float *ms, int64_t *launches);

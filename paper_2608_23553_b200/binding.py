@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(_PKG, "libchimera.so")
 _lib = None
 
 PROFILE_SLOTS = ("score_table", "probes", "gather", "centroid_interaction", "select", "residual_scores", "topk",
-                 "misc")
+                 "misc", "ci_exact")
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "CUDA_ERROR", 3: "WORKSPACE_TOO_SMALL", 4: "CAPACITY_OVERFLOW",
                 5: "TIMEOUT", 6: "UNSUPPORTED"}

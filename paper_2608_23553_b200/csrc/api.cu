@@ -220,12 +220,13 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             prof_mark(SLOT_CI, st);
             if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, st))) return rc;
             prof_mark(SLOT_SELECT, st);
-            if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, 2 * ix.sm_count, st))) return rc;
-            prof_mark(SLOT_CI, st);
+            if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, 2 * ix.sm_count, SLOT_CI_EXACT, st)))
+                return rc;
+            prof_mark(SLOT_CI_EXACT, st);
             if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else {
-            if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, 0, st))) return rc;
+            if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, 0, SLOT_CI, st))) return rc;
             prof_mark(SLOT_CI, st);
             if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
             prof_mark(SLOT_SELECT, st);
@@ -259,7 +260,8 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if (taps->ci) {
                 if (two_phase) {                   // the search only needed exact CI for the contenders: the tap asks
                                                    // for every candidate, so the exact kernel runs over all of them
-                    if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, taps->ci, 0, st))) return rc;
+                    if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, taps->ci, 0, SLOT_MISC, st)))
+                        return rc;
                 } else if ((rc = copy_d2d(taps->ci, ci, cand_bytes, st))) return rc;
             }
             if (taps->n_contenders &&

@@ -87,7 +87,7 @@ int fail(int code, const char *fmt, ...);
 // ---------------------------------------------------------------------------------------------------------------
 // Profiling hooks (api.cu).
 // ---------------------------------------------------------------------------------------------------------------
-enum Slot { SLOT_G1 = 0, SLOT_PROBE, SLOT_GATHER, SLOT_CI, SLOT_SELECT, SLOT_G4, SLOT_TOPK, SLOT_MISC };
+enum Slot { SLOT_G1 = 0, SLOT_PROBE, SLOT_GATHER, SLOT_CI, SLOT_SELECT, SLOT_G4, SLOT_TOPK, SLOT_MISC, SLOT_CI_EXACT };
 void count_launch(int slot, int n = 1);
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -112,7 +112,7 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
 int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
                       const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st);
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
-                                const int32_t *n_cand, int32_t *ci, int blocks_cap, cudaStream_t st);
+                                const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, cudaStream_t st);
 int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
                   int32_t *pruned, int32_t *n_pruned, cudaStream_t st);
 int launch_residual_scores(const Index &ix, const Params &p, const float *queries, const int32_t *table,

@@ -179,21 +179,41 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
     const int4 *tb = reinterpret_cast<const int4 *>(table8 + (int64_t)b * K * NQ) + sub;
     const int32_t *cb = cand + (int64_t)b * maxc;
     const int warps_per_query = gridDim.x * CI_WARPS;
-    for (int j = blockIdx.x * CI_WARPS + (threadIdx.x >> 5); j < n; j += warps_per_query) {
+    // The chain candidate id -> token range -> first centroid ids is three dependent loads: it is issued one document
+    // ahead, so it overlaps the row gathers of the current document.
+    int64_t nx_t0 = 0, nx_t1 = 0;
+    int32_t nx_cid[SLABS];
+    auto prefetch = [&](int j) {
         const int64_t d = cb[j];
-        const int64_t t0 = doc_off[d], t1 = doc_off[d + 1];
+        nx_t0 = doc_off[d];
+        nx_t1 = doc_off[d + 1];
+#pragma unroll
+        for (int k = 0; k < SLABS; ++k) {
+            const int64_t i = nx_t0 + 32 * k + lane;
+            nx_cid[k] = cids[i < nx_t1 - 1 ? i : nx_t1 - 1];
+        }
+    };
+    int j = blockIdx.x * CI_WARPS + (threadIdx.x >> 5);
+    if (j < n) prefetch(j);
+    for (; j < n; j += warps_per_query) {
+        const int64_t t0 = nx_t0, t1 = nx_t1;
+        int32_t cid[SLABS];
+#pragma unroll
+        for (int k = 0; k < SLABS; ++k) cid[k] = nx_cid[k];
+        if (j + warps_per_query < n) prefetch(j + warps_per_query);
         uint32_t m[8];
 #pragma unroll
         for (int r = 0; r < 8; ++r) m[r] = 0x64006400u;       // 1024 + 0 in both halves
         for (int64_t base = t0; base < t1; base += 32 * SLABS) {
             // up to SLABS 32-token slabs per iteration, all their row loads in flight together; lanes past the end
             // repeat the last token (harmless for a maximum)
-            const int64_t last = t1 - 1;
-            int32_t cid[SLABS];
+            if (base != t0) {
+                const int64_t last = t1 - 1;
 #pragma unroll
-            for (int k = 0; k < SLABS; ++k) {
-                const int64_t i = base + 32 * k + lane;
-                cid[k] = cids[i < last ? i : last];
+                for (int k = 0; k < SLABS; ++k) {
+                    const int64_t i = base + 32 * k + lane;
+                    cid[k] = cids[i < last ? i : last];
+                }
             }
             int4 v[SLABS * STEPS];
 #pragma unroll
@@ -294,7 +314,7 @@ int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, 
 
 // Exact CI of a list of documents.  blocks_cap bounds the blocks per query (0 = default).
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
-                                const int32_t *n_cand, int32_t *ci, int blocks_cap, cudaStream_t st)
+                                const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, cudaStream_t st)
 {
     int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
     int64_t cap = blocks_cap > 0 ? blocks_cap : (int64_t)ix.sm_count * 8;
@@ -313,7 +333,7 @@ int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t 
     else
         ci_kernel<4><<<grid, CI_THREADS, 0, st>>>(table, ix.K, p.nq, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
     CHIMERA_CUDA(cudaGetLastError());
-    count_launch(SLOT_CI);
+    count_launch(slot);
     return CHIMERA_OK;
 }
 
