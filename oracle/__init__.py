@@ -26,7 +26,7 @@ def build(force: bool = False) -> str:
     """Compile the oracle with gcc (plain -O2, no -march flags, no OpenMP)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + ".%d.tmp" % os.getpid()
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -131,6 +131,20 @@ def prune(cand: np.ndarray, ci: np.ndarray, n_prune: int) -> np.ndarray:
     return out[:n].copy()
 
 
+def partial_scores(S: np.ndarray, q, pr: np.ndarray, cand: np.ndarray, ix: Index) -> np.ndarray:
+    """O-8: int32 partial score F' (Algorithm 2) of every candidate, from the retrieved tokens only."""
+    S = _arr(S, np.int32)
+    q = _arr(q, np.float32)
+    pr = _arr(pr, np.int32)
+    cand = _arr(cand, np.int32)
+    out = np.empty(cand.shape[0], dtype=np.int32)
+    lib().oracle_partial_scores(_p(S), _p(q), ctypes.c_int32(q.shape[0]), ctypes.c_int32(ix.dim),
+                                ctypes.c_int32(ix.nbits), ctypes.c_float(ix.res_lo), ctypes.c_float(ix.res_hi),
+                                _p(pr), ctypes.c_int32(pr.shape[1]), _p(ix.cids), _p(ix.codes), _p(ix.doclens),
+                                ctypes.c_int64(ix.N), _p(cand), ctypes.c_int64(cand.shape[0]), _p(out))
+    return out
+
+
 def score_docs(q, docs: np.ndarray, ix: Index) -> np.ndarray:
     """O-5: float32 Chamfer score of each listed document on its decoded tokens."""
     q = _arr(q, np.float32)
@@ -188,12 +202,13 @@ class Result:
     scores: np.ndarray     # [k] float32
 
 
-def pipeline(q, ix: Index, nprobe: int, n_prune: int, k: int) -> Result:
-    """All stages for one query [nq, D]."""
+def pipeline(q, ix: Index, nprobe: int, n_prune: int, k: int, partial: bool = False) -> Result:
+    """All stages for one query [nq, D].  partial=True prunes with the paper's partial scores F' (Algorithm 2) instead
+    of the full centroid interaction; `ci` then holds F'."""
     S = score_table(q, ix.centroids)
     pr = probes(S, nprobe)
     cand = candidates(pr, ix)
-    ci = ci_scores(S, cand, ix)
+    ci = partial_scores(S, q, pr, cand, ix) if partial else ci_scores(S, cand, ix)
     pruned = prune(cand, ci, n_prune)
     s4 = score_docs(q, pruned, ix)
     ids, sc = topk(pruned, s4, k)

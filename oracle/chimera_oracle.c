@@ -17,6 +17,7 @@
  *   O-5 oracle_score_docs    Chamfer similarity on decoded tokens          (Def. 1)
  *   O-6 oracle_topk          top-k by score                                (Def. 2, Eq. 1)
  *   O-7 oracle_chamfer       Def. 1 on raw vectors;  oracle_recall  Def. 3
+ *   O-8 oracle_partial_scores  candidate refinement with partial scores F'(Q,V)  (Sec. 3.2 step 2, Algorithm 2)
  *
  * Pins: every function above is pinned by tests that do not call it to produce their expectation
  * (closed forms, library routines on special cases, set identities, hand-worked values).  Unpinned:
@@ -138,6 +139,71 @@ int64_t oracle_prune(const int32_t *cand, const int32_t *ci, int64_t n_cand, int
     qsort(pruned, (size_t)keep, sizeof(int32_t), cmp_i32_asc);
     free(v);
     return keep;
+}
+
+/* ---------------------------------------------------------------- O-8 ------------------------------------------ */
+/* Candidate refinement (Sec. 3.2 step 2, Algorithm 2): only the tokens retrieved in candidate generation contribute.
+ * For each query token i, L_i = the tokens assigned to one of its nprobe probed centroids; every document score
+ * starts at 0 per query token, each retrieved token raises doc.score[i] to max(score, dist(i, token)), and the
+ * partial score is F'(d) = sum_i doc.score[i]  (a query token that retrieved nothing of d contributes 0).
+ *
+ * dist(i, t) is the low-bit score <q_i, c_cid + r^(code_t)> in Q.24 fixed point, so that the refinement is exactly
+ * reproducible:  dist = S[cid_t, i] + llrint(delta*4*T + kappa*4*SQ_i),  T = sum_x Xq_i[x] u_t[x],
+ * SQ_i = sum_x Xq_i[x],  Xq = rint(q * 2^22),  delta = (hi - lo) / 2^b and kappa = lo + delta/2 evaluated in float,
+ * the two products and their sum in double (each exact or correctly rounded, no fused operations).
+ *
+ * cand: ascending candidate ids (O-3); fprime[j] = F' of cand[j].  Written as Algorithm 2's loops over a dense
+ * n_cand x nq score table. */
+void oracle_partial_scores(const int32_t *S, const float *q, int32_t nq, int32_t D, int32_t nbits, float lo, float hi,
+                           const int32_t *probes, int32_t nprobe, const int32_t *cids, const uint8_t *codes,
+                           const int32_t *doclens, int64_t N, const int32_t *cand, int64_t n_cand, int32_t *fprime)
+{
+    const int per_byte = 8 / nbits, mask = (1 << nbits) - 1;
+    const int64_t cb = (int64_t)D * nbits / 8;
+    const float delta = (hi - lo) / (float)(1 << nbits);
+    const float kappa = lo + 0.5f * delta;
+    int64_t *slot = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);   /* document -> row of the score table, or -1 */
+    for (int64_t d = 0; d < N; ++d) slot[d] = -1;
+    for (int64_t j = 0; j < n_cand; ++j) slot[cand[j]] = j;
+    int32_t *score = (int32_t *)calloc((size_t)(n_cand > 0 ? n_cand : 1) * nq, sizeof(int32_t));   /* init 0 */
+    int64_t *xq = (int64_t *)malloc(sizeof(int64_t) * (size_t)D);
+    int64_t K = 0;                                        /* centroid ids are < K = 1 + the largest id in use */
+    for (int64_t d = 0, t = 0; d < N; ++d)
+        for (int j = 0; j < doclens[d]; ++j, ++t)
+            if (cids[t] >= K) K = (int64_t)cids[t] + 1;
+    for (int e = 0; e < nq * nprobe; ++e)
+        if (probes[e] >= K) K = (int64_t)probes[e] + 1;
+    uint8_t *probed = (uint8_t *)malloc((size_t)K);       /* is this centroid probed by query token i? */
+    for (int i = 0; i < nq; ++i) {
+        int64_t sq = 0;
+        for (int x = 0; x < D; ++x) { xq[x] = (int64_t)rint((double)q[(int64_t)i * D + x] * Q22); sq += xq[x]; }
+        memset(probed, 0, (size_t)K);
+        for (int p = 0; p < nprobe; ++p) probed[probes[i * nprobe + p]] = 1;
+        int64_t t = 0;
+        for (int64_t d = 0; d < N; ++d) {
+            for (int j = 0; j < doclens[d]; ++j, ++t) {
+                if (!probed[cids[t]]) continue;           /* token t is in L_i iff its centroid is probed by i */
+                int64_t T = 0;
+                for (int x = 0; x < D; ++x) {
+                    int u = (codes[t * cb + x / per_byte] >> ((x % per_byte) * nbits)) & mask;
+                    T += xq[x] * u;
+                }
+                double r = (double)delta * 4.0 * (double)T + (double)kappa * 4.0 * (double)sq;
+                int64_t dist = (int64_t)S[(int64_t)cids[t] * nq + i] + (int64_t)llrint(r);
+                int32_t *cell = &score[slot[d] * nq + i];
+                if (dist > *cell) *cell = (int32_t)dist;
+            }
+        }
+    }
+    for (int64_t j = 0; j < n_cand; ++j) {
+        int64_t sum = 0;
+        for (int i = 0; i < nq; ++i) sum += score[j * nq + i];
+        fprime[j] = (int32_t)sum;
+    }
+    free(slot);
+    free(score);
+    free(xq);
+    free(probed);
 }
 
 /* ---------------------------------------------------------------- O-5 ------------------------------------------ */

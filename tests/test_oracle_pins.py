@@ -415,3 +415,82 @@ def test_tiny_config_candidate_count_matches_closed_form():
         assert len(r.pruned) == cfg.n_prune and np.all(np.diff(r.pruned) > 0)
         # the generating component is the nearest centroid: probe 0 of a query token scores ~ cos(noise angle)
         assert np.all(r.S[r.probes[:, 0], np.arange(cfg.q_len)] > 0.8 * 2 ** 24)
+
+
+# ------------------------------------------------------------------ O-8 candidate refinement (Algorithm 2) --------
+
+def test_partial_scores_handworked():
+    D = 8
+    cent = np.zeros((2, D), np.float32)
+    cent[0, 0] = 1.0
+    cent[1, 1] = 1.0
+    q = cent.copy()
+    cids = np.array([0, 0, 0, 0, 1, 1], np.int32)
+    codes = np.array([[1], [0], [1], [0], [2], [0]], np.uint8)
+    doclens = np.array([1, 2, 2, 1], np.int32)
+    ix = oracle.make_index(cent, cids, codes, doclens, 1)
+    S = oracle.score_table(q, cent)
+    pr = oracle.probes(S, 1)
+    assert pr.tolist() == [[0], [1]]
+    cand = oracle.candidates(pr, ix)
+    assert cand.tolist() == [0, 1, 2, 3]
+    want = [int(r.split()[1]) for r in _golden_rows("partial_score_handworked.txt")]
+    assert oracle.partial_scores(S, q, pr, cand, ix).tolist() == want
+
+
+def test_partial_scores_with_every_list_probed_equal_the_full_low_bit_maxsim():
+    # Sec. 3.2: F' only drops the tokens that were not retrieved; with every cluster probed V n L_q = V, so F' is the
+    # full score of the decoded document (here every per-query-token maximum is positive, so the 0 floor is inactive)
+    for nbits in (2, 1):
+        ix, q = _small_case(30 + nbits, N=60, K=8, D=32, nbits=nbits, nq=5)
+        S = oracle.score_table(q, ix.centroids)
+        pr = oracle.probes(S, ix.K)
+        cand = oracle.candidates(pr, ix)
+        fp = oracle.partial_scores(S, q, pr, cand, ix)
+        full = oracle.score_docs(q, cand, ix).astype(np.float64)
+        dec = ix.centroids[ix.cids] + levels(nbits)[unpack_codes(ix.codes, ix.dim, nbits)].astype(np.float32)
+        for j, d in enumerate(cand):
+            per_q = (q.astype(np.float64) @ dec[ix.doc_off[d]:ix.doc_off[d + 1]].astype(np.float64).T).max(axis=1)
+            if np.all(per_q > 1e-3):
+                assert fp[j] * 2.0 ** -24 == pytest.approx(full[j], abs=5e-6)
+            else:                                        # floor at 0 for query tokens whose best token is negative
+                assert fp[j] * 2.0 ** -24 == pytest.approx(np.maximum(per_q, 0).sum(), abs=5e-6)
+
+
+def test_partial_scores_brute_force_and_monotone_in_nprobe():
+    ix, q = _small_case(33, N=80, K=16, D=16, nbits=2, nq=6)
+    S = oracle.score_table(q, ix.centroids)
+    X = lambda a: int(round(float(a) * 2 ** 22))
+    delta = np.float32(0.5) / np.float32(4)
+    kappa = np.float32(-0.25) + np.float32(0.5) * delta
+    prev = None
+    for P in (1, 2, 5, 16):
+        pr = oracle.probes(S, P)
+        cand = oracle.candidates(pr, ix)
+        fp = oracle.partial_scores(S, q, pr, cand, ix)
+        # Algorithm 2 from Python dictionaries, integers and one rounding per token
+        score = {}
+        for i in range(len(q)):
+            xq = [X(v) for v in q[i]]
+            for d in range(ix.N):
+                for t in range(int(ix.doc_off[d]), int(ix.doc_off[d + 1])):
+                    if int(ix.cids[t]) not in pr[i].tolist():
+                        continue
+                    T = sum(xq[x] * ((int(ix.codes[t, x // 4]) >> (2 * (x % 4))) & 3) for x in range(16))
+                    r = float(delta) * 4.0 * float(T) + float(kappa) * 4.0 * float(sum(xq))
+                    dist = int(S[ix.cids[t], i]) + int(np.rint(r))
+                    score[(d, i)] = max(score.get((d, i), 0), dist)
+        want = [sum(score.get((int(d), i), 0) for i in range(len(q))) for d in cand]
+        assert fp.tolist() == want
+        cur = dict(zip(cand.tolist(), fp.tolist()))
+        if prev is not None:                                      # more retrieved tokens can only raise a maximum
+            assert all(cur[d] >= v for d, v in prev.items())
+        prev = cur
+
+
+def test_pipeline_with_partial_scores_prunes_by_f_prime():
+    ix, q = _small_case(34, N=150, K=24, D=16, nq=6)
+    r = oracle.pipeline(q, ix, 3, 20, 5, partial=True)
+    order = np.lexsort((r.cand, -r.ci.astype(np.int64)))[:20]
+    assert np.array_equal(r.pruned, np.sort(r.cand[order]))
+    assert np.array_equal(r.score4, oracle.score_docs(q, r.pruned, ix))
