@@ -155,6 +155,29 @@ int chimera_run_stages(const chimera_index *index, int32_t first_stage, int32_t 
                        int64_t max_candidates, void *workspace, size_t workspace_bytes, void *stream,
                        const chimera_taps *inout, int32_t *out_ids, float *out_scores);
 
+/* Build the token-level posting lists (per centroid: its tokens and their documents; Sec. 3.2 step 1 keeps posting
+ * lists at token level) that chimera_search_partial needs.  Allocates 8 bytes per token plus 8 per centroid inside the
+ * index (cudaMalloc), synchronises the stream.  Idempotent.  Workspace sizes grow afterwards (a score table of
+ * n_queries x max_candidates x q_len int32), so query chimera_workspace_bytes again.
+ * Errors: INVALID_ARG, UNSUPPORTED (more than 2^31 - 1 tokens), CUDA_ERROR (nothing stays allocated). */
+int chimera_index_enable_partial(chimera_index *index, void *stream);
+
+/* The search with the paper's own candidate refinement in place of stage 3 (Sec. 3.2 step 2, Algorithm 2; aggregation
+ * as in Algorithm 4): only the tokens retrieved in candidate generation are scored.  For query token i every token t of
+ * its nprobe probed posting lists raises score[doc(t), i] (initially 0) to
+ *     dist(i, t) = S[cid_t, i] + llrint(delta*4*T + kappa*4*SQ_i)          (Q.24 fixed point)
+ * with T = sum_x Xq_i[x] u_t[x], SQ_i = sum_x Xq_i[x], Xq = rint(q * 2^22), delta = (res_hi - res_lo) / 2^nbits and
+ * kappa = res_lo + delta / 2 in float, products and sum in double; F'(d) = sum_i score[d, i]; the n_prune candidates
+ * with the largest F' (ties: smaller id) go on to stages 4 and 5 unchanged.  It touches sum_i |L_i| tokens instead of
+ * every token of every candidate, and prunes by a different (cheaper, coarser) score than chimera_search, so results
+ * differ from chimera_search; they are exactly reproducible.
+ * Arguments as chimera_search_tapped (taps may be NULL); taps->ci receives F' of every candidate, taps->n_contenders
+ * the candidate counts.  Requires chimera_index_enable_partial. */
+int chimera_search_partial(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                           int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                           size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
+                           const chimera_taps *taps);
+
 /* Device-side status of the last search that used this workspace: synchronises the stream, then writes CHIMERA_OK,
  * CHIMERA_CAPACITY_OVERFLOW (some query had more than max_candidates candidates; its results are computed on the
  * first max_candidates of them and are not the specified output), CHIMERA_INVALID_ARG (a query element outside

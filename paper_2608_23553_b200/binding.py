@@ -178,9 +178,16 @@ class Index:
             pruned=torch.empty(B, n_prune, dtype=i32, device=dev), n_pruned=torch.empty(B, dtype=i32, device=dev),
             score4=torch.empty(B, n_prune, dtype=torch.float32, device=dev))
 
+    def enable_partial(self):
+        """Build the token-level posting lists needed by search(..., partial=True)."""
+        with torch.cuda.device(self.device):
+            _check(lib().chimera_index_enable_partial(self._h, _stream()))
+        self._ws = None
+
     def search(self, queries: torch.Tensor, nprobe: int, n_prune: int, k: int, max_candidates: int = 0,
-               taps: Optional[Taps] = None, out=None):
-        """queries: [B, q_len, dim] float32 CUDA tensor.  Returns (ids [B,k] int32, scores [B,k] float32)."""
+               taps: Optional[Taps] = None, out=None, partial: bool = False):
+        """queries: [B, q_len, dim] float32 CUDA tensor.  Returns (ids [B,k] int32, scores [B,k] float32).
+        partial=True prunes with the paper's partial scores (chimera_search_partial)."""
         assert queries.is_cuda and queries.dtype == torch.float32 and queries.is_contiguous()
         B, q_len, dim = queries.shape
         assert dim == self.dim
@@ -194,7 +201,10 @@ class Index:
         args = (self._h, _ptr(queries), ctypes.c_int32(B), ctypes.c_int32(q_len), ctypes.c_int32(nprobe),
                 ctypes.c_int32(n_prune), ctypes.c_int32(k), ctypes.c_int64(max_candidates), _ptr(ws),
                 ctypes.c_size_t(ws.numel()), _stream(), _ptr(ids), _ptr(scores))
-        if taps is None:
+        if partial:
+            c = taps._c() if taps is not None else None
+            _check(lib().chimera_search_partial(*args, ctypes.byref(c) if c is not None else None))
+        elif taps is None:
             _check(lib().chimera_search(*args))
         else:
             c = taps._c()

@@ -104,6 +104,8 @@ Layout make_layout(const Index &ix, const Params &p)
     L.cont = take(two_phase);
     L.n_cont = take(B * sizeof(int32_t));
     L.pruned = take(B * p.n_prune * sizeof(int32_t));
+    L.word_rank = take(B * (size_t)L.words * sizeof(int32_t));
+    L.partial_m = take(ix.tok_id ? B * (size_t)p.maxc * nq * sizeof(int32_t) : 0);
     L.n_pruned = take(B * sizeof(int32_t));
     L.score4 = take(B * p.n_prune * sizeof(float));
     L.total = o;
@@ -136,8 +138,11 @@ static int copy_d2d(void *dst, const void *src, size_t bytes, cudaStream_t st)
 }
 
 static int run(const Index &ix, const Params &p, int first, int last, const float *queries, void *workspace,
-               size_t workspace_bytes, cudaStream_t st, const chimera_taps *taps, int32_t *out_ids, float *out_scores)
+               size_t workspace_bytes, cudaStream_t st, const chimera_taps *taps, int32_t *out_ids, float *out_scores,
+               bool partial = false)
 {
+    if (partial && !ix.tok_id)
+        return fail(CHIMERA_INVALID_ARG, "partial-score refinement needs chimera_index_enable_partial first");
     if (!workspace || ((uintptr_t)workspace & 255)) return fail(CHIMERA_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
     const Layout L = make_layout(ix, p);
     if (workspace_bytes < L.total)
@@ -156,7 +161,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int32_t *cand = (int32_t *)(ws + L.cand);
     int32_t *n_cand = (int32_t *)(ws + L.n_cand);
     int32_t *ci = (int32_t *)(ws + L.ci);
-    const bool two_phase = coarse_supported(p.nq);
+    const bool two_phase = coarse_supported(p.nq) && !partial;
     uint8_t *table8 = two_phase ? (uint8_t *)(ws + L.table8) : nullptr;
     int32_t *lo = (int32_t *)(ws + L.lo);
     int32_t *hi = (int32_t *)(ws + L.hi);
@@ -164,6 +169,8 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int32_t *n_cont = (int32_t *)(ws + L.n_cont);
     int32_t *pruned = (int32_t *)(ws + L.pruned);
     int32_t *n_pruned = (int32_t *)(ws + L.n_pruned);
+    int32_t *word_rank = (int32_t *)(ws + L.word_rank);
+    int32_t *partial_m = (int32_t *)(ws + L.partial_m);
     float *score4 = (float *)(ws + L.score4);
 
     const size_t B = (size_t)p.B;
@@ -206,11 +213,19 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     if (first <= 2 && last >= 2) {
         if ((rc = launch_probes(ix, p, L, table, part, probes, st))) return rc;
         prof_mark(SLOT_PROBE, st);
-        if ((rc = launch_gather(ix, p, L, probes, bitmap, chunk_cnt, cand, n_cand, status, st))) return rc;
+        if ((rc = launch_gather(ix, p, L, probes, bitmap, chunk_cnt, cand, n_cand, word_rank, status, st))) return rc;
         prof_mark(SLOT_GATHER, st);
     }
     if (first <= 3 && last >= 3) {
-        if (two_phase) {
+        if (partial) {
+            // the paper's candidate refinement: partial scores from the retrieved tokens only, then the same selection
+            if ((rc = launch_partial_scores(ix, p, L, queries, table, probes, bitmap, word_rank, n_cand, partial_m, ci,
+                                            st)))
+                return rc;
+            prof_mark(SLOT_CI, st);
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
+            prof_mark(SLOT_SELECT, st);
+        } else if (two_phase) {
             if (first > 1) {                       // the table came from the caller: derive its coarse copy
                 if ((rc = launch_coarse_table(ix, p, table, table8, st))) return rc;
                 prof_mark(SLOT_MISC, st);
@@ -337,10 +352,33 @@ int chimera_build_index(const chimera_index_desc *desc, const float *centroids, 
     return CHIMERA_OK;
 }
 
+int chimera_index_enable_partial(chimera_index *index, void *stream)
+{
+    Index *ix = reinterpret_cast<Index *>(index);
+    if (!ix) return fail(CHIMERA_INVALID_ARG, "index is NULL");
+    return build_token_lists(*ix, (cudaStream_t)stream);
+}
+
+int chimera_search_partial(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                           int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, void *workspace,
+                           size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
+                           const chimera_taps *taps)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc) return rc;
+    return run(*ix, p, 1, 5, queries, workspace, workspace_bytes, (cudaStream_t)stream, taps, out_ids, out_scores,
+               true);
+}
+
 int chimera_destroy_index(chimera_index *index)
 {
     Index *ix = reinterpret_cast<Index *>(index);
     if (!ix) return CHIMERA_OK;
+    cudaFree(ix->tok_off);
+    cudaFree(ix->tok_id);
+    cudaFree(ix->tok_doc);
     cudaFree(ix->doc_off);
     cudaFree(ix->cdig);
     cudaFree(ix->ivf_off);

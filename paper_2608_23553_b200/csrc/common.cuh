@@ -25,6 +25,10 @@ struct Index {
     int32_t *ivf_doc = nullptr;       // [ivf_len]  owned: unique document ids per centroid, unordered
     int64_t ivf_len = 0;
     int32_t max_doclen = 0;
+    // token-level posting lists (only after chimera_index_enable_partial): per centroid its tokens and their documents
+    int64_t *tok_off = nullptr;       // [K+1]      owned
+    int32_t *tok_id = nullptr;        // [T]        owned: token ids per centroid, unordered
+    int32_t *tok_doc = nullptr;       // [T]        owned: document of each listed token
 };
 
 // Device status bits kept in the first word of a workspace.
@@ -58,6 +62,8 @@ struct Layout {
     size_t cont;          // int32  [B][maxc]         contender ids, ascending
     size_t n_cont;        // int32  [B]
     size_t pruned;        // int32  [B][n_prune]
+    size_t word_rank;     // int32  [B][words]        candidates before each bitmap word (document -> candidate index)
+    size_t partial_m;     // int32  [B][maxc][nq]     per (candidate, query token) best retrieved-token score
     size_t n_pruned;      // int32  [B]
     size_t score4;        // float  [B][n_prune]
     size_t total;
@@ -104,7 +110,15 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
 int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32_t *table, unsigned long long *part,
                   int32_t *probes, cudaStream_t st);
 int launch_gather(const Index &ix, const Params &p, const Layout &L, const int32_t *probes, uint32_t *bitmap,
-                  int32_t *chunk_cnt, int32_t *cand, int32_t *n_cand, uint32_t *status, cudaStream_t st);
+                  int32_t *chunk_cnt, int32_t *cand, int32_t *n_cand, int32_t *word_rank, uint32_t *status,
+                  cudaStream_t st);
+// Token-level posting lists for the partial-score refinement (allocates; index_build.cu).
+int build_token_lists(Index &ix, cudaStream_t st);
+// Candidate refinement with partial scores (Algorithm 2): fprime[b][j] for every candidate.
+int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, const float *queries,
+                          const int32_t *table, const int32_t *probes, const uint32_t *bitmap,
+                          const int32_t *word_rank, const int32_t *n_cand, int32_t *partial_m, int32_t *fprime,
+                          cudaStream_t st);
 bool coarse_supported(int nq);
 int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st);
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,

@@ -100,7 +100,8 @@ chunk_scan_kernel(int32_t *__restrict__ chunk_cnt, int n_chunks, int64_t maxc, i
 // grid (n_chunks, B): write the ids of the set bits of each chunk, ascending, at its scanned offset.
 __global__ void __launch_bounds__(CHUNK_THREADS)
 compact_kernel(const uint32_t *__restrict__ bitmap, int64_t words, int n_chunks,
-               const int32_t *__restrict__ chunk_cnt, int64_t maxc, int32_t *__restrict__ cand)
+               const int32_t *__restrict__ chunk_cnt, int64_t maxc, int32_t *__restrict__ cand,
+               int32_t *__restrict__ word_rank)
 {
     const int b = blockIdx.y;
     const uint32_t *bm = bitmap + (int64_t)b * words;
@@ -118,6 +119,7 @@ compact_kernel(const uint32_t *__restrict__ bitmap, int64_t words, int n_chunks,
 #pragma unroll
     for (int j = 0; j < WORDS_PER_THREAD; ++j) {
         uint32_t bits = w[j];
+        if (w0 + j < words) word_rank[(int64_t)b * words + w0 + j] = (int32_t)pos;
         while (bits) {
             int t = __ffs(bits) - 1;
             bits &= bits - 1;
@@ -128,7 +130,8 @@ compact_kernel(const uint32_t *__restrict__ bitmap, int64_t words, int n_chunks,
 }
 
 int launch_gather(const Index &ix, const Params &p, const Layout &L, const int32_t *probes, uint32_t *bitmap,
-                  int32_t *chunk_cnt, int32_t *cand, int32_t *n_cand, uint32_t *status, cudaStream_t st)
+                  int32_t *chunk_cnt, int32_t *cand, int32_t *n_cand, int32_t *word_rank, uint32_t *status,
+                  cudaStream_t st)
 {
     CHIMERA_CUDA(cudaMemsetAsync(bitmap, 0, sizeof(uint32_t) * (size_t)L.words * p.B, st));
     const int n_lists = p.nq * p.P;
@@ -140,7 +143,7 @@ int launch_gather(const Index &ix, const Params &p, const Layout &L, const int32
     CHIMERA_CUDA(cudaGetLastError());
     chunk_scan_kernel<<<(unsigned)p.B, 32, 0, st>>>(chunk_cnt, L.n_chunks, p.maxc, n_cand, status);
     CHIMERA_CUDA(cudaGetLastError());
-    compact_kernel<<<gc, CHUNK_THREADS, 0, st>>>(bitmap, L.words, L.n_chunks, chunk_cnt, p.maxc, cand);
+    compact_kernel<<<gc, CHUNK_THREADS, 0, st>>>(bitmap, L.words, L.n_chunks, chunk_cnt, p.maxc, cand, word_rank);
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_GATHER, 4);
     return CHIMERA_OK;

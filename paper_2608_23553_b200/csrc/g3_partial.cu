@@ -1,0 +1,132 @@
+// Candidate refinement with partial scores (Sec. 3.2 step 2, Algorithm 2; aggregation as in Algorithm 4): only the
+// tokens retrieved in candidate generation contribute.  For query token i and each of its probed centroids, every
+// token of that centroid's posting list raises M[document, i] to max(M, dist(i, token)); M starts at 0 and the partial
+// score is F'(d) = sum_i M[d, i].
+//
+// dist(i, t) = S[cid_t, i] + llrint(delta*4*T + kappa*4*SQ_i) in Q.24 fixed point, T = sum_x Xq_i[x] u_t[x],
+// SQ_i = sum_x Xq_i[x], Xq = rint(q * 2^22): integers plus one correctly rounded double expression, so the result does
+// not depend on the order in which tokens are visited (integer max) nor on the machine.
+//
+// As in the paper's design a block serves one (query token, posting list) pair: the query token's integers sit in
+// shared memory, one thread scores one document token, and the maximum goes to the score table with atomicMax while the
+// thread moves on to its next token.  The table is indexed by candidate rank (bitmap word prefix + popcount), so it has
+// one 4*q_len-byte row per candidate rather than per document.
+#include "common.cuh"
+
+namespace chimera {
+
+constexpr int PS_THREADS = 128;
+
+// grid (blocks, B): zero the first n_cand[b] rows of M.
+__global__ void __launch_bounds__(256)
+partial_clear_kernel(int32_t *__restrict__ M, const int32_t *__restrict__ n_cand, int64_t maxc, int nq)
+{
+    const int b = blockIdx.y;
+    const int64_t n = (int64_t)n_cand[b] * nq;
+    int32_t *row = M + (int64_t)b * maxc * nq;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
+        row[e] = 0;
+}
+
+// grid (nq * P, B): one block per (query token, probed list).
+template <int NBITS>
+__global__ void __launch_bounds__(PS_THREADS)
+partial_score_kernel(const float *__restrict__ queries, const int32_t *__restrict__ table, int64_t K, int nq, int D,
+                     int CW, int P, float delta, float kappa, const int32_t *__restrict__ probes,
+                     const int64_t *__restrict__ tok_off, const int32_t *__restrict__ tok_id,
+                     const int32_t *__restrict__ tok_doc, const uint32_t *__restrict__ codes,
+                     const uint32_t *__restrict__ bitmap, const int32_t *__restrict__ word_rank, int64_t words,
+                     int64_t maxc, int32_t *__restrict__ M)
+{
+    __shared__ int32_t xq[128];
+    __shared__ long long s_sq;
+    const int b = blockIdx.y;
+    const int i = blockIdx.x / P;
+    const int32_t c = probes[((int64_t)b * nq + i) * P + blockIdx.x % P];
+    const float *q = queries + ((int64_t)b * nq + i) * D;
+    for (int x = threadIdx.x; x < D; x += PS_THREADS) {
+        float v = fminf(fmaxf(q[x], -1.0f), 1.0f);
+        xq[x] = __float2int_rn(v * 4194304.0f);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long s = 0;
+        for (int x = 0; x < D; ++x) s += xq[x];
+        s_sq = s;
+    }
+    __syncthreads();
+    const int32_t s_c = table[((int64_t)b * K + c) * nq + i];
+    const double d4 = __dmul_rn((double)delta, 4.0);
+    const double kterm = __dmul_rn(__dmul_rn((double)kappa, 4.0), (double)s_sq);
+    const uint32_t *bm = bitmap + (int64_t)b * words;
+    const int32_t *wr = word_rank + (int64_t)b * words;
+    int32_t *Mb = M + (int64_t)b * maxc * nq;
+    constexpr int DPW = 32 / NBITS;
+    constexpr uint32_t MASK = (1u << NBITS) - 1u;
+    for (int64_t e = tok_off[c] + threadIdx.x; e < tok_off[c + 1]; e += PS_THREADS) {
+        const int64_t t = tok_id[e];
+        const uint32_t d = (uint32_t)tok_doc[e];
+        const uint32_t *cw = codes + t * CW;
+        int T = 0;                                     // |T| <= 3 * 2^22 * |q|_1 < 2^31 for unit-norm queries
+        for (int w = 0; w < CW; ++w) {
+            const uint32_t word = __ldg(cw + w);
+#pragma unroll
+            for (int s = 0; s < DPW; ++s) T += xq[w * DPW + s] * (int)((word >> (s * NBITS)) & MASK);
+        }
+        const double r = __dadd_rn(__dmul_rn(d4, (double)T), kterm);
+        const long long dist = (long long)s_c + __double2ll_rn(r);
+        if (dist > 0) {                                // the table starts at 0 (Algorithm 2)
+            const int64_t rank = wr[d >> 5] + __popc(bm[d >> 5] & ((1u << (d & 31)) - 1u));
+            if (rank < maxc) atomicMax(&Mb[rank * nq + i], (int32_t)dist);
+        }
+    }
+}
+
+// grid (blocks, B): F'[b][j] = sum_i M[b][j][i], one warp per candidate.
+__global__ void __launch_bounds__(256)
+partial_sum_kernel(const int32_t *__restrict__ M, const int32_t *__restrict__ n_cand, int64_t maxc, int nq,
+                   int32_t *__restrict__ fprime)
+{
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const int n = n_cand[b];
+    const int warps = gridDim.x * (blockDim.x >> 5);
+    for (int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); j < n; j += warps) {
+        const int32_t *row = M + ((int64_t)b * maxc + j) * nq;
+        int s = 0;
+        for (int i = lane; i < nq; i += 32) s += row[i];
+        s = warp_sum(s);
+        if (lane == 0) fprime[(int64_t)b * maxc + j] = s;
+    }
+}
+
+int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, const float *queries,
+                          const int32_t *table, const int32_t *probes, const uint32_t *bitmap,
+                          const int32_t *word_rank, const int32_t *n_cand, int32_t *partial_m, int32_t *fprime,
+                          cudaStream_t st)
+{
+    const float delta = (ix.res_hi - ix.res_lo) / (float)(1 << ix.nbits);
+    const float kappa = ix.res_lo + 0.5f * delta;
+    int64_t per_query = ((int64_t)ix.sm_count * 8 + p.B - 1) / p.B;
+    if (per_query < 1) per_query = 1;
+    dim3 gclr((unsigned)per_query, (unsigned)p.B);
+    partial_clear_kernel<<<gclr, 256, 0, st>>>(partial_m, n_cand, p.maxc, p.nq);
+    CHIMERA_CUDA(cudaGetLastError());
+    dim3 grid((unsigned)(p.nq * p.P), (unsigned)p.B);
+    const uint32_t *codes = reinterpret_cast<const uint32_t *>(ix.codes);
+    if (ix.nbits == 2)
+        partial_score_kernel<2><<<grid, PS_THREADS, 0, st>>>(queries, table, ix.K, p.nq, ix.D, ix.CB / 4, p.P, delta,
+                                                             kappa, probes, ix.tok_off, ix.tok_id, ix.tok_doc, codes,
+                                                             bitmap, word_rank, L.words, p.maxc, partial_m);
+    else
+        partial_score_kernel<1><<<grid, PS_THREADS, 0, st>>>(queries, table, ix.K, p.nq, ix.D, ix.CB / 4, p.P, delta,
+                                                             kappa, probes, ix.tok_off, ix.tok_id, ix.tok_doc, codes,
+                                                             bitmap, word_rank, L.words, p.maxc, partial_m);
+    CHIMERA_CUDA(cudaGetLastError());
+    partial_sum_kernel<<<gclr, 256, 0, st>>>(partial_m, n_cand, p.maxc, p.nq, fprime);
+    CHIMERA_CUDA(cudaGetLastError());
+    count_launch(SLOT_CI, 3);
+    return CHIMERA_OK;
+}
+
+}  // namespace chimera

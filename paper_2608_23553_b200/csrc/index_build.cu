@@ -175,6 +175,75 @@ __global__ void ivf_kernel(const int32_t *__restrict__ cids, const int64_t *__re
     }
 }
 
+// ------------------------------------------------------------------------------------------------ token lists ----
+// Per centroid the ids of its tokens and their documents (the posting lists P_i of Sec. 3.2 step 1 as the paper keeps
+// them: token level).  One warp per document; pass 0 counts, pass 1 writes through an atomic cursor.
+template <int PASS>
+__global__ void token_list_kernel(const int32_t *__restrict__ cids, const int64_t *__restrict__ doc_off, int64_t N,
+                                  int32_t *__restrict__ count, const int64_t *__restrict__ tok_off,
+                                  int32_t *__restrict__ tok_id, int32_t *__restrict__ tok_doc)
+{
+    int lane = threadIdx.x & 31;
+    int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t d = warp; d < N; d += n_warps) {
+        int64_t b = doc_off[d], e = doc_off[d + 1];
+        for (int64_t t = b + lane; t < e; t += 32) {
+            int32_t c = cids[t];
+            int32_t pos = atomicAdd(&count[c], 1);
+            if (PASS == 1) {
+                tok_id[tok_off[c] + pos] = (int32_t)t;
+                tok_doc[tok_off[c] + pos] = (int32_t)d;
+            }
+        }
+    }
+}
+
+int build_token_lists(Index &ix, cudaStream_t st)
+{
+    if (ix.tok_id) return CHIMERA_OK;
+    if (ix.T > 0x7fffffffLL) return fail(CHIMERA_UNSUPPORTED, "token ids must fit int32");
+    int32_t *count = nullptr;
+    int64_t *tmp = nullptr;
+    int64_t *off = nullptr;
+    int32_t *ids = nullptr, *docs = nullptr;
+    auto cleanup = [&](bool all) {
+        cudaFree(count);
+        cudaFree(tmp);
+        if (all) { cudaFree(off); cudaFree(ids); cudaFree(docs); }
+    };
+#define TL_CUDA(call)                                                                        \
+    do {                                                                                     \
+        cudaError_t e__ = (call);                                                            \
+        if (e__ != cudaSuccess) {                                                            \
+            cleanup(true);                                                                   \
+            return fail(CHIMERA_CUDA_ERROR, "%s: %s", #call, cudaGetErrorString(e__));      \
+        }                                                                                    \
+    } while (0)
+    TL_CUDA(cudaMalloc(&count, sizeof(int32_t) * ix.K));
+    TL_CUDA(cudaMalloc(&tmp, sizeof(int64_t) * ((ix.K + SCAN_TILE - 1) / SCAN_TILE + 1)));
+    TL_CUDA(cudaMalloc(&off, sizeof(int64_t) * (ix.K + 1)));
+    TL_CUDA(cudaMalloc(&ids, sizeof(int32_t) * ix.T));
+    TL_CUDA(cudaMalloc(&docs, sizeof(int32_t) * ix.T));
+    TL_CUDA(cudaMemsetAsync(count, 0, sizeof(int32_t) * ix.K, st));
+    int64_t warps_wanted = ix.N < (int64_t)ix.sm_count * 64 ? ix.N : (int64_t)ix.sm_count * 64;
+    unsigned blocks = (unsigned)((warps_wanted * 32 + 255) / 256);
+    token_list_kernel<0><<<blocks, 256, 0, st>>>(ix.cids, ix.doc_off, ix.N, count, nullptr, nullptr, nullptr);
+    TL_CUDA(cudaGetLastError());
+    int rc = exclusive_scan(count, ix.K, off, tmp, st);
+    if (rc) { cleanup(true); return rc; }
+    TL_CUDA(cudaMemsetAsync(count, 0, sizeof(int32_t) * ix.K, st));
+    token_list_kernel<1><<<blocks, 256, 0, st>>>(ix.cids, ix.doc_off, ix.N, count, off, ids, docs);
+    TL_CUDA(cudaGetLastError());
+    TL_CUDA(cudaStreamSynchronize(st));
+#undef TL_CUDA
+    cleanup(false);
+    ix.tok_off = off;
+    ix.tok_id = ids;
+    ix.tok_doc = docs;
+    return CHIMERA_OK;
+}
+
 // ------------------------------------------------------------------------------------------------ driver ---------
 int build_index_device(Index &ix, const float *centroids, const int32_t *doclens, cudaStream_t st)
 {

@@ -1,0 +1,81 @@
+"""GPU parity of the paper's candidate refinement (partial scores F', Algorithm 2) against the oracle: F' of every
+candidate and the pruned ids bit-exact, later stages by the usual rules."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import random_corpus, unit_rows
+from parity import check_query, taps_to_numpy
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(gix, oix, q, nprobe, n_prune, k, sample=None, max_diffs=0):
+    B, nq, _ = q.shape
+    taps = gix.alloc_taps(B, nq, nprobe, n_prune, table=False)
+    ids, sc = gix.search(torch.from_numpy(q).cuda(), nprobe, n_prune, k, taps=taps, partial=True)
+    assert gix.status() == 0
+    tn = taps_to_numpy(taps)
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    for b in (range(B) if sample is None else sample):
+        res = oracle.pipeline(q[b], oix, nprobe, n_prune, k, partial=True)
+        assert check_query(tn, b, res, ids[b], sc[b], k, n_prune, table=False) <= max_diffs
+
+
+@pytest.mark.parametrize("D,nbits,nq,K,N,nprobe,n_prune,k", [
+    (32, 2, 5, 16, 80, 2, 9, 3),
+    (128, 2, 32, 64, 500, 4, 60, 10),
+    (128, 1, 32, 64, 500, 4, 60, 10),
+    (96, 2, 64, 48, 300, 8, 40, 12),
+    (96, 1, 40, 48, 300, 3, 33, 5),
+    (64, 2, 100, 32, 200, 32, 64, 20),       # every list probed: F' is the full low-bit score
+])
+def test_partial_refinement_small_corpora(D, nbits, nq, K, N, nprobe, n_prune, k):
+    import paper_2608_23553_b200 as pkg
+    cent, cids, codes, doclens = random_corpus(300 + D + nq, N, K, D, nbits, len_lo=1, len_hi=60)
+    oix = oracle.make_index(cent, cids, codes, doclens, nbits)
+    dev = torch.device("cuda:0")
+    gix = pkg.Index(torch.from_numpy(cent).to(dev), torch.from_numpy(cids).to(dev), torch.from_numpy(codes).to(dev),
+                    torch.from_numpy(doclens).to(dev), nbits)
+    q = np.stack([unit_rows(np.random.default_rng(b), nq, D) for b in range(3)])
+    with pytest.raises(pkg.ChimeraError):                    # not enabled yet
+        gix.search(torch.from_numpy(q).cuda(), nprobe, n_prune, k, partial=True)
+    gix.enable_partial()
+    _check(gix, oix, q, nprobe, n_prune, k)
+    # the default search is unaffected by the extra lists
+    ids_a, _ = gix.search(torch.from_numpy(q).cuda(), nprobe, n_prune, k)
+    res = oracle.pipeline(q[0], oix, nprobe, n_prune, k)
+    assert np.array_equal(np.sort(ids_a[0].cpu().numpy()), np.sort(res.ids))
+
+
+def test_partial_refinement_tiny_config_and_batch_invariance():
+    import paper_2608_23553_b200 as pkg
+    from synth import CONFIGS, make_corpus, make_queries
+    cfg = CONFIGS["tiny"]
+    corp = make_corpus(cfg)
+    oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    gix = pkg.Index(corp.centroids.cuda(), corp.cids.cuda(), corp.codes.cuda(), corp.doclens.cuda(), cfg.nbits,
+                    cfg.res_lo, cfg.res_hi)
+    gix.enable_partial()
+    q = make_queries(cfg).numpy()
+    _check(gix, oix, q, cfg.nprobe, cfg.n_prune, cfg.k)
+    qd = torch.from_numpy(q).cuda()
+    ids16, sc16 = gix.search(qd, cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
+    ids16, sc16 = ids16.clone(), sc16.clone()
+    for b in (0, 7, 15):
+        i1, s1 = gix.search(qd[b:b + 1].contiguous(), cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
+        assert torch.equal(i1[0], ids16[b]) and torch.equal(s1[0], sc16[b])
+
+
+def test_partial_refinement_mid_batch256_sampled():
+    import paper_2608_23553_b200 as pkg
+    from synth import CONFIGS, make_corpus, make_queries
+    cfg = CONFIGS["mid"]
+    dev = torch.device("cuda:0")
+    corp = make_corpus(cfg, device=dev)
+    q = make_queries(cfg, 256, device=dev).cpu().numpy()
+    gix = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    gix.enable_partial()
+    oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    _check(gix, oix, q, cfg.nprobe, cfg.n_prune, cfg.k, sample=(0, 255), max_diffs=2)
