@@ -220,20 +220,24 @@ def run_sweep(args, cfg, pkg, index, corp, q):
         for n_prune in (256, 1024, 4096, 16384):
             for k in (10, 100, 1000):
                 out = (torch.empty(B, k, dtype=torch.int32, device=dev), torch.empty(B, k, dtype=torch.float32, device=dev))
-                index.search(batches[0], P, n_prune, k, max_candidates=maxc, out=out)
-                torch.cuda.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                for s in range(args.steps):
-                    index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out)
-                e1.record()
-                torch.cuda.synchronize()
-                ms = e0.elapsed_time(e1) / args.steps
-                assert index.status() == 0
-                ids, _ = index.search(qrec, P, n_prune, k, max_candidates=maxc)
-                hits = (ids[:, :, None] == truth_ids[:, None, :k]).any(dim=2).sum(dim=1).float()
-                print(json.dumps({"nprobe": P, "n_prune": n_prune, "k": k, "qps": B / (ms * 1e-3),
-                                  "ms_per_step": ms, "recall": float((hits / k).mean()), "max_candidates": maxc}))
+                point = {"nprobe": P, "n_prune": n_prune, "k": k, "max_candidates": maxc}
+                for mode, partial in (("", False), ("partial_", True)):
+                    index.search(batches[0], P, n_prune, k, max_candidates=maxc, out=out, partial=partial)
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for s in range(args.steps):
+                        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out,
+                                     partial=partial)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ms = e0.elapsed_time(e1) / args.steps
+                    assert index.status() == 0
+                    ids, _ = index.search(qrec, P, n_prune, k, max_candidates=maxc, partial=partial)
+                    hits = (ids[:, :, None] == truth_ids[:, None, :k]).any(dim=2).sum(dim=1).float()
+                    point.update({mode + "qps": B / (ms * 1e-3), mode + "ms_per_step": ms,
+                                  mode + "recall": float((hits / k).mean())})
+                print(json.dumps(point))
 
 
 def main():
@@ -244,6 +248,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="mid")
     ap.add_argument("--batch", type=int, default=0, help="queries per call (default 256; 64 for the long-document configs)")
+    ap.add_argument("--partial", action="store_true",
+                    help="prune with the paper's partial scores (chimera_search_partial) instead of stage 3")
     ap.add_argument("--sweep", action="store_true", help="QPS vs recall over nprobe x n_prune x k (see run_sweep)")
     ap.add_argument("--sweep-queries", type=int, default=200)
     ap.add_argument("--batch1-queries", type=int, default=200)
@@ -282,6 +288,8 @@ def main():
     index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
     build_s = time.time() - t0
     B, nq, P, n_prune, k = args.batch, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
+    if args.partial or args.sweep:
+        index.enable_partial()
     if args.sweep:
         if rank == 0:
             run_sweep(args, cfg, pkg, index, corp, q)
@@ -301,7 +309,7 @@ def main():
     work = []
     for bi in range(n_batches):
         taps = index.alloc_taps(B, nq, P, n_prune, max_candidates=maxc, table=False, ci=False)
-        index.search(batches[bi], P, n_prune, k, max_candidates=maxc, taps=taps)
+        index.search(batches[bi], P, n_prune, k, max_candidates=maxc, taps=taps, partial=args.partial)
         assert index.status() == 0
         mask = torch.arange(taps.cand.shape[1], device=device)[None, :] < taps.n_cand[:, None].to(torch.int64)
         toks = (doclens64[taps.cand.to(torch.int64).clamp_(0, index.N - 1)] * mask).sum()
@@ -314,7 +322,7 @@ def main():
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps ------------------------------------
     for s in range(args.warmup):
-        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out)
+        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out, partial=args.partial)
     barrier()
     pkg.profile_enable(True)
     pkg.profile_read()
@@ -323,7 +331,8 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for s in range(args.steps):
-        index.search(batches[(args.warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc, out=out)
+        index.search(batches[(args.warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc, out=out,
+                     partial=args.partial)
     e1.record()
     barrier()
     clocks = sampler.stop()
@@ -338,13 +347,24 @@ def main():
     qps = world * B * args.steps / (ms_total / 1e3)
 
     # ---- end to end through the host entry point: pinned host queries in, host ids/scores out -------------------
+    dq = torch.empty_like(batches[0])
+
+    def host_search(hq, hout, dbuf, dout):
+        if not args.partial:
+            index.search_host(hq, P, n_prune, k, max_candidates=maxc, out=hout)
+        else:       # the host entry point has no partial variant: pinned copies around chimera_search_partial
+            dbuf.copy_(hq, non_blocking=True)
+            index.search(dbuf, P, n_prune, k, max_candidates=maxc, out=dout, partial=True)
+            hout[0].copy_(dout[0], non_blocking=True)
+            hout[1].copy_(dout[1], non_blocking=True)
+            torch.cuda.synchronize()
+
     for s in range(2):
-        index.search_host(host_batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=host_out)
+        host_search(host_batches[s % n_batches], host_out, dq, out)
     barrier()
     w0 = time.perf_counter()
     for s in range(args.steps):
-        index.search_host(host_batches[(args.warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc,
-                          out=host_out)
+        host_search(host_batches[(args.warmup + s) % n_batches], host_out, dq, out)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - w0
     t = torch.tensor([e2e_s], device=device)
@@ -358,14 +378,14 @@ def main():
     n1 = min(args.batch1_queries, q.shape[0])
     out1 = (torch.empty(1, k, dtype=torch.int32, device=device), torch.empty(1, k, dtype=torch.float32, device=device))
     for i in range(5):
-        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1)
+        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, partial=args.partial)
     torch.cuda.synchronize()
     lat = []
     pkg.profile_enable(True)
     pkg.profile_read()
     for i in range(n1):
         a = time.perf_counter()
-        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1)
+        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, partial=args.partial)
         torch.cuda.synchronize()
         lat.append(time.perf_counter() - a)
     stage_ms1, _ = pkg.profile_read()
@@ -374,8 +394,9 @@ def main():
     host_q1 = q[:n1].cpu().pin_memory()
     hout1 = (torch.empty(1, k, dtype=torch.int32).pin_memory(), torch.empty(1, k, dtype=torch.float32).pin_memory())
     w0 = time.perf_counter()
+    dq1 = torch.empty_like(q[:1])
     for i in range(n1):
-        index.search_host(host_q1[i:i + 1], P, n_prune, k, max_candidates=maxc, out=hout1)
+        host_search(host_q1[i:i + 1], hout1, dq1, out1)
     e2e1_qps = n1 / (time.perf_counter() - w0)
 
     if rank != 0:
@@ -418,13 +439,16 @@ def main():
     }
 
     result = {
-        "metric": metric_name(cfg, B), "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": metric_name(cfg, B) + (" with partial-score refinement" if args.partial else ""), "value": qps,
+        "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32 fixed point (stages 1-3) + f32 (stage 4)", "data": "synthetic",
         "config": {"workload": cfg.name, "batch": B, "n_docs": cfg.n_docs, "n_tokens": corp.n_tokens,
                    "n_centroids": cfg.n_centroids, "dim": cfg.dim, "nbits": cfg.nbits, "q_len": nq, "nprobe": P,
                    "n_prune": n_prune, "k": k, "parallelism": "replicas only" if world > 1 else "single GPU",
                    "max_candidates": maxc if maxc else cfg.n_docs,
+                   "pruning": "partial scores of retrieved tokens (Algorithm 2)" if args.partial
+                   else "centroid interaction over every candidate token",
                    "l2": "inputs larger than L2 (index %.1f GB, score table %.1f GB per batch); no flush"
                          % ((corp.cids.numel() * 4 + corp.codes.numel()) / 1e9, B * cfg.n_centroids * nq * 4 / 1e9),
                    "gen_s": round(gen_s, 1), "index_build_s": round(build_s, 2)},
