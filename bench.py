@@ -123,6 +123,18 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def whole_job_qps(local_ms: float, queries_per_rank: int, dist=None, device="cpu"):
+    """(QPS over all ranks, slowest rank's milliseconds): every rank ran `queries_per_rank` queries on its own replica;
+    the job takes as long as its slowest rank."""
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    world = 1
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        world = dist.get_world_size()
+    ms = float(t.item())
+    return world * queries_per_rank / (ms / 1e3), ms
+
+
 def build_workload(cfg, device):
     t0 = time.time()
     corp = make_corpus(cfg, device=device)
@@ -339,12 +351,8 @@ def main():
     ms_total = e0.elapsed_time(e1)
     stage_ms, launches = pkg.profile_read()
     pkg.profile_enable(False)
-    t = torch.tensor([ms_total], device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    qps, ms_total = whole_job_qps(ms_total, B * args.steps, dist, device)
     ms_per_step = ms_total / args.steps
-    qps = world * B * args.steps / (ms_total / 1e3)
 
     # ---- end to end through the host entry point: pinned host queries in, host ids/scores out -------------------
     dq = torch.empty_like(batches[0])
@@ -367,10 +375,7 @@ def main():
         host_search(host_batches[(args.warmup + s) % n_batches], host_out, dq, out)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - w0
-    t = torch.tensor([e2e_s], device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_qps = world * B * args.steps / float(t.item())
+    e2e_qps, _ = whole_job_qps(e2e_s * 1e3, B * args.steps, dist, device)
     h2d = B * nq * cfg.dim * 4
     d2h = B * k * 8
 
