@@ -30,11 +30,13 @@ constexpr uint32_t G1_A_PLANE = G1_M * G1_ROW_BYTES;      // 16 KB
 constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;      // 6 KB
 constexpr uint32_t G1_SMEM = 3 * G1_A_PLANE + 2 * 3 * G1_B_PLANE + 1024 /* alignment slack */ + 64 /* barriers */;
 
+// floor((a0 + 2^8 a1 + 2^16 a2 + 2^24 a3 + 2^32 a4 + 2^19) / 2^20).  The two high terms are multiples of 2^20, so they
+// contribute 2^4 a3 + 2^12 a4 exactly (32-bit wrap-around is harmless: the result fits int32); only the low three need
+// 64 bits.
 __device__ __forceinline__ int32_t combine_digits(int32_t a0, int32_t a1, int32_t a2, int32_t a3, int32_t a4)
 {
-    long long T = (long long)a0 + (long long)a1 * 256LL + (long long)a2 * 65536LL + (long long)a3 * 16777216LL +
-                  (long long)a4 * 4294967296LL;
-    return (int32_t)((T + (1LL << 19)) >> 20);
+    const long long low = (long long)a0 + (long long)a1 * 256LL + (long long)a2 * 65536LL + (1LL << 19);
+    return (int32_t)(low >> 20) + a3 * 16 + a4 * 4096;
 }
 
 // grid (ceil(K / 128), n_splits).  Each CTA: centroid tile blockIdx.x, query-row tiles [blockIdx.y * tiles_per_split, ...).
@@ -141,8 +143,12 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
             int32_t out[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) out[e] = combine_digits(acc[0][e], acc[1][e], acc[2][e], acc[3][e], acc[4][e]);
-            const int64_t r0 = (int64_t)t * G1_N + chunk * 16;       // first query-token row of this chunk
-            if (table8 != nullptr && c < K && r0 < q_rows) {
+            // first query-token row of this chunk, and its (query, token) coordinates: one 32-bit division per chunk,
+            // then incremental (rows fit 32 bits: n_queries * q_len < 2^23)
+            const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)chunk * 16;
+            const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
+            uint32_t qb = r0 / unq, qi = r0 - qb * unq;
+            if (table8 != nullptr && c < K && r0 < rows32) {
                 // coarse copy for the bound phase of stage 3: min((S + 2^24 + 64) >> 17, 255); q_len is a multiple of
                 // 16 here, so the 16 rows of a chunk belong to one query and the store is 16-byte aligned
                 uint32_t w[4];
@@ -157,28 +163,23 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                     }
                     w[g] = pack;
                 }
-                const int64_t b = r0 / nq, i = r0 % nq;
-                *reinterpret_cast<uint4 *>(table8 + (b * K + c) * nq + i) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(table8 + ((int64_t)qb * K + c) * nq + qi) = make_uint4(w[0], w[1], w[2], w[3]);
             }
             if (c < K) {
                 if ((nq & 3) == 0) {
 #pragma unroll
                     for (int e = 0; e < 16; e += 4) {
-                        const int64_t r = r0 + e;
-                        if (r < q_rows) {                             // q_rows is a multiple of 4 here
-                            const int64_t b = r / nq, i = r % nq;
-                            *reinterpret_cast<int4 *>(table + (b * K + c) * nq + i) =
+                        if (r0 + e < rows32)                          // q_rows is a multiple of 4 here
+                            *reinterpret_cast<int4 *>(table + ((int64_t)qb * K + c) * nq + qi) =
                                 make_int4(out[e], out[e + 1], out[e + 2], out[e + 3]);
-                        }
+                        qi += 4;
+                        if (qi >= unq) { qi -= unq; ++qb; }           // groups of four never straddle two queries
                     }
                 } else {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
-                        const int64_t r = r0 + e;
-                        if (r < q_rows) {
-                            const int64_t b = r / nq, i = r % nq;
-                            table[(b * K + c) * nq + i] = out[e];
-                        }
+                        if (r0 + e < rows32) table[((int64_t)qb * K + c) * nq + qi] = out[e];
+                        if (++qi == unq) { qi = 0; ++qb; }
                     }
                 }
             }
