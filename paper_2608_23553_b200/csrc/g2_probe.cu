@@ -80,12 +80,26 @@ probe_final(const unsigned long long *__restrict__ part, int nq, int P, int n_pa
     unsigned long long *mine = lists + threadIdx.x;
     for (int j = 0; j < P; ++j) mine[j * PROBE_THREADS] = 0ull;
     if (col < nq) {
-        for (int l = warp; l < n_part; l += PROBE_WARPS) {
-            const unsigned long long *src = part + (((int64_t)b * n_part + l) * P) * nq + col;
-            for (int j = 0; j < P; ++j) {
-                unsigned long long key = src[(int64_t)j * nq];
-                if (key <= mine[(P - 1) * PROBE_THREADS]) break;      // source list is descending
-                list_insert(mine, P, key);
+        // the heads of four lists are loaded together (independent loads); a list is only walked further while its
+        // keys still beat this thread's current P-th best
+        for (int l0 = warp; l0 < n_part; l0 += 4 * PROBE_WARPS) {
+            unsigned long long head[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int l = l0 + u * PROBE_WARPS;
+                head[u] = l < n_part ? part[(((int64_t)b * n_part + l) * P) * nq + col] : 0ull;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int l = l0 + u * PROBE_WARPS;
+                if (l >= n_part || head[u] <= mine[(P - 1) * PROBE_THREADS]) continue;
+                list_insert(mine, P, head[u]);
+                const unsigned long long *src = part + (((int64_t)b * n_part + l) * P) * nq + col;
+                for (int j = 1; j < P; ++j) {
+                    unsigned long long key = src[(int64_t)j * nq];
+                    if (key <= mine[(P - 1) * PROBE_THREADS]) break;      // source list is descending
+                    list_insert(mine, P, key);
+                }
             }
         }
     }
