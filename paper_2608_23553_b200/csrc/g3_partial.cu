@@ -9,7 +9,8 @@
 //
 // As in the paper's design a block serves one (query token, posting list) pair: the query token's integers sit in
 // shared memory, one thread scores one document token, and the maximum goes to the score table with atomicMax while the
-// thread moves on to its next token.  The table is indexed by candidate rank (bitmap word prefix + popcount), so it has
+// thread moves on to its next token; every increase of a table entry is also added to the document's partial score, so
+// no separate summation pass is needed.  The table is indexed by candidate rank (bitmap word prefix + popcount), so it has
 // one 4*q_len-byte row per candidate rather than per document.
 #include "common.cuh"
 
@@ -17,15 +18,22 @@ namespace chimera {
 
 constexpr int PS_THREADS = 128;
 
-// grid (blocks, B): zero the first n_cand[b] rows of M.
+// grid (blocks, B): zero the first n_cand[b] rows of M and the first n_cand[b] partial scores.
 __global__ void __launch_bounds__(256)
-partial_clear_kernel(int32_t *__restrict__ M, const int32_t *__restrict__ n_cand, int64_t maxc, int nq)
+partial_clear_kernel(int32_t *__restrict__ M, int32_t *__restrict__ fprime, const int32_t *__restrict__ n_cand,
+                     int64_t maxc, int nq)
 {
     const int b = blockIdx.y;
     const int64_t n = (int64_t)n_cand[b] * nq;
-    int32_t *row = M + (int64_t)b * maxc * nq;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
-        row[e] = 0;
+    int4 *row = reinterpret_cast<int4 *>(M + (int64_t)b * maxc * nq);      // rows are 16-byte aligned when nq % 4 == 0
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (int64_t)gridDim.x * blockDim.x;
+    if ((nq & 3) == 0 && (maxc * nq) % 4 == 0) {
+        for (int64_t e = tid; e < n / 4; e += stride) row[e] = make_int4(0, 0, 0, 0);
+    } else {
+        int32_t *r1 = M + (int64_t)b * maxc * nq;
+        for (int64_t e = tid; e < n; e += stride) r1[e] = 0;
+    }
+    for (int64_t e = tid; e < n_cand[b]; e += stride) fprime[(int64_t)b * maxc + e] = 0;
 }
 
 // grid (nq * P, B): one block per (query token, probed list).
@@ -36,7 +44,7 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
                      const int64_t *__restrict__ tok_off, const int32_t *__restrict__ tok_id,
                      const int32_t *__restrict__ tok_doc, const uint32_t *__restrict__ codes,
                      const uint32_t *__restrict__ bitmap, const int32_t *__restrict__ word_rank, int64_t words,
-                     int64_t maxc, int32_t *__restrict__ M)
+                     int64_t maxc, int32_t *__restrict__ M, int32_t *__restrict__ fprime)
 {
     __shared__ int32_t xq[128];
     __shared__ long long s_sq;
@@ -77,26 +85,12 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
         const long long dist = (long long)s_c + __double2ll_rn(r);
         if (dist > 0) {                                // the table starts at 0 (Algorithm 2)
             const int64_t rank = wr[d >> 5] + __popc(bm[d >> 5] & ((1u << (d & 31)) - 1u));
-            if (rank < maxc) atomicMax(&Mb[rank * nq + i], (int32_t)dist);
+            if (rank < maxc) {
+                // F' = sum_i M[., i] is kept up to date with the increments: M only grows, integer adds commute
+                const int32_t old = atomicMax(&Mb[rank * nq + i], (int32_t)dist);
+                if ((int32_t)dist > old) atomicAdd(&fprime[(int64_t)b * maxc + rank], (int32_t)dist - old);
+            }
         }
-    }
-}
-
-// grid (blocks, B): F'[b][j] = sum_i M[b][j][i], one warp per candidate.
-__global__ void __launch_bounds__(256)
-partial_sum_kernel(const int32_t *__restrict__ M, const int32_t *__restrict__ n_cand, int64_t maxc, int nq,
-                   int32_t *__restrict__ fprime)
-{
-    const int b = blockIdx.y;
-    const int lane = threadIdx.x & 31;
-    const int n = n_cand[b];
-    const int warps = gridDim.x * (blockDim.x >> 5);
-    for (int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); j < n; j += warps) {
-        const int32_t *row = M + ((int64_t)b * maxc + j) * nq;
-        int s = 0;
-        for (int i = lane; i < nq; i += 32) s += row[i];
-        s = warp_sum(s);
-        if (lane == 0) fprime[(int64_t)b * maxc + j] = s;
     }
 }
 
@@ -110,22 +104,20 @@ int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, con
     int64_t per_query = ((int64_t)ix.sm_count * 8 + p.B - 1) / p.B;
     if (per_query < 1) per_query = 1;
     dim3 gclr((unsigned)per_query, (unsigned)p.B);
-    partial_clear_kernel<<<gclr, 256, 0, st>>>(partial_m, n_cand, p.maxc, p.nq);
+    partial_clear_kernel<<<gclr, 256, 0, st>>>(partial_m, fprime, n_cand, p.maxc, p.nq);
     CHIMERA_CUDA(cudaGetLastError());
     dim3 grid((unsigned)(p.nq * p.P), (unsigned)p.B);
     const uint32_t *codes = reinterpret_cast<const uint32_t *>(ix.codes);
     if (ix.nbits == 2)
         partial_score_kernel<2><<<grid, PS_THREADS, 0, st>>>(queries, table, ix.K, p.nq, ix.D, ix.CB / 4, p.P, delta,
                                                              kappa, probes, ix.tok_off, ix.tok_id, ix.tok_doc, codes,
-                                                             bitmap, word_rank, L.words, p.maxc, partial_m);
+                                                             bitmap, word_rank, L.words, p.maxc, partial_m, fprime);
     else
         partial_score_kernel<1><<<grid, PS_THREADS, 0, st>>>(queries, table, ix.K, p.nq, ix.D, ix.CB / 4, p.P, delta,
                                                              kappa, probes, ix.tok_off, ix.tok_id, ix.tok_doc, codes,
-                                                             bitmap, word_rank, L.words, p.maxc, partial_m);
+                                                             bitmap, word_rank, L.words, p.maxc, partial_m, fprime);
     CHIMERA_CUDA(cudaGetLastError());
-    partial_sum_kernel<<<gclr, 256, 0, st>>>(partial_m, n_cand, p.maxc, p.nq, fprime);
-    CHIMERA_CUDA(cudaGetLastError());
-    count_launch(SLOT_CI, 3);
+    count_launch(SLOT_CI, 2);
     return CHIMERA_OK;
 }
 
