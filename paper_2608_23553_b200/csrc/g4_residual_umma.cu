@@ -149,9 +149,25 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             const long long t = s_t0[dl] + (s - s_off[dl]);
             cid = cids[t];
             const uint32_t *src = codes + t * CW;
+            if ((CW & 3) == 0) {                          // 16-byte aligned codes: two wide loads for 32 bytes
 #pragma unroll
-            for (int w = 0; w < MAXCW; ++w)
-                if (w < CW) cw[w] = __ldg(src + w);
+                for (int w = 0; w < MAXCW; w += 4)
+                    if (w < CW) {
+                        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src + w));
+                        cw[w] = v.x; cw[w + 1] = v.y; cw[w + 2] = v.z; cw[w + 3] = v.w;
+                    }
+            } else if ((CW & 1) == 0) {
+#pragma unroll
+                for (int w = 0; w < MAXCW; w += 2)
+                    if (w < CW) {
+                        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src + w));
+                        cw[w] = v.x; cw[w + 1] = v.y;
+                    }
+            } else {
+#pragma unroll
+                for (int w = 0; w < MAXCW; ++w)
+                    if (w < CW) cw[w] = __ldg(src + w);
+            }
         }
     };
 

@@ -9,6 +9,7 @@
 namespace chimera {
 
 constexpr long long UMMA_WAIT_CYCLES = 2000000000LL;       // ~1 s at 2 GHz: every mbarrier wait gives up after this
+constexpr uint32_t UMMA_SUSPEND_HINT_NS = 20000u;          // one try_wait may sleep this long before re-checking
 
 // ------------------------------------------------------------------------------------------------ PTX wrappers ---
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -21,7 +22,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase with the given parity to complete.  false = gave up.
+// Bounded wait for the phase with the given parity to complete.  false = gave up.  Each try_wait may suspend the
+// thread in hardware for up to the hinted time (it returns early when the phase completes), so a waiting warp does not
+// burn issue slots; the loop around it enforces the overall limit.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
     const long long t0 = clock64();
@@ -29,10 +32,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.b32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(UMMA_SUSPEND_HINT_NS)
             : "memory");
         if (done) return true;
         if (clock64() - t0 > UMMA_WAIT_CYCLES) return false;
