@@ -145,6 +145,65 @@ def partial_scores(S: np.ndarray, q, pr: np.ndarray, cand: np.ndarray, ix: Index
     return out
 
 
+@dataclass
+class RabitqCodes:
+    """RaBitQ 1-bit codes of the corpus tokens (Sec. 2.2), as the oracle reads them."""
+    rotation: np.ndarray   # [D, D] float32
+    bits: np.ndarray       # [T, D/8] uint8
+    inv_dot: np.ndarray    # [T] float32
+
+
+def make_rabitq(rotation, bits, inv_dot) -> RabitqCodes:
+    return RabitqCodes(_arr(rotation, np.float32), _arr(bits, np.uint8), _arr(inv_dot, np.float32))
+
+
+def rotate(rotation, q) -> np.ndarray:
+    """O-9: q_p = P q per row, as a sequential fp32 fma chain."""
+    P = _arr(rotation, np.float32)
+    q = _arr(q, np.float32)
+    out = np.empty_like(q)
+    lib().oracle_rotate(_p(P), _p(q), ctypes.c_int64(q.shape[0]), ctypes.c_int32(q.shape[1]), _p(out))
+    return out
+
+
+def rabitq_score_docs(qp, docs, ix: Index, rq: RabitqCodes) -> np.ndarray:
+    """O-9: complete 1-bit Chamfer score of each listed document (qp = rotated query)."""
+    qp = _arr(qp, np.float32)
+    docs = _arr(docs, np.int32)
+    out = np.empty(docs.shape[0], dtype=np.float32)
+    lib().oracle_rabitq_score_docs(_p(qp), ctypes.c_int32(qp.shape[0]), ctypes.c_int32(ix.dim), _p(rq.bits),
+                                   _p(rq.inv_dot), _p(ix.doc_off), _p(docs), ctypes.c_int64(docs.shape[0]), _p(out))
+    return out
+
+
+def rabitq_partial(qp, pr, cand, ix: Index, rq: RabitqCodes) -> np.ndarray:
+    """O-9: float32 partial score F' (Algorithm 2 with the 1-bit estimate) of every candidate."""
+    qp = _arr(qp, np.float32)
+    pr = _arr(pr, np.int32)
+    cand = _arr(cand, np.int32)
+    out = np.empty(cand.shape[0], dtype=np.float32)
+    lib().oracle_rabitq_partial(_p(qp), ctypes.c_int32(qp.shape[0]), ctypes.c_int32(ix.dim), _p(rq.bits),
+                                _p(rq.inv_dot), _p(pr), ctypes.c_int32(pr.shape[1]), _p(ix.cids), _p(ix.doclens),
+                                ctypes.c_int64(ix.N), ctypes.c_int64(ix.K), _p(cand), ctypes.c_int64(cand.shape[0]),
+                                _p(out))
+    return out
+
+
+def pipeline_rabitq(q, ix: Index, rq: RabitqCodes, nprobe: int, k_refine: int, k: int) -> "Result":
+    """The paper's GPU pipeline on 1-bit codes (Algorithm 1 without its CPU half): centroid probes and candidates as
+    usual, candidate refinement by partial 1-bit scores, complete 1-bit scores of the survivors, top-k.  `ci` holds
+    F' (float32); ordering floats >= 0 equals ordering their bit patterns, so O-4b selects on the int32 view."""
+    S = score_table(q, ix.centroids)
+    pr = probes(S, nprobe)
+    cand = candidates(pr, ix)
+    qp = rotate(rq.rotation, q)
+    fp = rabitq_partial(qp, pr, cand, ix, rq)
+    pruned = prune(cand, fp.view(np.int32), k_refine)
+    s4 = rabitq_score_docs(qp, pruned, ix, rq)
+    ids, sc = topk(pruned, s4, k)
+    return Result(S, pr, cand, fp, pruned, s4, ids, sc)
+
+
 def score_docs(q, docs: np.ndarray, ix: Index) -> np.ndarray:
     """O-5: float32 Chamfer score of each listed document on its decoded tokens."""
     q = _arr(q, np.float32)

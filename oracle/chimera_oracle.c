@@ -18,6 +18,8 @@
  *   O-6 oracle_topk          top-k by score                                (Def. 2, Eq. 1)
  *   O-7 oracle_chamfer       Def. 1 on raw vectors;  oracle_recall  Def. 3
  *   O-8 oracle_partial_scores  candidate refinement with partial scores F'(Q,V)  (Sec. 3.2 step 2, Algorithm 2)
+ *   O-9 oracle_rotate, oracle_rabitq_score_docs, oracle_rabitq_partial   the same two steps on RaBitQ 1-bit codes
+ *       (Sec. 2.2: rotation, 1-bit code, estimator <q_p, o_p-bar> / <o_p, o_p-bar>, code form of <q_p, o_p-bar>)
  *
  * Pins: every function above is pinned by tests that do not call it to produce their expectation
  * (closed forms, library routines on special cases, set identities, hand-worked values).  Unpinned:
@@ -199,6 +201,104 @@ void oracle_partial_scores(const int32_t *S, const float *q, int32_t nq, int32_t
         int64_t sum = 0;
         for (int i = 0; i < nq; ++i) sum += score[j * nq + i];
         fprime[j] = (int32_t)sum;
+    }
+    free(slot);
+    free(score);
+    free(xq);
+    free(probed);
+}
+
+/* ---------------------------------------------------------------- O-9 ------------------------------------------ */
+/* Sec. 2.2: vectors are rotated by a random orthonormal matrix P before quantisation; inner products are preserved.
+ * q_p = P q, evaluated as one fp32 fused-multiply-add chain per output in increasing x, so that every implementation
+ * that follows this order gets the same bits.  P is [D][D] row-major, q is [n][D]. */
+void oracle_rotate(const float *P, const float *q, int64_t n, int32_t D, float *out)
+{
+    for (int64_t i = 0; i < n; ++i)
+        for (int r = 0; r < D; ++r) {
+            float acc = 0.0f;
+            for (int x = 0; x < D; ++x) acc = fmaf(P[(int64_t)r * D + x], q[i * D + x], acc);
+            out[i * D + r] = acc;
+        }
+}
+
+/* Estimator of Sec. 2.2 with B = 1:  <q, o> ~ <q_p, o_p-bar> / <o_p, o_p-bar>, and by the code equation
+ * <q_p, o_p-bar> = (1 / |y-bar|) (<q_p, o_b> - 1/2 sum q_p), |y-bar| = sqrt(D) / 2, o_b the 0/1 code.
+ * With Xq = rint(q_p * 2^22):  T = sum_x Xq[x] o_b[x],  A = 2 T - sum_x Xq[x]  (integers),
+ * est = inv_dot * (c * (float)A),  c = (float)(1 / (sqrt(D) * 2^22)),  two fp32 multiplications in that order.
+ * bits: bit t of byte g holds dimension 8g+t. */
+static float rabitq_est(const int64_t *xq, int64_t sq, const uint8_t *bits, int64_t t, int32_t D, float inv_dot)
+{
+    const int64_t cb = D / 8;
+    int64_t T = 0;
+    for (int x = 0; x < D; ++x)
+        if ((bits[t * cb + x / 8] >> (x % 8)) & 1) T += xq[x];
+    const float c = (float)(1.0 / (sqrt((double)D) * Q22));
+    const float a = (float)(2 * T - sq);
+    const float ca = c * a;
+    return inv_dot * ca;
+}
+
+/* Document scoring on the 1-bit codes (Sec. 3.2 step 3, GPU half): the complete 1-bit Chamfer score
+ * sum_i max_{t in d} est(i, t), query tokens summed in increasing i in fp32.  qp: rotated query [nq][D]. */
+void oracle_rabitq_score_docs(const float *qp, int32_t nq, int32_t D, const uint8_t *bits, const float *inv_dot,
+                              const int64_t *doc_off, const int32_t *docs, int64_t n_listed, float *scores)
+{
+    int64_t *xq = (int64_t *)malloc(sizeof(int64_t) * (size_t)nq * D);
+    int64_t *sq = (int64_t *)calloc((size_t)nq, sizeof(int64_t));
+    for (int i = 0; i < nq; ++i)
+        for (int x = 0; x < D; ++x) {
+            xq[(int64_t)i * D + x] = (int64_t)rint((double)qp[(int64_t)i * D + x] * Q22);
+            sq[i] += xq[(int64_t)i * D + x];
+        }
+    for (int64_t j = 0; j < n_listed; ++j) {
+        const int64_t d = docs[j];
+        if (d < 0) { scores[j] = -INFINITY; continue; }
+        float total = 0.0f;
+        for (int i = 0; i < nq; ++i) {
+            float best = -INFINITY;
+            for (int64_t t = doc_off[d]; t < doc_off[d + 1]; ++t) {
+                float e = rabitq_est(xq + (int64_t)i * D, sq[i], bits, t, D, inv_dot[t]);
+                if (e > best) best = e;
+            }
+            total = total + best;
+        }
+        scores[j] = total;
+    }
+    free(xq);
+    free(sq);
+}
+
+/* Candidate refinement (Algorithm 2) with the 1-bit estimate as the distance: doc.score[i] starts at 0 and is raised
+ * by every retrieved token; F' = sum_i doc.score[i] in increasing i in fp32.  fprime[j] belongs to cand[j]. */
+void oracle_rabitq_partial(const float *qp, int32_t nq, int32_t D, const uint8_t *bits, const float *inv_dot,
+                           const int32_t *probes, int32_t nprobe, const int32_t *cids, const int32_t *doclens,
+                           int64_t N, int64_t K, const int32_t *cand, int64_t n_cand, float *fprime)
+{
+    int64_t *slot = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    for (int64_t d = 0; d < N; ++d) slot[d] = -1;
+    for (int64_t j = 0; j < n_cand; ++j) slot[cand[j]] = j;
+    float *score = (float *)calloc((size_t)(n_cand > 0 ? n_cand : 1) * nq, sizeof(float));   /* init 0 */
+    int64_t *xq = (int64_t *)malloc(sizeof(int64_t) * (size_t)D);
+    uint8_t *probed = (uint8_t *)malloc((size_t)K);
+    for (int i = 0; i < nq; ++i) {
+        int64_t sq = 0;
+        for (int x = 0; x < D; ++x) { xq[x] = (int64_t)rint((double)qp[(int64_t)i * D + x] * Q22); sq += xq[x]; }
+        memset(probed, 0, (size_t)K);
+        for (int p = 0; p < nprobe; ++p) probed[probes[i * nprobe + p]] = 1;
+        int64_t t = 0;
+        for (int64_t d = 0; d < N; ++d)
+            for (int j = 0; j < doclens[d]; ++j, ++t) {
+                if (!probed[cids[t]]) continue;
+                float e = rabitq_est(xq, sq, bits, t, D, inv_dot[t]);
+                float *cell = &score[slot[d] * nq + i];
+                if (e > *cell) *cell = e;
+            }
+    }
+    for (int64_t j = 0; j < n_cand; ++j) {
+        float sum = 0.0f;
+        for (int i = 0; i < nq; ++i) sum = sum + score[j * nq + i];
+        fprime[j] = sum;
     }
     free(slot);
     free(score);

@@ -5,4 +5,5 @@ library consume.  It holds none of the retrieval method's arithmetic: no
 scoring, no selection, no decoding.  It imports neither `oracle` nor the
 CUDA package.
 """
-from .corpus import CONFIGS, CorpusConfig, Corpus, make_corpus, make_queries, doc_lengths  # noqa: F401
+from .corpus import (CONFIGS, CorpusConfig, Corpus, make_corpus, make_queries, doc_lengths,  # noqa: F401
+                     random_rotation, encode_rabitq_1bit)

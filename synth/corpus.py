@@ -30,7 +30,7 @@ import torch
 _CHUNK_TOKENS = 1 << 20
 
 # RNG stream tags
-_S_MEANS, _S_LENS, _S_COMP, _S_NOISE, _S_QCOMP, _S_QNOISE = range(6)
+_S_MEANS, _S_LENS, _S_COMP, _S_NOISE, _S_QCOMP, _S_QNOISE, _S_ROT = range(7)
 
 
 @dataclass(frozen=True)
@@ -86,6 +86,10 @@ class Corpus:
     codes: torch.Tensor          # [T, D*nbits/8] uint8, document-major
     doclens: torch.Tensor        # [N] int32
     raw: Optional[torch.Tensor] = None   # [T, D] float32 uncompressed tokens (small corpora only)
+    # RaBitQ 1-bit codes of the (unit-norm) tokens, when requested
+    rotation: Optional[torch.Tensor] = None   # [D, D] float32 random orthonormal matrix P
+    rq_bits: Optional[torch.Tensor] = None    # [T, D/8] uint8: bit t of byte g = (P o)[8g+t] > 0
+    rq_inv_dot: Optional[torch.Tensor] = None  # [T] float32: 1 / <o_p, o_p-bar> = sqrt(D) / sum_x |(P o)[x]|
 
     @property
     def n_tokens(self) -> int:
@@ -162,8 +166,31 @@ def encode_residual(r: torch.Tensor, nbits: int, lo: float, hi: float) -> torch.
     return (u << shifts).sum(dim=2).to(torch.uint8)
 
 
-def make_corpus(cfg: CorpusConfig, device="cpu", out_device=None, keep_raw: bool = False) -> Corpus:
-    """Generate the index arrays of `cfg` on `device`; results are moved to `out_device` (default: `device`)."""
+def random_rotation(cfg: CorpusConfig) -> torch.Tensor:
+    """[D, D] float32 random orthonormal matrix (QR of a Gaussian matrix, on the CPU in float64)."""
+    g = _gen(cfg.seed, _S_ROT, 0, "cpu")
+    a = torch.randn(cfg.dim, cfg.dim, generator=g, dtype=torch.float64)
+    qmat, r = torch.linalg.qr(a)
+    qmat = qmat * torch.sign(torch.diagonal(r))[None, :]
+    return qmat.to(torch.float32).contiguous()
+
+
+def encode_rabitq_1bit(x: torch.Tensor, rotation: torch.Tensor):
+    """RaBitQ with B = 1 on unit-norm rows x: rotate, keep the signs, and store 1 / <o_p, o_p-bar> where o_p-bar is
+    the nearest codeword (sign(o_p) / sqrt(D)).  Returns (bits [n, D/8] uint8, inv_dot [n] float32)."""
+    op = x @ rotation.t()
+    bits = (op > 0).to(torch.int32)
+    n, d = bits.shape
+    shifts = torch.arange(8, device=x.device, dtype=torch.int32).view(1, 1, 8)
+    packed = (bits.view(n, d // 8, 8) << shifts).sum(dim=2).to(torch.uint8)
+    inv_dot = (math.sqrt(d) / op.abs().sum(dim=1)).to(torch.float32)
+    return packed, inv_dot
+
+
+def make_corpus(cfg: CorpusConfig, device="cpu", out_device=None, keep_raw: bool = False,
+                rabitq: bool = False) -> Corpus:
+    """Generate the index arrays of `cfg` on `device`; results are moved to `out_device` (default: `device`).
+    rabitq=True also produces RaBitQ 1-bit codes of the tokens (rotation, rq_bits, rq_inv_dot)."""
     device = torch.device(device)
     out_device = torch.device(out_device) if out_device is not None else device
     assert cfg.dim % 8 == 0 and cfg.nbits in (1, 2)
@@ -174,6 +201,9 @@ def make_corpus(cfg: CorpusConfig, device="cpu", out_device=None, keep_raw: bool
     cids = torch.empty(T, dtype=torch.int32, device=out_device)
     codes = torch.empty(T, cfg.code_bytes, dtype=torch.uint8, device=out_device)
     raw = torch.empty(T, cfg.dim, dtype=torch.float32, device=out_device) if keep_raw else None
+    rot = random_rotation(cfg).to(device) if rabitq else None
+    rq_bits = torch.empty(T, cfg.dim // 8, dtype=torch.uint8, device=out_device) if rabitq else None
+    rq_inv = torch.empty(T, dtype=torch.float32, device=out_device) if rabitq else None
     for ci, t0 in enumerate(range(0, T, _CHUNK_TOKENS)):
         n = min(_CHUNK_TOKENS, T - t0)
         comp = torch.randint(0, cfg.n_centroids, (n,), generator=_gen(cfg.seed, _S_COMP, ci, device), device=device)
@@ -186,7 +216,12 @@ def make_corpus(cfg: CorpusConfig, device="cpu", out_device=None, keep_raw: bool
         codes[t0:t0 + n] = encode_residual(r, cfg.nbits, cfg.res_lo, cfg.res_hi).to(out_device)
         if keep_raw:
             raw[t0:t0 + n] = x.to(out_device)
-    return Corpus(cfg, cent.to(out_device).contiguous(), cids, codes, doclens.to(out_device), raw)
+        if rabitq:
+            b, f = encode_rabitq_1bit(x, rot)
+            rq_bits[t0:t0 + n] = b.to(out_device)
+            rq_inv[t0:t0 + n] = f.to(out_device)
+    return Corpus(cfg, cent.to(out_device).contiguous(), cids, codes, doclens.to(out_device), raw,
+                  rot.to(out_device) if rabitq else None, rq_bits, rq_inv)
 
 
 def make_queries(cfg: CorpusConfig, n_queries: Optional[int] = None, device="cpu", out_device=None) -> torch.Tensor:

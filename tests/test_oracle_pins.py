@@ -494,3 +494,114 @@ def test_pipeline_with_partial_scores_prunes_by_f_prime():
     order = np.lexsort((r.cand, -r.ci.astype(np.int64)))[:20]
     assert np.array_equal(r.pruned, np.sort(r.cand[order]))
     assert np.array_equal(r.score4, oracle.score_docs(q, r.pruned, ix))
+
+
+# ------------------------------------------------------------------ O-9 RaBitQ 1-bit codes (Sec. 2.2) --------------
+
+def _rabitq_case(seed, N=40, K=8, D=64, nq=5):
+    import torch
+    from synth import CONFIGS, encode_rabitq_1bit, random_rotation
+    rng = np.random.default_rng(seed)
+    cent, cids, codes, doclens = random_corpus(seed, N, K, D, 1, len_lo=1, len_hi=8)
+    raw = unit_rows(rng, len(cids), D)
+    P = random_rotation(CONFIGS["tiny"].replace(dim=D, seed=seed))
+    bits, inv = encode_rabitq_1bit(torch.from_numpy(raw), P)
+    ix = oracle.make_index(cent, cids, codes, doclens, 1)
+    rq = oracle.make_rabitq(P, bits, inv)
+    return ix, rq, raw, unit_rows(rng, nq, D)
+
+
+def test_rotation_is_orthonormal_and_rotate_matches_numpy():
+    ix, rq, raw, q = _rabitq_case(40)
+    P = rq.rotation.astype(np.float64)
+    assert np.allclose(P @ P.T, np.eye(P.shape[0]), atol=1e-6)
+    qp = oracle.rotate(rq.rotation, q)
+    assert np.allclose(qp, q.astype(np.float64) @ P.T, atol=1e-6)
+    assert np.allclose(np.linalg.norm(qp, axis=1), 1.0, atol=1e-6)
+    # inner products are preserved by the rotation (Sec. 2.2)
+    rp = oracle.rotate(rq.rotation, raw[:7])
+    assert np.allclose(qp.astype(np.float64) @ rp.astype(np.float64).T, q.astype(np.float64) @ raw[:7].T.astype(np.float64),
+                       atol=1e-6)
+
+
+def test_rabitq_estimate_equals_codeword_formula_and_is_exact_on_codewords():
+    ix, rq, raw, q = _rabitq_case(41, N=30, D=64)
+    D = ix.dim
+    qp = oracle.rotate(rq.rotation, q).astype(np.float64)
+    # one-token documents: the score of document d for a single query token is est(q, token d)
+    one = oracle.make_index(ix.centroids, ix.cids, ix.codes, np.ones(len(ix.cids), np.int32), 1)
+    op = raw.astype(np.float64) @ rq.rotation.astype(np.float64).T
+    obar = np.sign(op) / np.sqrt(D)                      # nearest codeword of G_r for B = 1
+    want = (qp[:1] @ obar.T)[0] / np.einsum("td,td->t", op, obar)      # <q_p, o-bar> / <o_p, o-bar>
+    got = oracle.rabitq_score_docs(qp[:1].astype(np.float32), np.arange(len(raw), dtype=np.int32), one, rq)
+    assert np.allclose(got, want, atol=3e-6)
+    # a token that IS a codeword is estimated exactly: est = <q, o>
+    signs = np.where(np.random.default_rng(1).random((5, D)) > 0.5, 1.0, -1.0) / np.sqrt(D)
+    tok = (signs @ rq.rotation.astype(np.float64)).astype(np.float32)          # o = P^T o_p
+    import torch
+    from synth import encode_rabitq_1bit
+    bits, inv = encode_rabitq_1bit(torch.from_numpy(tok), torch.from_numpy(rq.rotation))
+    rq2 = oracle.make_rabitq(rq.rotation, bits, inv)
+    one2 = oracle.make_index(ix.centroids, np.zeros(5, np.int32), np.zeros((5, D // 8), np.uint8), np.ones(5, np.int32), 1)
+    got2 = oracle.rabitq_score_docs(qp[:1].astype(np.float32), np.arange(5, dtype=np.int32), one2, rq2)
+    assert np.allclose(got2, (q[:1].astype(np.float64) @ tok.astype(np.float64).T)[0], atol=5e-6)
+
+
+def test_rabitq_estimator_is_unbiased_with_error_of_order_one_over_sqrt_d():
+    # Sec. 2.2: the estimator is unbiased with a tight error bound; over many random unit vectors the mean error is
+    # zero within its standard error and the error spread is a small multiple of 1/sqrt(D)
+    import torch
+    from synth import CONFIGS, encode_rabitq_1bit, random_rotation
+    D, n = 128, 4000
+    rng = np.random.default_rng(42)
+    raw = unit_rows(rng, n, D)
+    q = unit_rows(rng, 1, D)
+    P = random_rotation(CONFIGS["tiny"].replace(seed=5))
+    bits, inv = encode_rabitq_1bit(torch.from_numpy(raw), P)
+    rq = oracle.make_rabitq(P, bits, inv)
+    one = oracle.make_index(unit_rows(rng, 1, D), np.zeros(n, np.int32), np.zeros((n, D // 8), np.uint8),
+                            np.ones(n, np.int32), 1)
+    est = oracle.rabitq_score_docs(oracle.rotate(P.numpy(), q), np.arange(n, dtype=np.int32), one, rq).astype(np.float64)
+    err = est - (raw.astype(np.float64) @ q[0].astype(np.float64))
+    assert abs(err.mean()) < 4 * err.std() / np.sqrt(n)
+    assert 0.2 / np.sqrt(D) < err.std() < 1.5 / np.sqrt(D)
+
+
+def test_rabitq_lookup_table_identity():
+    # Sec. 4.1: <q, b> = sum_j T_q[j, b^(j)] with 4-bit chunks; it is the integer T of the estimate
+    ix, rq, raw, q = _rabitq_case(43, N=12, D=64)
+    D = ix.dim
+    qp = oracle.rotate(rq.rotation, q[:1])
+    xq = np.rint(qp[0].astype(np.float64) * 2 ** 22)
+    Tq = np.array([[sum(((u >> t) & 1) * xq[4 * j + t] for t in range(4)) for u in range(16)] for j in range(D // 4)])
+    one = oracle.make_index(ix.centroids, ix.cids, ix.codes, np.ones(len(ix.cids), np.int32), 1)
+    got = oracle.rabitq_score_docs(qp, np.arange(len(raw), dtype=np.int32), one, rq)
+    c = np.float32(1.0 / (np.sqrt(float(D)) * 2.0 ** 22))
+    for t in range(len(raw)):
+        nib = []
+        for byte in rq.bits[t]:
+            nib += [int(byte) & 15, int(byte) >> 4]
+        T = sum(Tq[j, nib[j]] for j in range(D // 4))
+        want = rq.inv_dot[t] * np.float32(c * np.float32(2 * T - xq.sum()))
+        assert got[t] == np.float32(want)
+
+
+def test_rabitq_partial_with_every_list_probed_is_the_complete_one_bit_score():
+    ix, rq, raw, q = _rabitq_case(44, N=50, K=8, D=64, nq=6)
+    S = oracle.score_table(q, ix.centroids)
+    pr = oracle.probes(S, ix.K)
+    cand = oracle.candidates(pr, ix)
+    qp = oracle.rotate(rq.rotation, q)
+    fp = oracle.rabitq_partial(qp, pr, cand, ix, rq)
+    # per query token max(0, max_t est), summed in fp32 in increasing i -- from one-token scores
+    one = oracle.make_index(ix.centroids, ix.cids, ix.codes, np.ones(len(ix.cids), np.int32), 1)
+    per_tok = np.stack([oracle.rabitq_score_docs(qp[i:i + 1], np.arange(len(ix.cids), dtype=np.int32), one, rq)
+                        for i in range(len(q))])
+    for j, d in enumerate(cand):
+        tot = np.float32(0)
+        for i in range(len(q)):
+            tot = np.float32(tot + max(np.float32(0), per_tok[i, ix.doc_off[d]:ix.doc_off[d + 1]].max()))
+        assert fp[j] == tot
+    r = oracle.pipeline_rabitq(q, ix, rq, 2, 10, 4)
+    assert len(r.pruned) == 10 and np.all(np.diff(r.pruned) > 0) and np.all(np.isin(r.ids, r.pruned))
+    assert np.array_equal(r.score4, oracle.rabitq_score_docs(qp, r.pruned, ix, rq))
