@@ -178,6 +178,31 @@ int chimera_search_partial(const chimera_index *index, const float *queries, int
                            size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
                            const chimera_taps *taps);
 
+/* Attach RaBitQ 1-bit codes of the corpus tokens (Sec. 2.2: unit-norm token o, o_p = P o, code bit x = (o_p[x] > 0),
+ * nearest codeword o_p-bar = sign(o_p) / sqrt(dim)) so that chimera_search_rabitq can run the paper's own GPU pipeline.
+ *   rotation  device, [dim, dim] float32 row-major orthonormal matrix P.  Copied (transposed).
+ *   bits      device, [T, dim/8] uint8, document-major: bit t of byte g is dimension 8g+t.  REFERENCED, not copied.
+ *   inv_dot   device, [T] float32, 1 / <o_p, o_p-bar> = sqrt(dim) / sum_x |o_p[x]|.  REFERENCED, not copied.
+ * Also builds the token-level posting lists (as chimera_index_enable_partial).  Synchronises the stream.
+ * Errors: INVALID_ARG, CUDA_ERROR. */
+int chimera_index_attach_rabitq(chimera_index *index, const float *rotation, const uint8_t *bits,
+                                const float *inv_dot, void *stream);
+
+/* The paper's GPU-resident pipeline on its own codec (Algorithm 1 without the CPU half): stage 1 and 2 as in
+ * chimera_search (centroid probes, candidate set); queries rotated (q_p = P q, one fp32 fma chain per output);
+ * candidate refinement by partial 1-bit scores (Algorithm 2: score[doc, i] starts at 0 and is raised by every
+ * retrieved token's estimate; F' = sum over i in increasing i, fp32) keeping k_refine documents; document scoring =
+ * the complete 1-bit Chamfer score sum_i max_t est(i, t) of the survivors; top-k.  The estimate (Sec. 2.2) is
+ *     est(i, t) = <q_p, o_p-bar> / <o_p, o_p-bar> = inv_dot_t * (c * (float)(2 T - SQ_i)),   c = 1 / (sqrt(dim) 2^22),
+ * T = sum_x Xq_i[x] bit_t[x], SQ_i = sum_x Xq_i[x], Xq = rint(q_p * 2^22): reproducible bit for bit.
+ * Arguments as chimera_search_tapped with k_refine in the place of n_prune (taps may be NULL); taps->ci receives the
+ * bit patterns of the float F' of every candidate, taps->score4 the complete 1-bit scores.  q_len <= 64.
+ * Requires chimera_index_attach_rabitq; query chimera_workspace_bytes after attaching. */
+int chimera_search_rabitq(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                          int32_t nprobe, int32_t k_refine, int32_t k, int64_t max_candidates, void *workspace,
+                          size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
+                          const chimera_taps *taps);
+
 /* Device-side status of the last search that used this workspace: synchronises the stream, then writes CHIMERA_OK,
  * CHIMERA_CAPACITY_OVERFLOW (some query had more than max_candidates candidates; its results are computed on the
  * first max_candidates of them and are not the specified output), CHIMERA_INVALID_ARG (a query element outside

@@ -184,8 +184,17 @@ class Index:
             _check(lib().chimera_index_enable_partial(self._h, _stream()))
         self._ws = None
 
+    def attach_rabitq(self, rotation: torch.Tensor, bits: torch.Tensor, inv_dot: torch.Tensor):
+        """Attach RaBitQ 1-bit codes (kept referenced) for search(..., rabitq=True)."""
+        self._rq = (rotation.contiguous().to(torch.float32), bits.contiguous().to(torch.uint8),
+                    inv_dot.contiguous().to(torch.float32))
+        with torch.cuda.device(self.device):
+            _check(lib().chimera_index_attach_rabitq(self._h, _ptr(self._rq[0]), _ptr(self._rq[1]), _ptr(self._rq[2]),
+                                                     _stream()))
+        self._ws = None
+
     def search(self, queries: torch.Tensor, nprobe: int, n_prune: int, k: int, max_candidates: int = 0,
-               taps: Optional[Taps] = None, out=None, partial: bool = False):
+               taps: Optional[Taps] = None, out=None, partial: bool = False, rabitq: bool = False):
         """queries: [B, q_len, dim] float32 CUDA tensor.  Returns (ids [B,k] int32, scores [B,k] float32).
         partial=True prunes with the paper's partial scores (chimera_search_partial)."""
         assert queries.is_cuda and queries.dtype == torch.float32 and queries.is_contiguous()
@@ -201,9 +210,10 @@ class Index:
         args = (self._h, _ptr(queries), ctypes.c_int32(B), ctypes.c_int32(q_len), ctypes.c_int32(nprobe),
                 ctypes.c_int32(n_prune), ctypes.c_int32(k), ctypes.c_int64(max_candidates), _ptr(ws),
                 ctypes.c_size_t(ws.numel()), _stream(), _ptr(ids), _ptr(scores))
-        if partial:
+        if partial or rabitq:
             c = taps._c() if taps is not None else None
-            _check(lib().chimera_search_partial(*args, ctypes.byref(c) if c is not None else None))
+            fn = lib().chimera_search_rabitq if rabitq else lib().chimera_search_partial
+            _check(fn(*args, ctypes.byref(c) if c is not None else None))
         elif taps is None:
             _check(lib().chimera_search(*args))
         else:

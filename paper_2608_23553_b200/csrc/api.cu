@@ -106,6 +106,8 @@ Layout make_layout(const Index &ix, const Params &p)
     L.pruned = take(B * p.n_prune * sizeof(int32_t));
     L.word_rank = take(B * (size_t)L.words * sizeof(int32_t));
     L.partial_m = take(ix.tok_id ? B * (size_t)p.maxc * nq * sizeof(int32_t) : 0);
+    L.q_rot = take(ix.rot_t ? B * nq * ix.D * sizeof(float) : 0);
+    L.qdig_rot = take(ix.rot_t ? 3 * B * nq * 128 : 0);
     L.n_pruned = take(B * sizeof(int32_t));
     L.score4 = take(B * p.n_prune * sizeof(float));
     L.total = o;
@@ -139,10 +141,12 @@ static int copy_d2d(void *dst, const void *src, size_t bytes, cudaStream_t st)
 
 static int run(const Index &ix, const Params &p, int first, int last, const float *queries, void *workspace,
                size_t workspace_bytes, cudaStream_t st, const chimera_taps *taps, int32_t *out_ids, float *out_scores,
-               bool partial = false)
+               bool partial = false, bool rabitq = false)
 {
     if (partial && !ix.tok_id)
         return fail(CHIMERA_INVALID_ARG, "partial-score refinement needs chimera_index_enable_partial first");
+    if (rabitq && (!ix.rot_t || !residual_umma_supported(p.nq)))
+        return fail(CHIMERA_INVALID_ARG, "the RaBitQ pipeline needs chimera_index_attach_rabitq and q_len <= 64");
     if (!workspace || ((uintptr_t)workspace & 255)) return fail(CHIMERA_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
     const Layout L = make_layout(ix, p);
     if (workspace_bytes < L.total)
@@ -161,7 +165,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int32_t *cand = (int32_t *)(ws + L.cand);
     int32_t *n_cand = (int32_t *)(ws + L.n_cand);
     int32_t *ci = (int32_t *)(ws + L.ci);
-    const bool two_phase = coarse_supported(p.nq) && !partial;
+    const bool two_phase = coarse_supported(p.nq) && !partial && !rabitq;
     uint8_t *table8 = two_phase ? (uint8_t *)(ws + L.table8) : nullptr;
     int32_t *lo = (int32_t *)(ws + L.lo);
     int32_t *hi = (int32_t *)(ws + L.hi);
@@ -171,6 +175,8 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int32_t *n_pruned = (int32_t *)(ws + L.n_pruned);
     int32_t *word_rank = (int32_t *)(ws + L.word_rank);
     int32_t *partial_m = (int32_t *)(ws + L.partial_m);
+    float *q_rot = (float *)(ws + L.q_rot);
+    int8_t *qdig_rot = (int8_t *)(ws + L.qdig_rot);
     float *score4 = (float *)(ws + L.score4);
 
     const size_t B = (size_t)p.B;
@@ -217,7 +223,18 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
         prof_mark(SLOT_GATHER, st);
     }
     if (first <= 3 && last >= 3) {
-        if (partial) {
+        if (rabitq) {
+            // the paper's pipeline on its own codec: rotate the queries, refine by partial 1-bit scores
+            if ((rc = launch_rotate(ix, p, queries, q_rot, st))) return rc;
+            if ((rc = launch_digits(q_rot, (int64_t)p.B * p.nq, ix.D, qdig_rot, status, st))) return rc;
+            count_launch(SLOT_G1);
+            prof_mark(SLOT_G1, st);
+            if ((rc = launch_rabitq_partial(ix, p, L, q_rot, probes, bitmap, word_rank, n_cand, partial_m, ci, st)))
+                return rc;
+            prof_mark(SLOT_CI, st);
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
+            prof_mark(SLOT_SELECT, st);
+        } else if (partial) {
             // the paper's candidate refinement: partial scores from the retrieved tokens only, then the same selection
             if ((rc = launch_partial_scores(ix, p, L, queries, table, probes, bitmap, word_rank, n_cand, partial_m, ci,
                                             st)))
@@ -248,7 +265,9 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
         }
     }
     if (first <= 4 && last >= 4) {
-        if (residual_umma_supported(p.nq)) {
+        if (rabitq) {
+            if ((rc = launch_rabitq_scores_umma(ix, p, q_rot, qdig_rot, pruned, score4, status, st))) return rc;
+        } else if (residual_umma_supported(p.nq)) {
             if (first > 1) {                       // stage 1 did not run in this call: build the query digit planes
                 if ((rc = launch_digits(queries, (int64_t)p.B * p.nq, ix.D, qdig, status, st))) return rc;
                 count_launch(SLOT_G4);
@@ -372,10 +391,39 @@ int chimera_search_partial(const chimera_index *index, const float *queries, int
                true);
 }
 
+int chimera_index_attach_rabitq(chimera_index *index, const float *rotation, const uint8_t *bits,
+                                const float *inv_dot, void *stream)
+{
+    Index *ix = reinterpret_cast<Index *>(index);
+    if (!ix || !rotation || !bits || !inv_dot) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if (((uintptr_t)bits & 15) || ((uintptr_t)inv_dot & 3)) return fail(CHIMERA_INVALID_ARG, "bits must be 16-byte aligned");
+    int rc = build_token_lists(*ix, (cudaStream_t)stream);
+    if (rc) return rc;
+    rc = attach_rabitq(*ix, rotation, (cudaStream_t)stream);
+    if (rc) return rc;
+    ix->rq_bits = bits;
+    ix->rq_inv = inv_dot;
+    return CHIMERA_OK;
+}
+
+int chimera_search_rabitq(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                          int32_t nprobe, int32_t k_refine, int32_t k, int64_t max_candidates, void *workspace,
+                          size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
+                          const chimera_taps *taps)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, k_refine, k, max_candidates, &p);
+    if (rc) return rc;
+    return run(*ix, p, 1, 5, queries, workspace, workspace_bytes, (cudaStream_t)stream, taps, out_ids, out_scores,
+               false, true);
+}
+
 int chimera_destroy_index(chimera_index *index)
 {
     Index *ix = reinterpret_cast<Index *>(index);
     if (!ix) return CHIMERA_OK;
+    cudaFree(ix->rot_t);
     cudaFree(ix->tok_off);
     cudaFree(ix->tok_id);
     cudaFree(ix->tok_doc);

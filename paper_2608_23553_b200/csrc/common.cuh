@@ -29,6 +29,10 @@ struct Index {
     int64_t *tok_off = nullptr;       // [K+1]      owned
     int32_t *tok_id = nullptr;        // [T]        owned: token ids per centroid, unordered
     int32_t *tok_doc = nullptr;       // [T]        owned: document of each listed token
+    // RaBitQ 1-bit codes (only after chimera_index_attach_rabitq)
+    const uint8_t *rq_bits = nullptr; // [T, D/8]   borrowed: sign bits of the rotated tokens
+    const float *rq_inv = nullptr;    // [T]        borrowed: 1 / <o_p, o_p-bar>
+    float *rot_t = nullptr;           // [D][D]     owned: transposed rotation, rot_t[x * D + r] = P[r][x]
 };
 
 // Device status bits kept in the first word of a workspace.
@@ -64,6 +68,8 @@ struct Layout {
     size_t pruned;        // int32  [B][n_prune]
     size_t word_rank;     // int32  [B][words]        candidates before each bitmap word (document -> candidate index)
     size_t partial_m;     // int32  [B][maxc][nq]     per (candidate, query token) best retrieved-token score
+    size_t q_rot;         // float  [B, nq, D]        rotated queries (RaBitQ pipeline)
+    size_t qdig_rot;      // int8   [3][B*nq][128]    their digit planes
     size_t n_pruned;      // int32  [B]
     size_t score4;        // float  [B][n_prune]
     size_t total;
@@ -136,6 +142,14 @@ bool residual_umma_supported(int nq);
 int launch_residual_scores_umma(const Index &ix, const Params &p, const float *queries, const int8_t *qdig,
                                 const int32_t *table, const int32_t *pruned, float *score4, uint32_t *status,
                                 cudaStream_t st);
+int launch_rabitq_scores_umma(const Index &ix, const Params &p, const float *q_rot, const int8_t *qdig_rot,
+                              const int32_t *pruned, float *score4, uint32_t *status, cudaStream_t st);
+// rabitq.cu
+int attach_rabitq(Index &ix, const float *rotation, cudaStream_t st);
+int launch_rotate(const Index &ix, const Params &p, const float *queries, float *q_rot, cudaStream_t st);
+int launch_rabitq_partial(const Index &ix, const Params &p, const Layout &L, const float *q_rot,
+                          const int32_t *probes, const uint32_t *bitmap, const int32_t *word_rank,
+                          const int32_t *n_cand, int32_t *partial_m, int32_t *fprime_bits, cudaStream_t st);
 int launch_topk(const Index &ix, const Params &p, const int32_t *pruned, const float *score4, int32_t *out_ids,
                 float *out_scores, cudaStream_t st);
 

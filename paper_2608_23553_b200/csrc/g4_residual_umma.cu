@@ -35,13 +35,18 @@ __device__ __forceinline__ float f_unorder(uint32_t o)
     return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
 }
 
-template <int NQP, int NBITS>
+// RQ = true scores RaBitQ 1-bit codes instead (Sec. 2.2; the GPU half of the paper's document scoring): the same
+// contraction T = sum_x Xq[x] b[x] against the digit planes of the ROTATED query, then
+// est = inv_dot_t * (c * (float)(2 T - SQ_i)) with SQ_i = sum_x Xq_i[x] and c = 1 / (sqrt(D) 2^22); no centroid term;
+// query tokens are summed in increasing order in fp32 so that the score is reproducible bit for bit.
+template <int NQP, int NBITS, bool RQ>
 __global__ void __launch_bounds__(G4U_THREADS)
 residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__restrict__ queries,
                      const int32_t *__restrict__ table, int64_t K, int nq, int D, int CW, float delta, float kappa,
                      const int32_t *__restrict__ pruned, int n_prune, int docs_per_cta,
                      const int32_t *__restrict__ cids, const uint32_t *__restrict__ codes,
-                     const int64_t *__restrict__ doc_off, float *__restrict__ score4, uint32_t *status)
+                     const float *__restrict__ factors, const int64_t *__restrict__ doc_off,
+                     float *__restrict__ score4, uint32_t *status)
 {
     constexpr int N = 3 * NQP;                               // MMA N: three digit planes side by side
     constexpr uint32_t TMEM_COLS = N <= 128 ? 128 : 256;
@@ -57,6 +62,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     __shared__ int s_off[G4U_MAX_DOCS + 1];                  // stream offset of each document
     __shared__ long long s_t0[G4U_MAX_DOCS];                 // first global token of each document
     __shared__ float s_sumq[NQP];
+    __shared__ int s_sq[NQP];                                // RQ: sum_x rint(q_p[x] * 2^22) per query token
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to the aligned area
     const uint32_t sA = base, sB = base + A_BYTES;
@@ -113,10 +119,16 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     // sum_x q_i[x] per query token (warp per row, coalesced)
     for (int i = warp; i < NQP; i += G4U_THREADS / 32) {
         float s = 0.f;
+        int si = 0;
         if (i < nq)
-            for (int x = lane; x < D; x += 32) s += queries[((int64_t)b * nq + i) * D + x];
+            for (int x = lane; x < D; x += 32) {
+                const float v = queries[((int64_t)b * nq + i) * D + x];
+                s += v;
+                si += __float2int_rn(fminf(fmaxf(v, -1.0f), 1.0f) * 4194304.0f);
+            }
         s = warp_sum(s);
-        if (lane == 0) s_sumq[i] = s;
+        si = warp_sum(si);
+        if (lane == 0) { s_sumq[i] = s; s_sq[i] = si; }
     }
     tc_fence_before();
     __syncthreads();
@@ -147,7 +159,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             while (dl_hint + 1 < nd && s_off[dl_hint + 1] <= s) ++dl_hint;    // positions only move forward
             dl = dl_hint;
             const long long t = s_t0[dl] + (s - s_off[dl]);
-            cid = cids[t];
+            cid = RQ ? __float_as_int(factors[t]) : cids[t];     // RQ: the slot carries the token's factor bits (> 0)
             const uint32_t *src = codes + t * CW;
             if ((CW & 3) == 0) {                          // 16-byte aligned codes: two wide loads for 32 bytes
 #pragma unroll
@@ -232,7 +244,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
 
         // ---- while the tensor core works: this token's row of the score table, and the next tile's token -----------
         int4 sv[NQP / 4];
-        if (cid >= 0) {
+        if (!RQ && cid >= 0) {
             const int32_t *srow = tb + (int64_t)cid * nq;
 #pragma unroll
             for (int g = 0; g < NQP / 4; ++g) {
@@ -271,14 +283,18 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             if (cid >= 0) {
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
-                    const int4 q4 = sv[ch * 4 + g];
+                    const int4 q4 = RQ ? make_int4(0, 0, 0, 0) : sv[ch * 4 + g];
                     const int32_t se[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int o = 4 * g + e;
                         // |sum_x u_x Xq_x| <= 3 * 2^22 * |q|_1 < 2^31: the plane recombination fits int32
                         const int32_t T = a0[o] + a1[o] * 256 + a2[o] * 65536;
-                        vrow[ch * 16 + o] = fmaf(code_scale, (float)T, (float)se[e] * (1.0f / 16777216.0f));
+                        if (RQ)
+                            vrow[ch * 16 + o] = __fmul_rn(__int_as_float(cid),
+                                                          __fmul_rn(kappa, (float)(2 * T - s_sq[ch * 16 + o])));
+                        else
+                            vrow[ch * 16 + o] = fmaf(code_scale, (float)T, (float)se[e] * (1.0f / 16777216.0f));
                     }
                 }
             }
@@ -319,7 +335,10 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         for (int dl = warp; dl < nd; dl += G4U_THREADS / 32) {
             const int32_t d = pruned[(int64_t)b * n_prune + j0 + dl];
             float v = 0.f;
-            if (d >= 0) {
+            if (RQ) {                                   // fixed summation order: reproducible bits
+                if (d >= 0 && lane == 0)
+                    for (int i = 0; i < nq; ++i) v = __fadd_rn(v, f_unorder(docmax[dl * NQP + i]));
+            } else if (d >= 0) {
                 if (lane < nq) v = f_unorder(docmax[dl * NQP + lane]) + kappa * s_sumq[lane];
                 if (NQP > 32 && 32 + lane < nq) v += f_unorder(docmax[dl * NQP + 32 + lane]) + kappa * s_sumq[32 + lane];
             }
@@ -333,19 +352,20 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     }
 }
 
-template <int NQP, int NBITS>
+template <int NQP, int NBITS, bool RQ>
 static int launch_g4_umma(const Index &ix, const Params &p, const float *queries, const int8_t *qdig,
                           const int32_t *table, const int32_t *pruned, float *score4, uint32_t *status, cudaStream_t st)
 {
     constexpr int N = 3 * NQP;
     const float delta = (ix.res_hi - ix.res_lo) / (float)(1 << ix.nbits);
-    const float kappa = ix.res_lo + 0.5f * delta;
+    // RQ: the kappa slot carries c = 1 / (sqrt(D) * 2^22)
+    const float kappa = RQ ? (float)(1.0 / (sqrt((double)ix.D) * 4194304.0)) : ix.res_lo + 0.5f * delta;
     CUtensorMap map_q;
     int rc = make_plane_map(&map_q, qdig, (int64_t)p.B * p.nq, NQP);
     if (rc) return rc;
     const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 + sizeof(float) * G4U_TOK * (NQP + 1) +
                         sizeof(uint32_t) * G4U_MAX_DOCS * NQP + sizeof(uint32_t) * (NBITS == 2 ? 256 : 512) + 32;
-    auto kern = residual_maxsim_umma<NQP, NBITS>;
+    auto kern = residual_maxsim_umma<NQP, NBITS, RQ>;
     CHIMERA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // documents per CTA: about four CTAs per SM in total, between 4 and 32 documents each
     int64_t dpc = ((int64_t)p.n_prune * p.B + 4LL * ix.sm_count - 1) / (4LL * ix.sm_count);
@@ -353,9 +373,10 @@ static int launch_g4_umma(const Index &ix, const Params &p, const float *queries
     if (dpc > G4U_MAX_DOCS) dpc = G4U_MAX_DOCS;
     if (dpc > p.n_prune) dpc = p.n_prune;
     dim3 grid((unsigned)((p.n_prune + dpc - 1) / dpc), (unsigned)p.B);
-    kern<<<grid, G4U_THREADS, smem, st>>>(map_q, queries, table, ix.K, p.nq, ix.D, ix.CB / 4, delta, kappa, pruned,
-                                          p.n_prune, (int)dpc, ix.cids, reinterpret_cast<const uint32_t *>(ix.codes),
-                                          ix.doc_off, score4, status);
+    const uint32_t *code_words = reinterpret_cast<const uint32_t *>(RQ ? ix.rq_bits : ix.codes);
+    kern<<<grid, G4U_THREADS, smem, st>>>(map_q, queries, table, ix.K, p.nq, ix.D, RQ ? ix.D / 32 : ix.CB / 4, delta,
+                                          kappa, pruned, p.n_prune, (int)dpc, ix.cids, code_words, ix.rq_inv, ix.doc_off,
+                                          score4, status);
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_G4);
     return CHIMERA_OK;
@@ -368,11 +389,19 @@ int launch_residual_scores_umma(const Index &ix, const Params &p, const float *q
                                 cudaStream_t st)
 {
     if (ix.nbits == 2) {
-        if (p.nq <= 32) return launch_g4_umma<32, 2>(ix, p, queries, qdig, table, pruned, score4, status, st);
-        return launch_g4_umma<64, 2>(ix, p, queries, qdig, table, pruned, score4, status, st);
+        if (p.nq <= 32) return launch_g4_umma<32, 2, false>(ix, p, queries, qdig, table, pruned, score4, status, st);
+        return launch_g4_umma<64, 2, false>(ix, p, queries, qdig, table, pruned, score4, status, st);
     }
-    if (p.nq <= 32) return launch_g4_umma<32, 1>(ix, p, queries, qdig, table, pruned, score4, status, st);
-    return launch_g4_umma<64, 1>(ix, p, queries, qdig, table, pruned, score4, status, st);
+    if (p.nq <= 32) return launch_g4_umma<32, 1, false>(ix, p, queries, qdig, table, pruned, score4, status, st);
+    return launch_g4_umma<64, 1, false>(ix, p, queries, qdig, table, pruned, score4, status, st);
+}
+
+// Complete 1-bit scores of the surviving documents on the RaBitQ codes; q_rot / qdig_rot belong to the rotated queries.
+int launch_rabitq_scores_umma(const Index &ix, const Params &p, const float *q_rot, const int8_t *qdig_rot,
+                              const int32_t *pruned, float *score4, uint32_t *status, cudaStream_t st)
+{
+    if (p.nq <= 32) return launch_g4_umma<32, 1, true>(ix, p, q_rot, qdig_rot, nullptr, pruned, score4, status, st);
+    return launch_g4_umma<64, 1, true>(ix, p, q_rot, qdig_rot, nullptr, pruned, score4, status, st);
 }
 
 }  // namespace chimera
