@@ -144,9 +144,9 @@ def whole_job_qps(local_ms: float, queries_per_rank: int, dist=None, device="cpu
     return world * queries_per_rank / (ms / 1e3), ms
 
 
-def build_workload(cfg, device):
+def build_workload(cfg, device, rabitq=False):
     t0 = time.time()
-    corp = make_corpus(cfg, device=device)
+    corp = make_corpus(cfg, device=device, rabitq=rabitq)
     q = make_queries(cfg, device=device)
     torch.cuda.synchronize() if device.type == "cuda" else None
     return corp, q, time.time() - t0
@@ -242,22 +242,24 @@ def run_sweep(args, cfg, pkg, index, corp, q):
             for k in (10, 100, 1000):
                 out = (torch.empty(B, k, dtype=torch.int32, device=dev), torch.empty(B, k, dtype=torch.float32, device=dev))
                 point = {"nprobe": P, "n_prune": n_prune, "k": k, "max_candidates": maxc}
-                for mode, partial in (("", False), ("partial_", True)):
-                    index.search(batches[0], P, n_prune, k, max_candidates=maxc, out=out, partial=partial)
+                for mode, kw in (("", {}), ("partial_", {"partial": True}), ("rabitq_", {"rabitq": True})):
+                    index.search(batches[0], P, n_prune, k, max_candidates=maxc, out=out, **kw)
                     torch.cuda.synchronize()
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
                     for s in range(args.steps):
-                        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out,
-                                     partial=partial)
+                        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out, **kw)
                     e1.record()
                     torch.cuda.synchronize()
                     ms = e0.elapsed_time(e1) / args.steps
                     assert index.status() == 0
-                    ids, _ = index.search(qrec, P, n_prune, k, max_candidates=maxc, partial=partial)
+                    ids, _ = index.search(qrec, P, n_prune, k, max_candidates=maxc, **kw)
                     hits = (ids[:, :, None] == truth_ids[:, None, :k]).any(dim=2).sum(dim=1).float()
+                    # how many of the ground-truth top-10 are among the k returned (the use of a GPU filter stage)
+                    top10 = (truth_ids[:, :10, None] == ids[:, None, :]).any(dim=2).sum(dim=1).float()
                     point.update({mode + "qps": B / (ms * 1e-3), mode + "ms_per_step": ms,
-                                  mode + "recall": float((hits / k).mean())})
+                                  mode + "recall": float((hits / k).mean()),
+                                  mode + "top10_in_k": float((top10 / 10).mean())})
                 print(json.dumps(point))
 
 
@@ -271,6 +273,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="queries per call (default 256; 64 for the long-document configs)")
     ap.add_argument("--partial", action="store_true",
                     help="prune with the paper's partial scores (chimera_search_partial) instead of stage 3")
+    ap.add_argument("--rabitq", action="store_true",
+                    help="the paper's pipeline on RaBitQ 1-bit codes (chimera_search_rabitq)")
     ap.add_argument("--sweep", action="store_true", help="QPS vs recall over nprobe x n_prune x k (see run_sweep)")
     ap.add_argument("--sweep-queries", type=int, default=200)
     ap.add_argument("--batch1-queries", type=int, default=200)
@@ -304,13 +308,16 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    corp, q, gen_s = build_workload(cfg, device)
+    corp, q, gen_s = build_workload(cfg, device, rabitq=args.rabitq or args.sweep)
     t0 = time.time()
     index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
     build_s = time.time() - t0
     B, nq, P, n_prune, k = args.batch, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
     if args.partial or args.sweep:
         index.enable_partial()
+    if args.rabitq or args.sweep:
+        index.attach_rabitq(corp.rotation, corp.rq_bits, corp.rq_inv_dot)
+    mode = {"partial": args.partial, "rabitq": args.rabitq}
     if args.sweep:
         if rank == 0:
             run_sweep(args, cfg, pkg, index, corp, q)
@@ -330,7 +337,7 @@ def main():
     work = []
     for bi in range(n_batches):
         taps = index.alloc_taps(B, nq, P, n_prune, max_candidates=maxc, table=False, ci=False)
-        index.search(batches[bi], P, n_prune, k, max_candidates=maxc, taps=taps, partial=args.partial)
+        index.search(batches[bi], P, n_prune, k, max_candidates=maxc, taps=taps, **mode)
         assert index.status() == 0
         mask = torch.arange(taps.cand.shape[1], device=device)[None, :] < taps.n_cand[:, None].to(torch.int64)
         toks = (doclens64[taps.cand.to(torch.int64).clamp_(0, index.N - 1)] * mask).sum()
@@ -343,7 +350,7 @@ def main():
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps ------------------------------------
     for s in range(args.warmup):
-        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out, partial=args.partial)
+        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out, **mode)
     barrier()
     pkg.profile_enable(True)
     pkg.profile_read()
@@ -353,7 +360,7 @@ def main():
     e0.record()
     for s in range(args.steps):
         index.search(batches[(args.warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc, out=out,
-                     partial=args.partial)
+                     **mode)
     e1.record()
     barrier()
     clocks = sampler.stop()
@@ -367,11 +374,11 @@ def main():
     dq = torch.empty_like(batches[0])
 
     def host_search(hq, hout, dbuf, dout):
-        if not args.partial:
+        if not (args.partial or args.rabitq):
             index.search_host(hq, P, n_prune, k, max_candidates=maxc, out=hout)
-        else:       # the host entry point has no partial variant: pinned copies around chimera_search_partial
+        else:       # the host entry point has no such variant: pinned copies around the device entry point
             dbuf.copy_(hq, non_blocking=True)
-            index.search(dbuf, P, n_prune, k, max_candidates=maxc, out=dout, partial=True)
+            index.search(dbuf, P, n_prune, k, max_candidates=maxc, out=dout, **mode)
             hout[0].copy_(dout[0], non_blocking=True)
             hout[1].copy_(dout[1], non_blocking=True)
             torch.cuda.synchronize()
@@ -392,14 +399,14 @@ def main():
     n1 = min(args.batch1_queries, q.shape[0])
     out1 = (torch.empty(1, k, dtype=torch.int32, device=device), torch.empty(1, k, dtype=torch.float32, device=device))
     for i in range(5):
-        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, partial=args.partial)
+        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, **mode)
     torch.cuda.synchronize()
     lat = []
     pkg.profile_enable(True)
     pkg.profile_read()
     for i in range(n1):
         a = time.perf_counter()
-        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, partial=args.partial)
+        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, **mode)
         torch.cuda.synchronize()
         lat.append(time.perf_counter() - a)
     stage_ms1, _ = pkg.profile_read()
@@ -472,7 +479,8 @@ def main():
     }
 
     result = {
-        "metric": metric_name(cfg, B) + (" with partial-score refinement" if args.partial else ""), "value": qps,
+        "metric": metric_name(cfg, B) + (" with partial-score refinement" if args.partial else "")
+        + (" on RaBitQ 1-bit codes (paper pipeline)" if args.rabitq else ""), "value": qps,
         "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32 fixed point (stages 1-3) + f32 (stage 4)", "data": "synthetic",
@@ -480,7 +488,8 @@ def main():
                    "n_centroids": cfg.n_centroids, "dim": cfg.dim, "nbits": cfg.nbits, "q_len": nq, "nprobe": P,
                    "n_prune": n_prune, "k": k, "parallelism": "replicas only" if world > 1 else "single GPU",
                    "max_candidates": maxc if maxc else cfg.n_docs,
-                   "pruning": "partial scores of retrieved tokens (Algorithm 2)" if args.partial
+                   "pruning": "partial 1-bit RaBitQ scores of retrieved tokens, then complete 1-bit scores" if args.rabitq
+                   else "partial scores of retrieved tokens (Algorithm 2)" if args.partial
                    else "centroid interaction over every candidate token",
                    "l2": "inputs larger than L2 (index %.1f GB, score table %.1f GB per batch); no flush"
                          % ((corp.cids.numel() * 4 + corp.codes.numel()) / 1e9, B * cfg.n_centroids * nq * 4 / 1e9),
