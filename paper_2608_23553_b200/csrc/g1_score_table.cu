@@ -240,11 +240,8 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     CUtensorMap map_c, map_q;
     if ((rc = make_plane_map(&map_c, ix.cdig, ix.K, G1_M))) return rc;
     if ((rc = make_plane_map(&map_q, qdig, rows, G1_N))) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G1_SMEM));
-        attr_set = true;
-    }
+    // per device, so set on every launch (it is a cheap host-side call)
+    CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G1_SMEM));
     const int c_tiles = (int)((ix.K + G1_M - 1) / G1_M);
     const int n_tiles = (int)((rows + G1_N - 1) / G1_N);
     // about eight waves of two CTAs per SM, so the last wave is mostly full
