@@ -79,3 +79,35 @@ def test_partial_refinement_mid_batch256_sampled():
     gix.enable_partial()
     oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
     _check(gix, oix, q, cfg.nprobe, cfg.n_prune, cfg.k, sample=(0, 255), max_diffs=2)
+
+
+def test_partial_and_rabitq_edge_cases():
+    """Few candidates (k_refine and k larger than the candidate set), and a candidate capacity that overflows."""
+    import paper_2608_23553_b200 as pkg
+    from synth import CONFIGS, encode_rabitq_1bit, random_rotation
+    D, K, N = 32, 16, 40
+    cent, cids, codes, doclens = random_corpus(77, N, K, D, 2, len_lo=1, len_hi=4)
+    rng = np.random.default_rng(78)
+    raw = unit_rows(rng, len(cids), D)
+    P = random_rotation(CONFIGS["tiny"].replace(dim=D, seed=9))
+    bits, inv = encode_rabitq_1bit(torch.from_numpy(raw), P)
+    oix = oracle.make_index(cent, cids, codes, doclens, 2)
+    rq = oracle.make_rabitq(P, bits, inv)
+    dev = torch.device("cuda:0")
+    gix = pkg.Index(torch.from_numpy(cent).to(dev), torch.from_numpy(cids).to(dev), torch.from_numpy(codes).to(dev),
+                    torch.from_numpy(doclens).to(dev), 2)
+    gix.attach_rabitq(P.to(dev), bits.to(dev), inv.to(dev))          # also builds the token lists
+    q = unit_rows(rng, 4, D)[None]
+    qd = torch.from_numpy(q).cuda()
+    for kw, ref in (({"partial": True}, lambda: oracle.pipeline(q[0], oix, 1, 100, 200, partial=True)),
+                    ({"rabitq": True}, lambda: oracle.pipeline_rabitq(q[0], oix, rq, 1, 100, 200))):
+        ids, sc = gix.search(qd, 1, 100, 200, **kw)
+        assert gix.status() == 0
+        res = ref()
+        n = int((res.ids >= 0).sum())
+        assert n < 100 and np.array_equal(ids[0].cpu().numpy(), res.ids)
+        assert np.all(np.isneginf(sc[0, n:].cpu().numpy()))
+        gix.search(qd, 8, 10, 5, max_candidates=4, **kw)             # more candidates than the capacity
+        assert gix.status() == 4
+        gix.search(qd, 8, 10, 5, **kw)
+        assert gix.status() == 0
