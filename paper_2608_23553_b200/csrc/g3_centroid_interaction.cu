@@ -162,12 +162,16 @@ __device__ __forceinline__ void coarse_accumulate(uint32_t (&m)[8], const int4 &
     }
 }
 
-template <int LPR>
-__global__ void __launch_bounds__(CI_THREADS)
+// SMEM = true: the query's whole 8-bit table (K * q_len bytes) is first staged in shared memory and the row lookups
+// are shared-memory loads (small K only); blocks are then larger (THREADS) because only one fits an SM.
+template <int LPR, bool SMEM, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *__restrict__ cand,
                  const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
                  const int64_t *__restrict__ doc_off, int32_t *__restrict__ lo, int32_t *__restrict__ hi)
 {
+    extern __shared__ int4 smem_table[];
+    constexpr int WARPS = THREADS / 32;
     constexpr int NQ = 16 * LPR;
     constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
     constexpr int STEPS = 32 / TPL;               // loads per 32-token slab (= LPR)
@@ -177,8 +181,14 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
     const int grp = lane / LPR, sub = lane % LPR;
     const int n = n_cand[b];
     const int4 *tb = reinterpret_cast<const int4 *>(table8 + (int64_t)b * K * NQ) + sub;
+    if (SMEM) {
+        const int4 *src = reinterpret_cast<const int4 *>(table8 + (int64_t)b * K * NQ);
+        for (int64_t e = threadIdx.x; e < K * LPR; e += THREADS) smem_table[e] = __ldg(src + e);
+        __syncthreads();
+    }
+    const int4 *ts = smem_table + sub;
     const int32_t *cb = cand + (int64_t)b * maxc;
-    const int warps_per_query = gridDim.x * CI_WARPS;
+    const int warps_per_query = gridDim.x * WARPS;
     // The chain candidate id -> token range -> first centroid ids is three dependent loads: it is issued one document
     // ahead, so it overlaps the row gathers of the current document.
     int64_t nx_t0 = 0, nx_t1 = 0;
@@ -193,7 +203,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
             nx_cid[k] = cids[i < nx_t1 - 1 ? i : nx_t1 - 1];
         }
     };
-    int j = blockIdx.x * CI_WARPS + (threadIdx.x >> 5);
+    int j = blockIdx.x * WARPS + (threadIdx.x >> 5);
     if (j < n) prefetch(j);
     for (; j < n; j += warps_per_query) {
         const int64_t t0 = nx_t0, t1 = nx_t1;
@@ -222,7 +232,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
 #pragma unroll
                     for (int s = 0; s < STEPS; ++s) {
                         const int32_t c = __shfl_sync(0xffffffffu, cid[k], s * TPL + grp);
-                        v[k * STEPS + s] = __ldg(tb + (int64_t)c * LPR);
+                        v[k * STEPS + s] = SMEM ? ts[c * LPR] : __ldg(tb + (int64_t)c * LPR);
                     }
                 }
             }
@@ -280,15 +290,42 @@ bool coarse_supported(int nq) { return nq == 32 || nq == 64; }
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
                          const int32_t *n_cand, int32_t *lo, int32_t *hi, cudaStream_t st)
 {
+    const size_t table_bytes = (size_t)ix.K * p.nq;
+    if (table_bytes <= 160 * 1024) {
+        // the whole 8-bit table of a query fits in shared memory: stage it once per block and look rows up there
+        constexpr int T = 512;
+        int64_t gx = (4LL * ix.sm_count + p.B - 1) / p.B;       // every block re-reads the table: few, long blocks
+        int64_t want = (p.maxc + T / 32 - 1) / (T / 32);
+        if (gx > want) gx = want;
+        if (gx > 64) gx = 64;
+        if (gx < 1) gx = 1;
+        dim3 grid((unsigned)gx, (unsigned)p.B);
+        if (p.nq == 32) {
+            CHIMERA_CUDA(cudaFuncSetAttribute(ci_coarse_kernel<2, true, T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)table_bytes));
+            ci_coarse_kernel<2, true, T><<<grid, T, table_bytes, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids,
+                                                                       ix.doc_off, lo, hi);
+        } else {
+            CHIMERA_CUDA(cudaFuncSetAttribute(ci_coarse_kernel<4, true, T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)table_bytes));
+            ci_coarse_kernel<4, true, T><<<grid, T, table_bytes, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids,
+                                                                       ix.doc_off, lo, hi);
+        }
+        CHIMERA_CUDA(cudaGetLastError());
+        count_launch(SLOT_CI);
+        return CHIMERA_OK;
+    }
     int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
     int64_t cap = (int64_t)ix.sm_count * 8;
     unsigned gx = (unsigned)(want < cap ? want : cap);
     if (gx < 1) gx = 1;
     dim3 grid(gx, (unsigned)p.B);
     if (p.nq == 32)
-        ci_coarse_kernel<2><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, lo, hi);
+        ci_coarse_kernel<2, false, CI_THREADS><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids,
+                                                                          ix.doc_off, lo, hi);
     else
-        ci_coarse_kernel<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, lo, hi);
+        ci_coarse_kernel<4, false, CI_THREADS><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids,
+                                                                          ix.doc_off, lo, hi);
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_CI);
     return CHIMERA_OK;
