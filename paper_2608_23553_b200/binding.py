@@ -263,6 +263,38 @@ class Index:
         return st.value
 
 
+class GraphedSearch:
+    """A search of fixed shape captured once into a CUDA graph and replayed (removes the per-kernel launch gaps of the
+    ~18 small kernels of a batch-1 search).  Plumbing only: the captured work is exactly one Index.search call.
+    Profiling must be off while capturing (events cannot be timed inside a graph)."""
+
+    def __init__(self, index: "Index", n_queries: int, q_len: int, nprobe: int, n_prune: int, k: int,
+                 max_candidates: int = 0, **mode):
+        dev = index.device
+        self.queries = torch.zeros(n_queries, q_len, index.dim, dtype=torch.float32, device=dev)
+        self.ids = torch.empty(n_queries, k, dtype=torch.int32, device=dev)
+        self.scores = torch.empty(n_queries, k, dtype=torch.float32, device=dev)
+        self.queries[..., 0] = 1.0                       # valid unit vectors for the warm-up call
+        self._index = index
+        args = (nprobe, n_prune, k)
+        stream = torch.cuda.Stream(device=dev)
+        stream.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.stream(stream):
+            index.search(self.queries, *args, max_candidates=max_candidates, out=(self.ids, self.scores), **mode)
+            stream.synchronize()
+            self.graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.graph, stream=stream):
+                index.search(self.queries, *args, max_candidates=max_candidates, out=(self.ids, self.scores), **mode)
+        torch.cuda.current_stream(dev).wait_stream(stream)
+
+    def __call__(self, queries: torch.Tensor):
+        """Copy `queries` (device or pinned host tensor of the captured shape) into the static input and replay.
+        Returns the static output tensors (overwritten by the next call)."""
+        self.queries.copy_(queries, non_blocking=True)
+        self.graph.replay()
+        return self.ids, self.scores
+
+
 def probes_static(score_table: torch.Tensor, nprobe: int) -> torch.Tensor:
     """Top-nprobe centroids per query token through chimera_probes_static: no workspace and no device allocation
     inside the library (its scratch is a fixed 4 MiB array in the library image).  For callers that must not allocate

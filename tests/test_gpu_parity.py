@@ -247,3 +247,15 @@ def test_tiny_config_recall_against_exhaustive(chimera, tiny):
         truth, _, _ = oracle.exhaustive(q[b], oix, cfg.k)
         res = oracle.pipeline(q[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
         assert oracle.recall(truth, ids[b]) == oracle.recall(truth, res.ids)
+
+
+def test_graphed_search_equals_eager(chimera, tiny):
+    cfg, oix, gix, q = tiny
+    qd = torch.from_numpy(q).cuda()
+    g = chimera.GraphedSearch(gix, 1, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k)
+    for b in (0, 5, 15):
+        ids_e, sc_e = gix.search(qd[b:b + 1].contiguous(), cfg.nprobe, cfg.n_prune, cfg.k)
+        ids_e, sc_e = ids_e.clone(), sc_e.clone()
+        ids_g, sc_g = g(qd[b:b + 1])
+        torch.cuda.synchronize()
+        assert torch.equal(ids_g, ids_e) and torch.equal(sc_g, sc_e)
