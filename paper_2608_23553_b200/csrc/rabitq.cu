@@ -65,8 +65,13 @@ rabitq_clear_kernel(int32_t *__restrict__ M, const int32_t *__restrict__ n_cand,
     const int b = blockIdx.y;
     const int64_t n = (int64_t)n_cand[b] * nq;
     int32_t *row = M + (int64_t)b * maxc * nq;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
-        row[e] = 0;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (int64_t)gridDim.x * blockDim.x;
+    if ((nq & 3) == 0) {                               // rows are 16-byte aligned
+        int4 *row4 = reinterpret_cast<int4 *>(row);
+        for (int64_t e = tid; e < n / 4; e += stride) row4[e] = make_int4(0, 0, 0, 0);
+    } else {
+        for (int64_t e = tid; e < n; e += stride) row[e] = 0;
+    }
 }
 
 // grid (nq * P, B): one block per (query token, probed list); M holds float bits (>= 0, so integer order = float order).
@@ -127,7 +132,18 @@ rabitq_sum_kernel(const int32_t *__restrict__ M, const int32_t *__restrict__ n_c
     for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
         const int32_t *row = M + ((int64_t)b * maxc + j) * nq;
         float s = 0.0f;
-        for (int i = 0; i < nq; ++i) s = __fadd_rn(s, __int_as_float(row[i]));
+        if ((nq & 3) == 0) {
+            const int4 *row4 = reinterpret_cast<const int4 *>(row);
+            for (int i = 0; i < nq / 4; ++i) {
+                const int4 v = row4[i];
+                s = __fadd_rn(s, __int_as_float(v.x));
+                s = __fadd_rn(s, __int_as_float(v.y));
+                s = __fadd_rn(s, __int_as_float(v.z));
+                s = __fadd_rn(s, __int_as_float(v.w));
+            }
+        } else {
+            for (int i = 0; i < nq; ++i) s = __fadd_rn(s, __int_as_float(row[i]));
+        }
         fprime_bits[(int64_t)b * maxc + j] = __float_as_int(s);
     }
 }
