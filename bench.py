@@ -79,6 +79,7 @@ def ncu_traffic(cfg, batch):
 
 
 NCU_CI_COARSE_MID_B8_BYTES = 467.2e6    # dram__bytes_read.sum + dram__bytes_write.sum of one launch at batch 8
+NCU_PARTIAL_MID_B64_BYTES = 1833e6      # the same for partial_score_kernel<2> at batch 64 (profiles/ncu_partial_score_mid.md)
 
 
 class ClockSampler:
@@ -334,6 +335,7 @@ def main():
 
     # algorithmic work per batch (outside the timed region): candidate documents and their tokens, from the taps
     doclens64 = corp.doclens.to(torch.int64)
+    list_len = torch.bincount(corp.cids.to(torch.int64).view(-1), minlength=cfg.n_centroids)   # posting-list sizes
     work = []
     for bi in range(n_batches):
         taps = index.alloc_taps(B, nq, P, n_prune, max_candidates=maxc, table=False, ci=False)
@@ -344,7 +346,8 @@ def main():
         pr = taps.pruned.to(torch.int64)
         toks4 = (doclens64[pr.clamp(min=0)] * (pr >= 0)).sum()
         work.append({"cand": int(taps.n_cand.sum()), "cand_tokens": int(toks), "pruned_tokens": int(toks4),
-                     "contenders": int(taps.n_contenders.sum())})
+                     "contenders": int(taps.n_contenders.sum()),
+                     "retrieved": int(list_len[taps.probes.to(torch.int64)].sum())})
         del taps, mask
     torch.cuda.empty_cache()
 
@@ -453,7 +456,8 @@ def main():
     lookup_roof = 148 * 1.965e9
     cont_frac = mean("contenders") / max(mean("cand"), 1.0)
     g4_ms = stage_ms["residual_scores"] / n_prof
-    g4_bytes = mean("pruned_tokens") * (4.0 + cfg.code_bytes)
+    # stage 4 reads per survivor token its centroid id + residual code (or its 1-bit code + scale on the RaBitQ path)
+    g4_bytes = mean("pruned_tokens") * ((cfg.dim // 8 + 4.0) if args.rabitq else (4.0 + cfg.code_bytes))
     stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
     roofline = {
         "kernel": "ci_coarse_kernel (stage 3 bound scan over every candidate token)", "bound": "hbm",
@@ -470,6 +474,26 @@ def main():
                    "code_gbs": g4_bytes / (g4_ms * 1e-3) / 1e9 if g4_ms > 0 else 0.0,
                    "int8_tops": 2.0 * 3.0 * mean("pruned_tokens") * nq * cfg.dim / (g4_ms * 1e-3) / 1e12 if g4_ms > 0 else 0.0},
     }
+    if args.partial or args.rabitq:
+        # candidate refinement by partial scores replaces the scan: the dominant stage-3 kernel visits every token of
+        # the nq * nprobe probed posting lists.  Algorithmic bytes per visit: the list entry (token id + document id,
+        # 8 B) and the token's code (residual code, or 1-bit code + its 4-byte scale); per candidate document one
+        # nq * 4-byte row of running maxima is cleared first.  The slot times the clear and the scoring kernel together.
+        code_b = (cfg.dim // 8 + 4.0) if args.rabitq else float(cfg.code_bytes)
+        ps_bytes = mean("retrieved") * (8.0 + code_b) + mean("cand") * nq * 4.0
+        ps_gbs = ps_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0
+        traffic = None
+        if cfg.name == "mid" and args.partial and not args.rabitq:
+            traffic = NCU_PARTIAL_MID_B64_BYTES * B / 64.0
+        for key in ("binding_roof", "contender_fraction"):
+            roofline.pop(key)
+        roofline.update({
+            "kernel": ("rabitq_partial_kernel" if args.rabitq else "partial_score_kernel")
+            + " (+ its clear kernel): partial scores of the retrieved tokens, Algorithm 2",
+            "achieved": ps_gbs, "frac": ps_gbs / peak, "traffic": traffic, "algorithmic_bytes_per_launch": ps_bytes,
+            "visits_per_launch": mean("retrieved"),
+            "note": "scattered 32-byte sectors (codes of random tokens, read-modify-write of 4-byte cells): the roof "
+                    "of such accesses is below the streaming-copy peak this fraction is taken against"})
     # per-stage achieved fraction of the roof that the stage's algorithmic work is measured against
     i8_peak, i8_kind = measured_int8_tops()
 
@@ -483,7 +507,8 @@ def main():
         "score_table": frac_entry("tensor (int8, %s)" % i8_kind, 2.0 * 9.0 * B * nq * cfg.n_centroids * cfg.dim / 1e12,
                                   g1_ms, i8_peak, "TOP/s"),
         "probes": frac_entry("hbm", B * nq * cfg.n_centroids * 4.0 / 1e9, pr_ms, peak, "GB/s"),
-        "centroid_interaction_bounds": frac_entry("hbm", ci_bytes / 1e9, ci_ms, peak, "GB/s"),
+        ("partial_scores" if args.partial or args.rabitq else "centroid_interaction_bounds"):
+            frac_entry("hbm", (ps_bytes if args.partial or args.rabitq else ci_bytes) / 1e9, ci_ms, peak, "GB/s"),
         "residual_scores": frac_entry("hbm (code + centroid-id bytes)", g4_bytes / 1e9, g4_ms, peak, "GB/s"),
         "residual_scores_tensor": frac_entry("tensor (int8, %s)" % i8_kind,
                                              2.0 * 3.0 * mean("pruned_tokens") * nq * cfg.dim / 1e12, g4_ms, i8_peak,
