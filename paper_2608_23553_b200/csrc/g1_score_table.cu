@@ -24,7 +24,7 @@ namespace chimera {
 constexpr int G1_M = 128;            // centroids per tile (MMA M)
 constexpr int G1_N = 48;             // query-token rows per tile (MMA N)
 constexpr int G1_ROW_BYTES = 128;    // digit-plane row pitch = padded dimension count
-constexpr int G1_THREADS = 128;
+constexpr int G1_THREADS = 256;        // two warps per tensor-memory lane quarter: both drain accumulators
 constexpr int G1_TMEM_COLS = 256;
 constexpr uint32_t G1_A_PLANE = G1_M * G1_ROW_BYTES;      // 16 KB
 constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;      // 6 KB
@@ -132,43 +132,46 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         __syncwarp();
-        const int64_t c = c0 + warp * 32 + lane;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        // warp w reads tensor-memory lanes 32 (w % 4) ... + 31 (its centroids); the two warps of a lane quarter take
+        // alternate chunks of eight query-token columns
+        const int quad = warp & 3;
+        const int64_t c = c0 + quad * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+        const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
 #pragma unroll 1
-        for (int chunk = 0; chunk < G1_N / 16; ++chunk) {
-            int32_t acc[5][16];
+        for (int chunk = warp >> 2; chunk < G1_N / 8; chunk += 2) {
+            int32_t acc[5][8];
 #pragma unroll
-            for (int w = 0; w < 5; ++w) tmem_ld16(lane_addr + w * G1_N + chunk * 16, acc[w]);
+            for (int w = 0; w < 5; ++w) tmem_ld8(lane_addr + w * G1_N + chunk * 8, acc[w]);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            int32_t out[16];
+            int32_t out[8];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) out[e] = combine_digits(acc[0][e], acc[1][e], acc[2][e], acc[3][e], acc[4][e]);
-            // first query-token row of this chunk, and its (query, token) coordinates: one 32-bit division per chunk,
-            // then incremental (rows fit 32 bits: n_queries * q_len < 2^23)
-            const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)chunk * 16;
-            const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
+            for (int e = 0; e < 8; ++e) out[e] = combine_digits(acc[0][e], acc[1][e], acc[2][e], acc[3][e], acc[4][e]);
+            // first query-token row of this chunk and its (query, token) coordinates (rows fit 32 bits:
+            // n_queries * q_len < 2^23)
+            const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)chunk * 8;
             uint32_t qb = r0 / unq, qi = r0 - qb * unq;
-            if (table8 != nullptr && c < K && r0 < rows32) {
-                // coarse copy for the bound phase of stage 3: min((S + 2^24 + 64) >> 17, 255); q_len is a multiple of
-                // 16 here, so the 16 rows of a chunk belong to one query and the store is 16-byte aligned
-                uint32_t w[4];
+            if (c < K && r0 < rows32) {
+                if (table8 != nullptr) {
+                    // coarse copy for the bound phase of stage 3: min((S + 2^24 + 64) >> 17, 255); q_len is a multiple
+                    // of 16 here, so the 8 rows of a chunk belong to one query and the store is 8-byte aligned
+                    uint32_t w[2];
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    uint32_t pack = 0;
+                    for (int g = 0; g < 2; ++g) {
+                        uint32_t pack = 0;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        int v = (out[4 * g + e] + (1 << 24) + 64) >> 17;
-                        v = v > 255 ? 255 : v;
-                        pack |= (uint32_t)v << (8 * e);
+                        for (int e = 0; e < 4; ++e) {
+                            int v = (out[4 * g + e] + (1 << 24) + 64) >> 17;
+                            v = v > 255 ? 255 : v;
+                            pack |= (uint32_t)v << (8 * e);
+                        }
+                        w[g] = pack;
                     }
-                    w[g] = pack;
+                    *reinterpret_cast<uint2 *>(table8 + ((int64_t)qb * K + c) * nq + qi) = make_uint2(w[0], w[1]);
                 }
-                *reinterpret_cast<uint4 *>(table8 + ((int64_t)qb * K + c) * nq + qi) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            if (c < K) {
                 if ((nq & 3) == 0) {
 #pragma unroll
-                    for (int e = 0; e < 16; e += 4) {
+                    for (int e = 0; e < 8; e += 4) {
                         if (r0 + e < rows32)                          // q_rows is a multiple of 4 here
                             *reinterpret_cast<int4 *>(table + ((int64_t)qb * K + c) * nq + qi) =
                                 make_int4(out[e], out[e + 1], out[e + 2], out[e + 3]);
@@ -177,7 +180,7 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                     }
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
+                    for (int e = 0; e < 8; ++e) {
                         if (r0 + e < rows32) table[((int64_t)qb * K + c) * nq + qi] = out[e];
                         if (++qi == unq) { qi = 0; ++qb; }
                     }
