@@ -11,18 +11,19 @@ namespace chimera {
 
 constexpr int PROBE_THREADS = PROBE_WARPS * 32;
 
+template <int STRIDE = PROBE_THREADS>
 __device__ __forceinline__ void list_insert(unsigned long long *list, int P, unsigned long long key)
 {
-    // list[j * PROBE_THREADS] is entry j of this thread's list, descending.
-    if (key <= list[(P - 1) * PROBE_THREADS]) return;
+    // list[j * STRIDE] is entry j of this thread's list, descending.
+    if (key <= list[(P - 1) * STRIDE]) return;
     int j = P - 1;
     while (j > 0) {
-        unsigned long long up = list[(j - 1) * PROBE_THREADS];
+        unsigned long long up = list[(j - 1) * STRIDE];
         if (up >= key) break;
-        list[j * PROBE_THREADS] = up;
+        list[j * STRIDE] = up;
         --j;
     }
-    list[j * PROBE_THREADS] = key;
+    list[j * STRIDE] = key;
 }
 
 // grid (probe_blocks, B, ceil(nq / 32)).  part: [B][n_part][P][nq], n_part = probe_blocks (one list per block).
@@ -69,71 +70,97 @@ probe_partial(const int32_t *__restrict__ table, int64_t K, int nq, int P, int r
     }
 }
 
-// grid (1, B, ceil(nq / 32)).  Folds n_part sorted lists per column into one; writes probes[b][col][0..P).
-__global__ void __launch_bounds__(PROBE_THREADS)
+// grid (1, B, ceil(nq / 32)), THREADS threads.  Folds n_part sorted lists per column into one; writes
+// probes[b][col][0..P).  Warp w takes lists w, w + W, ... (W = THREADS / 32 warps, lane = column); the warps' lists are
+// then folded pairwise in a tree.  With one query per call this kernel is a single block, so it is latency that counts:
+// up to eight list heads are loaded together, and 32 warps share the lists when nprobe is small enough for the
+// shared-memory lists of 1024 threads.
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
 probe_final(const unsigned long long *__restrict__ part, int nq, int P, int n_part, int32_t *__restrict__ probes)
 {
-    extern __shared__ unsigned long long lists[];
+    extern __shared__ unsigned long long lists[];      // [P][THREADS]
+    constexpr int W = THREADS / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int col = blockIdx.z * 32 + lane;
     const int b = blockIdx.y;
     unsigned long long *mine = lists + threadIdx.x;
-    for (int j = 0; j < P; ++j) mine[j * PROBE_THREADS] = 0ull;
+    for (int j = 0; j < P; ++j) mine[j * THREADS] = 0ull;
     if (col < nq) {
-        // the heads of four lists are loaded together (independent loads); a list is only walked further while its
-        // keys still beat this thread's current P-th best
-        for (int l0 = warp; l0 < n_part; l0 += 4 * PROBE_WARPS) {
-            unsigned long long head[4];
+        // a list is only walked further while its keys still beat this thread's current P-th best
+        for (int l0 = warp; l0 < n_part; l0 += 8 * W) {
+            unsigned long long head[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int l = l0 + u * PROBE_WARPS;
+            for (int u = 0; u < 8; ++u) {
+                const int l = l0 + u * W;
                 head[u] = l < n_part ? part[(((int64_t)b * n_part + l) * P) * nq + col] : 0ull;
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int l = l0 + u * PROBE_WARPS;
-                if (l >= n_part || head[u] <= mine[(P - 1) * PROBE_THREADS]) continue;
-                list_insert(mine, P, head[u]);
+            for (int u = 0; u < 8; ++u) {
+                const int l = l0 + u * W;
+                if (l >= n_part || head[u] <= mine[(P - 1) * THREADS]) continue;
+                list_insert<THREADS>(mine, P, head[u]);
                 const unsigned long long *src = part + (((int64_t)b * n_part + l) * P) * nq + col;
                 for (int j = 1; j < P; ++j) {
                     unsigned long long key = src[(int64_t)j * nq];
-                    if (key <= mine[(P - 1) * PROBE_THREADS]) break;      // source list is descending
-                    list_insert(mine, P, key);
+                    if (key <= mine[(P - 1) * THREADS]) break;      // source list is descending
+                    list_insert<THREADS>(mine, P, key);
                 }
             }
         }
     }
-    __syncthreads();
-    if (warp == 0 && col < nq) {
-        for (int w = 1; w < PROBE_WARPS; ++w) {
-            const unsigned long long *src = lists + w * 32 + lane;
+    for (int s = W / 2; s >= 1; s >>= 1) {
+        __syncthreads();
+        if (warp < s && col < nq) {
+            const unsigned long long *src = lists + (warp + s) * 32 + lane;
             for (int j = 0; j < P; ++j) {
-                unsigned long long key = src[j * PROBE_THREADS];
-                if (key <= mine[(P - 1) * PROBE_THREADS]) break;
-                list_insert(mine, P, key);
+                unsigned long long key = src[j * THREADS];
+                if (key <= mine[(P - 1) * THREADS]) break;
+                list_insert<THREADS>(mine, P, key);
             }
         }
-        int32_t *dst = probes + ((int64_t)b * nq + col) * P;
-        for (int j = 0; j < P; ++j) dst[j] = key_id(mine[j * PROBE_THREADS]);
     }
+    if (warp == 0 && col < nq) {
+        int32_t *dst = probes + ((int64_t)b * nq + col) * P;
+        for (int j = 0; j < P; ++j) dst[j] = key_id(mine[j * THREADS]);
+    }
+}
+
+// The widest block whose lists (nprobe keys of 8 bytes per thread) fit the default 48 KB of shared memory, at least
+// PROBE_THREADS (whose lists may need the opt-in limit: 128 KB at nprobe = 64).
+static int launch_probe_final(const unsigned long long *part, int B, int nq, int P, int n_part, int32_t *probes,
+                              cudaStream_t st)
+{
+    const dim3 grid(1, (unsigned)B, (unsigned)((nq + 31) / 32));
+    const size_t per_thread = sizeof(unsigned long long) * (size_t)P;
+    if (per_thread * 1024 <= 48 * 1024) {
+        probe_final<1024><<<grid, 1024, per_thread * 1024, st>>>(part, nq, P, n_part, probes);
+    } else if (per_thread * 512 <= 48 * 1024) {
+        probe_final<512><<<grid, 512, per_thread * 512, st>>>(part, nq, P, n_part, probes);
+    } else {
+        const size_t smem = per_thread * PROBE_THREADS;
+        if (smem > 48 * 1024)
+            CHIMERA_CUDA(cudaFuncSetAttribute(probe_final<PROBE_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)smem));
+        probe_final<PROBE_THREADS><<<grid, PROBE_THREADS, smem, st>>>(part, nq, P, n_part, probes);
+    }
+    CHIMERA_CUDA(cudaGetLastError());
+    return CHIMERA_OK;
 }
 
 int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32_t *table, unsigned long long *part,
                   int32_t *probes, cudaStream_t st)
 {
     const size_t smem = sizeof(unsigned long long) * (size_t)p.P * PROBE_THREADS;
-    if (smem > 48 * 1024) {
+    if (smem > 48 * 1024)
         CHIMERA_CUDA(cudaFuncSetAttribute(probe_partial, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CHIMERA_CUDA(cudaFuncSetAttribute(probe_final, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    }
     const int rows_per_block = (int)((ix.K + L.probe_blocks - 1) / L.probe_blocks);
     const unsigned col_groups = (unsigned)((p.nq + 31) / 32);
     dim3 g1((unsigned)L.probe_blocks, (unsigned)p.B, col_groups);
     probe_partial<<<g1, PROBE_THREADS, smem, st>>>(table, ix.K, p.nq, p.P, rows_per_block, L.n_part, part);
     CHIMERA_CUDA(cudaGetLastError());
-    dim3 g2(1, (unsigned)p.B, col_groups);
-    probe_final<<<g2, PROBE_THREADS, smem, st>>>(part, p.nq, p.P, L.n_part, probes);
-    CHIMERA_CUDA(cudaGetLastError());
+    const int rc = launch_probe_final(part, p.B, p.nq, p.P, L.n_part, probes, st);
+    if (rc) return rc;
     count_launch(SLOT_PROBE, 2);
     return CHIMERA_OK;
 }
@@ -200,10 +227,8 @@ extern "C" int chimera_probes_static(const int32_t *score_table, int64_t n_centr
 
     cudaStream_t st = (cudaStream_t)stream;
     const size_t smem = sizeof(unsigned long long) * (size_t)nprobe * PROBE_THREADS;
-    if (smem > 48 * 1024) {
+    if (smem > 48 * 1024)
         CHIMERA_CUDA(cudaFuncSetAttribute(probe_partial, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CHIMERA_CUDA(cudaFuncSetAttribute(probe_final, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    }
     const int rows_per_block = (int)((n_centroids + blocks - 1) / blocks);
     const unsigned col_groups = (unsigned)((q_len + 31) / 32);
     // probe_partial writes every entry probe_final reads (all n_part lists x nprobe keys x q_len columns), so nothing
@@ -211,8 +236,5 @@ extern "C" int chimera_probes_static(const int32_t *score_table, int64_t n_centr
     probe_partial<<<dim3((unsigned)blocks, (unsigned)n_queries, col_groups), PROBE_THREADS, smem, st>>>(
         score_table, n_centroids, q_len, nprobe, rows_per_block, n_part, part);
     CHIMERA_CUDA(cudaGetLastError());
-    probe_final<<<dim3(1, (unsigned)n_queries, col_groups), PROBE_THREADS, smem, st>>>(part, q_len, nprobe, n_part,
-                                                                                        out_probes);
-    CHIMERA_CUDA(cudaGetLastError());
-    return CHIMERA_OK;
+    return launch_probe_final(part, n_queries, q_len, nprobe, n_part, out_probes, st);
 }

@@ -518,18 +518,22 @@ select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_ca
 
 // grid (B).  Contenders for the top n_prune: with tau = the n_prune-th largest lower bound, every document of the
 // true top n_prune has hi >= CI >= (n_prune-th largest CI) >= tau.  Writes their ids (ascending) and their number.
+// The lower bounds are lo = (sum - 128 nq) 2^17 - 64 nq with sum = the sum of nq 8-bit maxima (ci_coarse_kernel), so
+// sum itself is a key of at most 14 bits: one histogram sweep over CONT_BINS bins (two neighbouring sums share a bin
+// for q_len 64; tau is then the smaller of the two, still a valid lower threshold) finds tau without radix passes.
+constexpr int CONT_BINS = 8192;
 __global__ void __launch_bounds__(SEL_THREADS)
 contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, const int32_t *__restrict__ lo,
-                 const int32_t *__restrict__ hi, int64_t maxc, int n_prune, int32_t *__restrict__ cont,
+                 const int32_t *__restrict__ hi, int64_t maxc, int n_prune, int nq, int32_t *__restrict__ cont,
                  int32_t *__restrict__ n_cont)
 {
-    __shared__ int hist[2048];
+    __shared__ int hist[CONT_BINS];
     __shared__ int warp_part[32];
-    __shared__ uint32_t s_prefix;
-    __shared__ int s_want;
+    __shared__ int s_bin;
     const int b = blockIdx.x;
     const int n = n_cand[b];
     const int32_t *cb = cand + (int64_t)b * maxc;
+    const int32_t *lb = lo + (int64_t)b * maxc;
     const int32_t *hb = hi + (int64_t)b * maxc;
     int32_t *out = cont + (int64_t)b * maxc;
     if (n <= n_prune) {
@@ -537,28 +541,57 @@ contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n
         if (threadIdx.x == 0) n_cont[b] = n;
         return;
     }
-    int need_eq;
-    const uint32_t thr = radix_select(lo + (int64_t)b * maxc, n, n_prune, hist, warp_part, &s_prefix, &s_want, &need_eq);
-    const int32_t tau = (int32_t)(thr ^ 0x80000000u);
-    int run = 0;
-    for (int base = 0; base < n; base += 4 * SEL_THREADS) {
-        const int j0 = base + 4 * threadIdx.x;
-        int32_t h[4], id[4];
+    const int bin_shift = 255 * nq < CONT_BINS ? 0 : 1;            // q_len 32: one sum per bin; q_len 64: two
+    for (int i = threadIdx.x; i < CONT_BINS; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    for (int base = 0; base < n; base += 16 * SEL_THREADS) {
+        int32_t v[16];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int j = j0 + e;
-            h[e] = j < n ? hb[j] : INT_MIN;
-            id[e] = j < n ? cb[j] : 0;
+        for (int e = 0; e < 16; ++e) {
+            const int j = base + e * SEL_THREADS + threadIdx.x;
+            v[e] = j < n ? lb[j] : 0;
         }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const int j = base + e * SEL_THREADS + threadIdx.x;
+            if (j < n) atomicAdd(&hist[(((v[e] + 64 * nq) >> 17) + 128 * nq) >> bin_shift], 1);
+        }
+    }
+    __syncthreads();
+    // descending bins, CONT_BINS / SEL_THREADS consecutive bins per thread
+    constexpr int PER = CONT_BINS / SEL_THREADS;
+    const int first_bin = CONT_BINS - 1 - PER * (int)threadIdx.x;  // this thread owns first_bin, first_bin - 1, ...
+    int h[PER], mine = 0;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) { h[e] = hist[first_bin - e]; mine += h[e]; }
+    int total;
+    int before = sel_block_scan(mine, &total, warp_part);
+    if (before < n_prune && n_prune <= before + mine) {
+#pragma unroll
+        for (int e = 0; e < PER; ++e) {
+            if (before < n_prune && n_prune <= before + h[e]) s_bin = first_bin - e;
+            before += h[e];
+        }
+    }
+    __syncthreads();
+    const int32_t tau = ((s_bin << bin_shift) - 128 * nq) * (1 << 17) - 64 * nq;   // smallest lower bound in that bin
+    // ordered compaction, eight consecutive entries per thread and round (one block scan per 8192 entries); the ids
+    // are only read for the few entries that are kept
+    int run = 0;
+    for (int base = 0; base < n; base += 8 * SEL_THREADS) {
+        const int j0 = base + 8 * threadIdx.x;
+        int32_t hv[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) hv[e] = j0 + e < n ? hb[j0 + e] : INT_MIN;
         int keep = 0;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) keep += (j0 + e < n && h[e] >= tau) ? 1 : 0;
-        int total;
-        int pos = run + sel_block_scan(keep, &total, warp_part);
+        for (int e = 0; e < 8; ++e) keep += (j0 + e < n && hv[e] >= tau) ? 1 : 0;
+        int tot;
+        int pos = run + sel_block_scan(keep, &tot, warp_part);
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if (j0 + e < n && h[e] >= tau) out[pos++] = id[e];
-        run += total;
+        for (int e = 0; e < 8; ++e)
+            if (j0 + e < n && hv[e] >= tau) out[pos++] = cb[j0 + e];
+        run += tot;
     }
     if (threadIdx.x == 0) n_cont[b] = run;
 }
@@ -567,7 +600,8 @@ int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, con
                       const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st)
 {
     (void)ix;
-    contender_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, lo, hi, p.maxc, p.n_prune, cont, n_cont);
+    contender_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, lo, hi, p.maxc, p.n_prune, p.nq, cont,
+                                                            n_cont);
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_SELECT);
     return CHIMERA_OK;
