@@ -102,7 +102,8 @@ int chimera_workspace_bytes(const chimera_index *index, int32_t n_queries, int32
                             int32_t n_prune, int32_t k, int64_t max_candidates, size_t *out);
 
 /* Stages 1-5 for a batch of queries (Algorithm 1 with the stage list at the top of this file).
- *   queries     device, [n_queries, q_len, dim] float32, unit-norm rows (the library does not normalise).
+ *   queries     device, 16-byte aligned, [n_queries, q_len, dim] float32, unit-norm rows (the library does not
+ *               normalise).
  *   workspace   device, 256-byte aligned, at least chimera_workspace_bytes(...) bytes; contents are scratch.  Two
  *               calls that may overlap on the device need distinct workspaces.
  *   out_ids     device, [n_queries, k] int32: best first; -1 where fewer than k documents survive.

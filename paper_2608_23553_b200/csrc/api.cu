@@ -151,7 +151,8 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     const Layout L = make_layout(ix, p);
     if (workspace_bytes < L.total)
         return fail(CHIMERA_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
-    if ((first <= 1 || (first <= 4 && last >= 4)) && !queries) return fail(CHIMERA_INVALID_ARG, "queries is NULL");
+    if ((first <= 1 || (first <= 4 && last >= 4)) && (!queries || ((uintptr_t)queries & 15)))
+        return fail(CHIMERA_INVALID_ARG, "queries is NULL or not 16-byte aligned");
     if (last >= 5 && (!out_ids || !out_scores)) return fail(CHIMERA_INVALID_ARG, "out_ids / out_scores is NULL");
 
     char *ws = (char *)workspace;

@@ -83,20 +83,29 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         mbar_init(bar_mma, 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // stream offsets of this CTA's documents (padding slots have id -1 and no tokens)
-        int run = 0;
-        for (int dl = 0; dl < nd; ++dl) {
-            const int32_t d = pruned[(int64_t)b * n_prune + j0 + dl];
-            s_off[dl] = run;
-            if (d >= 0) {
-                const long long t0 = doc_off[d];
-                s_t0[dl] = t0;
-                run += (int)(doc_off[d + 1] - t0);
-            } else {
-                s_t0[dl] = 0;
-            }
+    }
+    if (warp == 1) {
+        // stream offsets of this CTA's documents (padding slots have id -1 and no tokens): lane = document, one
+        // round of loads, then a prefix sum of the lengths
+        int32_t d = -1;
+        if (lane < nd) d = pruned[(int64_t)b * n_prune + j0 + lane];
+        long long t0 = 0;
+        int len = 0;
+        if (d >= 0) {
+            t0 = doc_off[d];
+            len = (int)(doc_off[d + 1] - t0);
         }
-        s_off[nd] = run;
+        int incl = len;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane < nd) {
+            s_off[lane] = incl - len;
+            s_t0[lane] = t0;
+        }
+        if (lane == 31) s_off[nd] = incl;          // lanes past nd add nothing
     }
     if (warp == 0) {
         __syncwarp();
@@ -116,19 +125,27 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         }
     }
     for (int e = tid; e < G4U_MAX_DOCS * NQP; e += G4U_THREADS) docmax[e] = 0u;     // below every real value
-    // sum_x q_i[x] per query token (warp per row, coalesced)
-    for (int i = warp; i < NQP; i += G4U_THREADS / 32) {
-        float s = 0.f;
+    // sum_x q_i[x] per query token: four threads per row, each a quarter of the row with 16-byte loads
+    for (int i = tid >> 2; i < NQP; i += G4U_THREADS / 4) {
+        float sum = 0.f;
         int si = 0;
-        if (i < nq)
-            for (int x = lane; x < D; x += 32) {
-                const float v = queries[((int64_t)b * nq + i) * D + x];
-                s += v;
-                si += __float2int_rn(fminf(fmaxf(v, -1.0f), 1.0f) * 4194304.0f);
+        if (i < nq) {
+            const int quarter = D >> 2;               // D is a multiple of 32
+            const float4 *src = reinterpret_cast<const float4 *>(queries + ((int64_t)b * nq + i) * D + (tid & 3) * quarter);
+            for (int x = 0; x < (quarter >> 2); ++x) {
+                const float4 v = __ldg(src + x);
+                sum += (v.x + v.y) + (v.z + v.w);
+                si += __float2int_rn(fminf(fmaxf(v.x, -1.0f), 1.0f) * 4194304.0f) +
+                      __float2int_rn(fminf(fmaxf(v.y, -1.0f), 1.0f) * 4194304.0f) +
+                      __float2int_rn(fminf(fmaxf(v.z, -1.0f), 1.0f) * 4194304.0f) +
+                      __float2int_rn(fminf(fmaxf(v.w, -1.0f), 1.0f) * 4194304.0f);
             }
-        s = warp_sum(s);
-        si = warp_sum(si);
-        if (lane == 0) { s_sumq[i] = s; s_sq[i] = si; }
+        }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        si += __shfl_xor_sync(0xffffffffu, si, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        si += __shfl_xor_sync(0xffffffffu, si, 2);
+        if ((tid & 3) == 0) { s_sumq[i] = sum; s_sq[i] = si; }
     }
     tc_fence_before();
     __syncthreads();
@@ -367,9 +384,10 @@ static int launch_g4_umma(const Index &ix, const Params &p, const float *queries
                         sizeof(uint32_t) * G4U_MAX_DOCS * NQP + sizeof(uint32_t) * (NBITS == 2 ? 256 : 512) + 32;
     auto kern = residual_maxsim_umma<NQP, NBITS, RQ>;
     CHIMERA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    // documents per CTA: about four CTAs per SM in total, between 4 and 32 documents each
+    // documents per CTA: about four CTAs per SM in total, at most 32 documents each (with few queries per call a CTA
+    // gets one or two documents, so that the call's latency is a tile or two and not a chain of them)
     int64_t dpc = ((int64_t)p.n_prune * p.B + 4LL * ix.sm_count - 1) / (4LL * ix.sm_count);
-    if (dpc < 4) dpc = 4;
+    if (dpc < 1) dpc = 1;
     if (dpc > G4U_MAX_DOCS) dpc = G4U_MAX_DOCS;
     if (dpc > p.n_prune) dpc = p.n_prune;
     dim3 grid((unsigned)((p.n_prune + dpc - 1) / dpc), (unsigned)p.B);

@@ -3,7 +3,9 @@
 //
 // One block per query.  Each (score, id) becomes a 64-bit key whose unsigned order is (score desc, id asc); the keys
 // are sorted descending with a bitonic network in shared memory (n_prune <= 16384 keys = 128 KB) and the first k are
-// decoded back.
+// decoded back.  For k <= 16 the keys stay in registers instead and the block extracts its maximum k times (two
+// barriers per result instead of the network's log^2 stages): the shorter chain matters when one query is served at
+// a time.
 #include <math.h>
 
 #include "common.cuh"
@@ -64,10 +66,74 @@ topk_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ score4
     }
 }
 
+template <int KPT>      // keys per thread: n_prune <= KPT * TOPK_THREADS
+__global__ void __launch_bounds__(TOPK_THREADS)
+topk_small_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ score4, int n_prune, int k,
+                  int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
+{
+    __shared__ unsigned long long warp_max[32];
+    __shared__ unsigned long long s_win;
+    const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long keys[KPT];
+#pragma unroll
+    for (int e = 0; e < KPT; ++e) {
+        const int j = e * TOPK_THREADS + threadIdx.x;
+        keys[e] = 0ull;
+        if (j < n_prune) {
+            const int32_t id = pruned[(int64_t)b * n_prune + j];
+            if (id >= 0)
+                keys[e] = ((unsigned long long)float_order(score4[(int64_t)b * n_prune + j]) << 32) |
+                          (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
+        }
+    }
+    for (int r = 0; r < k; ++r) {
+        unsigned long long m = keys[0];
+#pragma unroll
+        for (int e = 1; e < KPT; ++e) m = keys[e] > m ? keys[e] : m;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long t = __shfl_xor_sync(0xffffffffu, m, o);
+            m = t > m ? t : m;
+        }
+        if (lane == 0) warp_max[warp] = m;
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long v = warp_max[lane];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o);
+                v = t > v ? t : v;
+            }
+            if (lane == 0) {
+                s_win = v;
+                out_ids[(int64_t)b * k + r] = v ? (int32_t)(0xFFFFFFFFu - (uint32_t)v) : -1;
+                out_scores[(int64_t)b * k + r] = v ? float_unorder((uint32_t)(v >> 32)) : -INFINITY;
+            }
+        }
+        __syncthreads();
+        const unsigned long long win = s_win;       // keys are distinct (the id is part of the key): one owner
+#pragma unroll
+        for (int e = 0; e < KPT; ++e)
+            if (keys[e] == win) keys[e] = 0ull;
+    }
+}
+
 int launch_topk(const Index &ix, const Params &p, const int32_t *pruned, const float *score4, int32_t *out_ids,
                 float *out_scores, cudaStream_t st)
 {
     (void)ix;
+    if (p.k <= 16) {
+        const unsigned B = (unsigned)p.B;
+        if (p.n_prune <= TOPK_THREADS)
+            topk_small_kernel<1><<<B, TOPK_THREADS, 0, st>>>(pruned, score4, p.n_prune, p.k, out_ids, out_scores);
+        else if (p.n_prune <= 4 * TOPK_THREADS)
+            topk_small_kernel<4><<<B, TOPK_THREADS, 0, st>>>(pruned, score4, p.n_prune, p.k, out_ids, out_scores);
+        else
+            topk_small_kernel<16><<<B, TOPK_THREADS, 0, st>>>(pruned, score4, p.n_prune, p.k, out_ids, out_scores);
+        CHIMERA_CUDA(cudaGetLastError());
+        count_launch(SLOT_TOPK);
+        return CHIMERA_OK;
+    }
     int n_pow2 = 2;
     while (n_pow2 < p.n_prune) n_pow2 <<= 1;
     const size_t smem = sizeof(unsigned long long) * (size_t)n_pow2;
