@@ -252,6 +252,36 @@ int chimera_profile_read(float *ms, int64_t *launches);
 int chimera_probes_static(const int32_t *score_table, int64_t n_centroids, int32_t n_queries, int32_t q_len,
                           int32_t nprobe, void *stream, int32_t *out_probes);
 
+/* ---- Document-sharded search over several GPUs (the scaling sketch of Sec. 3.3) -----------------------------------
+ * The documents are partitioned into `world` contiguous id ranges in rank order; rank r builds an index of its own
+ * documents (local ids 0 .. n_local-1 = global ids doc_base .. doc_base+n_local-1) and of ALL centroids.  Queries are
+ * the same on every rank.  Only ids and scores cross GPUs (the caller moves them, e.g. with an all-gather):
+ *   1. chimera_shard_local   stages 1-3 on the local shard; exports the local top n_prune (global ids ascending,
+ *                            -1 padded) and their stage-3 scores (INT_MIN padded): int32 [n_queries, n_prune] each.
+ *   2. all-gather both arrays over the ranks, in rank order: [world, n_queries, n_prune].
+ *   3. chimera_shard_finish  the global top n_prune of the gathered lists by (score descending, global id ascending)
+ *                            -- the set a single index of all documents prunes to, because stage-3 scores are
+ *                            integers that do not depend on the shard --, of which this rank keeps its own documents,
+ *                            scores them (stage 4) and emits its local top-k with GLOBAL ids: [n_queries, k].
+ *   4. all-gather ids and scores: [world, n_queries, k].
+ *   5. chimera_shard_merge_topk  the best k of the union, (score descending, id ascending): equal to the single-index
+ *                            result (a document's stage-4 score does not depend on the shard it is scored in).
+ * mode: 0 = stage 3 by centroid interaction, 1 = by partial scores (needs chimera_index_enable_partial), 2 = the
+ * RaBitQ pipeline (needs chimera_index_attach_rabitq).  Steps 1 and 3 must use the same workspace and the same
+ * parameters, with no other call on that workspace in between (step 3 continues from what step 1 left there);
+ * check chimera_workspace_status after step 1.  All pointers device; everything is enqueued on `stream`.
+ * world * k <= 16384 in step 5 (CHIMERA_UNSUPPORTED otherwise). */
+int chimera_shard_local(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                        int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, int32_t mode,
+                        int64_t doc_base, void *workspace, size_t workspace_bytes, void *stream, int32_t *out_ids,
+                        int32_t *out_scores3);
+int chimera_shard_finish(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                         int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, int32_t mode,
+                         int64_t doc_base, int32_t world, const int32_t *all_ids, const int32_t *all_scores3,
+                         void *workspace, size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores);
+int chimera_shard_merge_topk(const int32_t *all_ids, const float *all_scores, int32_t world, int32_t n_queries,
+                             int32_t k, void *stream, int32_t *out_ids, float *out_scores);
+
 #ifdef __cplusplus
 }
 #endif

@@ -5,3 +5,4 @@ memory and the stream).  There is no CPU fallback: importing the binding without
 """
 from .binding import (ChimeraError, GraphedSearch, Index, Taps, lib, library_path, probes_static, profile_enable, profile_read,  # noqa: F401
                       PROFILE_SLOTS)
+from .sharded import ShardEngine, ShardedSearcher, all_gather_stack, shard_ranges  # noqa: F401

@@ -109,6 +109,7 @@ Layout make_layout(const Index &ix, const Params &p)
     L.q_rot = take(ix.rot_t ? B * nq * ix.D * sizeof(float) : 0);
     L.qdig_rot = take(ix.rot_t ? 3 * B * nq * 128 : 0);
     L.n_pruned = take(B * sizeof(int32_t));
+    L.pruned_ci = take(B * p.n_prune * sizeof(int32_t));
     L.score4 = take(B * p.n_prune * sizeof(float));
     L.total = o;
     return L;
@@ -141,8 +142,10 @@ static int copy_d2d(void *dst, const void *src, size_t bytes, cudaStream_t st)
 
 static int run(const Index &ix, const Params &p, int first, int last, const float *queries, void *workspace,
                size_t workspace_bytes, cudaStream_t st, const chimera_taps *taps, int32_t *out_ids, float *out_scores,
-               bool partial = false, bool rabitq = false)
+               bool partial = false, bool rabitq = false, bool resume = false)
 {
+    // resume: stages before `first` ran in an earlier call on this workspace with the same parameters and their
+    // results are still there (document-sharded search: the exchange happens between the two calls)
     if (partial && !ix.tok_id)
         return fail(CHIMERA_INVALID_ARG, "partial-score refinement needs chimera_index_enable_partial first");
     if (rabitq && (!ix.rot_t || !residual_umma_supported(p.nq)))
@@ -174,6 +177,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int32_t *n_cont = (int32_t *)(ws + L.n_cont);
     int32_t *pruned = (int32_t *)(ws + L.pruned);
     int32_t *n_pruned = (int32_t *)(ws + L.n_pruned);
+    int32_t *pruned_ci = (int32_t *)(ws + L.pruned_ci);
     int32_t *word_rank = (int32_t *)(ws + L.word_rank);
     int32_t *partial_m = (int32_t *)(ws + L.partial_m);
     float *q_rot = (float *)(ws + L.q_rot);
@@ -190,7 +194,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     CHIMERA_CUDA(cudaMemsetAsync(status, 0, 64 * sizeof(uint32_t), st));
 
     // results of the stages that do not run come from the caller
-    if (first > 1) {
+    if (first > 1 && !resume) {
         if (!taps) return fail(CHIMERA_INVALID_ARG, "taps are required when first_stage > 1");
         if (first <= 4) {       // stages 2-4 read the score table
             if (!taps->score_table) return fail(CHIMERA_INVALID_ARG, "taps->score_table is required");
@@ -233,7 +237,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if ((rc = launch_rabitq_partial(ix, p, L, q_rot, probes, bitmap, word_rank, n_cand, partial_m, ci, st)))
                 return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else if (partial) {
             // the paper's candidate refinement: partial scores from the retrieved tokens only, then the same selection
@@ -241,7 +245,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
                                             st)))
                 return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else if (two_phase) {
             if (first > 1) {                       // the table came from the caller: derive its coarse copy
@@ -256,12 +260,12 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, 2 * ix.sm_count, SLOT_CI_EXACT, st)))
                 return rc;
             prof_mark(SLOT_CI_EXACT, st);
-            if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, st))) return rc;
+            if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, pruned_ci, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else {
             if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, 0, SLOT_CI, st))) return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, st))) return rc;
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         }
     }
@@ -418,6 +422,75 @@ int chimera_search_rabitq(const chimera_index *index, const float *queries, int3
     if (rc) return rc;
     return run(*ix, p, 1, 5, queries, workspace, workspace_bytes, (cudaStream_t)stream, taps, out_ids, out_scores,
                false, true);
+}
+
+// ---- document-sharded search ------------------------------------------------------------------------------------
+static int shard_mode(int32_t mode, bool *partial, bool *rabitq)
+{
+    if (mode < 0 || mode > 2) return fail(CHIMERA_INVALID_ARG, "mode must be 0 (centroid interaction), 1 (partial scores) or 2 (RaBitQ)");
+    *partial = mode == 1;
+    *rabitq = mode == 2;
+    return CHIMERA_OK;
+}
+
+int chimera_shard_local(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                        int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, int32_t mode,
+                        int64_t doc_base, void *workspace, size_t workspace_bytes, void *stream, int32_t *out_ids,
+                        int32_t *out_scores3)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    bool partial, rabitq;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc || (rc = shard_mode(mode, &partial, &rabitq))) return rc;
+    if (!out_ids || !out_scores3) return fail(CHIMERA_INVALID_ARG, "out_ids / out_scores3 is NULL");
+    if (doc_base < 0 || doc_base + ix->N > 0x7fffffffLL) return fail(CHIMERA_INVALID_ARG, "global document ids must fit int32");
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = run(*ix, p, 1, 3, queries, workspace, workspace_bytes, st, nullptr, nullptr, nullptr, partial, rabitq)))
+        return rc;
+    const Layout L = make_layout(*ix, p);
+    char *ws = (char *)workspace;
+    return launch_shard_export(p, (const int32_t *)(ws + L.pruned), (const int32_t *)(ws + L.pruned_ci), doc_base,
+                               out_ids, out_scores3, st);
+}
+
+int chimera_shard_finish(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                         int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, int32_t mode,
+                         int64_t doc_base, int32_t world, const int32_t *all_ids, const int32_t *all_scores3,
+                         void *workspace, size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    bool partial, rabitq;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc || (rc = shard_mode(mode, &partial, &rabitq))) return rc;
+    if (world < 1 || (int64_t)world * n_prune > 0x7fffffffLL) return fail(CHIMERA_INVALID_ARG, "world out of range");
+    if (!all_ids || !all_scores3 || !out_ids || !out_scores) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if (!workspace || ((uintptr_t)workspace & 255)) return fail(CHIMERA_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
+    const Layout L = make_layout(*ix, p);
+    if (workspace_bytes < L.total)
+        return fail(CHIMERA_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = (char *)workspace;
+    if ((rc = launch_shard_select(p, all_ids, all_scores3, world, doc_base, ix->N, (int32_t *)(ws + L.pruned),
+                                  (int32_t *)(ws + L.n_pruned), st)))
+        return rc;
+    if ((rc = run(*ix, p, 4, 5, queries, workspace, workspace_bytes, st, nullptr, out_ids, out_scores, partial, rabitq,
+                  true)))
+        return rc;
+    return launch_add_base(out_ids, (int64_t)p.B * p.k, doc_base, st);
+}
+
+int chimera_shard_merge_topk(const int32_t *all_ids, const float *all_scores, int32_t world, int32_t n_queries,
+                             int32_t k, void *stream, int32_t *out_ids, float *out_scores)
+{
+    if (!all_ids || !all_scores || !out_ids || !out_scores) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if (world < 1 || n_queries < 1 || n_queries > 65535 || k < 1 || k > CHIMERA_MAX_K)
+        return fail(CHIMERA_INVALID_ARG, "world, n_queries or k out of range");
+    if ((int64_t)world * k > 16384)
+        return fail(CHIMERA_UNSUPPORTED, "world * k = %lld entries per query exceed the 16384 the merge holds",
+                    (long long)world * k);
+    return launch_shard_merge_topk(all_ids, all_scores, world, n_queries, k, out_ids, out_scores, (cudaStream_t)stream);
 }
 
 int chimera_destroy_index(chimera_index *index)

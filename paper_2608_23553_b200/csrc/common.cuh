@@ -71,6 +71,7 @@ struct Layout {
     size_t q_rot;         // float  [B, nq, D]        rotated queries (RaBitQ pipeline)
     size_t qdig_rot;      // int8   [3][B*nq][128]    their digit planes
     size_t n_pruned;      // int32  [B]
+    size_t pruned_ci;     // int32  [B][n_prune] stage-3 score of each survivor (document-sharded search)
     size_t score4;        // float  [B][n_prune]
     size_t total;
     // derived sizes
@@ -133,8 +134,17 @@ int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, con
                       const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st);
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
                                 const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, cudaStream_t st);
+// pruned_ci (may be NULL): the score of each kept document, INT_MIN in the padding.
 int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
-                  int32_t *pruned, int32_t *n_pruned, cudaStream_t st);
+                  int32_t *pruned, int32_t *n_pruned, int32_t *pruned_ci, cudaStream_t st);
+// Document-sharded search: the global top-n_prune of the shards' lists and the final top-k merge.
+int launch_shard_export(const Params &p, const int32_t *pruned, const int32_t *pruned_ci, int64_t doc_base,
+                        int32_t *out_ids, int32_t *out_ci, cudaStream_t st);
+int launch_shard_select(const Params &p, const int32_t *all_ids, const int32_t *all_ci, int world, int64_t doc_base,
+                        int64_t n_local, int32_t *pruned, int32_t *n_pruned, cudaStream_t st);
+int launch_add_base(int32_t *ids, int64_t n, int64_t doc_base, cudaStream_t st);
+int launch_shard_merge_topk(const int32_t *all_ids, const float *all_scores, int world, int B, int k, int32_t *out_ids,
+                            float *out_scores, cudaStream_t st);
 int launch_residual_scores(const Index &ix, const Params &p, const float *queries, const int32_t *table,
                            const int32_t *pruned, float *score4, cudaStream_t st);
 // Tensor-core variant of stage 4 for q_len <= 64; qdig = the query digit planes of stage 1.

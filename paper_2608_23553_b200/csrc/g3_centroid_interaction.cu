@@ -405,8 +405,9 @@ __device__ __forceinline__ int sel_block_scan(int v, int *total, int *warp_part 
 // Radix select (11 + 11 + 10 bits, most significant first) of the `want`-th largest value of sb[0..n) in the order of
 // u = value ^ 0x80000000.  Needs n >= want >= 1.  Returns that value's u; *need_eq = how many entries equal to it
 // belong to the top `want` (the rest of the top `want` are strictly greater).  Whole block, uniform.
-__device__ __forceinline__ uint32_t radix_select(const int32_t *__restrict__ sb, int n, int want_in, int *hist,
-                                                 int *warp_part, uint32_t *s_prefix, int *s_want, int *need_eq)
+template <class Load>     // load(j) = value j (int32)
+__device__ __forceinline__ uint32_t radix_select(Load load, int n, int want_in, int *hist, int *warp_part,
+                                                 uint32_t *s_prefix, int *s_want, int *need_eq)
 {
     if (threadIdx.x == 0) { *s_prefix = 0u; *s_want = want_in; }
     const int shifts[3] = {21, 10, 0};
@@ -424,7 +425,7 @@ __device__ __forceinline__ uint32_t radix_select(const int32_t *__restrict__ sb,
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const int j = base + e * SEL_THREADS + threadIdx.x;
-                u[e] = j < n ? ((uint32_t)sb[j] ^ 0x80000000u) : 0u;
+                u[e] = j < n ? ((uint32_t)load(j) ^ 0x80000000u) : 0u;
             }
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -456,10 +457,12 @@ __device__ __forceinline__ uint32_t radix_select(const int32_t *__restrict__ sb,
     return *s_prefix;
 }
 
-// grid (B).  pruned[b][0..n_prune) ascending ids, -1 padded; n_pruned[b].  
+// grid (B).  pruned[b][0..n_prune) ascending ids, -1 padded; n_pruned[b]; pruned_ci (optional): the score of each
+// kept document, INT_MIN beside every -1.
 __global__ void __launch_bounds__(SEL_THREADS)
 select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, const int32_t *__restrict__ ci,
-              int64_t maxc, int n_prune, int32_t *__restrict__ pruned, int32_t *__restrict__ n_pruned)
+              int64_t maxc, int n_prune, int32_t *__restrict__ pruned, int32_t *__restrict__ n_pruned,
+              int32_t *__restrict__ pruned_ci)
 {
     __shared__ int hist[2048];
     __shared__ int warp_part[32];
@@ -470,14 +473,19 @@ select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_ca
     const int32_t *cb = cand + (int64_t)b * maxc;
     const int32_t *sb = ci + (int64_t)b * maxc;
     int32_t *out = pruned + (int64_t)b * n_prune;
+    int32_t *out_ci = pruned_ci ? pruned_ci + (int64_t)b * n_prune : nullptr;
 
     if (n <= n_prune) {
-        for (int j = threadIdx.x; j < n_prune; j += SEL_THREADS) out[j] = j < n ? cb[j] : -1;
+        for (int j = threadIdx.x; j < n_prune; j += SEL_THREADS) {
+            out[j] = j < n ? cb[j] : -1;
+            if (out_ci) out_ci[j] = j < n ? sb[j] : INT_MIN;
+        }
         if (threadIdx.x == 0) n_pruned[b] = n;
         return;
     }
     int need_eq;
-    const uint32_t thr = radix_select(sb, n, n_prune, hist, warp_part, &s_prefix, &s_want, &need_eq);
+    const uint32_t thr = radix_select([&](int j) { return sb[j]; }, n, n_prune, hist, warp_part, &s_prefix, &s_want,
+                                      &need_eq);
 
     // Ordered compaction: keep u > thr, and the first need_eq entries with u == thr.  Each thread owns four
     // consecutive entries per round, so one block scan covers 4096 entries.
@@ -505,8 +513,11 @@ select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_ca
         for (int e = 0; e < 4; ++e) {
             if (j0 + e >= n) break;
             const bool is_gt = u[e] > thr, is_eq = u[e] == thr;
-            if (is_gt || (is_eq && eq_before < need_eq))
-                out[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = id[e];
+            if (is_gt || (is_eq && eq_before < need_eq)) {
+                const int pos = gt_before + (eq_before < need_eq ? eq_before : need_eq);
+                out[pos] = id[e];
+                if (out_ci) out_ci[pos] = (int32_t)(u[e] ^ 0x80000000u);
+            }
             gt_before += is_gt ? 1 : 0;
             eq_before += is_eq ? 1 : 0;
         }
@@ -596,6 +607,89 @@ contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n
     if (threadIdx.x == 0) n_cont[b] = run;
 }
 
+// Document-sharded search, grid (B): the global top n_prune of the shards' local top-n_prune lists.  all_ids / all_ci
+// are [world][B][n_prune] (global document ids ascending within a shard, -1 / INT_MIN padded); shards own ascending,
+// disjoint id ranges in rank order, so walking rank by rank visits the valid entries in ascending id order and ties
+// resolve towards the smaller id exactly as in select_kernel.  Of the selected documents this shard keeps its own
+// (ids in [doc_base, doc_base + n_local)) as local ids: pruned[b][0..n_prune) ascending, -1 padded; n_pruned[b].
+__global__ void __launch_bounds__(SEL_THREADS)
+shard_select_kernel(const int32_t *__restrict__ all_ids, const int32_t *__restrict__ all_ci, int world, int B,
+                    int n_prune, long long doc_base, long long n_local, int32_t *__restrict__ pruned,
+                    int32_t *__restrict__ n_pruned)
+{
+    __shared__ int hist[2048];
+    __shared__ int warp_part[32];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_want;
+    const int b = blockIdx.x;
+    const int n = world * n_prune;
+    auto at = [&](int j) { return ((int64_t)(j / n_prune) * B + b) * n_prune + j % n_prune; };
+    int32_t *out = pruned + (int64_t)b * n_prune;
+
+    // number of valid entries
+    int valid = 0;
+    for (int j = threadIdx.x; j < n; j += SEL_THREADS) valid += all_ids[at(j)] >= 0 ? 1 : 0;
+    int total_valid;
+    sel_block_scan(valid, &total_valid, warp_part);
+    uint32_t thr = 0u;              // keep everything valid
+    int need_eq = 0;
+    if (total_valid > n_prune)
+        thr = radix_select([&](int j) { return all_ci[at(j)]; }, n, n_prune, hist, warp_part, &s_prefix, &s_want,
+                           &need_eq);
+    const bool keep_all = total_valid <= n_prune;
+
+    int run_eq = 0, run_own = 0;
+    for (int base = 0; base < n; base += 4 * SEL_THREADS) {
+        const int j0 = base + 4 * threadIdx.x;
+        uint32_t u[4];
+        int32_t id[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = j0 + e;
+            id[e] = j < n ? all_ids[at(j)] : -1;
+            u[e] = id[e] >= 0 ? ((uint32_t)all_ci[at(j)] ^ 0x80000000u) : 0u;
+        }
+        int eq = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) eq += (id[e] >= 0 && !keep_all && u[e] == thr) ? 1 : 0;
+        int total_eq;
+        int eq_before = run_eq + sel_block_scan(eq, &total_eq, warp_part);
+        bool own[4];
+        int n_own = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            bool kept = id[e] >= 0;
+            if (kept && !keep_all) {
+                const bool is_eq = u[e] == thr;
+                kept = u[e] > thr || (is_eq && eq_before < need_eq);
+                eq_before += is_eq ? 1 : 0;
+            }
+            own[e] = kept && id[e] >= doc_base && id[e] < doc_base + n_local;
+            n_own += own[e] ? 1 : 0;
+        }
+        int total_own;
+        int pos = run_own + sel_block_scan(n_own, &total_own, warp_part);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (own[e]) out[pos++] = (int32_t)(id[e] - doc_base);
+        run_eq += total_eq;
+        run_own += total_own;
+    }
+    for (int j = run_own + threadIdx.x; j < n_prune; j += SEL_THREADS) out[j] = -1;
+    if (threadIdx.x == 0) n_pruned[b] = run_own;
+}
+
+int launch_shard_select(const Params &p, const int32_t *all_ids, const int32_t *all_ci, int world, int64_t doc_base,
+                        int64_t n_local, int32_t *pruned, int32_t *n_pruned, cudaStream_t st)
+{
+    shard_select_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(all_ids, all_ci, world, p.B, p.n_prune,
+                                                               (long long)doc_base, (long long)n_local, pruned,
+                                                               n_pruned);
+    CHIMERA_CUDA(cudaGetLastError());
+    count_launch(SLOT_SELECT);
+    return CHIMERA_OK;
+}
+
 int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
                       const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st)
 {
@@ -608,10 +702,11 @@ int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, con
 }
 
 int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
-                  int32_t *pruned, int32_t *n_pruned, cudaStream_t st)
+                  int32_t *pruned, int32_t *n_pruned, int32_t *pruned_ci, cudaStream_t st)
 {
     (void)ix;
-    select_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, ci, p.maxc, p.n_prune, pruned, n_pruned);
+    select_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, ci, p.maxc, p.n_prune, pruned, n_pruned,
+                                                         pruned_ci);
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_SELECT);
     return CHIMERA_OK;

@@ -25,19 +25,26 @@ __device__ __forceinline__ float float_unorder(uint32_t o)
     return __uint_as_float(u);
 }
 
+// Entry j of query b.  A query's entries are one run of n_prune (seg_len = n_prune) or, for the merge of several
+// shards' lists laid out [shard][query][seg_len], one run of seg_len per shard, seg_stride apart.
+__device__ __forceinline__ int64_t entry_index(int j, int b, int seg_len, long long seg_stride)
+{
+    return (int64_t)(j / seg_len) * seg_stride + (int64_t)b * seg_len + j % seg_len;
+}
+
 __global__ void __launch_bounds__(TOPK_THREADS)
 topk_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ score4, int n_prune, int n_pow2, int k,
-            int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
+            int seg_len, long long seg_stride, int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
 {
     extern __shared__ unsigned long long keys[];
     const int b = blockIdx.x;
     for (int j = threadIdx.x; j < n_pow2; j += TOPK_THREADS) {
         unsigned long long key = 0ull;
         if (j < n_prune) {
-            int32_t id = pruned[(int64_t)b * n_prune + j];
+            const int64_t at = entry_index(j, b, seg_len, seg_stride);
+            int32_t id = pruned[at];
             if (id >= 0)
-                key = ((unsigned long long)float_order(score4[(int64_t)b * n_prune + j]) << 32) |
-                      (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
+                key = ((unsigned long long)float_order(score4[at]) << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
         }
         keys[j] = key;
     }
@@ -69,7 +76,7 @@ topk_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ score4
 template <int KPT>      // keys per thread: n_prune <= KPT * TOPK_THREADS
 __global__ void __launch_bounds__(TOPK_THREADS)
 topk_small_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ score4, int n_prune, int k,
-                  int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
+                  int seg_len, long long seg_stride, int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
 {
     __shared__ unsigned long long warp_max[32];
     __shared__ unsigned long long s_win;
@@ -80,10 +87,10 @@ topk_small_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ 
         const int j = e * TOPK_THREADS + threadIdx.x;
         keys[e] = 0ull;
         if (j < n_prune) {
-            const int32_t id = pruned[(int64_t)b * n_prune + j];
+            const int64_t at = entry_index(j, b, seg_len, seg_stride);
+            const int32_t id = pruned[at];
             if (id >= 0)
-                keys[e] = ((unsigned long long)float_order(score4[(int64_t)b * n_prune + j]) << 32) |
-                          (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
+                keys[e] = ((unsigned long long)float_order(score4[at]) << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
         }
     }
     for (int r = 0; r < k; ++r) {
@@ -118,30 +125,52 @@ topk_small_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ 
     }
 }
 
+// n entries per query (laid out by entry_index) -> the best k.
+static int launch_topk_entries(const int32_t *ids, const float *scores, int B, int n, int k, int seg_len,
+                               long long seg_stride, int32_t *out_ids, float *out_scores, cudaStream_t st)
+{
+    if (k <= 16 && n <= 16 * TOPK_THREADS) {
+        if (n <= TOPK_THREADS)
+            topk_small_kernel<1><<<(unsigned)B, TOPK_THREADS, 0, st>>>(ids, scores, n, k, seg_len, seg_stride, out_ids,
+                                                                       out_scores);
+        else if (n <= 4 * TOPK_THREADS)
+            topk_small_kernel<4><<<(unsigned)B, TOPK_THREADS, 0, st>>>(ids, scores, n, k, seg_len, seg_stride, out_ids,
+                                                                       out_scores);
+        else
+            topk_small_kernel<16><<<(unsigned)B, TOPK_THREADS, 0, st>>>(ids, scores, n, k, seg_len, seg_stride, out_ids,
+                                                                        out_scores);
+        CHIMERA_CUDA(cudaGetLastError());
+        return CHIMERA_OK;
+    }
+    int n_pow2 = 2;
+    while (n_pow2 < n) n_pow2 <<= 1;
+    const size_t smem = sizeof(unsigned long long) * (size_t)n_pow2;
+    if (smem > 128 * 1024) return fail(CHIMERA_UNSUPPORTED, "top-k over %d entries per query does not fit shared memory", n);
+    if (smem > 48 * 1024)
+        CHIMERA_CUDA(cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    topk_kernel<<<(unsigned)B, TOPK_THREADS, smem, st>>>(ids, scores, n, n_pow2, k, seg_len, seg_stride, out_ids,
+                                                         out_scores);
+    CHIMERA_CUDA(cudaGetLastError());
+    return CHIMERA_OK;
+}
+
 int launch_topk(const Index &ix, const Params &p, const int32_t *pruned, const float *score4, int32_t *out_ids,
                 float *out_scores, cudaStream_t st)
 {
     (void)ix;
-    if (p.k <= 16) {
-        const unsigned B = (unsigned)p.B;
-        if (p.n_prune <= TOPK_THREADS)
-            topk_small_kernel<1><<<B, TOPK_THREADS, 0, st>>>(pruned, score4, p.n_prune, p.k, out_ids, out_scores);
-        else if (p.n_prune <= 4 * TOPK_THREADS)
-            topk_small_kernel<4><<<B, TOPK_THREADS, 0, st>>>(pruned, score4, p.n_prune, p.k, out_ids, out_scores);
-        else
-            topk_small_kernel<16><<<B, TOPK_THREADS, 0, st>>>(pruned, score4, p.n_prune, p.k, out_ids, out_scores);
-        CHIMERA_CUDA(cudaGetLastError());
-        count_launch(SLOT_TOPK);
-        return CHIMERA_OK;
-    }
-    int n_pow2 = 2;
-    while (n_pow2 < p.n_prune) n_pow2 <<= 1;
-    const size_t smem = sizeof(unsigned long long) * (size_t)n_pow2;
-    if (smem > 48 * 1024)
-        CHIMERA_CUDA(cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    topk_kernel<<<(unsigned)p.B, TOPK_THREADS, smem, st>>>(pruned, score4, p.n_prune, n_pow2, p.k, out_ids,
-                                                           out_scores);
-    CHIMERA_CUDA(cudaGetLastError());
+    const int rc = launch_topk_entries(pruned, score4, p.B, p.n_prune, p.k, p.n_prune, 0, out_ids, out_scores, st);
+    if (rc) return rc;
+    count_launch(SLOT_TOPK);
+    return CHIMERA_OK;
+}
+
+// Final merge of a document-sharded search: all_ids / all_scores are the shards' top-k lists, [world][B][k] (global
+// ids, -1 / -inf padded); out = the best k of their union per query, (score desc, id asc).
+int launch_shard_merge_topk(const int32_t *all_ids, const float *all_scores, int world, int B, int k, int32_t *out_ids,
+                            float *out_scores, cudaStream_t st)
+{
+    const int rc = launch_topk_entries(all_ids, all_scores, B, world * k, k, k, (long long)B * k, out_ids, out_scores, st);
+    if (rc) return rc;
     count_launch(SLOT_TOPK);
     return CHIMERA_OK;
 }
