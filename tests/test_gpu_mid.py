@@ -68,3 +68,29 @@ def test_mid_score_table_sampled_rows_match_oracle(mid):
     gix.run_stages(1, 1, q[5:7].contiguous(), B, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k, taps)
     S = oracle.score_table(q[5].cpu().numpy(), oix.centroids)
     assert np.array_equal(taps.score_table[0].cpu().numpy(), S)
+
+
+def test_mid_batch256_four_document_shards_equal_the_single_index(mid):
+    """The document-sharded search at the benchmark's size: four shards of 125k documents, their phases run one after
+    the other on this GPU, merged ids and scores equal the single index's for every query."""
+    import paper_2608_23553_b200 as pkg
+    from paper_2608_23553_b200.sharded import ShardEngine, shard_ranges
+    cfg, corp, gix, oix, q = mid
+    qb = q[:256].contiguous()
+    ref_ids, ref_sc = gix.search(qb, cfg.nprobe, cfg.n_prune, cfg.k)
+    off = torch.cat([torch.zeros(1, dtype=torch.int64, device=qb.device), torch.cumsum(corp.doclens.to(torch.int64), 0)])
+    engines = []
+    for lo, hi in shard_ranges(cfg.n_docs, 4):
+        t0, t1 = int(off[lo]), int(off[hi])
+        ix = pkg.Index(corp.centroids, corp.cids[t0:t1].contiguous(), corp.codes[t0:t1].contiguous(),
+                       corp.doclens[lo:hi].contiguous(), cfg.nbits, cfg.res_lo, cfg.res_hi)
+        engines.append(ShardEngine(ix, lo, "ci"))
+    local = [e.local_phase(qb, cfg.nprobe, cfg.n_prune, cfg.k) for e in engines]
+    for e in engines:
+        e.check()
+    all_ids = torch.stack([l[0] for l in local]).contiguous()
+    all_sc3 = torch.stack([l[1] for l in local]).contiguous()
+    tops = [e.finish_phase(qb, cfg.nprobe, cfg.n_prune, cfg.k, all_ids, all_sc3) for e in engines]
+    ids, sc = engines[0].merge_phase(torch.stack([t[0] for t in tops]).contiguous(),
+                                     torch.stack([t[1] for t in tops]).contiguous())
+    assert torch.equal(ids, ref_ids) and torch.equal(sc, ref_sc)
