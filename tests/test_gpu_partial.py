@@ -30,6 +30,7 @@ def _check(gix, oix, q, nprobe, n_prune, k, sample=None, max_diffs=0):
     (96, 2, 64, 48, 300, 8, 40, 12),
     (96, 1, 40, 48, 300, 3, 33, 5),
     (64, 2, 100, 32, 200, 32, 64, 20),       # every list probed: F' is the full low-bit score
+    (32, 2, 6, 4, 1500, 2, 50, 10),          # four long lists of ~2,500 tokens each
 ])
 def test_partial_refinement_small_corpora(D, nbits, nq, K, N, nprobe, n_prune, k):
     import paper_2608_23553_b200 as pkg
