@@ -8,8 +8,8 @@
 // int32; the three planes are recombined in fp32 (relative error 2^-24).
 //
 // A CTA owns one query and a run of its surviving documents, whose tokens form one stream cut into tiles of 128
-// (MMA M).  Per tile: every thread expands the packed code of one token through a 256-entry byte table into a 128-byte
-// int8 row and stores it, 128-byte swizzled, into the A tile; one thread issues D/32 MMAs (N = 3 * padded q_len: the
+// (MMA M).  Per tile: every thread expands the packed code of one token into a 128-byte int8 row (two integer
+// multiplications and two masks per four dimensions) and stores it, 128-byte swizzled, into the A tile; one thread issues D/32 MMAs (N = 3 * padded q_len: the
 // three digit planes side by side, loaded once per CTA by TMA); the accumulators come back with tcgen05.ld, get the
 // centroid term from the stage-1 table, and go to shared memory, where each warp folds its 32 tokens into per-document
 // maxima.  Tensor memory: 128 or 256 columns per CTA, so several CTAs share an SM and overlap each other's phases.
@@ -34,6 +34,17 @@ __device__ __forceinline__ float f_unorder(uint32_t o)
 {
     return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
 }
+
+// One code byte (four 2-bit bucket indices, dimension 4g+t in bits [2t, 2t+1]) -> four int8 values, one per byte.
+// Both multiplications only place copies at disjoint bit positions, so they are shifts-and-ors without carries.
+__device__ __forceinline__ uint32_t spread2(uint32_t byte)
+{
+    const uint32_t x = (byte * 0x1001u) & 0x000F000Fu;       // low nibble at bit 0, high nibble at bit 16
+    return (x * 0x41u) & 0x03030303u;                        // second index of each nibble moved up one byte
+}
+// Four 1-bit codes (a nibble, dimension t in bit t) -> four int8 values 0/1: bit t lands at bit 8t of the product
+// (the other copies fall on bits that the mask drops; all partial products occupy distinct bits).
+__device__ __forceinline__ uint32_t spread1(uint32_t nibble) { return (nibble * 0x00204081u) & 0x01010101u; }
 
 // RQ = true scores RaBitQ 1-bit codes instead (Sec. 2.2; the GPU half of the paper's document scoring): the same
 // contraction T = sum_x Xq[x] b[x] against the digit planes of the ROTATED query, then
@@ -68,8 +79,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     const uint32_t sA = base, sB = base + A_BYTES;
     float *vals = reinterpret_cast<float *>(gen + A_BYTES + B_BYTES);                       // [128][VP]
     uint32_t *docmax = reinterpret_cast<uint32_t *>(vals + G4U_TOK * VP);                  // [MAX_DOCS][NQP]
-    uint32_t *lut = docmax + G4U_MAX_DOCS * NQP;                                           // 256 or 512 words
-    const uint32_t bars = smem_u32(lut + (NBITS == 2 ? 256 : 512));
+    const uint32_t bars = smem_u32(docmax + G4U_MAX_DOCS * NQP);
     const uint32_t bar_b = (bars + 7u) & ~7u, bar_mma = bar_b + 8;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -110,19 +120,6 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     if (warp == 0) {
         __syncwarp();
         tmem_alloc(&s_tmem_base, TMEM_COLS);
-    }
-    // byte -> int8 bucket indices
-    if (NBITS == 2) {
-        for (int v = tid; v < 256; v += G4U_THREADS)
-            lut[v] = (uint32_t)(v & 3) | ((uint32_t)((v >> 2) & 3) << 8) | ((uint32_t)((v >> 4) & 3) << 16) |
-                     ((uint32_t)((v >> 6) & 3) << 24);
-    } else {
-        for (int v = tid; v < 256; v += G4U_THREADS) {
-            lut[2 * v] = (uint32_t)(v & 1) | ((uint32_t)((v >> 1) & 1) << 8) | ((uint32_t)((v >> 2) & 1) << 16) |
-                         ((uint32_t)((v >> 3) & 1) << 24);
-            lut[2 * v + 1] = (uint32_t)((v >> 4) & 1) | ((uint32_t)((v >> 5) & 1) << 8) |
-                             ((uint32_t)((v >> 6) & 1) << 16) | ((uint32_t)((v >> 7) & 1) << 24);
-        }
     }
     for (int e = tid; e < G4U_MAX_DOCS * NQP; e += G4U_THREADS) docmax[e] = 0u;     // below every real value
     // sum_x q_i[x] per query token: four threads per row, each a quarter of the row with 16-byte loads
@@ -220,21 +217,20 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                 if (w < CW) {
                     const uint32_t word = cw[w];
                     if (NBITS == 2) {
-                        const uint32_t c0 = lut[word & 255u], c1 = lut[(word >> 8) & 255u],
-                                       c2 = lut[(word >> 16) & 255u], c3 = lut[word >> 24];
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)w ^ sw) << 4)),
-                                     "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                                     "r"(spread2(word & 255u)), "r"(spread2((word >> 8) & 255u)),
+                                     "r"(spread2((word >> 16) & 255u)), "r"(spread2(word >> 24))
                                      : "memory");
                     } else {
-                        const uint32_t b0 = word & 255u, b1 = (word >> 8) & 255u, b2 = (word >> 16) & 255u,
-                                       b3 = word >> 24;
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(
                                          row + (((uint32_t)(2 * w) ^ sw) << 4)),
-                                     "r"(lut[2 * b0]), "r"(lut[2 * b0 + 1]), "r"(lut[2 * b1]), "r"(lut[2 * b1 + 1])
+                                     "r"(spread1(word & 15u)), "r"(spread1((word >> 4) & 15u)),
+                                     "r"(spread1((word >> 8) & 15u)), "r"(spread1((word >> 12) & 15u))
                                      : "memory");
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(
                                          row + (((uint32_t)(2 * w + 1) ^ sw) << 4)),
-                                     "r"(lut[2 * b2]), "r"(lut[2 * b2 + 1]), "r"(lut[2 * b3]), "r"(lut[2 * b3 + 1])
+                                     "r"(spread1((word >> 16) & 15u)), "r"(spread1((word >> 20) & 15u)),
+                                     "r"(spread1((word >> 24) & 15u)), "r"(spread1(word >> 28))
                                      : "memory");
                     }
                 }
@@ -381,7 +377,7 @@ static int launch_g4_umma(const Index &ix, const Params &p, const float *queries
     int rc = make_plane_map(&map_q, qdig, (int64_t)p.B * p.nq, NQP);
     if (rc) return rc;
     const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 + sizeof(float) * G4U_TOK * (NQP + 1) +
-                        sizeof(uint32_t) * G4U_MAX_DOCS * NQP + sizeof(uint32_t) * (NBITS == 2 ? 256 : 512) + 32;
+                        sizeof(uint32_t) * G4U_MAX_DOCS * NQP + 32;
     auto kern = residual_maxsim_umma<NQP, NBITS, RQ>;
     CHIMERA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // documents per CTA: about four CTAs per SM in total, at most 32 documents each (with few queries per call a CTA
