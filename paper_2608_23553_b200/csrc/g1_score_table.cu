@@ -30,13 +30,15 @@ constexpr uint32_t G1_A_PLANE = G1_M * G1_ROW_BYTES;      // 16 KB
 constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;      // 6 KB
 constexpr uint32_t G1_SMEM = 3 * G1_A_PLANE + 2 * 3 * G1_B_PLANE + 1024 /* alignment slack */ + 64 /* barriers */;
 
-// floor((a0 + 2^8 a1 + 2^16 a2 + 2^24 a3 + 2^32 a4 + 2^19) / 2^20).  The two high terms are multiples of 2^20, so they
-// contribute 2^4 a3 + 2^12 a4 exactly (32-bit wrap-around is harmless: the result fits int32); only the low three need
-// 64 bits.
+// floor((a0 + 2^8 a1 + 2^16 a2 + 2^24 a3 + 2^32 a4 + 2^19) / 2^20) in 32-bit arithmetic.  The two high terms are
+// multiples of 2^20 and contribute 2^4 a3 + 2^12 a4.  With a1 = 2^12 h1 + l1 (0 <= l1 < 2^12) and a2 = 2^4 h2 + l2
+// (0 <= l2 < 2^4) -- arithmetic shifts, so this also holds for negative values -- the middle terms are
+// 2^20 (h1 + h2) + 2^8 l1 + 2^16 l2, and what is left under the floor, a0 + 2^8 l1 + 2^16 l2 + 2^19, is below 2^24
+// in magnitude (|a0| < 2^23).  32-bit wrap-around of the sum is harmless: the result fits int32.
 __device__ __forceinline__ int32_t combine_digits(int32_t a0, int32_t a1, int32_t a2, int32_t a3, int32_t a4)
 {
-    const long long low = (long long)a0 + (long long)a1 * 256LL + (long long)a2 * 65536LL + (1LL << 19);
-    return (int32_t)(low >> 20) + a3 * 16 + a4 * 4096;
+    const int32_t inner = a0 + ((a1 & 4095) << 8) + ((a2 & 15) << 16) + (1 << 19);
+    return (inner >> 20) + (a1 >> 12) + (a2 >> 4) + a3 * 16 + a4 * 4096;
 }
 
 // grid (ceil(K / 128), n_splits).  Each CTA: centroid tile blockIdx.x, query-row tiles [blockIdx.y * tiles_per_split, ...).
@@ -138,19 +140,19 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
         const int64_t c = c0 + quad * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
         const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
-#pragma unroll 1
-        for (int chunk = warp >> 2; chunk < G1_N / 8; chunk += 2) {
-            int32_t acc[5][8];
-#pragma unroll
-            for (int w = 0; w < 5; ++w) tmem_ld8(lane_addr + w * G1_N + chunk * 8, acc[w]);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        // (query, token) coordinates of the tile's first row: one 32-bit division per tile
+        const uint32_t tile_qb = ((uint32_t)t * G1_N) / unq, tile_qi = (uint32_t)t * G1_N - tile_qb * unq;
+        // The two warps of a lane quarter take alternate chunks (three each).  The tensor-memory loads of the next
+        // chunk are issued before the current one is recombined and stored, so their latency hides behind that work.
+        auto emit = [&](const int32_t (&acc)[5][8], const int chunk) {
             int32_t out[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) out[e] = combine_digits(acc[0][e], acc[1][e], acc[2][e], acc[3][e], acc[4][e]);
             // first query-token row of this chunk and its (query, token) coordinates (rows fit 32 bits:
             // n_queries * q_len < 2^23)
             const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)chunk * 8;
-            uint32_t qb = r0 / unq, qi = r0 - qb * unq;
+            uint32_t qb = tile_qb, qi = tile_qi + (uint32_t)chunk * 8;      // chunk * 8 < 48: few subtractions
+            while (qi >= unq) { qi -= unq; ++qb; }
             if (c < K && r0 < rows32) {
                 if (table8 != nullptr) {
                     // coarse copy for the bound phase of stage 3: min((S + 2^24 + 64) >> 17, 255); q_len is a multiple
@@ -158,14 +160,10 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                     uint32_t w[2];
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
-                        uint32_t pack = 0;
+                        uint32_t v[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            int v = (out[4 * g + e] + (1 << 24) + 64) >> 17;
-                            v = v > 255 ? 255 : v;
-                            pack |= (uint32_t)v << (8 * e);
-                        }
-                        w[g] = pack;
+                        for (int e = 0; e < 4; ++e) v[e] = (uint32_t)min((out[4 * g + e] + (1 << 24) + 64) >> 17, 255);
+                        w[g] = __byte_perm(__byte_perm(v[0], v[1], 0x0040), __byte_perm(v[2], v[3], 0x0040), 0x5410);
                     }
                     *reinterpret_cast<uint2 *>(table8 + ((int64_t)qb * K + c) * nq + qi) = make_uint2(w[0], w[1]);
                 }
@@ -186,6 +184,21 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                     }
                 }
             }
+        };
+        constexpr int CHUNKS_PER_WARP = G1_N / 16;
+        const int first_chunk = warp >> 2;
+        int32_t accs[2][5][8];
+#pragma unroll
+        for (int w = 0; w < 5; ++w) tmem_ld8(lane_addr + w * G1_N + first_chunk * 8, accs[0][w]);
+#pragma unroll
+        for (int it = 0; it < CHUNKS_PER_WARP; ++it) {
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (it + 1 < CHUNKS_PER_WARP) {
+#pragma unroll
+                for (int w = 0; w < 5; ++w)
+                    tmem_ld8(lane_addr + w * G1_N + (first_chunk + 2 * (it + 1)) * 8, accs[(it + 1) & 1][w]);
+            }
+            emit(accs[it & 1], first_chunk + 2 * it);
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();                   // accumulators drained before the next tile overwrites them
