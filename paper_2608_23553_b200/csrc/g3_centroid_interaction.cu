@@ -270,13 +270,12 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
         }
         // every lane now holds the maxima of two columns; sum over columns (skipping duplicate lanes)
         const float2 f = __half22float2(*reinterpret_cast<__half2 *>(&m[0]));
-        int sum = 0, sat = 0;
-        if ((lane & dup_mask) == 0) {
-            sum = (int)(f.x + f.y) - 2048;                      // two halves of 1024 + u, exact
-            sat = (f.x >= 1279.0f) + (f.y >= 1279.0f);
-        }
-        sum = warp_sum(sum);
-        sat = warp_sum(sat);
+        int packed = 0;                                         // sum of maxima | saturated count << 20
+        if ((lane & dup_mask) == 0)
+            packed = ((int)(f.x + f.y) - 2048)                  // two halves of 1024 + u, exact
+                     + (((f.x >= 1279.0f) + (f.y >= 1279.0f)) << 20);
+        packed = __reduce_add_sync(0xffffffffu, packed);        // sum <= 255 * 64 < 2^20, count <= 64
+        const int sum = packed & 0xfffff, sat = packed >> 20;
         if (lane == 0) {
             const int l = (sum - 128 * NQ) * (1 << 17) - 64 * NQ;
             lo[(int64_t)b * maxc + j] = l;
