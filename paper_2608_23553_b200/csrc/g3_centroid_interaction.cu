@@ -15,7 +15,6 @@
 // select_kernel: one block per query.  Radix select (11 + 11 + 10 bits) of the n_prune-th largest CI, then an
 // ordered compaction of the candidate list (which is ascending in id), so equal scores are resolved towards smaller
 // ids and the survivors come out ascending.
-#include <cuda_fp16.h>
 #include <limits.h>
 
 #include "common.cuh"
@@ -115,11 +114,11 @@ ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__re
                     v[u] = __ldg(tb + (int64_t)c * LPR);
                 }
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    m.x = max(m.x, v[u].x);
-                    m.y = max(m.y, v[u].y);
-                    m.z = max(m.z, v[u].z);
-                    m.w = max(m.w, v[u].w);
+                for (int u = 0; u < UNROLL; u += 2) {          // three-input integer maximum: two rows per instruction
+                    m.x = __vimax3_s32(m.x, v[u].x, v[u + 1].x);
+                    m.y = __vimax3_s32(m.y, v[u].y, v[u + 1].y);
+                    m.z = __vimax3_s32(m.z, v[u].z, v[u + 1].z);
+                    m.w = __vimax3_s32(m.w, v[u].w, v[u + 1].w);
                 }
             }
         }
@@ -145,23 +144,18 @@ ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__re
 //     lo(d) = sum_i (2^17 m_i - 2^24 - 64)  <=  CI(d)  <=  lo(d) + nq (2^17 - 1) + 2^18 #{i : m_i = 255} = hi(d)
 // (the last term covers the saturated top bucket).  A row of U8 is q_len bytes -- one 32-byte sector for 32 query
 // tokens instead of four -- and a lane's 16-byte load covers 16 query tokens, so one warp load covers 32 / LPR tokens
-// (LPR = q_len / 16 lanes per row).  Bytes are widened to fp16 with one byte-permute per pair (0x64xx = 1024 + x,
-// exact) so that the running maxima use the native packed-half max.
-__device__ __forceinline__ uint32_t hmax2_bits(uint32_t a, uint32_t b)
+// (LPR = q_len / 16 lanes per row).  Bytes are widened to pairs of 16-bit integers with one byte-permute per pair and
+// the running maxima fold two rows per instruction with the three-input packed 16-bit integer maximum.
+__device__ __forceinline__ void coarse_accumulate2(uint32_t (&m)[8], const int4 &va, const int4 &vb)
 {
-    __half2 r = __hmax2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b));
-    return *reinterpret_cast<uint32_t *>(&r);
-}
-__device__ __forceinline__ void coarse_accumulate(uint32_t (&m)[8], const int4 &v)
-{
-    const uint32_t w[4] = {(uint32_t)v.x, (uint32_t)v.y, (uint32_t)v.z, (uint32_t)v.w};
+    const uint32_t a[4] = {(uint32_t)va.x, (uint32_t)va.y, (uint32_t)va.z, (uint32_t)va.w};
+    const uint32_t b[4] = {(uint32_t)vb.x, (uint32_t)vb.y, (uint32_t)vb.z, (uint32_t)vb.w};
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        m[2 * k] = hmax2_bits(m[2 * k], __byte_perm(w[k], 0x64646464u, 0x4140));         // bytes 0, 1
-        m[2 * k + 1] = hmax2_bits(m[2 * k + 1], __byte_perm(w[k], 0x64646464u, 0x4342)); // bytes 2, 3
+        m[2 * k] = __vimax3_u16x2(m[2 * k], __byte_perm(a[k], 0u, 0x4140), __byte_perm(b[k], 0u, 0x4140));
+        m[2 * k + 1] = __vimax3_u16x2(m[2 * k + 1], __byte_perm(a[k], 0u, 0x4342), __byte_perm(b[k], 0u, 0x4342));
     }
 }
-
 // SMEM = true: the query's whole 8-bit table (K * q_len bytes) is first staged in shared memory and the row lookups
 // are shared-memory loads (small K only); blocks are then larger (THREADS) because only one fits an SM.
 template <int LPR, bool SMEM, int THREADS>
@@ -213,7 +207,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
         if (j + warps_per_query < n) prefetch(j + warps_per_query);
         uint32_t m[8];
 #pragma unroll
-        for (int r = 0; r < 8; ++r) m[r] = 0x64006400u;       // 1024 + 0 in both halves
+        for (int r = 0; r < 8; ++r) m[r] = 0u;
         for (int64_t base = t0; base < t1; base += 32 * SLABS) {
             // up to SLABS 32-token slabs per iteration, all their row loads in flight together; lanes past the end
             // repeat the last token (harmless for a maximum)
@@ -240,7 +234,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
             for (int k = 0; k < SLABS; ++k) {
                 if (k == 0 || base + 32 * k < t1) {
 #pragma unroll
-                    for (int s = 0; s < STEPS; ++s) coarse_accumulate(m, v[k * STEPS + s]);
+                    for (int s = 0; s < STEPS; s += 2) coarse_accumulate2(m, v[k * STEPS + s], v[k * STEPS + s + 1]);
                 }
             }
         }
@@ -259,21 +253,20 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
                     if (r < half) {
                         const uint32_t send = up ? m[r] : m[r + half];
                         const uint32_t keep = up ? m[r + half] : m[r];
-                        m[r] = hmax2_bits(keep, __shfl_xor_sync(0xffffffffu, send, o));
+                        m[r] = __vmaxu2(keep, __shfl_xor_sync(0xffffffffu, send, o));
                     }
                 }
                 nreg = half;
             } else {
-                m[0] = hmax2_bits(m[0], __shfl_xor_sync(0xffffffffu, m[0], o));
+                m[0] = __vmaxu2(m[0], __shfl_xor_sync(0xffffffffu, m[0], o));
                 dup_mask |= (uint32_t)o;
             }
         }
         // every lane now holds the maxima of two columns; sum over columns (skipping duplicate lanes)
-        const float2 f = __half22float2(*reinterpret_cast<__half2 *>(&m[0]));
+        const int u_lo = (int)(m[0] & 0xffffu), u_hi = (int)(m[0] >> 16);
         int packed = 0;                                         // sum of maxima | saturated count << 20
         if ((lane & dup_mask) == 0)
-            packed = ((int)(f.x + f.y) - 2048)                  // two halves of 1024 + u, exact
-                     + (((f.x >= 1279.0f) + (f.y >= 1279.0f)) << 20);
+            packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 20);
         packed = __reduce_add_sync(0xffffffffu, packed);        // sum <= 255 * 64 < 2^20, count <= 64
         const int sum = packed & 0xfffff, sat = packed >> 20;
         if (lane == 0) {
