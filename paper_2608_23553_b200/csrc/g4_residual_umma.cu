@@ -276,7 +276,8 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             fetch(tile + 1, dl_next, cid_next, cw_next);
             // the next token's score-table row is a scattered 4 * q_len-byte read that misses L2 (a batch's tables
             // are far larger): ask for it now so that HBM latency passes during this tile's epilogue
-            if (!RQ && cid_next >= 0) {
+            // (measured: a gain for q_len <= 32, a loss for the two-line rows of longer queries)
+            if (!RQ && NQP == 32 && cid_next >= 0) {
                 const char *row = reinterpret_cast<const char *>(tb + (int64_t)cid_next * nq);
                 for (int off = 0; off < nq * 4; off += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + off));
             }
