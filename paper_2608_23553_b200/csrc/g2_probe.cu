@@ -43,14 +43,13 @@ probe_partial(const int32_t *__restrict__ table, int64_t K, int nq, int P, int r
     if (col < nq) {
         const int32_t *tb = table + (int64_t)b * K * nq + col;
         int64_t r = r0 + warp;
-        // four independent loads in flight per thread
-        for (; r + 3 * PROBE_WARPS < r1; r += 4 * PROBE_WARPS) {
-            int32_t s0 = tb[r * nq], s1 = tb[(r + PROBE_WARPS) * nq], s2 = tb[(r + 2 * PROBE_WARPS) * nq],
-                    s3 = tb[(r + 3 * PROBE_WARPS) * nq];
-            list_insert(mine, P, key_int(s0, (int32_t)r));
-            list_insert(mine, P, key_int(s1, (int32_t)(r + PROBE_WARPS)));
-            list_insert(mine, P, key_int(s2, (int32_t)(r + 2 * PROBE_WARPS)));
-            list_insert(mine, P, key_int(s3, (int32_t)(r + 3 * PROBE_WARPS)));
+        // sixteen independent loads in flight per thread (the stream is bound by bytes in flight)
+        for (; r + 15 * PROBE_WARPS < r1; r += 16 * PROBE_WARPS) {
+            int32_t sc[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) sc[u] = tb[(r + u * PROBE_WARPS) * nq];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) list_insert(mine, P, key_int(sc[u], (int32_t)(r + u * PROBE_WARPS)));
         }
         for (; r < r1; r += PROBE_WARPS) list_insert(mine, P, key_int(tb[r * nq], (int32_t)r));
     }
