@@ -71,16 +71,39 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
     int32_t *Mb = M + (int64_t)b * maxc * nq;
     constexpr int DPW = 32 / NBITS;
     constexpr uint32_t MASK = (1u << NBITS) - 1u;
-    for (int64_t e = tok_off[c] + threadIdx.x; e < tok_off[c + 1]; e += PS_THREADS) {
-        const int64_t t = tok_id[e];
-        const uint32_t d = (uint32_t)tok_doc[e];
+    // One visit: the token's packed code (16-byte loads where the code size allows) against the query token's integers.
+    auto code_dot = [&](int64_t t) -> int {
         const uint32_t *cw = codes + t * CW;
-        int T = 0;                                     // |T| <= 3 * 2^22 * |q|_1 < 2^31 for unit-norm queries
-        for (int w = 0; w < CW; ++w) {
-            const uint32_t word = __ldg(cw + w);
+        uint32_t word[8];                              // at most 32 code bytes per token
+        if ((CW & 3) == 0) {
 #pragma unroll
-            for (int s = 0; s < DPW; ++s) T += xq[w * DPW + s] * (int)((word >> (s * NBITS)) & MASK);
+            for (int w = 0; w < 8; w += 4)
+                if (w < CW) {
+                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(cw + w));
+                    word[w] = v.x; word[w + 1] = v.y; word[w + 2] = v.z; word[w + 3] = v.w;
+                }
+        } else if ((CW & 1) == 0) {
+#pragma unroll
+            for (int w = 0; w < 8; w += 2)
+                if (w < CW) {
+                    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(cw + w));
+                    word[w] = v.x; word[w + 1] = v.y;
+                }
+        } else {
+#pragma unroll
+            for (int w = 0; w < 8; ++w)
+                if (w < CW) word[w] = __ldg(cw + w);
         }
+        int T = 0;                                     // |T| <= 3 * 2^22 * |q|_1 < 2^31 for unit-norm queries
+#pragma unroll
+        for (int w = 0; w < 8; ++w)
+            if (w < CW) {
+#pragma unroll
+                for (int s = 0; s < DPW; ++s) T += xq[w * DPW + s] * (int)((word[w] >> (s * NBITS)) & MASK);
+            }
+        return T;
+    };
+    auto update = [&](uint32_t d, int T) {
         const double r = __dadd_rn(__dmul_rn(d4, (double)T), kterm);
         const long long dist = (long long)s_c + __double2ll_rn(r);
         if (dist > 0) {                                // the table starts at 0 (Algorithm 2)
@@ -91,7 +114,18 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
                 if ((int32_t)dist > old) atomicAdd(&fprime[(int64_t)b * maxc + rank], (int32_t)dist - old);
             }
         }
+    };
+    // two visits per thread and iteration, their loads issued together
+    const int64_t e1 = tok_off[c + 1];
+    int64_t e = tok_off[c] + threadIdx.x;
+    for (; e + PS_THREADS < e1; e += 2 * PS_THREADS) {
+        const int64_t ta = tok_id[e], tb2 = tok_id[e + PS_THREADS];
+        const uint32_t da = (uint32_t)tok_doc[e], db = (uint32_t)tok_doc[e + PS_THREADS];
+        const int Ta = code_dot(ta), Tb = code_dot(tb2);
+        update(da, Ta);
+        update(db, Tb);
     }
+    if (e < e1) update((uint32_t)tok_doc[e], code_dot(tok_id[e]));
 }
 
 int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, const float *queries,
