@@ -82,7 +82,12 @@ rabitq_partial_kernel(const float *__restrict__ q_rot, int nq, int D, int P, flo
                       const float *__restrict__ inv_dot, const uint32_t *__restrict__ bitmap,
                       const int32_t *__restrict__ word_rank, int64_t words, int64_t maxc, int32_t *__restrict__ M)
 {
+    // Sec. 4.1's look-up-table form of the binary inner product: for every group of four dimensions the 16 partial
+    // sums of the query token's integers are tabulated once per block (D/4 * 16 entries: cheap next to a list of a few
+    // hundred tokens), so a token costs D/4 table reads and adds instead of a data-dependent loop over its set bits.
+    // Integer sums: the same T in any order.
     __shared__ int32_t xq[128];
+    __shared__ int32_t lut[32 * 16];
     __shared__ int s_sq;
     const int b = blockIdx.y;
     const int i = blockIdx.x / P;
@@ -96,29 +101,56 @@ rabitq_partial_kernel(const float *__restrict__ q_rot, int nq, int D, int P, flo
         for (int x = 0; x < D; ++x) s += xq[x];
         s_sq = s;
     }
+    for (int e = threadIdx.x; e < (D >> 2) * 16; e += RP_THREADS) {
+        const int g = e >> 4, v = e & 15;
+        int s = 0;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) s += ((v >> t) & 1) ? xq[4 * g + t] : 0;
+        lut[e] = s;
+    }
     __syncthreads();
     const int sq = s_sq;
     const int CW = D >> 5;
     const uint32_t *bm = bitmap + (int64_t)b * words;
     const int32_t *wr = word_rank + (int64_t)b * words;
     int32_t *Mb = M + (int64_t)b * maxc * nq;
-    for (int64_t e = tok_off[cen] + threadIdx.x; e < tok_off[cen + 1]; e += RP_THREADS) {
-        const int64_t t = tok_id[e];
-        const uint32_t d = (uint32_t)tok_doc[e];
-        int T = 0;
-        for (int w = 0; w < CW; ++w) {
-            uint32_t word = __ldg(bits + t * CW + w);
-            while (word) {
-                const int s = __ffs(word) - 1;
-                word &= word - 1;
-                T += xq[w * 32 + s];
-            }
+    auto code_dot = [&](int64_t t) -> int {
+        uint32_t word[4];                              // D <= 128: at most four words
+        if (CW == 4) {                                 // 16-byte rows (the attach call checks the alignment)
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(bits + t * 4));
+            word[0] = v.x; word[1] = v.y; word[2] = v.z; word[3] = v.w;
+        } else {
+#pragma unroll
+            for (int w = 0; w < 4; ++w) word[w] = w < CW ? __ldg(bits + t * CW + w) : 0u;
         }
+        int T = 0;
+#pragma unroll
+        for (int w = 0; w < 4; ++w)
+            if (w < CW) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) T += lut[(8 * w + k) * 16 + ((word[w] >> (4 * k)) & 15u)];
+            }
+        return T;
+    };
+    auto update = [&](uint32_t d, int64_t t, int T) {
         const float est = __fmul_rn(inv_dot[t], __fmul_rn(c, (float)(2 * T - sq)));
         if (est > 0.0f) {                              // the table starts at 0 (Algorithm 2)
             const int64_t rank = wr[d >> 5] + __popc(bm[d >> 5] & ((1u << (d & 31)) - 1u));
             if (rank < maxc) atomicMax(&Mb[rank * nq + i], __float_as_int(est));
         }
+    };
+    const int64_t e1 = tok_off[cen + 1];
+    int64_t e = tok_off[cen] + threadIdx.x;
+    for (; e + RP_THREADS < e1; e += 2 * RP_THREADS) {         // two visits per iteration, their loads issued together
+        const int64_t ta = tok_id[e], tb = tok_id[e + RP_THREADS];
+        const uint32_t da = (uint32_t)tok_doc[e], db = (uint32_t)tok_doc[e + RP_THREADS];
+        const int Ta = code_dot(ta), Tb = code_dot(tb);
+        update(da, ta, Ta);
+        update(db, tb, Tb);
+    }
+    if (e < e1) {
+        const int64_t t = tok_id[e];
+        update((uint32_t)tok_doc[e], t, code_dot(t));
     }
 }
 
