@@ -231,7 +231,8 @@ def test_tiny_config_stage_isolated(chimera, tiny):
 
 def test_tiny_config_parameter_grid(chimera, tiny):
     cfg, oix, gix, q = tiny
-    for nprobe, n_prune, k in [(1, 256, 10), (2, 1024, 100), (8, 64, 10), (32, 4096, 1000), (16, 16384, 10)]:
+    for nprobe, n_prune, k in [(1, 256, 10), (2, 1024, 100), (8, 64, 10), (32, 4096, 1000), (16, 16384, 10),
+                               (4, 2048, 16), (6, 300, 17)]:
         # check_topk (inside) allows position swaps only between scores within the tolerance; with k = 1000 of 4096
         # survivors a few fp32 near-ties are expected
         diffs, _, _ = _run_and_check(chimera, gix, oix, q[:2], nprobe, n_prune, k, table=False)
@@ -259,3 +260,13 @@ def test_graphed_search_equals_eager(chimera, tiny):
         ids_g, sc_g = g(qd[b:b + 1])
         torch.cuda.synchronize()
         assert torch.equal(ids_g, ids_e) and torch.equal(sc_g, sc_e)
+
+
+def test_unaligned_queries_are_rejected(chimera, tiny):
+    """The query pointer must be 16-byte aligned (the kernels read rows with 16-byte loads)."""
+    cfg, oix, gix, q = tiny
+    flat = torch.zeros(q[:1].size + 1, dtype=torch.float32, device="cuda")
+    shifted = flat[1:].view(1, cfg.q_len, cfg.dim)            # 4 bytes past an aligned address
+    shifted.copy_(torch.from_numpy(q[:1]))
+    with pytest.raises(chimera.ChimeraError):
+        gix.search(shifted, cfg.nprobe, cfg.n_prune, cfg.k)
