@@ -24,7 +24,9 @@ namespace chimera {
 constexpr int G1_M = 128;            // centroids per tile (MMA M)
 constexpr int G1_N = 48;             // query-token rows per tile (MMA N)
 constexpr int G1_ROW_BYTES = 128;    // digit-plane row pitch = padded dimension count
-constexpr int G1_THREADS = 256;        // two warps per tensor-memory lane quarter: both drain accumulators
+constexpr int G1_WPQ = 3;              // warps per tensor-memory lane quarter that drain the accumulators (2: 1.53 ms,
+                                       // 3: 1.43 ms, 6: 1.76 ms on the Mid corpus at batch 256)
+constexpr int G1_THREADS = 128 * G1_WPQ;
 constexpr int G1_TMEM_COLS = 256;
 constexpr uint32_t G1_A_PLANE = G1_M * G1_ROW_BYTES;      // 16 KB
 constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;      // 6 KB
@@ -134,15 +136,15 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         __syncwarp();
-        // warp w reads tensor-memory lanes 32 (w % 4) ... + 31 (its centroids); the two warps of a lane quarter take
-        // alternate chunks of eight query-token columns
+        // warp w reads tensor-memory lanes 32 (w % 4) ... + 31 (its centroids); the G1_WPQ warps of a lane quarter
+        // take the chunks of eight query-token columns in turn
         const int quad = warp & 3;
         const int64_t c = c0 + quad * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
         const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
         // (query, token) coordinates of the tile's first row: one 32-bit division per tile
         const uint32_t tile_qb = ((uint32_t)t * G1_N) / unq, tile_qi = (uint32_t)t * G1_N - tile_qb * unq;
-        // The two warps of a lane quarter take alternate chunks (three each).  The tensor-memory loads of the next
+        // Each warp takes every G1_WPQ-th chunk.  The tensor-memory loads of the next
         // chunk are issued before the current one is recombined and stored, so their latency hides behind that work.
         auto emit = [&](const int32_t (&acc)[5][8], const int chunk) {
             int32_t out[8];
@@ -185,7 +187,7 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                 }
             }
         };
-        constexpr int CHUNKS_PER_WARP = G1_N / 16;
+        constexpr int CHUNKS_PER_WARP = (G1_N / 8) / G1_WPQ;
         const int first_chunk = warp >> 2;
         int32_t accs[2][5][8];
 #pragma unroll
@@ -196,9 +198,9 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
             if (it + 1 < CHUNKS_PER_WARP) {
 #pragma unroll
                 for (int w = 0; w < 5; ++w)
-                    tmem_ld8(lane_addr + w * G1_N + (first_chunk + 2 * (it + 1)) * 8, accs[(it + 1) & 1][w]);
+                    tmem_ld8(lane_addr + w * G1_N + (first_chunk + G1_WPQ * (it + 1)) * 8, accs[(it + 1) & 1][w]);
             }
-            emit(accs[it & 1], first_chunk + 2 * it);
+            emit(accs[it & 1], first_chunk + G1_WPQ * it);
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();                   // accumulators drained before the next tile overwrites them
