@@ -87,7 +87,7 @@ ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__re
 {
     constexpr int NQ = 4 * LPR;
     constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
-    constexpr int UNROLL = 4;
+    constexpr int UNROLL = 8;
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int grp = lane / LPR, sub = lane % LPR;
