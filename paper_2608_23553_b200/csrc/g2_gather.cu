@@ -26,6 +26,7 @@ mark_kernel(const int32_t *__restrict__ probes, int n_lists, const int64_t *__re
 
 constexpr int CHUNK_THREADS = 256;
 constexpr int WORDS_PER_THREAD = BITMAP_CHUNK_WORDS / CHUNK_THREADS;   // 4 consecutive words per thread
+constexpr int COMPACT_STAGE = 8192;      // ids a chunk stages in shared memory (a chunk covers 32,768 documents)
 
 __device__ __forceinline__ int block_exclusive_scan_256(int v, int *total)
 {
@@ -114,18 +115,32 @@ compact_kernel(const uint32_t *__restrict__ bitmap, int64_t words, int n_chunks,
         c += __popc(w[j]);
     }
     int total;
-    int64_t pos = chunk_cnt[(int64_t)b * (n_chunks + 1) + blockIdx.x] + block_exclusive_scan_256(c, &total);
+    const int local = block_exclusive_scan_256(c, &total);
+    const int64_t base = chunk_cnt[(int64_t)b * (n_chunks + 1) + blockIdx.x];
     int32_t *out = cand + (int64_t)b * maxc;
+    // A thread's ids are consecutive in the output but the threads' runs are ~30 ids apart, so direct stores are
+    // scattered 4-byte writes: when the chunk's ids fit, they are staged in shared memory and copied out coalesced.
+    __shared__ int32_t staged[COMPACT_STAGE];
+    const bool use_stage = total <= COMPACT_STAGE;
+    int64_t pos = use_stage ? local : base + local;
 #pragma unroll
     for (int j = 0; j < WORDS_PER_THREAD; ++j) {
         uint32_t bits = w[j];
-        if (w0 + j < words) word_rank[(int64_t)b * words + w0 + j] = (int32_t)pos;
+        if (w0 + j < words)
+            word_rank[(int64_t)b * words + w0 + j] = (int32_t)(use_stage ? base + pos : pos);
         while (bits) {
             int t = __ffs(bits) - 1;
             bits &= bits - 1;
-            if (pos < maxc) out[pos] = (int32_t)(((w0 + j) << 5) + t);
+            const int32_t id = (int32_t)(((w0 + j) << 5) + t);
+            if (use_stage) staged[pos] = id;
+            else if (pos < maxc) out[pos] = id;
             ++pos;
         }
+    }
+    if (use_stage) {
+        __syncthreads();
+        for (int e = threadIdx.x; e < total; e += CHUNK_THREADS)
+            if (base + e < maxc) out[base + e] = staged[e];
     }
 }
 
