@@ -17,10 +17,21 @@ mark_kernel(const int32_t *__restrict__ probes, int n_lists, const int64_t *__re
     const int32_t c = probes[(int64_t)b * n_lists + blockIdx.x];
     uint32_t *bm = bitmap + (int64_t)b * words;
     const int64_t lo = ivf_off[c], hi = ivf_off[c + 1];
-    for (int64_t e = lo + threadIdx.x; e < hi; e += blockDim.x) {
-        uint32_t d = (uint32_t)ivf_doc[e];
-        uint32_t bit = 1u << (d & 31);
-        if (!(bm[d >> 5] & bit)) atomicOr(&bm[d >> 5], bit);
+    // four list entries per thread and iteration: their loads and the bitmap reads they lead to are in flight together
+    for (int64_t e0 = lo + threadIdx.x; e0 < hi; e0 += 4 * (int64_t)blockDim.x) {
+        uint32_t d[4], cur[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t e = e0 + u * (int64_t)blockDim.x;
+            d[u] = e < hi ? (uint32_t)ivf_doc[e] : 0xffffffffu;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) cur[u] = d[u] != 0xffffffffu ? bm[d[u] >> 5] : 0xffffffffu;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t bit = 1u << (d[u] & 31);
+            if (!(cur[u] & bit)) atomicOr(&bm[d[u] >> 5], bit);
+        }
     }
 }
 
