@@ -307,10 +307,20 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
         count_launch(SLOT_CI);
         return CHIMERA_OK;
     }
-    int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
-    int64_t cap = (int64_t)ix.sm_count * 8;
-    unsigned gx = (unsigned)(want < cap ? want : cap);
-    if (gx < 1) gx = 1;
+    // Blocks per query.  Four blocks are resident per SM and the blocks of a query are adjacent in the grid, so
+    // (resident blocks) / (blocks per query) queries are scanned at the same time and their 8-bit tables compete for
+    // L2: enough blocks per query to keep those tables within COARSE_L2_TABLES bytes, at least enough to fill the GPU
+    // when the batch is small, never more than one warp per candidate.  Measured on the Mid corpus at batch 256
+    // (2 MB tables): 4 blocks per query 57 ms, 16: 23.4, 24: 18.9, 37: 16.5, 74: 16.6, 148: 16.7, 1184: 17.6.
+    constexpr int64_t COARSE_L2_TABLES = 32LL << 20;
+    const int64_t resident = 4LL * ix.sm_count;
+    const int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
+    int64_t per_query = (resident * (int64_t)table_bytes + COARSE_L2_TABLES - 1) / COARSE_L2_TABLES;
+    const int64_t to_fill = (2 * resident + p.B - 1) / p.B;      // two waves when the batch is small
+    if (per_query < to_fill) per_query = to_fill;
+    if (per_query > want) per_query = want;
+    if (per_query < 1) per_query = 1;
+    const unsigned gx = (unsigned)per_query;
     dim3 grid(gx, (unsigned)p.B);
     if (p.nq == 32)
         ci_coarse_kernel<2, false, CI_THREADS><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids,
