@@ -257,7 +257,11 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             prof_mark(SLOT_CI, st);
             if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, st))) return rc;
             prof_mark(SLOT_SELECT, st);
-            if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, 2 * ix.sm_count, SLOT_CI_EXACT, st)))
+            // blocks per query for the few contenders: one per SM in a large batch (measured best), four per SM
+            // when a single query has the GPU to itself
+            int exact_blocks = (4 * ix.sm_count + p.B - 1) / p.B;
+            if (exact_blocks < ix.sm_count) exact_blocks = ix.sm_count;
+            if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, exact_blocks, SLOT_CI_EXACT, st)))
                 return rc;
             prof_mark(SLOT_CI_EXACT, st);
             if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, pruned_ci, st))) return rc;
