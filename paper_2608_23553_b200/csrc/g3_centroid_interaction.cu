@@ -311,8 +311,9 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
     // (resident blocks) / (blocks per query) queries are scanned at the same time and their 8-bit tables compete for
     // L2: enough blocks per query to keep those tables within COARSE_L2_TABLES bytes, at least enough to fill the GPU
     // when the batch is small, never more than one warp per candidate.  Measured on the Mid corpus at batch 256
-    // (2 MB tables): 4 blocks per query 57 ms, 16: 23.4, 24: 18.9, 37: 16.5, 74: 16.6, 148: 16.7, 1184: 17.6.
-    constexpr int64_t COARSE_L2_TABLES = 32LL << 20;
+    // (2 MB tables): 4 blocks per query 57 ms, 16: 23.4, 24: 18.9, 37: 16.5, 74: 16.6, 148: 16.7, 1184: 17.6; a budget
+    // of 16 MB against 32 MB: Mid 16.56 / 16.52 ms, Large (8 MB tables) 36.6 / 37.2 ms; 64 MB: 21.3 and 46.7 ms.
+    constexpr int64_t COARSE_L2_TABLES = 16LL << 20;
     const int64_t resident = 4LL * ix.sm_count;
     const int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
     int64_t per_query = (resident * (int64_t)table_bytes + COARSE_L2_TABLES - 1) / COARSE_L2_TABLES;
