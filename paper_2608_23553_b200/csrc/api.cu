@@ -255,7 +255,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             // bounds for every candidate, contenders for the top n_prune, exact CI and selection among those
             if ((rc = launch_coarse_bounds(ix, p, table8, cand, n_cand, lo, hi, st))) return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, st))) return rc;
+            if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, ci, st))) return rc;
             prof_mark(SLOT_SELECT, st);
             // blocks per query for the few contenders: one per SM in a large batch (measured best), four per SM
             // when a single query has the GPU to itself

@@ -130,8 +130,9 @@ bool coarse_supported(int nq);
 int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st);
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
                          const int32_t *n_cand, int32_t *lo, int32_t *hi, cudaStream_t st);
+// scratch: an int32 [B][maxc] array that is free during this step.
 int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
-                      const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st);
+                      const int32_t *hi, int32_t *cont, int32_t *n_cont, int32_t *scratch, cudaStream_t st);
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
                                 const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, cudaStream_t st);
 // pruned_ci (may be NULL): the score of each kept document, INT_MIN in the padding.

@@ -693,10 +693,135 @@ int launch_shard_select(const Params &p, const int32_t *all_ids, const int32_t *
     return CHIMERA_OK;
 }
 
-int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
-                      const int32_t *hi, int32_t *cont, int32_t *n_cont, cudaStream_t st)
+// The same selection spread over CONT_SPLIT blocks per query, for calls with few queries: one block reads its arrays
+// at one SM's bandwidth (about 40 us for 100k candidates), which is most of the stage's latency when a single query is
+// served.  Three kernels: slice histograms added into a global one; every block finds tau from it and counts its
+// slice's contenders; every block writes its contenders behind those of the slices before it (ascending ids kept).
+// Scratch: `scratch[b * maxc ...]` holds the histogram (CONT_BINS), the slice counts (CONT_SPLIT) and tau.
+constexpr int CONT_SPLIT = 32;
+
+__device__ __forceinline__ void cont_slice(int n, int g, int *j0, int *j1)
 {
-    (void)ix;
+    const int per = (n + CONT_SPLIT - 1) / CONT_SPLIT;
+    *j0 = g * per < n ? g * per : n;
+    *j1 = (g + 1) * per < n ? (g + 1) * per : n;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+contender_hist_kernel(const int32_t *__restrict__ n_cand, const int32_t *__restrict__ lo, int64_t maxc, int n_prune,
+                      int nq, int32_t *__restrict__ scratch)
+{
+    __shared__ int hist[CONT_BINS];
+    const int b = blockIdx.y, n = n_cand[b];
+    if (n <= n_prune) return;                          // everything is a contender: no threshold needed
+    int j0, j1;
+    cont_slice(n, blockIdx.x, &j0, &j1);
+    const int32_t *lb = lo + (int64_t)b * maxc;
+    const int bin_shift = 255 * nq < CONT_BINS ? 0 : 1;
+    for (int i = threadIdx.x; i < CONT_BINS; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    for (int j = j0 + threadIdx.x; j < j1; j += SEL_THREADS)
+        atomicAdd(&hist[(((lb[j] + 64 * nq) >> 17) + 128 * nq) >> bin_shift], 1);
+    __syncthreads();
+    int32_t *gh = scratch + (int64_t)b * maxc;
+    for (int i = threadIdx.x; i < CONT_BINS; i += SEL_THREADS)
+        if (hist[i]) atomicAdd(&gh[i], hist[i]);
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+contender_count_kernel(const int32_t *__restrict__ n_cand, const int32_t *__restrict__ hi, int64_t maxc, int n_prune,
+                       int nq, int32_t *__restrict__ scratch)
+{
+    __shared__ int warp_part[32];
+    __shared__ int s_bin;
+    const int b = blockIdx.y, n = n_cand[b];
+    int32_t *gh = scratch + (int64_t)b * maxc;
+    int32_t tau = INT_MIN;
+    if (n > n_prune) {
+        const int bin_shift = 255 * nq < CONT_BINS ? 0 : 1;
+        constexpr int PER = CONT_BINS / SEL_THREADS;
+        const int first_bin = CONT_BINS - 1 - PER * (int)threadIdx.x;
+        int h[PER], mine = 0;
+#pragma unroll
+        for (int e = 0; e < PER; ++e) { h[e] = gh[first_bin - e]; mine += h[e]; }
+        int total;
+        int before = sel_block_scan(mine, &total, warp_part);
+        if (before < n_prune && n_prune <= before + mine) {
+#pragma unroll
+            for (int e = 0; e < PER; ++e) {
+                if (before < n_prune && n_prune <= before + h[e]) s_bin = first_bin - e;
+                before += h[e];
+            }
+        }
+        __syncthreads();
+        tau = ((s_bin << bin_shift) - 128 * nq) * (1 << 17) - 64 * nq;
+    }
+    int j0, j1;
+    cont_slice(n, blockIdx.x, &j0, &j1);
+    const int32_t *hb = hi + (int64_t)b * maxc;
+    int keep = 0;
+    for (int j = j0 + threadIdx.x; j < j1; j += SEL_THREADS) keep += hb[j] >= tau ? 1 : 0;
+    int total;
+    sel_block_scan(keep, &total, warp_part);
+    if (threadIdx.x == 0) {
+        gh[CONT_BINS + blockIdx.x] = total;
+        if (blockIdx.x == 0) gh[CONT_BINS + CONT_SPLIT] = tau;
+    }
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+contender_write_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand,
+                       const int32_t *__restrict__ hi, int64_t maxc, const int32_t *__restrict__ scratch,
+                       int32_t *__restrict__ cont, int32_t *__restrict__ n_cont)
+{
+    __shared__ int warp_part[32];
+    const int b = blockIdx.y, n = n_cand[b], g = blockIdx.x;
+    const int32_t *gh = scratch + (int64_t)b * maxc;
+    const int32_t tau = gh[CONT_BINS + CONT_SPLIT];
+    int offset = 0;
+    for (int s = 0; s < g; ++s) offset += gh[CONT_BINS + s];
+    int j0, j1;
+    cont_slice(n, g, &j0, &j1);
+    const int32_t *cb = cand + (int64_t)b * maxc;
+    const int32_t *hb = hi + (int64_t)b * maxc;
+    int32_t *out = cont + (int64_t)b * maxc;
+    int run = offset;
+    for (int base = j0; base < j1; base += 4 * SEL_THREADS) {
+        const int q0 = base + 4 * threadIdx.x;
+        int32_t hv[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) hv[e] = q0 + e < j1 ? hb[q0 + e] : INT_MIN;
+        int keep = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) keep += (q0 + e < j1 && hv[e] >= tau) ? 1 : 0;
+        int tot;
+        int pos = run + sel_block_scan(keep, &tot, warp_part);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (q0 + e < j1 && hv[e] >= tau) out[pos++] = cb[q0 + e];
+        run += tot;
+    }
+    if (g == CONT_SPLIT - 1 && threadIdx.x == 0) n_cont[b] = run;
+}
+
+// scratch: an int32 [B][maxc] array that is free during this step (the exact-CI output buffer).
+int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
+                      const int32_t *hi, int32_t *cont, int32_t *n_cont, int32_t *scratch, cudaStream_t st)
+{
+    if (4 * p.B <= ix.sm_count && p.maxc >= CONT_BINS + CONT_SPLIT + 1) {
+        // few queries: CONT_SPLIT blocks each
+        CHIMERA_CUDA(cudaMemset2DAsync(scratch, sizeof(int32_t) * (size_t)p.maxc, 0, sizeof(int32_t) * CONT_BINS,
+                                       (size_t)p.B, st));
+        const dim3 grid(CONT_SPLIT, (unsigned)p.B);
+        contender_hist_kernel<<<grid, SEL_THREADS, 0, st>>>(n_cand, lo, p.maxc, p.n_prune, p.nq, scratch);
+        CHIMERA_CUDA(cudaGetLastError());
+        contender_count_kernel<<<grid, SEL_THREADS, 0, st>>>(n_cand, hi, p.maxc, p.n_prune, p.nq, scratch);
+        CHIMERA_CUDA(cudaGetLastError());
+        contender_write_kernel<<<grid, SEL_THREADS, 0, st>>>(cand, n_cand, hi, p.maxc, scratch, cont, n_cont);
+        CHIMERA_CUDA(cudaGetLastError());
+        count_launch(SLOT_SELECT, 3);
+        return CHIMERA_OK;
+    }
     contender_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, lo, hi, p.maxc, p.n_prune, p.nq, cont,
                                                             n_cont);
     CHIMERA_CUDA(cudaGetLastError());
