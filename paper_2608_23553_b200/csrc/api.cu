@@ -102,6 +102,7 @@ Layout make_layout(const Index &ix, const Params &p)
     L.lo = take(two_phase);
     L.hi = take(two_phase);
     L.cont = take(two_phase);
+    L.cand_rng = take(2 * two_phase);
     L.n_cont = take(B * sizeof(int32_t));
     L.pruned = take(B * p.n_prune * sizeof(int32_t));
     L.word_rank = take(B * (size_t)L.words * sizeof(int32_t));
@@ -253,7 +254,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
                 prof_mark(SLOT_MISC, st);
             }
             // bounds for every candidate, contenders for the top n_prune, exact CI and selection among those
-            if ((rc = launch_coarse_bounds(ix, p, table8, cand, n_cand, lo, hi, st))) return rc;
+            if ((rc = launch_coarse_bounds(ix, p, table8, cand, n_cand, lo, hi, (int2 *)(ws + L.cand_rng), st))) return rc;
             prof_mark(SLOT_CI, st);
             if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, ci, st))) return rc;
             prof_mark(SLOT_SELECT, st);

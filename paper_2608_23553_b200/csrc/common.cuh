@@ -64,6 +64,7 @@ struct Layout {
     size_t lo;            // int32  [B][maxc]         lower bound on CI of every candidate
     size_t hi;            // int32  [B][maxc]         upper bound
     size_t cont;          // int32  [B][maxc]         contender ids, ascending
+    size_t cand_rng;      // int2   [B][maxc]         (first token, length) of each candidate (bound scan)
     size_t n_cont;        // int32  [B]
     size_t pruned;        // int32  [B][n_prune]
     size_t word_rank;     // int32  [B][words]        candidates before each bitmap word (document -> candidate index)
@@ -128,8 +129,9 @@ int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, con
                           cudaStream_t st);
 bool coarse_supported(int nq);
 int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st);
+// rng: int2 [B][maxc] scratch for the candidates' token ranges (may be NULL: per-document offset lookups instead).
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
-                         const int32_t *n_cand, int32_t *lo, int32_t *hi, cudaStream_t st);
+                         const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, cudaStream_t st);
 // scratch: an int32 [B][maxc] array that is free during this step.
 int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
                       const int32_t *hi, int32_t *cont, int32_t *n_cont, int32_t *scratch, cudaStream_t st);

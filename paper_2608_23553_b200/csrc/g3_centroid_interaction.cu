@@ -277,10 +277,155 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
     }
 }
 
+// Token range (first token, length) of every candidate, written once per search: the scan then finds a document's
+// tokens with one coalesced load per 32 documents instead of the dependent chain id -> offsets per document.
+__global__ void __launch_bounds__(256)
+cand_range_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, int64_t maxc,
+                  const int64_t *__restrict__ doc_off, int2 *__restrict__ rng)
+{
+    const int b = blockIdx.y;
+    const int n = n_cand[b];
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
+        const int64_t d = cand[(int64_t)b * maxc + j];
+        const int64_t t0 = doc_off[d];
+        rng[(int64_t)b * maxc + j] = make_int2((int)t0, (int)(doc_off[d + 1] - t0));
+    }
+}
+
+// The bound scan over precomputed token ranges (corpora with fewer than 2^31 tokens).  A warp owns a contiguous run of
+// the query's candidates and takes them 32 at a time: lane i loads the range of document i of the group (one coalesced
+// load), the ranges are handed out by shuffle, and while document i is scanned the first centroid ids of document
+// i + 1 are already being fetched -- a one-level prefetch where the per-document chain used to have three levels.
+// The 32 results of a group are written back coalesced.
+template <int LPR>
+__global__ void __launch_bounds__(CI_THREADS)
+ci_coarse_rng_kernel(const uint8_t *__restrict__ table8, int64_t K, const int2 *__restrict__ rng,
+                     const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
+                     int32_t *__restrict__ lo, int32_t *__restrict__ hi)
+{
+    constexpr int NQ = 16 * LPR;
+    constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
+    constexpr int STEPS = 32 / TPL;               // loads per 32-token slab (= LPR)
+    constexpr int SLABS = 2;                      // 32-token slabs per iteration
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const int grp = lane / LPR, sub = lane % LPR;
+    const int n = n_cand[b];
+    const int4 *tb = reinterpret_cast<const int4 *>(table8 + (int64_t)b * K * NQ) + sub;
+    const int2 *rb = rng + (int64_t)b * maxc;
+    const int warps_per_query = gridDim.x * CI_WARPS;
+    const int per_warp = (n + warps_per_query - 1) / warps_per_query;
+    const int wq = blockIdx.x * CI_WARPS + (threadIdx.x >> 5);
+    const int j_begin = wq * per_warp < n ? wq * per_warp : n;
+    const int j_end = j_begin + per_warp < n ? j_begin + per_warp : n;
+
+    for (int jb = j_begin; jb < j_end; jb += 32) {
+        const int cnt = j_end - jb < 32 ? j_end - jb : 32;
+        const int2 mine = lane < cnt ? rb[jb + lane] : make_int2(0, 1);
+        int my_lo = 0, my_hi = 0;
+        int32_t nx_cid[SLABS];
+        {
+            const int t0 = __shfl_sync(0xffffffffu, mine.x, 0), len = __shfl_sync(0xffffffffu, mine.y, 0);
+#pragma unroll
+            for (int k = 0; k < SLABS; ++k) {
+                const int i = 32 * k + lane;
+                nx_cid[k] = cids[(int64_t)t0 + (i < len - 1 ? i : len - 1)];
+            }
+        }
+        for (int di = 0; di < cnt; ++di) {
+            const int t0 = __shfl_sync(0xffffffffu, mine.x, di), len = __shfl_sync(0xffffffffu, mine.y, di);
+            int32_t cid[SLABS];
+#pragma unroll
+            for (int k = 0; k < SLABS; ++k) cid[k] = nx_cid[k];
+            if (di + 2 < cnt) {                        // two documents ahead: pull the centroid ids into L2
+                const int p0 = __shfl_sync(0xffffffffu, mine.x, di + 2), pl = __shfl_sync(0xffffffffu, mine.y, di + 2);
+                if (lane * 32 < pl) asm volatile("prefetch.global.L2 [%0];" ::"l"(cids + (int64_t)p0 + lane * 32));
+            }
+            if (di + 1 < cnt) {
+                const int n0 = __shfl_sync(0xffffffffu, mine.x, di + 1), nl = __shfl_sync(0xffffffffu, mine.y, di + 1);
+#pragma unroll
+                for (int k = 0; k < SLABS; ++k) {
+                    const int i = 32 * k + lane;
+                    nx_cid[k] = cids[(int64_t)n0 + (i < nl - 1 ? i : nl - 1)];
+                }
+            }
+            uint32_t m[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) m[r] = 0u;
+            for (int base = 0; base < len; base += 32 * SLABS) {
+                // lanes past the end repeat the last token (harmless for a maximum)
+                int4 v[SLABS * STEPS];
+#pragma unroll
+                for (int k = 0; k < SLABS; ++k) {
+                    if (k == 0 || base + 32 * k < len) {
+#pragma unroll
+                        for (int s = 0; s < STEPS; ++s) {
+                            const int32_t c = __shfl_sync(0xffffffffu, cid[k], s * TPL + grp);
+                            v[k * STEPS + s] = __ldg(tb + (int64_t)c * LPR);
+                        }
+                    }
+                }
+                // the centroid ids of the next iteration travel while this iteration's rows do
+                if (base + 32 * SLABS < len) {
+#pragma unroll
+                    for (int k = 0; k < SLABS; ++k) {
+                        const int i = base + 32 * SLABS + 32 * k + lane;
+                        cid[k] = cids[(int64_t)t0 + (i < len - 1 ? i : len - 1)];
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < SLABS; ++k) {
+                    if (k == 0 || base + 32 * k < len) {
+#pragma unroll
+                        for (int s = 0; s < STEPS; s += 2)
+                            coarse_accumulate2(m, v[k * STEPS + s], v[k * STEPS + s + 1]);
+                    }
+                }
+            }
+            // merge the lane groups (same columns, different tokens): each exchange keeps one half of the registers
+            int nreg = 8;
+            uint32_t dup_mask = 0;
+#pragma unroll
+            for (int o = 16; o >= LPR; o >>= 1) {
+                if (nreg > 1) {
+                    const int half = nreg >> 1;
+                    const bool up = (lane & o) != 0;
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        if (r < half) {
+                            const uint32_t send = up ? m[r] : m[r + half];
+                            const uint32_t keep = up ? m[r + half] : m[r];
+                            m[r] = __vmaxu2(keep, __shfl_xor_sync(0xffffffffu, send, o));
+                        }
+                    }
+                    nreg = half;
+                } else {
+                    m[0] = __vmaxu2(m[0], __shfl_xor_sync(0xffffffffu, m[0], o));
+                    dup_mask |= (uint32_t)o;
+                }
+            }
+            const int u_lo = (int)(m[0] & 0xffffu), u_hi = (int)(m[0] >> 16);
+            int packed = 0;                                         // sum of maxima | saturated count << 20
+            if ((lane & dup_mask) == 0)
+                packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 20);
+            packed = __reduce_add_sync(0xffffffffu, packed);
+            if (lane == di) {                                       // lane di keeps the result of document di
+                const int sum = packed & 0xfffff, sat = packed >> 20;
+                my_lo = (sum - 128 * NQ) * (1 << 17) - 64 * NQ;
+                my_hi = my_lo + NQ * ((1 << 17) - 1) + sat * (1 << 18);
+            }
+        }
+        if (lane < cnt) {
+            lo[(int64_t)b * maxc + jb + lane] = my_lo;
+            hi[(int64_t)b * maxc + jb + lane] = my_hi;
+        }
+    }
+}
+
 bool coarse_supported(int nq) { return nq == 32 || nq == 64; }
 
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
-                         const int32_t *n_cand, int32_t *lo, int32_t *hi, cudaStream_t st)
+                         const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, cudaStream_t st)
 {
     const size_t table_bytes = (size_t)ix.K * p.nq;
     if (table_bytes <= 160 * 1024) {
@@ -323,6 +468,21 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
     if (per_query < 1) per_query = 1;
     const unsigned gx = (unsigned)per_query;
     dim3 grid(gx, (unsigned)p.B);
+    if (ix.T < 0x7fffffffLL && rng != nullptr) {
+        int64_t rb = ((int64_t)ix.sm_count * 8 + p.B - 1) / p.B;
+        const int64_t rwant = (p.maxc + 255) / 256;
+        if (rb > rwant) rb = rwant;
+        if (rb < 1) rb = 1;
+        cand_range_kernel<<<dim3((unsigned)rb, (unsigned)p.B), 256, 0, st>>>(cand, n_cand, p.maxc, ix.doc_off, rng);
+        CHIMERA_CUDA(cudaGetLastError());
+        if (p.nq == 32)
+            ci_coarse_rng_kernel<2><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
+        else
+            ci_coarse_rng_kernel<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
+        CHIMERA_CUDA(cudaGetLastError());
+        count_launch(SLOT_CI, 2);
+        return CHIMERA_OK;
+    }
     if (p.nq == 32)
         ci_coarse_kernel<2, false, CI_THREADS><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, cand, n_cand, p.maxc, ix.cids,
                                                                           ix.doc_off, lo, hi);
