@@ -78,7 +78,7 @@ def ncu_traffic(cfg, batch):
     return None
 
 
-NCU_CI_COARSE_MID_B8_BYTES = 463.8e6    # dram__bytes_read.sum + dram__bytes_write.sum of one launch at batch 8
+NCU_CI_COARSE_MID_B8_BYTES = 443.2e6    # dram__bytes_read.sum + dram__bytes_write.sum of one launch at batch 8
 NCU_PARTIAL_MID_B64_BYTES = 1833e6      # the same for partial_score_kernel<2> at batch 64 (profiles/ncu_partial_score_mid.md)
 
 
@@ -440,7 +440,7 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel: the stage-3 bound scan over every candidate token (ci_coarse_kernel) -------
+    # ---- roofline of the dominant kernel: the stage-3 bound scan over every candidate token (ci_coarse_rng_kernel) ---
     peak, peak_kind = measured_peaks()
     used = [work[(args.warmup + s) % n_batches] for s in range(args.steps)]
     mean = lambda key: float(np.mean([u[key] for u in used]))       # noqa: E731
@@ -460,7 +460,7 @@ def main():
     g4_bytes = mean("pruned_tokens") * ((cfg.dim // 8 + 4.0) if args.rabitq else (4.0 + cfg.code_bytes))
     stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
     roofline = {
-        "kernel": "ci_coarse_kernel (stage 3 bound scan over every candidate token)", "bound": "hbm",
+        "kernel": "ci_coarse_rng_kernel (stage 3 bound scan over every candidate token)", "bound": "hbm",
         "achieved": ci_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
         "frac": ci_gbs / peak, "traffic": ncu_traffic(cfg, B), "ms_per_launch": ci_ms,
         "algorithmic_bytes_per_launch": ci_bytes, "contender_fraction": cont_frac,
