@@ -75,17 +75,18 @@ const char *chimera_last_error(void);
 
 /* Build the device-resident index (offline step; Sec. 3.1: centroids, posting lists, per-token codes).
  *   desc       host pointer.
- *   centroids  device, [K, dim] float32 row-major, unit-norm rows (every |element| <= 1).  Copied (as fixed-point
+ *   centroids  device, 16-byte aligned, [K, dim] float32 row-major, unit-norm rows (every |element| <= 1).  Copied (as fixed-point
  *              digits); may be freed after the call returns.
  *   cids       device, [T] int32 in [0, K), document-major (document 0's tokens first).  REFERENCED, not copied:
  *              must outlive the index.
- *   codes      device, [T, dim*nbits/8] uint8, document-major.  REFERENCED, not copied: must outlive the index.
+ *   codes      device, 32-byte aligned, [T, dim*nbits/8] uint8, document-major.  REFERENCED, not copied: must outlive
+ *              the index.
  *   doclens    device, [N] int32, each >= 1, summing to T.  Copied (as prefix sums).
  *   stream     work is enqueued on it and the call synchronises it before returning.
  *   out        host pointer receiving the handle.
  * Allocates (cudaMalloc) prefix sums, centroid digits and an inverted file: for each centroid the unique ids of the
  * documents owning a token assigned to it, in unspecified order.
- * Errors: INVALID_ARG (null pointer, sizes < 1, a cid outside [0,K), a doclen < 1, lengths not summing to T),
+ * Errors: INVALID_ARG (null or misaligned pointer, sizes < 1, a cid outside [0,K), a doclen < 1, lengths not summing to T),
  * UNSUPPORTED (dim / nbits), CUDA_ERROR.  On error nothing stays allocated and *out is NULL. */
 int chimera_build_index(const chimera_index_desc *desc, const float *centroids, const int32_t *cids,
                         const uint8_t *codes, const int32_t *doclens, void *stream, chimera_index **out);

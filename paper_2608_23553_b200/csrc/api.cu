@@ -345,8 +345,8 @@ int chimera_build_index(const chimera_index_desc *desc, const float *centroids, 
     if (desc->dim < 32 || desc->dim > 128 || desc->dim % 32) return fail(CHIMERA_UNSUPPORTED, "dim must be 32, 64, 96 or 128, got %d", desc->dim);
     if (desc->nbits != 1 && desc->nbits != 2) return fail(CHIMERA_UNSUPPORTED, "nbits must be 1 or 2, got %d", desc->nbits);
     if (!(desc->res_hi > desc->res_lo)) return fail(CHIMERA_INVALID_ARG, "res_hi must exceed res_lo");
-    if (((uintptr_t)cids & 3) || ((uintptr_t)codes & 15) || ((uintptr_t)centroids & 15))
-        return fail(CHIMERA_INVALID_ARG, "centroids and codes must be 16-byte aligned");
+    if (((uintptr_t)cids & 3) || ((uintptr_t)codes & 31) || ((uintptr_t)centroids & 15))
+        return fail(CHIMERA_INVALID_ARG, "centroids must be 16-byte aligned and codes 32-byte aligned");
 
     Index *ix = new (std::nothrow) Index();
     if (!ix) return fail(CHIMERA_CUDA_ERROR, "out of host memory");

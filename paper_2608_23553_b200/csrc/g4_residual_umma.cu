@@ -158,6 +158,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
 
     const int32_t *tb = table + (int64_t)b * K * nq;
     const bool vec_rows = (nq & 3) == 0;
+    const bool wide_rows = (nq & 7) == 0;          // rows are then 32-byte aligned (the table is 256-byte aligned)
     const int k_steps = D >> 5;
     const float code_scale = delta * (1.0f / 4194304.0f);    // delta * 2^-22
     bool alive = true;
@@ -175,7 +176,12 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             const long long t = s_t0[dl] + (s - s_off[dl]);
             cid = RQ ? __float_as_int(factors[t]) : cids[t];     // RQ: the slot carries the token's factor bits (> 0)
             const uint32_t *src = codes + t * CW;
-            if ((CW & 3) == 0) {                          // 16-byte aligned codes: two wide loads for 32 bytes
+            if (NBITS == 2 && CW == 8) {                  // 32-byte codes (32-byte aligned): one load
+                asm volatile("ld.global.nc.v8.u32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                             : "=r"(cw[0]), "=r"(cw[1]), "=r"(cw[2]), "=r"(cw[3]), "=r"(cw[4]), "=r"(cw[5]), "=r"(cw[6]),
+                               "=r"(cw[7])
+                             : "l"(src));
+            } else if ((CW & 3) == 0) {                   // 16-byte aligned codes
 #pragma unroll
                 for (int w = 0; w < MAXCW; w += 4)
                     if (w < CW) {
@@ -262,7 +268,16 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
 #pragma unroll
             for (int g = 0; g < NQP / 4; ++g) {
                 const int col = 4 * g;
-                if (vec_rows && col + 3 < nq) {
+                if (wide_rows && col + 7 < nq) {
+                    // 32 bytes per load: half as many line lookups per row as with 16-byte pieces
+                    if ((g & 1) == 0)
+                        asm volatile("ld.global.nc.v8.s32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                     : "=r"(sv[g].x), "=r"(sv[g].y), "=r"(sv[g].z), "=r"(sv[g].w), "=r"(sv[g + 1].x),
+                                       "=r"(sv[g + 1].y), "=r"(sv[g + 1].z), "=r"(sv[g + 1].w)
+                                     : "l"(srow + col));
+                } else if (wide_rows && (g & 1) == 1 && col + 3 < nq) {
+                    // second half of a 32-byte load issued at g - 1
+                } else if (vec_rows && col + 3 < nq) {
                     sv[g] = __ldg(reinterpret_cast<const int4 *>(srow + col));
                 } else {
                     sv[g].x = col + 0 < nq ? __ldg(srow + col + 0) : 0;
