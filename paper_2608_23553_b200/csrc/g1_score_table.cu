@@ -169,7 +169,15 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                     }
                     *reinterpret_cast<uint2 *>(table8 + ((int64_t)qb * K + c) * nq + qi) = make_uint2(w[0], w[1]);
                 }
-                if ((nq & 3) == 0) {
+                if ((nq & 7) == 0) {
+                    // the chunk's eight values are consecutive tokens of one query, 32-byte aligned: one store
+                    if (r0 < rows32)                                  // q_rows is a multiple of 8 here
+                        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(
+                                         table + ((int64_t)qb * K + c) * nq + qi),
+                                     "r"(out[0]), "r"(out[1]), "r"(out[2]), "r"(out[3]), "r"(out[4]), "r"(out[5]),
+                                     "r"(out[6]), "r"(out[7])
+                                     : "memory");
+                } else if ((nq & 3) == 0) {
 #pragma unroll
                     for (int e = 0; e < 8; e += 4) {
                         if (r0 + e < rows32)                          // q_rows is a multiple of 4 here
