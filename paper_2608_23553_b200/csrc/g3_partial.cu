@@ -75,7 +75,12 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
     auto code_dot = [&](int64_t t) -> int {
         const uint32_t *cw = codes + t * CW;
         uint32_t word[8];                              // at most 32 code bytes per token
-        if ((CW & 3) == 0) {
+        if (NBITS == 2 && CW == 8) {                   // 32-byte codes (32-byte aligned): one load
+            asm volatile("ld.global.nc.v8.u32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(word[0]), "=r"(word[1]), "=r"(word[2]), "=r"(word[3]), "=r"(word[4]), "=r"(word[5]),
+                           "=r"(word[6]), "=r"(word[7])
+                         : "l"(cw));
+        } else if ((CW & 3) == 0) {
 #pragma unroll
             for (int w = 0; w < 8; w += 4)
                 if (w < CW) {
