@@ -63,7 +63,8 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     constexpr uint32_t TMEM_COLS = N <= 128 ? 128 : 256;
     constexpr uint32_t A_BYTES = G4U_TOK * 128;              // 16 KB
     constexpr uint32_t B_BYTES = N * 128;
-    constexpr int VP = NQP + 1;                              // pitch of the value rows (floats)
+    constexpr int VP = NQP + 4;                              // pitch of the value rows (floats): 16-byte aligned rows;
+                                                             // a row is read with lane = column, so any pitch is conflict-free
     constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) |
                                ((uint32_t)(G4U_TOK >> 4) << 24);
 
@@ -322,17 +323,18 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                 for (int g = 0; g < 4; ++g) {
                     const int4 q4 = RQ ? make_int4(0, 0, 0, 0) : sv[ch * 4 + g];
                     const int32_t se[4] = {q4.x, q4.y, q4.z, q4.w};
+                    float val[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int o = 4 * g + e;
                         // |sum_x u_x Xq_x| <= 3 * 2^22 * |q|_1 < 2^31: the plane recombination fits int32
                         const int32_t T = a0[o] + a1[o] * 256 + a2[o] * 65536;
                         if (RQ)
-                            vrow[ch * 16 + o] = __fmul_rn(__int_as_float(cid),
-                                                          __fmul_rn(kappa, (float)(2 * T - s_sq[ch * 16 + o])));
+                            val[e] = __fmul_rn(__int_as_float(cid), __fmul_rn(kappa, (float)(2 * T - s_sq[ch * 16 + o])));
                         else
-                            vrow[ch * 16 + o] = fmaf(code_scale, (float)T, (float)se[e] * (1.0f / 16777216.0f));
+                            val[e] = fmaf(code_scale, (float)T, (float)se[e] * (1.0f / 16777216.0f));
                     }
+                    *reinterpret_cast<float4 *>(vrow + ch * 16 + 4 * g) = make_float4(val[0], val[1], val[2], val[3]);
                 }
             }
         }
@@ -400,7 +402,7 @@ static int launch_g4_umma(const Index &ix, const Params &p, const float *queries
     CUtensorMap map_q;
     int rc = make_plane_map(&map_q, qdig, (int64_t)p.B * p.nq, NQP);
     if (rc) return rc;
-    const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 + sizeof(float) * G4U_TOK * (NQP + 1) +
+    const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 + sizeof(float) * G4U_TOK * (NQP + 4) +
                         sizeof(uint32_t) * G4U_MAX_DOCS * NQP + 32;
     auto kern = residual_maxsim_umma<NQP, NBITS, RQ>;
     CHIMERA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
