@@ -111,6 +111,7 @@ Layout make_layout(const Index &ix, const Params &p)
     L.qdig_rot = take(ix.rot_t ? 3 * B * nq * 128 : 0);
     L.n_pruned = take(B * sizeof(int32_t));
     L.pruned_ci = take(B * p.n_prune * sizeof(int32_t));
+    L.sel_scratch = take(select_split_scratch_bytes(ix, p));
     L.score4 = take(B * p.n_prune * sizeof(float));
     L.total = o;
     return L;
@@ -179,6 +180,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int32_t *pruned = (int32_t *)(ws + L.pruned);
     int32_t *n_pruned = (int32_t *)(ws + L.n_pruned);
     int32_t *pruned_ci = (int32_t *)(ws + L.pruned_ci);
+    int32_t *sel_scratch = select_split_used(ix, p) ? (int32_t *)(ws + L.sel_scratch) : nullptr;
     int32_t *word_rank = (int32_t *)(ws + L.word_rank);
     int32_t *partial_m = (int32_t *)(ws + L.partial_m);
     float *q_rot = (float *)(ws + L.q_rot);
@@ -238,7 +240,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if ((rc = launch_rabitq_partial(ix, p, L, q_rot, probes, bitmap, word_rank, n_cand, partial_m, ci, st)))
                 return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, st))) return rc;
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, sel_scratch, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else if (partial) {
             // the paper's candidate refinement: partial scores from the retrieved tokens only, then the same selection
@@ -246,7 +248,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
                                             st)))
                 return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, st))) return rc;
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, sel_scratch, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else if (two_phase) {
             if (first > 1) {                       // the table came from the caller: derive its coarse copy
@@ -265,12 +267,12 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, exact_blocks, SLOT_CI_EXACT, st)))
                 return rc;
             prof_mark(SLOT_CI_EXACT, st);
-            if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, pruned_ci, st))) return rc;
+            if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, pruned_ci, nullptr, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else {
             if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, 0, SLOT_CI, st))) return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, st))) return rc;
+            if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, sel_scratch, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         }
     }

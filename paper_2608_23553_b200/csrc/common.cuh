@@ -73,6 +73,7 @@ struct Layout {
     size_t qdig_rot;      // int8   [3][B*nq][128]    their digit planes
     size_t n_pruned;      // int32  [B]
     size_t pruned_ci;     // int32  [B][n_prune] stage-3 score of each survivor (document-sharded search)
+    size_t sel_scratch;   // int32  histograms and slice counts of the multi-block selection (few queries per call)
     size_t score4;        // float  [B][n_prune]
     size_t total;
     // derived sizes
@@ -138,8 +139,11 @@ int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, con
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
                                 const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, cudaStream_t st);
 // pruned_ci (may be NULL): the score of each kept document, INT_MIN in the padding.
+// scratch: select_split_scratch_bytes() bytes (few queries per call: several blocks per query), or NULL.
+bool select_split_used(const Index &ix, const Params &p);
+size_t select_split_scratch_bytes(const Index &ix, const Params &p);
 int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
-                  int32_t *pruned, int32_t *n_pruned, int32_t *pruned_ci, cudaStream_t st);
+                  int32_t *pruned, int32_t *n_pruned, int32_t *pruned_ci, int32_t *scratch, cudaStream_t st);
 // Document-sharded search: the global top-n_prune of the shards' lists and the final top-k merge.
 int launch_shard_export(const Params &p, const int32_t *pruned, const int32_t *pruned_ci, int64_t doc_base,
                         int32_t *out_ids, int32_t *out_ci, cudaStream_t st);

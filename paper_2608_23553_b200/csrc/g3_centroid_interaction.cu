@@ -989,10 +989,223 @@ int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, con
     return CHIMERA_OK;
 }
 
-int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
-                  int32_t *pruned, int32_t *n_pruned, int32_t *pruned_ci, cudaStream_t st)
+// ------------------------------------------------------------------------------------------------------------------
+// The same selection spread over SELS_SPLIT blocks per query, for calls with few queries (one block reads its arrays at
+// one SM's bandwidth; with a single query that is most of the stage's latency).  Five kernels, each block working on a
+// contiguous slice of the candidates: three radix passes whose slice histograms are added into global ones (every block
+// of the next kernel re-derives the chosen digit from the global histogram, which is cheap), a count of the entries
+// above and at the threshold per slice, and the ordered write behind the slices before it.
+// Scratch per query (int32): hist[0] 2048, hist[1] 2048, hist[2] 1024, greater[SELS_SPLIT], equal[SELS_SPLIT].
+constexpr int SELS_SPLIT = 32;
+constexpr int SELS_SCRATCH = 2048 + 2048 + 1024 + 2 * SELS_SPLIT;
+
+__device__ __forceinline__ void sels_slice(int n, int g, int *j0, int *j1)
 {
-    (void)ix;
+    const int per = (n + SELS_SPLIT - 1) / SELS_SPLIT;
+    *j0 = g * per < n ? g * per : n;
+    *j1 = (g + 1) * per < n ? (g + 1) * per : n;
+}
+
+// The digit (bin) of `bins` descending-cumulative bins that holds rank `want`, and the rank left inside it.
+// Whole block, uniform result.
+__device__ __forceinline__ void sels_find(const int32_t *__restrict__ hist, int bins, int want, int *warp_part,
+                                          int *s_out /* [2] */, int *bin, int *want_rest)
+{
+    const int hi_bin = bins - 1 - 2 * (int)threadIdx.x, lo_bin = hi_bin - 1;
+    const int h_hi = hi_bin >= 0 ? hist[hi_bin] : 0;
+    const int h_lo = lo_bin >= 0 ? hist[lo_bin] : 0;
+    int total;
+    const int before = sel_block_scan(h_hi + h_lo, &total, warp_part);
+    if (before < want && want <= before + h_hi + h_lo) {
+        if (want <= before + h_hi) { s_out[0] = hi_bin; s_out[1] = want - before; }
+        else { s_out[0] = lo_bin; s_out[1] = want - before - h_hi; }
+    }
+    __syncthreads();
+    *bin = s_out[0];
+    *want_rest = s_out[1];
+    __syncthreads();
+}
+
+// PASS 0, 1, 2: histogram of the pass's digit over the slice's entries that match the digits chosen so far.
+template <int PASS>
+__global__ void __launch_bounds__(SEL_THREADS)
+sels_hist_kernel(const int32_t *__restrict__ n_cand, const int32_t *__restrict__ ci, int64_t maxc, int n_prune,
+                 int32_t *__restrict__ scratch)
+{
+    __shared__ int hist[2048];
+    __shared__ int warp_part[32];
+    __shared__ int s_out[2];
+    const int b = blockIdx.y, n = n_cand[b];
+    if (n <= n_prune) return;
+    int32_t *sc = scratch + (int64_t)b * SELS_SCRATCH;
+    uint32_t prefix = 0u, mask = 0u;
+    int want = n_prune;
+    if (PASS >= 1) {
+        int bin;
+        sels_find(sc, 2048, want, warp_part, s_out, &bin, &want);
+        prefix = (uint32_t)bin << 21;
+        mask = 0x7ffu << 21;
+    }
+    if (PASS >= 2) {
+        int bin;
+        sels_find(sc + 2048, 2048, want, warp_part, s_out, &bin, &want);
+        prefix |= (uint32_t)bin << 10;
+        mask |= 0x7ffu << 10;
+    }
+    constexpr int SHIFT = PASS == 0 ? 21 : PASS == 1 ? 10 : 0;
+    constexpr int BINS = PASS == 2 ? 1024 : 2048;
+    for (int i = threadIdx.x; i < BINS; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    int j0, j1;
+    sels_slice(n, blockIdx.x, &j0, &j1);
+    const int32_t *sb = ci + (int64_t)b * maxc;
+    for (int j = j0 + threadIdx.x; j < j1; j += SEL_THREADS) {
+        const uint32_t u = (uint32_t)sb[j] ^ 0x80000000u;
+        if ((u & mask) == prefix) atomicAdd(&hist[(u >> SHIFT) & (BINS - 1)], 1);
+    }
+    __syncthreads();
+    int32_t *gh = sc + (PASS == 0 ? 0 : PASS == 1 ? 2048 : 4096);
+    for (int i = threadIdx.x; i < BINS; i += SEL_THREADS)
+        if (hist[i]) atomicAdd(&gh[i], hist[i]);
+}
+
+// The threshold (all three digits) and how many entries equal to it belong to the top n_prune.
+__device__ __forceinline__ uint32_t sels_threshold(const int32_t *sc, int n_prune, int *warp_part, int *s_out, int *need_eq)
+{
+    int b1, b2, b3, want = n_prune;
+    sels_find(sc, 2048, want, warp_part, s_out, &b1, &want);
+    sels_find(sc + 2048, 2048, want, warp_part, s_out, &b2, &want);
+    sels_find(sc + 4096, 1024, want, warp_part, s_out, &b3, &want);
+    *need_eq = want;
+    return ((uint32_t)b1 << 21) | ((uint32_t)b2 << 10) | (uint32_t)b3;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+sels_count_kernel(const int32_t *__restrict__ n_cand, const int32_t *__restrict__ ci, int64_t maxc, int n_prune,
+                  int32_t *__restrict__ scratch)
+{
+    __shared__ int warp_part[32];
+    __shared__ int s_out[2];
+    const int b = blockIdx.y, n = n_cand[b];
+    if (n <= n_prune) return;
+    int32_t *sc = scratch + (int64_t)b * SELS_SCRATCH;
+    int need_eq;
+    const uint32_t thr = sels_threshold(sc, n_prune, warp_part, s_out, &need_eq);
+    int j0, j1;
+    sels_slice(n, blockIdx.x, &j0, &j1);
+    const int32_t *sb = ci + (int64_t)b * maxc;
+    int gt = 0, eq = 0;
+    for (int j = j0 + threadIdx.x; j < j1; j += SEL_THREADS) {
+        const uint32_t u = (uint32_t)sb[j] ^ 0x80000000u;
+        gt += u > thr ? 1 : 0;
+        eq += u == thr ? 1 : 0;
+    }
+    int total;
+    sel_block_scan((gt << 16) | eq, &total, warp_part);        // a slice has fewer than 2^15 entries (launcher)
+    if (threadIdx.x == 0) {
+        sc[5120 + blockIdx.x] = total >> 16;
+        sc[5120 + SELS_SPLIT + blockIdx.x] = total & 0xffff;
+    }
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+sels_write_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, const int32_t *__restrict__ ci,
+                  int64_t maxc, int n_prune, const int32_t *__restrict__ scratch, int32_t *__restrict__ pruned,
+                  int32_t *__restrict__ n_pruned, int32_t *__restrict__ pruned_ci)
+{
+    __shared__ int warp_part[32];
+    __shared__ int s_out[2];
+    const int b = blockIdx.y, n = n_cand[b], g = blockIdx.x;
+    const int32_t *cb = cand + (int64_t)b * maxc;
+    const int32_t *sb = ci + (int64_t)b * maxc;
+    int32_t *out = pruned + (int64_t)b * n_prune;
+    int32_t *out_ci = pruned_ci ? pruned_ci + (int64_t)b * n_prune : nullptr;
+    int j0, j1;
+    sels_slice(n, g, &j0, &j1);
+    if (n <= n_prune) {                                     // everything survives; the last block pads
+        for (int j = j0 + threadIdx.x; j < j1; j += SEL_THREADS) {
+            out[j] = cb[j];
+            if (out_ci) out_ci[j] = sb[j];
+        }
+        if (g == SELS_SPLIT - 1) {
+            for (int j = n + threadIdx.x; j < n_prune; j += SEL_THREADS) {
+                out[j] = -1;
+                if (out_ci) out_ci[j] = INT_MIN;
+            }
+            if (threadIdx.x == 0) n_pruned[b] = n;
+        }
+        return;
+    }
+    const int32_t *sc = scratch + (int64_t)b * SELS_SCRATCH;
+    int need_eq;
+    const uint32_t thr = sels_threshold(sc, n_prune, warp_part, s_out, &need_eq);
+    int run_gt = 0, run_eq = 0;
+    for (int s = 0; s < g; ++s) {
+        run_gt += sc[5120 + s];
+        run_eq += sc[5120 + SELS_SPLIT + s];
+    }
+    for (int base = j0; base < j1; base += 4 * SEL_THREADS) {
+        const int q0 = base + 4 * threadIdx.x;
+        uint32_t u[4];
+        int32_t id[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = q0 + e;
+            u[e] = j < j1 ? ((uint32_t)sb[j] ^ 0x80000000u) : 0u;
+            id[e] = j < j1 ? cb[j] : 0;
+        }
+        int gt = 0, eq = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            gt += (q0 + e < j1 && u[e] > thr) ? 1 : 0;
+            eq += (q0 + e < j1 && u[e] == thr) ? 1 : 0;
+        }
+        int total;
+        const int before = sel_block_scan((gt << 16) | eq, &total, warp_part);
+        int gt_before = run_gt + (before >> 16), eq_before = run_eq + (before & 0xffff);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (q0 + e >= j1) break;
+            const bool is_gt = u[e] > thr, is_eq = u[e] == thr;
+            if (is_gt || (is_eq && eq_before < need_eq)) {
+                const int pos = gt_before + (eq_before < need_eq ? eq_before : need_eq);
+                out[pos] = id[e];
+                if (out_ci) out_ci[pos] = (int32_t)(u[e] ^ 0x80000000u);
+            }
+            gt_before += is_gt ? 1 : 0;
+            eq_before += is_eq ? 1 : 0;
+        }
+        run_gt += total >> 16;
+        run_eq += total & 0xffff;
+    }
+    if (g == 0 && threadIdx.x == 0) n_pruned[b] = n_prune;
+}
+
+// Queries per call up to which the selection is spread over several blocks, and the scratch it needs.
+bool select_split_used(const Index &ix, const Params &p) { return 4 * p.B <= ix.sm_count; }
+size_t select_split_scratch_bytes(const Index &ix, const Params &p)
+{
+    return select_split_used(ix, p) ? sizeof(int32_t) * (size_t)p.B * SELS_SCRATCH : 0;
+}
+
+// scratch: select_split_scratch_bytes() bytes, or NULL (one block per query then).
+int launch_select(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *ci,
+                  int32_t *pruned, int32_t *n_pruned, int32_t *pruned_ci, int32_t *scratch, cudaStream_t st)
+{
+    // the slices must stay below 2^15 entries (two counters packed in an int) and be worth five launches
+    if (scratch != nullptr && select_split_used(ix, p) && p.maxc >= 16384 && p.maxc < (int64_t)SELS_SPLIT * 32767) {
+        CHIMERA_CUDA(cudaMemsetAsync(scratch, 0, select_split_scratch_bytes(ix, p), st));
+        const dim3 grid(SELS_SPLIT, (unsigned)p.B);
+        sels_hist_kernel<0><<<grid, SEL_THREADS, 0, st>>>(n_cand, ci, p.maxc, p.n_prune, scratch);
+        sels_hist_kernel<1><<<grid, SEL_THREADS, 0, st>>>(n_cand, ci, p.maxc, p.n_prune, scratch);
+        sels_hist_kernel<2><<<grid, SEL_THREADS, 0, st>>>(n_cand, ci, p.maxc, p.n_prune, scratch);
+        sels_count_kernel<<<grid, SEL_THREADS, 0, st>>>(n_cand, ci, p.maxc, p.n_prune, scratch);
+        sels_write_kernel<<<grid, SEL_THREADS, 0, st>>>(cand, n_cand, ci, p.maxc, p.n_prune, scratch, pruned, n_pruned,
+                                                        pruned_ci);
+        CHIMERA_CUDA(cudaGetLastError());
+        count_launch(SLOT_SELECT, 5);
+        return CHIMERA_OK;
+    }
     select_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, ci, p.maxc, p.n_prune, pruned, n_pruned,
                                                          pruned_ci);
     CHIMERA_CUDA(cudaGetLastError());

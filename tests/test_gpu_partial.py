@@ -80,6 +80,14 @@ def test_partial_refinement_mid_batch256_sampled():
     gix.enable_partial()
     oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
     _check(gix, oix, q, cfg.nprobe, cfg.n_prune, cfg.k, sample=(0, 255), max_diffs=2)
+    # few queries per call: the selection runs over several blocks per query (another code path); against the oracle,
+    # and bit-identical to the same queries inside the batch of 256
+    _check(gix, oix, q[254:256], cfg.nprobe, cfg.n_prune, cfg.k, max_diffs=2)
+    qd = torch.from_numpy(q).cuda()
+    big = gix.search(qd, cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
+    for lo, hi in ((0, 1), (100, 103)):
+        small = gix.search(qd[lo:hi].contiguous(), cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
+        assert torch.equal(small[0], big[0][lo:hi]) and torch.equal(small[1], big[1][lo:hi])
 
 
 def test_partial_and_rabitq_edge_cases():

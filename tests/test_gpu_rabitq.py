@@ -80,3 +80,9 @@ def test_rabitq_pipeline_mid_batch256_sampled():
     oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
     rq = oracle.make_rabitq(corp.rotation, corp.rq_bits, corp.rq_inv_dot)
     _run(gix, oix, rq, q, cfg.nprobe, cfg.n_prune, cfg.k, sample=(0, 255))
+    # few queries per call: the selection runs over several blocks per query (another code path)
+    _run(gix, oix, rq, q[254:256], cfg.nprobe, cfg.n_prune, cfg.k)
+    qd = torch.from_numpy(q).cuda()
+    big = gix.search(qd, cfg.nprobe, cfg.n_prune, cfg.k, rabitq=True)
+    small = gix.search(qd[7:10].contiguous(), cfg.nprobe, cfg.n_prune, cfg.k, rabitq=True)
+    assert torch.equal(small[0], big[0][7:10]) and torch.equal(small[1], big[1][7:10])
