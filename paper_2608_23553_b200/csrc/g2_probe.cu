@@ -86,24 +86,45 @@ probe_final(const unsigned long long *__restrict__ part, int nq, int P, int n_pa
     unsigned long long *mine = lists + threadIdx.x;
     for (int j = 0; j < P; ++j) mine[j * THREADS] = 0ull;
     if (col < nq) {
-        // a list is only walked further while its keys still beat this thread's current P-th best
-        for (int l0 = warp; l0 < n_part; l0 += 8 * W) {
-            unsigned long long head[8];
+        if (P <= 4 && n_part <= 8 * W) {
+            // Few lists per warp (one query per call): walking a list key by key is a chain of dependent loads, and
+            // with an empty running list every key of every list qualifies anyway -- so all keys of four lists are
+            // loaded together (16 independent loads), twice.
+            for (int l0 = warp; l0 < n_part; l0 += 4 * W) {
+                unsigned long long k[4][4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int l = l0 + u * W;
-                head[u] = l < n_part ? part[(((int64_t)b * n_part + l) * P) * nq + col] : 0ull;
+                for (int u = 0; u < 4; ++u) {
+                    const int l = l0 + u * W;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        k[u][j] = (l < n_part && j < P) ? part[((((int64_t)b * n_part + l) * P) + j) * nq + col] : 0ull;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (k[u][j] > mine[(P - 1) * THREADS]) list_insert<THREADS>(mine, P, k[u][j]);
             }
+        } else {
+            // a list is only walked further while its keys still beat this thread's current P-th best
+            for (int l0 = warp; l0 < n_part; l0 += 8 * W) {
+                unsigned long long head[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int l = l0 + u * W;
-                if (l >= n_part || head[u] <= mine[(P - 1) * THREADS]) continue;
-                list_insert<THREADS>(mine, P, head[u]);
-                const unsigned long long *src = part + (((int64_t)b * n_part + l) * P) * nq + col;
-                for (int j = 1; j < P; ++j) {
-                    unsigned long long key = src[(int64_t)j * nq];
-                    if (key <= mine[(P - 1) * THREADS]) break;      // source list is descending
-                    list_insert<THREADS>(mine, P, key);
+                for (int u = 0; u < 8; ++u) {
+                    const int l = l0 + u * W;
+                    head[u] = l < n_part ? part[(((int64_t)b * n_part + l) * P) * nq + col] : 0ull;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int l = l0 + u * W;
+                    if (l >= n_part || head[u] <= mine[(P - 1) * THREADS]) continue;
+                    list_insert<THREADS>(mine, P, head[u]);
+                    const unsigned long long *src = part + (((int64_t)b * n_part + l) * P) * nq + col;
+                    for (int j = 1; j < P; ++j) {
+                        unsigned long long key = src[(int64_t)j * nq];
+                        if (key <= mine[(P - 1) * THREADS]) break;      // source list is descending
+                        list_insert<THREADS>(mine, P, key);
+                    }
                 }
             }
         }
