@@ -4,17 +4,21 @@
 //                                                tokens -- applied to the centroid scores; integers, order-free)
 //   keep the n_prune candidates with the largest CI, ties towards the smaller document id.
 //
-// Two phases when q_len is 32, 64 or 128: cheap bounds lo(d) <= CI(d) <= hi(d) for every candidate from an 8-bit
-// copy of the table (ci_coarse_kernel), the documents whose hi reaches the n_prune-th largest lo (contender_kernel),
-// then exact CI and exact selection among those only.  Other q_len: exact CI for every candidate.
+// Two phases when q_len is 32 or 64: cheap bounds lo(d) <= CI(d) <= hi(d) for every candidate from an 8-bit copy of
+// the table (cand_range_kernel + ci_coarse_rng_kernel; ci_coarse_kernel for tables staged in shared memory and for
+// corpora of 2^31 tokens or more), the documents whose hi reaches the n_prune-th largest lo (contender kernels), then
+// exact CI (ci_wide_kernel) and the exact selection among those only.  Other q_len: exact CI for every candidate
+// (ci_kernel).
 //
 // ci_kernel: one warp per candidate document.  The document's centroid ids are streamed with coalesced 128-byte
 // loads (lane = token), each is broadcast with a shuffle, and the warp gathers the table row S[cid, :] with
 // lane = query token (one 128-byte line for 32 query tokens), keeping a running maximum per lane.
 //
-// select_kernel: one block per query.  Radix select (11 + 11 + 10 bits) of the n_prune-th largest CI, then an
+// select_kernel: one block per query.  Radix select (11 + 11 + 10 bits) of the n_prune-th largest score, then an
 // ordered compaction of the candidate list (which is ascending in id), so equal scores are resolved towards smaller
-// ids and the survivors come out ascending.
+// ids and the survivors come out ascending.  With few queries per call the contender and selection steps run over 32
+// blocks per query instead (contender_hist/count/write kernels, sels_* kernels), and shard_select_kernel merges the
+// lists of a document-sharded search.
 #include <limits.h>
 
 #include "common.cuh"
