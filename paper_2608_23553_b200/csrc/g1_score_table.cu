@@ -4,7 +4,7 @@
 // Each 23-bit integer is split into three balanced base-256 digits, so T = sum_{a,b} 256^(a+b) P_ab with the nine
 // digit-plane products P_ab = sum_d qa[d] * cb[d] being int8 x int8 -> int32 contractions (exact in any order).
 // Products of equal weight a+b share an accumulator (five accumulators, each |.| < 2^23); the epilogue recombines
-// them with shifts in int64 and rounds.
+// them with shifts (in 32-bit arithmetic, see combine_digits) and rounds.
 //
 // The contraction runs on the 5th-generation tensor cores: tcgen05.mma kind::i8 (int8 operands, int32 accumulators in
 // tensor memory), M = 128 centroids x N = 48 query tokens x K = 32 dimensions per instruction.  Both operands are
@@ -12,7 +12,8 @@
 // memory by TMA (plain per-CTA cp.async.bulk.tensor loads, no multicast).  One CTA owns a tile of 128 centroids (its
 // three digit planes stay in shared memory) and walks over tiles of 48 query-token rows, double-buffering the query
 // planes.  The five accumulators take 240 of the 256 tensor-memory columns a CTA allocates, so two CTAs share an SM and
-// one's epilogue overlaps the other's MMAs.  Every wait on an mbarrier is bounded; a wait that gives up sets the
+// one's epilogue overlaps the other's MMAs.  Twelve warps drain the accumulators (three per tensor-memory lane quarter,
+// chunks of eight columns, the next chunk's tcgen05.ld issued ahead) and store 32 bytes of the table per chunk.  Every wait on an mbarrier is bounded; a wait that gives up sets the
 // workspace's TIMEOUT status bit and the CTA frees its tensor memory and returns.
 #include <cuda.h>
 
