@@ -103,6 +103,7 @@ Layout make_layout(const Index &ix, const Params &p)
     L.hi = take(two_phase);
     L.cont = take(two_phase);
     L.cand_rng = take(2 * two_phase);
+    L.cont_rng = take(2 * two_phase);
     L.n_cont = take(B * sizeof(int32_t));
     L.pruned = take(B * p.n_prune * sizeof(int32_t));
     L.word_rank = take(B * (size_t)L.words * sizeof(int32_t));
@@ -258,19 +259,21 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             // bounds for every candidate, contenders for the top n_prune, exact CI and selection among those
             if ((rc = launch_coarse_bounds(ix, p, table8, cand, n_cand, lo, hi, (int2 *)(ws + L.cand_rng), st))) return rc;
             prof_mark(SLOT_CI, st);
-            if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, ci, st))) return rc;
+            if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, ci, (const int2 *)(ws + L.cand_rng),
+                                        (int2 *)(ws + L.cont_rng), st))) return rc;
             prof_mark(SLOT_SELECT, st);
             // blocks per query for the few contenders: one per SM in a large batch (measured best), four per SM
             // when a single query has the GPU to itself
             int exact_blocks = (4 * ix.sm_count + p.B - 1) / p.B;
             if (exact_blocks < ix.sm_count) exact_blocks = ix.sm_count;
-            if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, exact_blocks, SLOT_CI_EXACT, st)))
+            if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, exact_blocks, SLOT_CI_EXACT,
+                                                  ix.T < 0x7fffffffLL ? (const int2 *)(ws + L.cont_rng) : nullptr, st)))
                 return rc;
             prof_mark(SLOT_CI_EXACT, st);
             if ((rc = launch_select(ix, p, cont, n_cont, ci, pruned, n_pruned, pruned_ci, nullptr, st))) return rc;
             prof_mark(SLOT_SELECT, st);
         } else {
-            if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, 0, SLOT_CI, st))) return rc;
+            if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, ci, 0, SLOT_CI, nullptr, st))) return rc;
             prof_mark(SLOT_CI, st);
             if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, sel_scratch, st))) return rc;
             prof_mark(SLOT_SELECT, st);
@@ -306,7 +309,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if (taps->ci) {
                 if (two_phase) {                   // the search only needed exact CI for the contenders: the tap asks
                                                    // for every candidate, so the exact kernel runs over all of them
-                    if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, taps->ci, 0, SLOT_MISC, st)))
+                    if ((rc = launch_centroid_interaction(ix, p, table, cand, n_cand, taps->ci, 0, SLOT_MISC, nullptr, st)))
                         return rc;
                 } else if ((rc = copy_d2d(taps->ci, ci, cand_bytes, st))) return rc;
             }

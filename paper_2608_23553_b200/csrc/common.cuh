@@ -65,6 +65,7 @@ struct Layout {
     size_t hi;            // int32  [B][maxc]         upper bound
     size_t cont;          // int32  [B][maxc]         contender ids, ascending
     size_t cand_rng;      // int2   [B][maxc]         (first token, length) of each candidate (bound scan)
+    size_t cont_rng;      // int2   [B][maxc]         the same for the contenders
     size_t n_cont;        // int32  [B]
     size_t pruned;        // int32  [B][n_prune]
     size_t word_rank;     // int32  [B][words]        candidates before each bitmap word (document -> candidate index)
@@ -134,10 +135,14 @@ int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, 
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
                          const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, cudaStream_t st);
 // scratch: an int32 [B][maxc] array that is free during this step.
+// rng / cont_rng (may be NULL): the candidates' token ranges and where to put those of the contenders.
 int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
-                      const int32_t *hi, int32_t *cont, int32_t *n_cont, int32_t *scratch, cudaStream_t st);
+                      const int32_t *hi, int32_t *cont, int32_t *n_cont, int32_t *scratch, const int2 *rng,
+                      int2 *cont_rng, cudaStream_t st);
+// rng (may be NULL): the token ranges of the listed documents, in list order.
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
-                                const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, cudaStream_t st);
+                                const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, const int2 *rng,
+                                cudaStream_t st);
 // pruned_ci (may be NULL): the score of each kept document, INT_MIN in the padding.
 // scratch: select_split_scratch_bytes() bytes (few queries per call: several blocks per query), or NULL.
 bool select_split_used(const Index &ix, const Params &p);

@@ -142,6 +142,87 @@ ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__re
     }
 }
 
+// The wide variant over precomputed token ranges (first token, length) of the documents to score: a warp owns a
+// contiguous run of them and takes them 32 at a time -- one coalesced load of the ranges, handed out by shuffle, and the
+// first centroid ids of the next document fetched while the current one is scored -- instead of the dependent chain
+// id -> offsets -> centroid ids per document.
+template <int LPR>
+__global__ void __launch_bounds__(CI_THREADS)
+ci_wide_rng_kernel(const int32_t *__restrict__ table, int64_t K, const int2 *__restrict__ rng,
+                   const int32_t *__restrict__ n_docs, int64_t maxc, const int32_t *__restrict__ cids,
+                   int32_t *__restrict__ ci)
+{
+    constexpr int NQ = 4 * LPR;
+    constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
+    constexpr int UNROLL = 8;
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const int grp = lane / LPR, sub = lane % LPR;
+    const int n = n_docs[b];
+    const int4 *tb = reinterpret_cast<const int4 *>(table + (int64_t)b * K * NQ) + sub;
+    const int2 *rb = rng + (int64_t)b * maxc;
+    int32_t *out = ci + (int64_t)b * maxc;
+    const int warps_per_query = gridDim.x * CI_WARPS;
+    const int per_warp = (n + warps_per_query - 1) / warps_per_query;
+    const int wq = blockIdx.x * CI_WARPS + (threadIdx.x >> 5);
+    const int j_begin = wq * per_warp < n ? wq * per_warp : n;
+    const int j_end = j_begin + per_warp < n ? j_begin + per_warp : n;
+    for (int jb = j_begin; jb < j_end; jb += 32) {
+        const int cnt_docs = j_end - jb < 32 ? j_end - jb : 32;
+        const int2 mine = lane < cnt_docs ? rb[jb + lane] : make_int2(0, 1);
+        int my_sum = 0;
+        int32_t nx_cid;
+        {
+            const int t0 = __shfl_sync(0xffffffffu, mine.x, 0), len = __shfl_sync(0xffffffffu, mine.y, 0);
+            nx_cid = cids[(int64_t)t0 + (lane < len - 1 ? lane : len - 1)];
+        }
+        for (int di = 0; di < cnt_docs; ++di) {
+            const int t0 = __shfl_sync(0xffffffffu, mine.x, di), len = __shfl_sync(0xffffffffu, mine.y, di);
+            int32_t cidv = nx_cid;
+            if (di + 1 < cnt_docs) {
+                const int n0 = __shfl_sync(0xffffffffu, mine.x, di + 1), nl = __shfl_sync(0xffffffffu, mine.y, di + 1);
+                nx_cid = cids[(int64_t)n0 + (lane < nl - 1 ? lane : nl - 1)];
+            }
+            int4 m = make_int4(INT_MIN, INT_MIN, INT_MIN, INT_MIN);
+            for (int base = 0; base < len; base += 32) {
+                const int cnt = len - base < 32 ? len - base : 32;
+                // lanes past the end repeat the last token: a duplicate cannot change a maximum
+                if (base != 0) cidv = cids[(int64_t)t0 + base + (lane < cnt ? lane : cnt - 1)];
+                for (int s = 0; s * TPL < cnt; s += UNROLL) {
+                    int4 v[UNROLL];
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        int src = (s + u) * TPL + grp;
+                        src = src < 32 ? src : 31;    // lane 31 holds a valid (possibly repeated) token
+                        const int32_t c = __shfl_sync(0xffffffffu, cidv, src);
+                        v[u] = __ldg(tb + (int64_t)c * LPR);
+                    }
+#pragma unroll
+                    for (int u = 0; u < UNROLL; u += 2) {
+                        m.x = __vimax3_s32(m.x, v[u].x, v[u + 1].x);
+                        m.y = __vimax3_s32(m.y, v[u].y, v[u + 1].y);
+                        m.z = __vimax3_s32(m.z, v[u].z, v[u + 1].z);
+                        m.w = __vimax3_s32(m.w, v[u].w, v[u + 1].w);
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = LPR; o < 32; o <<= 1) {           // merge the TPL lane groups
+                m.x = max(m.x, __shfl_xor_sync(0xffffffffu, m.x, o));
+                m.y = max(m.y, __shfl_xor_sync(0xffffffffu, m.y, o));
+                m.z = max(m.z, __shfl_xor_sync(0xffffffffu, m.z, o));
+                m.w = max(m.w, __shfl_xor_sync(0xffffffffu, m.w, o));
+            }
+            int sum = m.x + m.y + m.z + m.w;
+#pragma unroll
+            for (int o = LPR >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            sum = __shfl_sync(0xffffffffu, sum, 0);
+            if (lane == di) my_sum = sum;
+        }
+        if (lane < cnt_docs) out[jb + lane] = my_sum;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ coarse bounds --
 // Bounds on CI from the 8-bit table U8[c, i] = min((S[c, i] + 2^24 + 64) >> 17, 255) (stage 1 writes it next to the
 // exact table; S + 2^24 + 64 > 0 always).  The map is monotone, so with m_i = max_t U8[cid_t, i]
@@ -432,6 +513,17 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
                          const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, cudaStream_t st)
 {
     const size_t table_bytes = (size_t)ix.K * p.nq;
+    // the candidates' token ranges, for this scan and for the exact scoring of the contenders afterwards
+    const bool use_rng = ix.T < 0x7fffffffLL && rng != nullptr;
+    if (use_rng) {
+        int64_t rb = ((int64_t)ix.sm_count * 8 + p.B - 1) / p.B;
+        const int64_t rwant = (p.maxc + 255) / 256;
+        if (rb > rwant) rb = rwant;
+        if (rb < 1) rb = 1;
+        cand_range_kernel<<<dim3((unsigned)rb, (unsigned)p.B), 256, 0, st>>>(cand, n_cand, p.maxc, ix.doc_off, rng);
+        CHIMERA_CUDA(cudaGetLastError());
+        count_launch(SLOT_CI);
+    }
     if (table_bytes <= 160 * 1024) {
         // the whole 8-bit table of a query fits in shared memory: stage it once per block and look rows up there
         constexpr int T = 512;
@@ -472,19 +564,13 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
     if (per_query < 1) per_query = 1;
     const unsigned gx = (unsigned)per_query;
     dim3 grid(gx, (unsigned)p.B);
-    if (ix.T < 0x7fffffffLL && rng != nullptr) {
-        int64_t rb = ((int64_t)ix.sm_count * 8 + p.B - 1) / p.B;
-        const int64_t rwant = (p.maxc + 255) / 256;
-        if (rb > rwant) rb = rwant;
-        if (rb < 1) rb = 1;
-        cand_range_kernel<<<dim3((unsigned)rb, (unsigned)p.B), 256, 0, st>>>(cand, n_cand, p.maxc, ix.doc_off, rng);
-        CHIMERA_CUDA(cudaGetLastError());
+    if (use_rng) {
         if (p.nq == 32)
             ci_coarse_rng_kernel<2><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
         else
             ci_coarse_rng_kernel<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
         CHIMERA_CUDA(cudaGetLastError());
-        count_launch(SLOT_CI, 2);
+        count_launch(SLOT_CI);
         return CHIMERA_OK;
     }
     if (p.nq == 32)
@@ -518,7 +604,8 @@ int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, 
 
 // Exact CI of a list of documents.  blocks_cap bounds the blocks per query (0 = default).
 int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t *table, const int32_t *cand,
-                                const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, cudaStream_t st)
+                                const int32_t *n_cand, int32_t *ci, int blocks_cap, int slot, const int2 *rng,
+                                cudaStream_t st)
 {
     int64_t want = (p.maxc + CI_WARPS - 1) / CI_WARPS;
     int64_t cap = blocks_cap > 0 ? blocks_cap : (int64_t)ix.sm_count * 8;
@@ -526,6 +613,15 @@ int launch_centroid_interaction(const Index &ix, const Params &p, const int32_t 
     if (gx < 1) gx = 1;
     dim3 grid(gx, (unsigned)p.B);
     const int nqw = (p.nq + 31) / 32;
+    if (rng != nullptr && (p.nq == 32 || p.nq == 64)) {       // the listed documents' token ranges are known
+        if (p.nq == 32)
+            ci_wide_rng_kernel<8><<<grid, CI_THREADS, 0, st>>>(table, ix.K, rng, n_cand, p.maxc, ix.cids, ci);
+        else
+            ci_wide_rng_kernel<16><<<grid, CI_THREADS, 0, st>>>(table, ix.K, rng, n_cand, p.maxc, ix.cids, ci);
+        CHIMERA_CUDA(cudaGetLastError());
+        count_launch(slot);
+        return CHIMERA_OK;
+    }
     if (p.nq == 32)
         ci_wide_kernel<8><<<grid, CI_THREADS, 0, st>>>(table, ix.K, cand, n_cand, p.maxc, ix.cids, ix.doc_off, ci);
     else if (p.nq == 64)
@@ -703,7 +799,7 @@ constexpr int CONT_BINS = 8192;
 __global__ void __launch_bounds__(SEL_THREADS)
 contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, const int32_t *__restrict__ lo,
                  const int32_t *__restrict__ hi, int64_t maxc, int n_prune, int nq, int32_t *__restrict__ cont,
-                 int32_t *__restrict__ n_cont)
+                 int32_t *__restrict__ n_cont, const int2 *__restrict__ rng, int2 *__restrict__ cont_rng)
 {
     __shared__ int hist[CONT_BINS];
     __shared__ int warp_part[32];
@@ -714,8 +810,13 @@ contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n
     const int32_t *lb = lo + (int64_t)b * maxc;
     const int32_t *hb = hi + (int64_t)b * maxc;
     int32_t *out = cont + (int64_t)b * maxc;
+    const int2 *rb = rng ? rng + (int64_t)b * maxc : nullptr;
+    int2 *orng = cont_rng ? cont_rng + (int64_t)b * maxc : nullptr;
     if (n <= n_prune) {
-        for (int j = threadIdx.x; j < n; j += SEL_THREADS) out[j] = cb[j];
+        for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
+            out[j] = cb[j];
+            if (orng) orng[j] = rb[j];
+        }
         if (threadIdx.x == 0) n_cont[b] = n;
         return;
     }
@@ -768,7 +869,11 @@ contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n
         int pos = run + sel_block_scan(keep, &tot, warp_part);
 #pragma unroll
         for (int e = 0; e < 8; ++e)
-            if (j0 + e < n && hv[e] >= tau) out[pos++] = cb[j0 + e];
+            if (j0 + e < n && hv[e] >= tau) {
+                out[pos] = cb[j0 + e];
+                if (orng) orng[pos] = rb[j0 + e];
+                ++pos;
+            }
         run += tot;
     }
     if (threadIdx.x == 0) n_cont[b] = run;
@@ -936,7 +1041,8 @@ contender_count_kernel(const int32_t *__restrict__ n_cand, const int32_t *__rest
 __global__ void __launch_bounds__(SEL_THREADS)
 contender_write_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand,
                        const int32_t *__restrict__ hi, int64_t maxc, const int32_t *__restrict__ scratch,
-                       int32_t *__restrict__ cont, int32_t *__restrict__ n_cont)
+                       int32_t *__restrict__ cont, int32_t *__restrict__ n_cont, const int2 *__restrict__ rng,
+                       int2 *__restrict__ cont_rng)
 {
     __shared__ int warp_part[32];
     const int b = blockIdx.y, n = n_cand[b], g = blockIdx.x;
@@ -949,6 +1055,8 @@ contender_write_kernel(const int32_t *__restrict__ cand, const int32_t *__restri
     const int32_t *cb = cand + (int64_t)b * maxc;
     const int32_t *hb = hi + (int64_t)b * maxc;
     int32_t *out = cont + (int64_t)b * maxc;
+    const int2 *rb = rng ? rng + (int64_t)b * maxc : nullptr;
+    int2 *orng = cont_rng ? cont_rng + (int64_t)b * maxc : nullptr;
     int run = offset;
     for (int base = j0; base < j1; base += 4 * SEL_THREADS) {
         const int q0 = base + 4 * threadIdx.x;
@@ -962,7 +1070,11 @@ contender_write_kernel(const int32_t *__restrict__ cand, const int32_t *__restri
         int pos = run + sel_block_scan(keep, &tot, warp_part);
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-            if (q0 + e < j1 && hv[e] >= tau) out[pos++] = cb[q0 + e];
+            if (q0 + e < j1 && hv[e] >= tau) {
+                out[pos] = cb[q0 + e];
+                if (orng) orng[pos] = rb[q0 + e];
+                ++pos;
+            }
         run += tot;
     }
     if (g == CONT_SPLIT - 1 && threadIdx.x == 0) n_cont[b] = run;
@@ -970,8 +1082,10 @@ contender_write_kernel(const int32_t *__restrict__ cand, const int32_t *__restri
 
 // scratch: an int32 [B][maxc] array that is free during this step (the exact-CI output buffer).
 int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,
-                      const int32_t *hi, int32_t *cont, int32_t *n_cont, int32_t *scratch, cudaStream_t st)
+                      const int32_t *hi, int32_t *cont, int32_t *n_cont, int32_t *scratch, const int2 *rng,
+                      int2 *cont_rng, cudaStream_t st)
 {
+    if (ix.T >= 0x7fffffffLL) { rng = nullptr; cont_rng = nullptr; }      // the bound scan wrote no ranges
     if (4 * p.B <= ix.sm_count && p.maxc >= CONT_BINS + CONT_SPLIT + 1) {
         // few queries: CONT_SPLIT blocks each
         CHIMERA_CUDA(cudaMemset2DAsync(scratch, sizeof(int32_t) * (size_t)p.maxc, 0, sizeof(int32_t) * CONT_BINS,
@@ -981,13 +1095,13 @@ int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, con
         CHIMERA_CUDA(cudaGetLastError());
         contender_count_kernel<<<grid, SEL_THREADS, 0, st>>>(n_cand, hi, p.maxc, p.n_prune, p.nq, scratch);
         CHIMERA_CUDA(cudaGetLastError());
-        contender_write_kernel<<<grid, SEL_THREADS, 0, st>>>(cand, n_cand, hi, p.maxc, scratch, cont, n_cont);
+        contender_write_kernel<<<grid, SEL_THREADS, 0, st>>>(cand, n_cand, hi, p.maxc, scratch, cont, n_cont, rng, cont_rng);
         CHIMERA_CUDA(cudaGetLastError());
         count_launch(SLOT_SELECT, 3);
         return CHIMERA_OK;
     }
     contender_kernel<<<(unsigned)p.B, SEL_THREADS, 0, st>>>(cand, n_cand, lo, hi, p.maxc, p.n_prune, p.nq, cont,
-                                                            n_cont);
+                                                            n_cont, rng, cont_rng);
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_SELECT);
     return CHIMERA_OK;
