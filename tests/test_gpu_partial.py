@@ -88,6 +88,13 @@ def test_partial_refinement_mid_batch256_sampled():
     for lo, hi in ((0, 1), (100, 103)):
         small = gix.search(qd[lo:hi].contiguous(), cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
         assert torch.equal(small[0], big[0][lo:hi]) and torch.equal(small[1], big[1][lo:hi])
+    # and the same single-query search replayed from a CUDA graph (the multi-block selection clears its histograms
+    # with a memset node)
+    g = pkg.GraphedSearch(gix, 1, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
+    for b in (0, 17):
+        ids_g, sc_g = g(qd[b:b + 1])
+        torch.cuda.synchronize()
+        assert torch.equal(ids_g, big[0][b:b + 1]) and torch.equal(sc_g, big[1][b:b + 1])
 
 
 def test_partial_and_rabitq_edge_cases():
