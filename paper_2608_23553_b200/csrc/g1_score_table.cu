@@ -145,8 +145,9 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
         const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
         // (query, token) coordinates of the tile's first row: one 32-bit division per tile
         const uint32_t tile_qb = ((uint32_t)t * G1_N) / unq, tile_qi = (uint32_t)t * G1_N - tile_qb * unq;
-        // Each warp takes every G1_WPQ-th chunk.  The tensor-memory loads of the next
+        // Each warp takes one pair of adjacent chunks.  The tensor-memory loads of the next
         // chunk are issued before the current one is recombined and stored, so their latency hides behind that work.
+        uint32_t w8_carry[2] = {0u, 0u};                  // 8-bit words of the even chunk of a pair
         auto emit = [&](const int32_t (&acc)[5][8], const int chunk) {
             int32_t out[8];
 #pragma unroll
@@ -168,7 +169,14 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                         for (int e = 0; e < 4; ++e) v[e] = (uint32_t)min((out[4 * g + e] + (1 << 24) + 64) >> 17, 255);
                         w[g] = __byte_perm(__byte_perm(v[0], v[1], 0x0040), __byte_perm(v[2], v[3], 0x0040), 0x5410);
                     }
-                    *reinterpret_cast<uint2 *>(table8 + ((int64_t)qb * K + c) * nq + qi) = make_uint2(w[0], w[1]);
+                    // a warp's two chunks are adjacent (16 query tokens of one query): one 16-byte store for the pair
+                    if ((chunk & 1) == 0) {
+                        w8_carry[0] = w[0];
+                        w8_carry[1] = w[1];
+                    } else {
+                        *reinterpret_cast<uint4 *>(table8 + ((int64_t)qb * K + c) * nq + qi - 8) =
+                            make_uint4(w8_carry[0], w8_carry[1], w[0], w[1]);
+                    }
                 }
                 if ((nq & 7) == 0) {
                     // the chunk's eight values are consecutive tokens of one query, 32-byte aligned: one store
@@ -197,7 +205,8 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
             }
         };
         constexpr int CHUNKS_PER_WARP = (G1_N / 8) / G1_WPQ;
-        const int first_chunk = warp >> 2;
+        static_assert(CHUNKS_PER_WARP == 2, "a warp drains one pair of adjacent chunks");
+        const int first_chunk = 2 * (warp >> 2);
         int32_t accs[2][5][8];
 #pragma unroll
         for (int w = 0; w < 5; ++w) tmem_ld8(lane_addr + w * G1_N + first_chunk * 8, accs[0][w]);
@@ -207,9 +216,9 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
             if (it + 1 < CHUNKS_PER_WARP) {
 #pragma unroll
                 for (int w = 0; w < 5; ++w)
-                    tmem_ld8(lane_addr + w * G1_N + (first_chunk + G1_WPQ * (it + 1)) * 8, accs[(it + 1) & 1][w]);
+                    tmem_ld8(lane_addr + w * G1_N + (first_chunk + (it + 1)) * 8, accs[(it + 1) & 1][w]);
             }
-            emit(accs[it & 1], first_chunk + G1_WPQ * it);
+            emit(accs[it & 1], first_chunk + it);
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();                   // accumulators drained before the next tile overwrites them
