@@ -159,14 +159,14 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
             while (qi >= unq) { qi -= unq; ++qb; }
             if (c < K && r0 < rows32) {
                 if (table8 != nullptr) {
-                    // coarse copy for the bound phase of stage 3: min((S + 2^24 + 64) >> 17, 255); q_len is a multiple
+                    // coarse copy for the bound phase of stage 3: clamp(S >> 16, 0, 255); q_len is a multiple
                     // of 16 here, so the 8 rows of a chunk belong to one query and the store is 8-byte aligned
                     uint32_t w[2];
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
                         uint32_t v[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) v[e] = (uint32_t)min((out[4 * g + e] + (1 << 24) + 64) >> 17, 255);
+                        for (int e = 0; e < 4; ++e) v[e] = (uint32_t)min(max(out[4 * g + e] >> 16, 0), 255);
                         w[g] = __byte_perm(__byte_perm(v[0], v[1], 0x0040), __byte_perm(v[2], v[3], 0x0040), 0x5410);
                     }
                     // a warp's two chunks are adjacent (16 query tokens of one query): one 16-byte store for the pair

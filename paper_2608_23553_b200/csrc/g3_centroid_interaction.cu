@@ -224,13 +224,31 @@ ci_wide_rng_kernel(const int32_t *__restrict__ table, int64_t K, const int2 *__r
 }
 
 // ------------------------------------------------------------------------------------------------ coarse bounds --
-// Bounds on CI from the 8-bit table U8[c, i] = min((S[c, i] + 2^24 + 64) >> 17, 255) (stage 1 writes it next to the
-// exact table; S + 2^24 + 64 > 0 always).  The map is monotone, so with m_i = max_t U8[cid_t, i]
-//     lo(d) = sum_i (2^17 m_i - 2^24 - 64)  <=  CI(d)  <=  lo(d) + nq (2^17 - 1) + 2^18 #{i : m_i = 255} = hi(d)
-// (the last term covers the saturated top bucket).  A row of U8 is q_len bytes -- one 32-byte sector for 32 query
+// Bounds on CI from the 8-bit table U8[c, i] = clamp(S[c, i] >> 16, 0, 255) (stage 1 writes it next to the exact
+// table): 256 buckets of width 2^16 over [0, 2^24), everything negative in bucket 0, everything from 255 * 2^16 up in
+// bucket 255 (|S| <= 2^24 + 64).  The map is monotone, so m_i = max_t U8[cid_t, i] is the bucket of the exact maximum:
+//     2^16 m_i <= max_t S <= 2^16 m_i + 2^16 - 1        for 0 < m_i < 255,
+// the lower end drops to -(2^24 + 64) for m_i = 0 and the upper end rises to 2^24 + 64 for m_i = 255.  With
+// sum = sum_i m_i, zeros = #{i : m_i = 0}, sat = #{i : m_i = 255}:
+//     lo(d) = 2^16 sum - zeros (2^24 + 64)  <=  CI(d)  <=  2^16 sum + nq (2^16 - 1) + 65 sat = hi(d).
+// (The scores that decide a maximum are positive -- a document token close to the query token -- so the buckets are
+// spent on [0, 1) and a column whose best score is negative only loosens lo.)  A row of U8 is q_len bytes -- one
+// 32-byte sector for 32 query
 // tokens instead of four -- and a lane's 16-byte load covers 16 query tokens, so one warp load covers 32 / LPR tokens
 // (LPR = q_len / 16 lanes per row).  Bytes are widened to pairs of 16-bit integers with one byte-permute per pair and
 // the running maxima fold two rows per instruction with the three-input packed 16-bit integer maximum.
+// packed = sum | sat << 16 | zeros << 24 (see above)
+__device__ __forceinline__ int32_t coarse_lo(int packed)
+{
+    return ((packed & 0xffff) << 16) - (packed >> 24) * ((1 << 24) + 64);
+}
+__device__ __forceinline__ int32_t coarse_hi(int packed, int nq)
+{
+    return ((packed & 0xffff) << 16) + nq * ((1 << 16) - 1) + ((packed >> 16) & 0xff) * 65;
+}
+// The histogram key of a lower bound in the contender step: floor(lo / 2^16) clamped at 0 -- a valid, slightly smaller
+// lower bound (documents with an empty column fall to the bottom, which only lowers the threshold).
+__device__ __forceinline__ int coarse_key(int32_t lo) { return lo < 0 ? 0 : lo >> 16; }
 __device__ __forceinline__ void coarse_accumulate2(uint32_t (&m)[8], const int4 &va, const int4 &vb)
 {
     const uint32_t a[4] = {(uint32_t)va.x, (uint32_t)va.y, (uint32_t)va.z, (uint32_t)va.w};
@@ -349,15 +367,13 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
         }
         // every lane now holds the maxima of two columns; sum over columns (skipping duplicate lanes)
         const int u_lo = (int)(m[0] & 0xffffu), u_hi = (int)(m[0] >> 16);
-        int packed = 0;                                         // sum of maxima | saturated count << 20
+        int packed = 0;                                         // sum of maxima | saturated << 16 | zeros << 24
         if ((lane & dup_mask) == 0)
-            packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 20);
-        packed = __reduce_add_sync(0xffffffffu, packed);        // sum <= 255 * 64 < 2^20, count <= 64
-        const int sum = packed & 0xfffff, sat = packed >> 20;
+            packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 16) + (((u_lo == 0) + (u_hi == 0)) << 24);
+        packed = __reduce_add_sync(0xffffffffu, packed);        // sum <= 255 * 64 < 2^16, counts <= 64
         if (lane == 0) {
-            const int l = (sum - 128 * NQ) * (1 << 17) - 64 * NQ;
-            lo[(int64_t)b * maxc + j] = l;
-            hi[(int64_t)b * maxc + j] = l + NQ * ((1 << 17) - 1) + sat * (1 << 18);
+            lo[(int64_t)b * maxc + j] = coarse_lo(packed);
+            hi[(int64_t)b * maxc + j] = coarse_hi(packed, NQ);
         }
     }
 }
@@ -490,14 +506,13 @@ ci_coarse_rng_kernel(const uint8_t *__restrict__ table8, int64_t K, const int2 *
                 }
             }
             const int u_lo = (int)(m[0] & 0xffffu), u_hi = (int)(m[0] >> 16);
-            int packed = 0;                                         // sum of maxima | saturated count << 20
+            int packed = 0;                                         // sum of maxima | saturated << 16 | zeros << 24
             if ((lane & dup_mask) == 0)
-                packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 20);
+                packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 16) + (((u_lo == 0) + (u_hi == 0)) << 24);
             packed = __reduce_add_sync(0xffffffffu, packed);
             if (lane == di) {                                       // lane di keeps the result of document di
-                const int sum = packed & 0xfffff, sat = packed >> 20;
-                my_lo = (sum - 128 * NQ) * (1 << 17) - 64 * NQ;
-                my_hi = my_lo + NQ * ((1 << 17) - 1) + sat * (1 << 18);
+                my_lo = coarse_lo(packed);
+                my_hi = coarse_hi(packed, NQ);
             }
         }
         if (lane < cnt) {
@@ -589,8 +604,8 @@ __global__ void coarse_table_kernel(const int32_t *__restrict__ table, int64_t n
 {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) {
-        int v = (table[i] + (1 << 24) + 64) >> 17;
-        table8[i] = (uint8_t)(v > 255 ? 255 : v);
+        const int v = table[i] >> 16;
+        table8[i] = (uint8_t)(v < 0 ? 0 : v > 255 ? 255 : v);
     }
 }
 int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st)
@@ -792,9 +807,10 @@ select_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_ca
 
 // grid (B).  Contenders for the top n_prune: with tau = the n_prune-th largest lower bound, every document of the
 // true top n_prune has hi >= CI >= (n_prune-th largest CI) >= tau.  Writes their ids (ascending) and their number.
-// The lower bounds are lo = (sum - 128 nq) 2^17 - 64 nq with sum = the sum of nq 8-bit maxima (ci_coarse_kernel), so
-// sum itself is a key of at most 14 bits: one histogram sweep over CONT_BINS bins (two neighbouring sums share a bin
-// for q_len 64; tau is then the smaller of the two, still a valid lower threshold) finds tau without radix passes.
+// The lower bounds are lo = 2^16 sum - zeros (2^24 + 64) with sum = the sum of nq 8-bit maxima (coarse_lo), so
+// coarse_key(lo) = floor(lo / 2^16), clamped at 0, is a key of at most 14 bits and 2^16 key <= lo: one histogram sweep
+// over CONT_BINS bins (two neighbouring keys share a bin for q_len 64; tau is then the smaller of the two, still a
+// valid lower threshold) finds tau without radix passes.
 constexpr int CONT_BINS = 8192;
 __global__ void __launch_bounds__(SEL_THREADS)
 contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n_cand, const int32_t *__restrict__ lo,
@@ -833,7 +849,7 @@ contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
             const int j = base + e * SEL_THREADS + threadIdx.x;
-            if (j < n) atomicAdd(&hist[(((v[e] + 64 * nq) >> 17) + 128 * nq) >> bin_shift], 1);
+            if (j < n) atomicAdd(&hist[coarse_key(v[e]) >> bin_shift], 1);
         }
     }
     __syncthreads();
@@ -853,7 +869,7 @@ contender_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ n
         }
     }
     __syncthreads();
-    const int32_t tau = ((s_bin << bin_shift) - 128 * nq) * (1 << 17) - 64 * nq;   // smallest lower bound in that bin
+    const int32_t tau = (s_bin << bin_shift) << 16;                 // smallest lower bound of that bin
     // ordered compaction, eight consecutive entries per thread and round (one block scan per 8192 entries); the ids
     // are only read for the few entries that are kept
     int run = 0;
@@ -990,7 +1006,7 @@ contender_hist_kernel(const int32_t *__restrict__ n_cand, const int32_t *__restr
     for (int i = threadIdx.x; i < CONT_BINS; i += SEL_THREADS) hist[i] = 0;
     __syncthreads();
     for (int j = j0 + threadIdx.x; j < j1; j += SEL_THREADS)
-        atomicAdd(&hist[(((lb[j] + 64 * nq) >> 17) + 128 * nq) >> bin_shift], 1);
+        atomicAdd(&hist[coarse_key(lb[j]) >> bin_shift], 1);
     __syncthreads();
     int32_t *gh = scratch + (int64_t)b * maxc;
     for (int i = threadIdx.x; i < CONT_BINS; i += SEL_THREADS)
@@ -1023,7 +1039,7 @@ contender_count_kernel(const int32_t *__restrict__ n_cand, const int32_t *__rest
             }
         }
         __syncthreads();
-        tau = ((s_bin << bin_shift) - 128 * nq) * (1 << 17) - 64 * nq;
+        tau = (s_bin << bin_shift) << 16;
     }
     int j0, j1;
     cont_slice(n, blockIdx.x, &j0, &j1);
