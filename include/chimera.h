@@ -24,6 +24,9 @@
  *   - Every function returns a chimera_status; chimera_last_error() gives a text for the calling thread's last
  *     failure.  No function throws, traps the device, or leaves a kernel waiting on anything.
  *   - Search calls only enqueue work (they are asynchronous to the host) unless stated otherwise.
+ *   - Searches on one index from several host threads are safe when each uses its own workspace and stream (the
+ *     index is read-only after its build / enable / attach calls, which must not overlap a search); the profiling
+ *     calls are for one thread.
  */
 #ifndef CHIMERA_H
 #define CHIMERA_H

@@ -3,6 +3,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
 #include <new>
 
 #include "common.cuh"
@@ -32,10 +33,12 @@ struct ProfCall {
 static bool g_prof_on = false;
 static ProfCall g_calls[CHIMERA_PROFILE_MAX_CALLS];
 static int g_n_calls = 0;
-static int64_t g_launches[CHIMERA_PROFILE_SLOTS] = {0};
+// launch counters are bumped by every search, from whichever host thread calls it; the per-call timing marks below
+// belong to one profiling thread (chimera_profile_enable's caller)
+static std::atomic<int64_t> g_launches[CHIMERA_PROFILE_SLOTS];
 static ProfCall *g_cur = nullptr;
 
-void count_launch(int slot, int n) { g_launches[slot] += n; }
+void count_launch(int slot, int n) { g_launches[slot].fetch_add(n, std::memory_order_relaxed); }
 
 static void prof_begin(cudaStream_t st)
 {
@@ -630,7 +633,7 @@ int chimera_profile_enable(int32_t on)
 int chimera_profile_read(float *ms, int64_t *launches)
 {
     if (!ms || !launches) return fail(CHIMERA_INVALID_ARG, "NULL argument");
-    for (int s = 0; s < CHIMERA_PROFILE_SLOTS; ++s) { ms[s] = 0.f; launches[s] = g_launches[s]; g_launches[s] = 0; }
+    for (int s = 0; s < CHIMERA_PROFILE_SLOTS; ++s) { ms[s] = 0.f; launches[s] = g_launches[s].exchange(0, std::memory_order_relaxed); }
     for (int c = 0; c < g_n_calls; ++c) {
         ProfCall &pc = g_calls[c];
         if (pc.n < 2) continue;
