@@ -4,8 +4,9 @@
 // One block per query.  Each (score, id) becomes a 64-bit key whose unsigned order is (score desc, id asc); the keys
 // are sorted descending with a bitonic network in shared memory (n_prune <= 16384 keys = 128 KB) and the first k are
 // decoded back.  For k <= 16 the keys stay in registers instead and the block extracts its maximum k times (two
-// barriers per result instead of the network's log^2 stages): the shorter chain matters when one query is served at
-// a time.
+// barriers per result instead of the network's log^2 stages), and for k <= 128 over at most 4096 entries the warps sort
+// 128-key runs in registers and merge them pairwise, keeping the better half each time: the shorter chains matter
+// when one query is served at a time.
 #include <math.h>
 
 #include "common.cuh"
@@ -17,6 +18,7 @@ constexpr int TOPK_THREADS = 1024;
 __device__ __forceinline__ uint32_t float_order(float f)
 {
     uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;        // -0 and +0 are the same score (the tie goes to the smaller id)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 __device__ __forceinline__ float float_unorder(uint32_t o)
@@ -125,6 +127,106 @@ topk_small_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ 
     }
 }
 
+// 16 < k <= 128 and at most 4096 entries: the full network's ~80 block barriers are what a single query waits for, so
+// here every warp sorts its own 128 keys in registers (element e * 32 + lane in register e; strides below 32 are
+// shuffles, 32 and 64 are register pairs), and the 32 sorted runs are then merged pairwise in five rounds through
+// shared memory, each merge keeping only the 128 best of its 256 keys: max(A[i], B[127 - i]) of two descending runs is
+// a bitonic sequence holding exactly those, and one bitonic merge sorts it again.  Six block barriers in all.
+constexpr int RUN = 128;                 // keys per warp and per run
+
+__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long v, int o)
+{
+    return __shfl_xor_sync(0xffffffffu, v, o);
+}
+// one compare-exchange stage with partner index i ^ stride over the warp's 128 keys; desc[e] = the direction of the
+// block that element e * 32 + lane lies in
+__device__ __forceinline__ void run_stage(unsigned long long (&key)[4], int stride, const bool (&desc)[4], int lane)
+{
+    if (stride < 32) {
+        const bool lower = (lane & stride) == 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const unsigned long long other = shfl_xor_u64(key[e], stride);
+            const bool take_max = lower == desc[e];
+            const unsigned long long hi = key[e] > other ? key[e] : other, lo = key[e] > other ? other : key[e];
+            key[e] = take_max ? hi : lo;
+        }
+    } else {
+        const int d = stride >> 5;       // 1: pairs (0,1), (2,3); 2: pairs (0,2), (1,3)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if ((e & d) == 0) {
+                unsigned long long &a = key[e], &b = key[e | d];
+                const unsigned long long hi = a > b ? a : b, lo = a > b ? b : a;
+                a = desc[e] ? hi : lo;
+                b = desc[e] ? lo : hi;
+            }
+        }
+    }
+}
+// bitonic merge of a bitonic 128-key sequence into descending order
+__device__ __forceinline__ void run_merge_desc(unsigned long long (&key)[4], int lane)
+{
+    const bool desc[4] = {true, true, true, true};
+#pragma unroll
+    for (int stride = 64; stride > 0; stride >>= 1) run_stage(key, stride, desc, lane);
+}
+
+__global__ void __launch_bounds__(TOPK_THREADS)
+topk_runs_kernel(const int32_t *__restrict__ pruned, const float *__restrict__ score4, int n_prune, int k, int seg_len,
+                 long long seg_stride, int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
+{
+    extern __shared__ unsigned long long runs[];           // [32][RUN] then [16][RUN]
+    unsigned long long *buf0 = runs, *buf1 = runs + 32 * RUN;
+    const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long key[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = warp * RUN + e * 32 + lane;
+        key[e] = 0ull;
+        if (j < n_prune) {
+            const int64_t at = entry_index(j, b, seg_len, seg_stride);
+            const int32_t id = pruned[at];
+            if (id >= 0)
+                key[e] = ((unsigned long long)float_order(score4[at]) << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
+        }
+    }
+    // the warp's 128 keys, descending
+#pragma unroll
+    for (int size = 2; size <= RUN; size <<= 1) {
+        bool desc[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) desc[e] = ((e * 32 + lane) & size) == 0;
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) run_stage(key, stride, desc, lane);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) buf0[warp * RUN + e * 32 + lane] = key[e];
+    __syncthreads();
+    unsigned long long *src = buf0, *dst = buf1;
+    for (int n_runs = 32; n_runs > 1; n_runs >>= 1) {
+        if (warp < (n_runs >> 1)) {
+            const unsigned long long *A = src + (2 * warp) * RUN, *B = src + (2 * warp + 1) * RUN;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int i = e * 32 + lane;
+                const unsigned long long a = A[i], c = B[RUN - 1 - i];
+                key[e] = a > c ? a : c;
+            }
+            run_merge_desc(key, lane);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) dst[warp * RUN + e * 32 + lane] = key[e];
+        }
+        __syncthreads();
+        unsigned long long *t = src; src = dst; dst = t;
+    }
+    for (int r = threadIdx.x; r < k; r += TOPK_THREADS) {
+        const unsigned long long v = src[r];
+        out_ids[(int64_t)b * k + r] = v ? (int32_t)(0xFFFFFFFFu - (uint32_t)v) : -1;
+        out_scores[(int64_t)b * k + r] = v ? float_unorder((uint32_t)(v >> 32)) : -INFINITY;
+    }
+}
+
 // n entries per query (laid out by entry_index) -> the best k.
 static int launch_topk_entries(const int32_t *ids, const float *scores, int B, int n, int k, int seg_len,
                                long long seg_stride, int32_t *out_ids, float *out_scores, cudaStream_t st)
@@ -139,6 +241,12 @@ static int launch_topk_entries(const int32_t *ids, const float *scores, int B, i
         else
             topk_small_kernel<16><<<(unsigned)B, TOPK_THREADS, 0, st>>>(ids, scores, n, k, seg_len, seg_stride, out_ids,
                                                                         out_scores);
+        CHIMERA_CUDA(cudaGetLastError());
+        return CHIMERA_OK;
+    }
+    if (k <= RUN && n <= 32 * RUN) {
+        topk_runs_kernel<<<(unsigned)B, TOPK_THREADS, sizeof(unsigned long long) * 48 * RUN, st>>>(
+            ids, scores, n, k, seg_len, seg_stride, out_ids, out_scores);
         CHIMERA_CUDA(cudaGetLastError());
         return CHIMERA_OK;
     }

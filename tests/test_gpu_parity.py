@@ -229,6 +229,40 @@ def test_tiny_config_stage_isolated(chimera, tiny):
         assert np.array_equal(ids[b].cpu().numpy(), r.ids) and np.array_equal(sc[b].cpu().numpy(), r.scores)
 
 
+@pytest.mark.parametrize("n_prune,k", [(17, 17), (100, 128), (128, 100), (129, 64), (1000, 100), (2048, 50),
+                                        (4096, 100), (4096, 128), (4097, 100), (5000, 129), (3000, 10), (300, 1000)])
+def test_topk_stage_alone_equals_a_plain_sort(chimera, tiny, n_prune, k):
+    """Stage 5 on crafted survivors (every kernel variant: k <= 16, k <= 128 over <= 4096 entries, the full network):
+    many equal scores, -1 padding inside the valid count's tail, fewer survivors than k.  Expected = Definition 2
+    written as a sort by (score descending, id ascending)."""
+    cfg, oix, gix, q = tiny
+    B = 3
+    rng = np.random.default_rng(n_prune * 1000 + k)
+    dev = torch.device("cuda:0")
+    pruned = np.full((B, n_prune), -1, dtype=np.int32)
+    score4 = np.full((B, n_prune), -np.inf, dtype=np.float32)
+    n_pruned = np.array([n_prune, max(1, n_prune // 3), min(n_prune, 5)], dtype=np.int32)
+    for b in range(B):
+        m = int(n_pruned[b])
+        pruned[b, :m] = np.sort(rng.choice(oix.N, size=m, replace=False)).astype(np.int32)
+        # few distinct values (ties decided by id), both signs, and exact zeros
+        score4[b, :m] = rng.choice(np.array([-3.5, -0.0, 0.0, 1.25, 1.25000012, 7.0, 19.75], dtype=np.float32), size=m)
+    t = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, n_prune)
+    t.pruned, t.n_pruned = torch.from_numpy(pruned).to(dev), torch.from_numpy(n_pruned).to(dev)
+    t.score4 = torch.from_numpy(score4).to(dev)
+    ids, sc = gix.run_stages(5, 5, None, B, cfg.q_len, cfg.nprobe, n_prune, k, t)
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    for b in range(B):
+        m = int(n_pruned[b])
+        order = np.lexsort((pruned[b, :m], -score4[b, :m].astype(np.float64)))[:k]
+        want_ids = np.full(k, -1, dtype=np.int32)
+        want_sc = np.full(k, -np.inf, dtype=np.float32)
+        want_ids[:len(order)] = pruned[b, order]
+        want_sc[:len(order)] = score4[b, order]
+        assert np.array_equal(ids[b], want_ids)
+        assert np.array_equal(sc[b], want_sc)
+
+
 def test_tiny_config_parameter_grid(chimera, tiny):
     cfg, oix, gix, q = tiny
     for nprobe, n_prune, k in [(1, 256, 10), (2, 1024, 100), (8, 64, 10), (32, 4096, 1000), (16, 16384, 10),
