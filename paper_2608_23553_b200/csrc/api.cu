@@ -453,7 +453,7 @@ int chimera_shard_local(const chimera_index *index, const float *queries, int32_
 {
     const Index *ix = reinterpret_cast<const Index *>(index);
     Params p;
-    bool partial, rabitq;
+    bool partial = false, rabitq = false;
     int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
     if (rc || (rc = shard_mode(mode, &partial, &rabitq))) return rc;
     if (!out_ids || !out_scores3) return fail(CHIMERA_INVALID_ARG, "out_ids / out_scores3 is NULL");
@@ -474,7 +474,7 @@ int chimera_shard_finish(const chimera_index *index, const float *queries, int32
 {
     const Index *ix = reinterpret_cast<const Index *>(index);
     Params p;
-    bool partial, rabitq;
+    bool partial = false, rabitq = false;
     int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
     if (rc || (rc = shard_mode(mode, &partial, &rabitq))) return rc;
     if (world < 1 || (int64_t)world * n_prune > 0x7fffffffLL) return fail(CHIMERA_INVALID_ARG, "world out of range");
