@@ -3,7 +3,6 @@ gloo ranks on the CPU."""
 import os
 import sys
 
-import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 

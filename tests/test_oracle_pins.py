@@ -4,7 +4,6 @@ No expectation in this file is produced by calling the oracle function under tes
 hand-worked value under tests/golden/, a numpy library routine on a special case, a set identity, or a brute-force
 enumeration written straight from the definition.
 """
-import itertools
 import os
 
 import numpy as np
