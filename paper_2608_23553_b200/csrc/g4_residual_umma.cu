@@ -63,8 +63,15 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     constexpr uint32_t TMEM_COLS = N <= 128 ? 128 : 256;
     constexpr uint32_t A_BYTES = G4U_TOK * 128;              // 16 KB
     constexpr uint32_t B_BYTES = N * 128;
-    constexpr int VP = NQP + 4;                              // pitch of the value rows (floats): 16-byte aligned rows;
-                                                             // a row is read with lane = column, so any pitch is conflict-free
+    // Value rows (one per token, floats).  ON_A (q_len <= 32, residual codes): a row is 128 bytes and lies on the
+    // token's own row of the A tile, which is free between the MMAs' completion and the next expansion; its 16-byte
+    // groups are XOR-swizzled like the A rows, so the row-per-thread writes and the lane = column reads are both
+    // conflict-free.  18 KB less shared memory per CTA lets the SM run with a smaller shared-memory carve-out, i.e.
+    // more L1 for the scattered score-table rows (Mid, batch 256: 2.72 -> 2.41 ms; forcing the largest carve-out
+    // brings 2.71 ms back).  The RaBitQ variant gathers no rows and is slower that way (1.45 -> 1.56 ms).  Otherwise
+    // the rows have their own buffer with pitch NQP + 4 (read with lane = column: conflict-free).
+    constexpr bool ON_A = NQP == 32 && !RQ;
+    constexpr int VP = ON_A ? 32 : NQP + 4;
     constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) |
                                ((uint32_t)(G4U_TOK >> 4) << 24);
 
@@ -78,8 +85,9 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to the aligned area
     const uint32_t sA = base, sB = base + A_BYTES;
-    float *vals = reinterpret_cast<float *>(gen + A_BYTES + B_BYTES);                       // [128][VP]
-    uint32_t *docmax = reinterpret_cast<uint32_t *>(vals + G4U_TOK * VP);                  // [MAX_DOCS][NQP]
+    float *vals = reinterpret_cast<float *>(ON_A ? gen : gen + A_BYTES + B_BYTES);          // [128][VP]
+    uint32_t *docmax = reinterpret_cast<uint32_t *>(
+        gen + A_BYTES + B_BYTES + (ON_A ? 0 : sizeof(float) * G4U_TOK * VP));              // [MAX_DOCS][NQP]
     const uint32_t bars = smem_u32(docmax + G4U_MAX_DOCS * NQP);
     const uint32_t bar_b = (bars + 7u) & ~7u, bar_mma = bar_b + 8;
 
@@ -334,7 +342,9 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                         else
                             val[e] = fmaf(code_scale, (float)T, (float)se[e] * (1.0f / 16777216.0f));
                     }
-                    *reinterpret_cast<float4 *>(vrow + ch * 16 + 4 * g) = make_float4(val[0], val[1], val[2], val[3]);
+                    const int grp = ch * 4 + g;               // 16-byte group of the row
+                    *reinterpret_cast<float4 *>(vrow + 4 * (ON_A ? grp ^ (tid & 7) : grp)) =
+                        make_float4(val[0], val[1], val[2], val[3]);
                 }
             }
         }
@@ -352,12 +362,21 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                 starts &= starts - 1;
                 const int e = starts ? __ffs(starts) - 1 : n_rows;
                 const int doc = __shfl_sync(0xffffffffu, dl, a);
-                const float *vp = vals + (warp * 32 + a) * VP + lane;
-                float m0 = vp[0], m1 = NQP > 32 ? vp[32] : 0.f;
-                for (int r = a + 1; r < e; ++r) {
-                    vp += VP;
-                    m0 = fmaxf(m0, vp[0]);
-                    if (NQP > 32) m1 = fmaxf(m1, vp[32]);
+                float m0, m1 = 0.f;
+                if (ON_A) {
+                    // column `lane` of row r sits in group (lane / 4) ^ (r & 7)
+                    const float *vw = vals + warp * 32 * VP + (lane & 3);
+                    m0 = vw[a * VP + ((((lane >> 2) ^ a) & 7) << 2)];
+                    for (int r = a + 1; r < e; ++r) m0 = fmaxf(m0, vw[r * VP + ((((lane >> 2) ^ r) & 7) << 2)]);
+                } else {
+                    const float *vp = vals + (warp * 32 + a) * VP + lane;
+                    m0 = vp[0];
+                    m1 = NQP > 32 ? vp[32] : 0.f;
+                    for (int r = a + 1; r < e; ++r) {
+                        vp += VP;
+                        m0 = fmaxf(m0, vp[0]);
+                        if (NQP > 32) m1 = fmaxf(m1, vp[32]);
+                    }
                 }
                 atomicMax(&docmax[doc * NQP + lane], f_order(m0));
                 if (NQP > 32) atomicMax(&docmax[doc * NQP + 32 + lane], f_order(m1));
@@ -402,7 +421,9 @@ static int launch_g4_umma(const Index &ix, const Params &p, const float *queries
     CUtensorMap map_q;
     int rc = make_plane_map(&map_q, qdig, (int64_t)p.B * p.nq, NQP);
     if (rc) return rc;
-    const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 + sizeof(float) * G4U_TOK * (NQP + 4) +
+    // (q_len <= 32 with residual codes: the value rows lie on the A tile)
+    const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 +
+                        (NQP == 32 && !RQ ? 0 : sizeof(float) * G4U_TOK * (NQP + 4)) +
                         sizeof(uint32_t) * G4U_MAX_DOCS * NQP + 32;
     auto kern = residual_maxsim_umma<NQP, NBITS, RQ>;
     CHIMERA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
