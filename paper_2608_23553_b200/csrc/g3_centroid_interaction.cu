@@ -399,15 +399,20 @@ cand_range_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ 
 // i + 1 are already being fetched -- a one-level prefetch where the per-document chain used to have three levels.
 // The 32 results of a group are written back coalesced.
 template <int LPR>
-__global__ void __launch_bounds__(CI_THREADS)
-ci_coarse_rng_kernel(const uint8_t *__restrict__ table8, int64_t K, const int2 *__restrict__ rng,
+__device__ __forceinline__ void
+ci_coarse_rng_body(const uint8_t *__restrict__ table8, int64_t K, const int2 *__restrict__ rng,
                      const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
                      int32_t *__restrict__ lo, int32_t *__restrict__ hi)
 {
     constexpr int NQ = 16 * LPR;
     constexpr int TPL = 32 / LPR;                 // tokens per warp-wide load
     constexpr int STEPS = 32 / TPL;               // loads per 32-token slab (= LPR)
-    constexpr int SLABS = 2;                      // 32-token slabs per iteration
+    // 32-token slabs per iteration, and whether the centroid ids of the document after next are pulled into L2.
+    // Measured (bound scan, batch 256): for 32-byte rows one slab without that prefetch is the fastest of the four
+    // combinations (Mid 14.21 ms against 14.45 ms for two slabs with it, 14.54 / 14.75 ms for the mixed ones; Large
+    // 28.2 against 28.7 ms); for 64-byte rows two slabs with the prefetch are (long documents: 28.8 against 29.1 ms).
+    constexpr int SLABS = LPR == 2 ? 1 : 2;
+    constexpr bool PREFETCH_L2 = LPR != 2;
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int grp = lane / LPR, sub = lane % LPR;
@@ -438,7 +443,7 @@ ci_coarse_rng_kernel(const uint8_t *__restrict__ table8, int64_t K, const int2 *
             int32_t cid[SLABS];
 #pragma unroll
             for (int k = 0; k < SLABS; ++k) cid[k] = nx_cid[k];
-            if (di + 2 < cnt) {                        // two documents ahead: pull the centroid ids into L2
+            if (PREFETCH_L2 && di + 2 < cnt) {         // two documents ahead: pull the centroid ids into L2
                 const int p0 = __shfl_sync(0xffffffffu, mine.x, di + 2), pl = __shfl_sync(0xffffffffu, mine.y, di + 2);
                 if (lane * 32 < pl) asm volatile("prefetch.global.L2 [%0];" ::"l"(cids + (int64_t)p0 + lane * 32));
             }
@@ -522,6 +527,26 @@ ci_coarse_rng_kernel(const uint8_t *__restrict__ table8, int64_t K, const int2 *
     }
 }
 
+// Two launch forms of the scan.  32-byte rows: no occupancy hint (the compiler's own 64 registers, four blocks per SM;
+// any hint measured slower).  64-byte rows: four blocks per SM instead of the three that the unhinted 75 registers
+// give (long-document corpus: 27.1 against 28.4 ms).
+template <int LPR>
+__global__ void __launch_bounds__(CI_THREADS)
+ci_coarse_rng_kernel(const uint8_t *__restrict__ table8, int64_t K, const int2 *__restrict__ rng,
+                     const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
+                     int32_t *__restrict__ lo, int32_t *__restrict__ hi)
+{
+    ci_coarse_rng_body<LPR>(table8, K, rng, n_cand, maxc, cids, lo, hi);
+}
+template <int LPR>
+__global__ void __launch_bounds__(CI_THREADS, 4)
+ci_coarse_rng_kernel_b4(const uint8_t *__restrict__ table8, int64_t K, const int2 *__restrict__ rng,
+                        const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
+                        int32_t *__restrict__ lo, int32_t *__restrict__ hi)
+{
+    ci_coarse_rng_body<LPR>(table8, K, rng, n_cand, maxc, cids, lo, hi);
+}
+
 bool coarse_supported(int nq) { return nq == 32 || nq == 64; }
 
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
@@ -583,7 +608,7 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
         if (p.nq == 32)
             ci_coarse_rng_kernel<2><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
         else
-            ci_coarse_rng_kernel<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
+            ci_coarse_rng_kernel_b4<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
         CHIMERA_CUDA(cudaGetLastError());
         count_launch(SLOT_CI);
         return CHIMERA_OK;
