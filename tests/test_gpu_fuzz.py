@@ -28,7 +28,26 @@ def _cases(n, seed):
     return out
 
 
-@pytest.mark.parametrize("case", _cases(24, 2024))
+def _larger_cases(n, seed):
+    """Corpora of thousands to tens of thousands of documents: long candidate lists, the multi-block selections that
+    serve small batches, n_prune and k in the thousands."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        D = int(rng.choice([32, 64, 96, 128]))
+        nbits = int(rng.choice([1, 2]))
+        nq = int(rng.choice([8, 32, 32, 64, 33, 100]))
+        K = int(rng.choice([64, 300, 1024, 4096]))
+        N = int(rng.choice([3000, 9000, 20000, 40000, 70000]))
+        nprobe = min(int(rng.choice([1, 2, 4, 8, 32])), K)
+        n_prune = int(rng.choice([10, 256, 1024, 5000]))
+        k = int(rng.choice([1, 10, 100, 1000]))
+        len_hi = int(rng.choice([3, 20, 60]))
+        out.append((D, nbits, nq, K, N, nprobe, n_prune, k, len_hi, int(rng.integers(1 << 30))))
+    return out
+
+
+@pytest.mark.parametrize("case", _cases(24, 2024) + _larger_cases(10, 77))
 def test_random_configuration_all_pipelines(case):
     import paper_2608_23553_b200 as pkg
     from synth import CONFIGS, encode_rabitq_1bit, random_rotation
