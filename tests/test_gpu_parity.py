@@ -284,6 +284,29 @@ def test_tiny_config_recall_against_exhaustive(chimera, tiny):
         assert oracle.recall(truth, ids[b]) == oracle.recall(truth, res.ids)
 
 
+def test_sweep_ground_truth_equals_the_oracles_exhaustive_scores(chimera, tiny):
+    """The recall sweeps of bench.py take their ground truth from the library's stage 4 run over every document in
+    chunks (bench.exhaustive_truth); here that procedure is compared with the oracle's exhaustive MaxSim on the whole
+    Tiny corpus: the same documents except for swaps between scores within the tolerance, scores within it."""
+    import bench
+    from parity import score_tol
+    cfg, oix, gix, q = tiny
+    k = 100
+    qd = torch.from_numpy(q).cuda()
+    ids, sc = bench.exhaustive_truth(gix, qd, cfg, k, chunk=4096)      # 10,000 documents: two full chunks and a ragged one
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    for b in range(q.shape[0]):
+        t_ids, t_sc, all_sc = oracle.exhaustive(q[b], oix, k)
+        tau = float(t_sc[-1])
+        tol = float(score_tol(tau, cfg.q_len))
+        assert len(set(ids[b].tolist())) == k
+        assert np.all(np.abs(sc[b] - all_sc[ids[b]]) <= score_tol(all_sc[ids[b]], cfg.q_len))
+        assert np.all(all_sc[ids[b]] >= tau - tol)
+        sure = t_ids[t_sc > tau + tol]
+        assert np.all(np.isin(sure, ids[b]))
+        assert oracle.recall(t_ids, ids[b]) >= 0.98
+
+
 def test_graphed_search_equals_eager(chimera, tiny):
     cfg, oix, gix, q = tiny
     qd = torch.from_numpy(q).cuda()
