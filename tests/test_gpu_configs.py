@@ -70,14 +70,14 @@ def test_large_corpus_full_size_sampled_queries():
     ids_np, sc_np, q_np = ids.cpu().numpy(), sc.cpu().numpy(), q.cpu().numpy()
     for b in range(B):
         _properties(tn, ids_np, sc_np, b, cfg, cfg.n_docs, cfg.k)
-    # stage 1 for one query, on its own
-    t1 = gix.alloc_taps(1, cfg.q_len, cfg.nprobe, cfg.n_prune, max_candidates=1024, table=True)
-    gix.run_stages(1, 1, q[77:78].contiguous(), 1, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k, t1, max_candidates=1024)
-    table77 = t1.score_table[0].cpu().numpy()
+    # stage 1 for the two sampled queries, on its own: 64 query tokens x all 262,144 centroids
+    t1 = gix.alloc_taps(2, cfg.q_len, cfg.nprobe, cfg.n_prune, max_candidates=1024, table=True)
+    q2 = torch.stack([q[77], q[255]]).contiguous()
+    gix.run_stages(1, 1, q2, 2, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k, t1, max_candidates=1024)
+    tables = {77: t1.score_table[0].cpu().numpy(), 255: t1.score_table[1].cpu().numpy()}
     oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
     for b in (77, 255):
         res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
-        if b == 77:
-            assert np.array_equal(table77, res.S)
+        assert np.array_equal(tables[b], res.S)
         # check_query enforces the tolerance rule; with k = 100 a swap between two fp32 near-ties can move positions
         assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) <= 4

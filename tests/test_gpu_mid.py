@@ -70,6 +70,22 @@ def test_mid_score_table_sampled_rows_match_oracle(mid):
     assert np.array_equal(taps.score_table[0].cpu().numpy(), S)
 
 
+def test_mid_score_table_in_the_batch256_launch_matches_oracle(mid):
+    """Stage 1 in the configuration the benchmark times (256 queries per call: the 48-row query tiles straddle query
+    boundaries and the grid is split over query tiles): every entry of the tables of eight queries spread over the
+    batch, 8 x 32 query tokens x 65,536 centroids."""
+    cfg, corp, gix, oix, q = mid
+    B = 256
+    taps = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, cfg.n_prune, max_candidates=1024, table=True, ci=False)
+    gix.run_stages(1, 1, q[:B].contiguous(), B, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k, taps, max_candidates=1024)
+    q_np = q[:B].cpu().numpy()
+    for b in (0, 1, 2, 37, 100, 191, 254, 255):
+        S = oracle.score_table(q_np[b], oix.centroids)
+        assert np.array_equal(taps.score_table[b].cpu().numpy(), S), "query %d" % b
+    del taps
+    torch.cuda.empty_cache()
+
+
 def test_mid_batch256_four_document_shards_equal_the_single_index(mid):
     """The document-sharded search at the benchmark's size: four shards of 125k documents, their phases run one after
     the other on this GPU, merged ids and scores equal the single index's for every query."""
