@@ -1,6 +1,6 @@
 """Parity on the other workload shapes: the long-document precision variants (512-token documents, 64-token queries,
-dim 96/128, 1/2 residual bits) at reduced document count, and the passage-corpus-shaped Large corpus (8.8M documents,
-~600M tokens, 262,144 centroids) at full size with sampled queries."""
+dim 96/128, 1/2 residual bits) at reduced document count and one of them at full size, and the passage-corpus-shaped
+Large corpus (8.8M documents, ~600M tokens, 262,144 centroids) at full size with sampled queries."""
 import numpy as np
 import pytest
 import torch
@@ -45,6 +45,35 @@ def test_long_document_variants_reduced(name):
         assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune) == 0
     for b in range(B):
         _properties(tn, ids_np, sc_np, b, cfg, oix.N, cfg.k)
+
+
+def test_long_document_corpus_full_size_sampled_query():
+    """The long-document workload at full size in the launch configuration the benchmark times (200,000 documents of
+    512 tokens, 64-token queries, batch 64, nprobe 8: nearly every document is a candidate): one sampled query against
+    the oracle stage by stage, every query for the properties that hold at any size."""
+    import psutil
+    import paper_2608_23553_b200 as pkg
+    from synth import CONFIGS, make_corpus, make_queries
+    if psutil.virtual_memory().available < 16e9:
+        pytest.skip("needs ~8 GB of host memory for the oracle's copy of the corpus")
+    cfg = CONFIGS["long_d128_b2"]
+    dev = torch.device("cuda:0")
+    corp = make_corpus(cfg, device=dev)
+    assert corp.n_tokens == 200_000 * 512
+    B = 64
+    q = make_queries(cfg, B, device=dev)
+    gix = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    taps = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, cfg.n_prune, table=False)
+    ids, sc = gix.search(q, cfg.nprobe, cfg.n_prune, cfg.k, taps=taps)
+    assert gix.status() == 0
+    tn = taps_to_numpy(taps)
+    ids_np, sc_np, q_np = ids.cpu().numpy(), sc.cpu().numpy(), q.cpu().numpy()
+    for b in range(B):
+        _properties(tn, ids_np, sc_np, b, cfg, cfg.n_docs, cfg.k)
+    oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    b = 41
+    res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
+    assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) <= 2
 
 
 def test_large_corpus_full_size_sampled_queries():
