@@ -265,10 +265,13 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, ci, (const int2 *)(ws + L.cand_rng),
                                         (int2 *)(ws + L.cont_rng), st))) return rc;
             prof_mark(SLOT_SELECT, st);
-            // blocks per query for the few contenders: one per SM in a large batch (measured best), four per SM
-            // when a single query has the GPU to itself
+            // blocks per query for the few contenders (typically two to three times n_prune documents): one per SM
+            // in a large batch, more when n_prune is large (about one block per eight survivors wanted; Large,
+            // n_prune 4096: 2.75 ms with 444-592 blocks against 3.26 ms with 148, Mid unchanged), four per SM when a
+            // single query has the GPU to itself
             int exact_blocks = (4 * ix.sm_count + p.B - 1) / p.B;
             if (exact_blocks < ix.sm_count) exact_blocks = ix.sm_count;
+            if (exact_blocks < p.n_prune / 8) exact_blocks = p.n_prune / 8;
             if ((rc = launch_centroid_interaction(ix, p, table, cont, n_cont, ci, exact_blocks, SLOT_CI_EXACT,
                                                   ix.T < 0x7fffffffLL ? (const int2 *)(ws + L.cont_rng) : nullptr, st)))
                 return rc;
