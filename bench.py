@@ -264,6 +264,69 @@ def run_sweep(args, cfg, pkg, index, corp, q):
                 print(json.dumps(point))
 
 
+def run_sharded(args, cfg, pkg, rank, world, local_rank, device):
+    """Document-sharded search (the scaling sketch of Sec. 3.3): every rank indexes its contiguous range of the
+    documents, the queries are the same everywhere, and one step is ShardedSearcher.search -- local stages 1-3,
+    all-gather of ids and integer scores, global selection, stages 4-5 on the rank's own survivors, all-gather, merge.
+    The corpus is fixed while ranks are added, so scaling is strong.  With one rank the result is also compared with
+    the plain search.  Prints one JSON line on rank 0."""
+    import torch.distributed as dist
+    from paper_2608_23553_b200.sharded import ShardEngine, ShardedSearcher, shard_ranges
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29533")
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=device)
+    corp, q, gen_s = build_workload(cfg, device, rabitq=args.rabitq)
+    lo, hi = shard_ranges(cfg.n_docs, world)[rank]
+    off = torch.cat([torch.zeros(1, dtype=torch.int64, device=device), torch.cumsum(corp.doclens.to(torch.int64), 0)])
+    t0, t1 = int(off[lo]), int(off[hi])
+    index = pkg.Index(corp.centroids, corp.cids[t0:t1].contiguous(), corp.codes[t0:t1].contiguous(),
+                      corp.doclens[lo:hi].contiguous(), cfg.nbits, cfg.res_lo, cfg.res_hi)
+    mode = "rabitq" if args.rabitq else ("partial" if args.partial else "ci")
+    if args.partial or args.rabitq:
+        index.enable_partial()
+    if args.rabitq:
+        index.attach_rabitq(corp.rotation, corp.rq_bits[t0:t1].contiguous(), corp.rq_inv_dot[t0:t1].contiguous())
+    searcher = ShardedSearcher(ShardEngine(index, lo, mode))
+    B, nq, P, n_prune, k = args.batch, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
+    n_batches = max(1, min(args.steps + args.warmup, (q.shape[0] + B - 1) // B + 1))
+    idx = (torch.arange(n_batches * B, device=device) % q.shape[0]).view(n_batches, B)
+    batches = q[idx].contiguous()
+    equal = None
+    if world == 1:                       # one shard holding everything: must equal the plain search bit for bit
+        ids_s, sc_s = searcher.search(batches[0], P, n_prune, k)
+        ids_p, sc_p = index.search(batches[0], P, n_prune, k, partial=args.partial, rabitq=args.rabitq)
+        equal = bool(torch.equal(ids_s, ids_p) and torch.equal(sc_s, sc_p))
+    for s in range(args.warmup):
+        searcher.search(batches[s % n_batches], P, n_prune, k)
+    dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(args.steps):
+        searcher.search(batches[(args.warmup + s) % n_batches], P, n_prune, k)
+    e1.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    if rank == 0:
+        qps = B * args.steps / (ms_total / 1e3)        # every rank works on the same queries: the job's rate
+        print(json.dumps({
+            "metric": metric_name(cfg, B) + ", document-sharded", "value": qps, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "int32 fixed point (stages 1-3) + f32 (stage 4)",
+            "data": "synthetic",
+            "config": {"workload": cfg.name, "batch": B, "pruning": mode,
+                       "parallelism": "documents sharded over %d ranks, two all-gathers of ids and scores per step" % world,
+                       "docs_per_rank": hi - lo, "equals_plain_search": equal},
+            "clocks": clocks}))
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -280,6 +343,8 @@ def main():
     ap.add_argument("--sweep-queries", type=int, default=200)
     ap.add_argument("--batch1-queries", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="document-sharded search over the ranks (one JSON line; see run_sharded) instead of replicas")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -299,6 +364,9 @@ def main():
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
+    if args.sharded:
+        run_sharded(args, cfg, pkg, rank, world, local_rank, device)
+        return
     dist = None
     if world > 1:
         import torch.distributed as dist
