@@ -108,11 +108,13 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
             }
         return T;
     };
-    auto update = [&](uint32_t d, int T) {
+    // (the document's bitmap word and its rank come as arguments: they depend on the list entry alone, so their loads
+    // are issued with the code loads instead of after the score is known -- one memory latency less per visit)
+    auto update = [&](uint32_t d, int T, uint32_t bm_word, int32_t wr_word) {
         const double r = __dadd_rn(__dmul_rn(d4, (double)T), kterm);
         const long long dist = (long long)s_c + __double2ll_rn(r);
         if (dist > 0) {                                // the table starts at 0 (Algorithm 2)
-            const int64_t rank = wr[d >> 5] + __popc(bm[d >> 5] & ((1u << (d & 31)) - 1u));
+            const int64_t rank = wr_word + __popc(bm_word & ((1u << (d & 31)) - 1u));
             if (rank < maxc) {
                 // F' = sum_i M[., i] is kept up to date with the increments: M only grows, integer adds commute
                 const int32_t old = atomicMax(&Mb[rank * nq + i], (int32_t)dist);
@@ -126,11 +128,18 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
     for (; e + PS_THREADS < e1; e += 2 * PS_THREADS) {
         const int64_t ta = tok_id[e], tb2 = tok_id[e + PS_THREADS];
         const uint32_t da = (uint32_t)tok_doc[e], db = (uint32_t)tok_doc[e + PS_THREADS];
+        const uint32_t bma = __ldg(bm + (da >> 5)), bmb = __ldg(bm + (db >> 5));
+        const int32_t wra = __ldg(wr + (da >> 5)), wrb = __ldg(wr + (db >> 5));
         const int Ta = code_dot(ta), Tb = code_dot(tb2);
-        update(da, Ta);
-        update(db, Tb);
+        update(da, Ta, bma, wra);
+        update(db, Tb, bmb, wrb);
     }
-    if (e < e1) update((uint32_t)tok_doc[e], code_dot(tok_id[e]));
+    if (e < e1) {
+        const uint32_t d = (uint32_t)tok_doc[e];
+        const uint32_t bmd = __ldg(bm + (d >> 5));
+        const int32_t wrd = __ldg(wr + (d >> 5));
+        update(d, code_dot(tok_id[e]), bmd, wrd);
+    }
 }
 
 int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, const float *queries,

@@ -132,10 +132,12 @@ rabitq_partial_kernel(const float *__restrict__ q_rot, int nq, int D, int P, flo
             }
         return T;
     };
-    auto update = [&](uint32_t d, int64_t t, int T) {
-        const float est = __fmul_rn(inv_dot[t], __fmul_rn(c, (float)(2 * T - sq)));
+    // (the token's factor, the document's bitmap word and its rank come as arguments: they depend on the list entry
+    // alone, so their loads are issued with the code loads instead of one after the other behind the score)
+    auto update = [&](uint32_t d, float factor, int T, uint32_t bm_word, int32_t wr_word) {
+        const float est = __fmul_rn(factor, __fmul_rn(c, (float)(2 * T - sq)));
         if (est > 0.0f) {                              // the table starts at 0 (Algorithm 2)
-            const int64_t rank = wr[d >> 5] + __popc(bm[d >> 5] & ((1u << (d & 31)) - 1u));
+            const int64_t rank = wr_word + __popc(bm_word & ((1u << (d & 31)) - 1u));
             if (rank < maxc) atomicMax(&Mb[rank * nq + i], __float_as_int(est));
         }
     };
@@ -144,13 +146,20 @@ rabitq_partial_kernel(const float *__restrict__ q_rot, int nq, int D, int P, flo
     for (; e + RP_THREADS < e1; e += 2 * RP_THREADS) {         // two visits per iteration, their loads issued together
         const int64_t ta = tok_id[e], tb = tok_id[e + RP_THREADS];
         const uint32_t da = (uint32_t)tok_doc[e], db = (uint32_t)tok_doc[e + RP_THREADS];
+        const float fa = __ldg(inv_dot + ta), fb = __ldg(inv_dot + tb);
+        const uint32_t bma = __ldg(bm + (da >> 5)), bmb = __ldg(bm + (db >> 5));
+        const int32_t wra = __ldg(wr + (da >> 5)), wrb = __ldg(wr + (db >> 5));
         const int Ta = code_dot(ta), Tb = code_dot(tb);
-        update(da, ta, Ta);
-        update(db, tb, Tb);
+        update(da, fa, Ta, bma, wra);
+        update(db, fb, Tb, bmb, wrb);
     }
     if (e < e1) {
         const int64_t t = tok_id[e];
-        update((uint32_t)tok_doc[e], t, code_dot(t));
+        const uint32_t d = (uint32_t)tok_doc[e];
+        const float f = __ldg(inv_dot + t);
+        const uint32_t bmd = __ldg(bm + (d >> 5));
+        const int32_t wrd = __ldg(wr + (d >> 5));
+        update(d, f, code_dot(t), bmd, wrd);
     }
 }
 
