@@ -7,7 +7,8 @@
 // Two phases when q_len is 32 or 64: cheap bounds lo(d) <= CI(d) <= hi(d) for every candidate from an 8-bit copy of
 // the table (cand_range_kernel + ci_coarse_rng_kernel; ci_coarse_kernel for tables staged in shared memory and for
 // corpora of 2^31 tokens or more), the documents whose hi reaches the n_prune-th largest lo (contender kernels), then
-// exact CI (ci_wide_kernel) and the exact selection among those only.  Other q_len: exact CI for every candidate
+// exact CI (ci_wide_rng_kernel over the contenders' token ranges; ci_wide_kernel without ranges) and the exact
+// selection among those only.  Other q_len: exact CI for every candidate
 // (ci_kernel).
 //
 // ci_kernel: one warp per candidate document.  The document's centroid ids are streamed with coalesced 128-byte
