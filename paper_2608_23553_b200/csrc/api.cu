@@ -110,7 +110,16 @@ Layout make_layout(const Index &ix, const Params &p)
     L.n_cont = take(B * sizeof(int32_t));
     L.pruned = take(B * p.n_prune * sizeof(int32_t));
     L.word_rank = take(B * (size_t)L.words * sizeof(int32_t));
-    L.partial_m = take(ix.tok_id ? B * (size_t)p.maxc * nq * sizeof(int32_t) : 0);
+    // partial-score table: dense rows per candidate (always for the RaBitQ refinement), or the hashed form
+    L.hash_slots = partial_hash_slots(ix, p);
+    {
+        const size_t dense = B * (size_t)p.maxc * nq * sizeof(int32_t);
+        const size_t hashed = B * (size_t)L.hash_slots * sizeof(unsigned long long);
+        size_t bytes = 0;
+        if (ix.tok_id) bytes = L.hash_slots ? hashed : dense;
+        if (ix.rot_t && bytes < dense) bytes = dense;
+        L.partial_m = take(bytes);
+    }
     L.q_rot = take(ix.rot_t ? B * nq * ix.D * sizeof(float) : 0);
     L.qdig_rot = take(ix.rot_t ? 3 * B * nq * 128 : 0);
     L.n_pruned = take(B * sizeof(int32_t));
@@ -249,7 +258,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
         } else if (partial) {
             // the paper's candidate refinement: partial scores from the retrieved tokens only, then the same selection
             if ((rc = launch_partial_scores(ix, p, L, queries, table, probes, bitmap, word_rank, n_cand, partial_m, ci,
-                                            st)))
+                                            status, st)))
                 return rc;
             prof_mark(SLOT_CI, st);
             if ((rc = launch_select(ix, p, cand, n_cand, ci, pruned, n_pruned, pruned_ci, sel_scratch, st))) return rc;

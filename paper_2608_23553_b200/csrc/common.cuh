@@ -29,6 +29,7 @@ struct Index {
     int64_t *tok_off = nullptr;       // [K+1]      owned
     int32_t *tok_id = nullptr;        // [T]        owned: token ids per centroid, unordered
     int32_t *tok_doc = nullptr;       // [T]        owned: document of each listed token
+    int64_t max_tok_list = 0;         // longest token list
     // RaBitQ 1-bit codes (only after chimera_index_attach_rabitq)
     const uint8_t *rq_bits = nullptr; // [T, D/8]   borrowed: sign bits of the rotated tokens
     const float *rq_inv = nullptr;    // [T]        borrowed: 1 / <o_p, o_p-bar>
@@ -69,7 +70,9 @@ struct Layout {
     size_t n_cont;        // int32  [B]
     size_t pruned;        // int32  [B][n_prune]
     size_t word_rank;     // int32  [B][words]        candidates before each bitmap word (document -> candidate index)
-    size_t partial_m;     // int32  [B][maxc][nq]     per (candidate, query token) best retrieved-token score
+    size_t partial_m;     // int32  [B][maxc][nq]     per (candidate, query token) best retrieved-token score, or
+                          // uint64 [B][hash_slots]   the same as an open-addressing table (see partial_hash_slots)
+    int64_t hash_slots;   // slots per query of that table; 0 = the dense form
     size_t q_rot;         // float  [B, nq, D]        rotated queries (RaBitQ pipeline)
     size_t qdig_rot;      // int8   [3][B*nq][128]    their digit planes
     size_t n_pruned;      // int32  [B]
@@ -125,9 +128,13 @@ int launch_gather(const Index &ix, const Params &p, const Layout &L, const int32
 // Token-level posting lists for the partial-score refinement (allocates; index_build.cu).
 int build_token_lists(Index &ix, cudaStream_t st);
 // Candidate refinement with partial scores (Algorithm 2): fprime[b][j] for every candidate.
+// Slots per query (a power of two) of the hashed score table of the partial-score refinement, 0 when the dense table
+// is used (no token lists, few queries per call, keys that do not fit 32 bits, or a dense table less than four times
+// as large).
+int64_t partial_hash_slots(const Index &ix, const Params &p);
 int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, const float *queries,
                           const int32_t *table, const int32_t *probes, const uint32_t *bitmap,
-                          const int32_t *word_rank, const int32_t *n_cand, int32_t *partial_m, int32_t *fprime,
+                          const int32_t *word_rank, const int32_t *n_cand, int32_t *partial_m, int32_t *fprime, uint32_t *status,
                           cudaStream_t st);
 bool coarse_supported(int nq);
 int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st);

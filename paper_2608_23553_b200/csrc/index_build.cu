@@ -199,6 +199,21 @@ __global__ void token_list_kernel(const int32_t *__restrict__ cids, const int64_
     }
 }
 
+// out[0] = max_c (off[c + 1] - off[c])
+__global__ void max_list_kernel(const int64_t *__restrict__ off, int64_t K, unsigned long long *__restrict__ out)
+{
+    unsigned long long m = 0;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < K; c += (int64_t)gridDim.x * blockDim.x) {
+        const unsigned long long len = (unsigned long long)(off[c + 1] - off[c]);
+        m = len > m ? len : m;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long t = __shfl_xor_sync(0xffffffffu, m, o);
+        m = t > m ? t : m;
+    }
+    if ((threadIdx.x & 31) == 0) atomicMax(out, m);
+}
+
 int build_token_lists(Index &ix, cudaStream_t st)
 {
     if (ix.tok_id) return CHIMERA_OK;
@@ -235,9 +250,17 @@ int build_token_lists(Index &ix, cudaStream_t st)
     TL_CUDA(cudaMemsetAsync(count, 0, sizeof(int32_t) * ix.K, st));
     token_list_kernel<1><<<blocks, 256, 0, st>>>(ix.cids, ix.doc_off, ix.N, count, off, ids, docs);
     TL_CUDA(cudaGetLastError());
+    // the longest list (sizes the hashed score table of the refinement); tmp is free again: its first word holds it
+    TL_CUDA(cudaMemsetAsync(tmp, 0, sizeof(int64_t), st));
+    max_list_kernel<<<(unsigned)((ix.K + 255) / 256 < 1024 ? (ix.K + 255) / 256 : 1024), 256, 0, st>>>(
+        off, ix.K, reinterpret_cast<unsigned long long *>(tmp));
+    TL_CUDA(cudaGetLastError());
+    long long longest = 0;
+    TL_CUDA(cudaMemcpyAsync(&longest, tmp, sizeof(longest), cudaMemcpyDeviceToHost, st));
     TL_CUDA(cudaStreamSynchronize(st));
 #undef TL_CUDA
     cleanup(false);
+    ix.max_tok_list = longest;
     ix.tok_off = off;
     ix.tok_id = ids;
     ix.tok_doc = docs;

@@ -50,6 +50,44 @@ def test_partial_refinement_small_corpora(D, nbits, nq, K, N, nprobe, n_prune, k
     assert np.array_equal(np.sort(ids_a[0].cpu().numpy()), np.sort(res.ids))
 
 
+@pytest.mark.parametrize("nbits", [2, 1])
+def test_partial_refinement_hashed_table_equals_dense_and_oracle(nbits):
+    """With enough queries per call and a corpus large enough, the (candidate, query token) maxima live in an
+    open-addressing table instead of dense rows.  40 queries (on a B200) on 30,000 documents take that path; the same queries one
+    at a time take the dense path; both must agree bit for bit in F' of every candidate, pruned ids and final results,
+    and sampled queries must match the oracle."""
+    import paper_2608_23553_b200 as pkg
+    D, nq, K, N, nprobe, n_prune, k = 64, 32, 4096, 30000, 2, 300, 20
+    cent, cids, codes, doclens = random_corpus(4242 + nbits, N, K, D, nbits, len_lo=1, len_hi=40)
+    oix = oracle.make_index(cent, cids, codes, doclens, nbits)
+    dev = torch.device("cuda:0")
+    gix = pkg.Index(torch.from_numpy(cent).to(dev), torch.from_numpy(cids).to(dev), torch.from_numpy(codes).to(dev),
+                    torch.from_numpy(doclens).to(dev), nbits)
+    gix.enable_partial()
+    # calls of up to (SM count / 4) queries keep dense rows; three more queries and the table is hashed, which shows in
+    # the workspace: more queries, yet fewer bytes
+    small = torch.cuda.get_device_properties(0).multi_processor_count // 4
+    B = small + 3
+    assert gix.workspace_bytes(B, nq, nprobe, n_prune, k) < gix.workspace_bytes(small, nq, nprobe, n_prune, k)
+    q = np.stack([unit_rows(np.random.default_rng(900 + b), nq, D) for b in range(B)])
+    qd = torch.from_numpy(q).cuda()
+    taps = gix.alloc_taps(B, nq, nprobe, n_prune, table=False)
+    ids, sc = gix.search(qd, nprobe, n_prune, k, taps=taps, partial=True)
+    assert gix.status() == 0
+    tn = taps_to_numpy(taps)
+    ids_np, sc_np = ids.cpu().numpy(), sc.cpu().numpy()
+    for b in (0, 17, B - 1):
+        res = oracle.pipeline(q[b], oix, nprobe, n_prune, k, partial=True)
+        assert check_query(tn, b, res, ids_np[b], sc_np[b], k, n_prune, table=False) == 0
+    for b in range(B):
+        t1 = gix.alloc_taps(1, nq, nprobe, n_prune, table=False)
+        i1, s1 = gix.search(qd[b:b + 1].contiguous(), nprobe, n_prune, k, taps=t1, partial=True)
+        n = int(t1.n_cand[0])
+        assert n == int(taps.n_cand[b])
+        assert torch.equal(t1.ci[0, :n], taps.ci[b, :n]) and torch.equal(t1.pruned[0], taps.pruned[b])
+        assert torch.equal(i1[0], ids[b]) and torch.equal(s1[0], sc[b])
+
+
 def test_partial_refinement_tiny_config_and_batch_invariance():
     import paper_2608_23553_b200 as pkg
     from synth import CONFIGS, make_corpus, make_queries
