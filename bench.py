@@ -79,7 +79,7 @@ def ncu_traffic(cfg, batch):
 
 
 NCU_CI_COARSE_MID_B8_BYTES = 443.5e6    # dram__bytes_read.sum + dram__bytes_write.sum of one launch at batch 8
-NCU_PARTIAL_MID_B64_BYTES = 1833e6      # the same for partial_score_kernel<2> at batch 64 (profiles/ncu_partial_score_mid.md)
+NCU_PARTIAL_MID_B64_BYTES = 1527e6      # the same for partial_score_kernel<2> at batch 64 (profiles/ncu_partial_score_mid.md)
 
 
 class ClockSampler:
