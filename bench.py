@@ -545,10 +545,11 @@ def main():
     if args.partial or args.rabitq:
         # candidate refinement by partial scores replaces the scan: the dominant stage-3 kernel visits every token of
         # the nq * nprobe probed posting lists.  Algorithmic bytes per visit: the list entry (token id + document id,
-        # 8 B) and the token's code (residual code, or 1-bit code + its 4-byte scale); per candidate document one
-        # nq * 4-byte row of running maxima is cleared first.  The slot times the clear and the scoring kernel together.
+        # 8 B) and the token's code (residual code, or 1-bit code + its 4-byte scale); per candidate document its
+        # partial score (4 B).  The table of running maxima is the implementation's, not the method's, and is not
+        # counted.  The slot times the clear, the scoring kernel and (RaBitQ) the summation together.
         code_b = (cfg.dim // 8 + 4.0) if args.rabitq else float(cfg.code_bytes)
-        ps_bytes = mean("retrieved") * (8.0 + code_b) + mean("cand") * nq * 4.0
+        ps_bytes = mean("retrieved") * (8.0 + code_b) + mean("cand") * 4.0
         ps_gbs = ps_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0
         traffic = None
         if cfg.name == "mid" and args.partial and not args.rabitq:
