@@ -604,3 +604,62 @@ def test_rabitq_partial_with_every_list_probed_is_the_complete_one_bit_score():
     r = oracle.pipeline_rabitq(q, ix, rq, 2, 10, 4)
     assert len(r.pruned) == 10 and np.all(np.diff(r.pruned) > 0) and np.all(np.isin(r.ids, r.pruned))
     assert np.array_equal(r.score4, oracle.rabitq_score_docs(qp, r.pruned, ix, rq))
+
+
+def test_rabitq_partial_handworked_with_unprobed_lists():
+    # golden/rabitq_partial_handworked.txt: nprobe = 1 < K = 3, a query token that retrieves nothing of a document, a
+    # token in a list only the OTHER query token probes, and a token in a list nobody probes
+    D = 8
+    toks = [[(0, 0x01, 1.0)], [(0, 0x00, 2.0), (0, 0x03, 1.0)], [(0, 0x00, 1.0), (1, 0x02, 2.0)],
+            [(1, 0x03, 4.0), (2, 0x03, 4.0)], [(1, 0x01, 2.0)], [(2, 0x03, 1.0)]]
+    flat = [t for d in toks for t in d]
+    cids = np.array([t[0] for t in flat], np.int32)
+    bits = np.array([[t[1]] for t in flat], np.uint8)
+    inv = np.array([t[2] for t in flat], np.float32)
+    ix = oracle.make_index(np.eye(3, D, dtype=np.float32), cids, np.zeros((len(flat), 1), np.uint8),
+                           np.array([len(d) for d in toks], np.int32), 1)
+    rq = oracle.make_rabitq(np.eye(D, dtype=np.float32), bits, inv)
+    q = np.eye(2, D, dtype=np.float32)
+    pr = np.array([[0], [1]], np.int32)
+    cand = oracle.candidates(pr, ix)
+    assert cand.tolist() == [0, 1, 2, 3, 4]
+    fp = oracle.rabitq_partial(oracle.rotate(rq.rotation, q), pr, cand, ix, rq)
+    rows = [r.split() for r in _golden_rows("rabitq_partial_handworked.txt")]
+    assert [int(r[0]) for r in rows] == cand.tolist()
+    assert fp.tolist() == [float(np.float32(float(r[1]))) for r in rows]
+
+
+def test_rabitq_partial_brute_force_below_full_probing():
+    # Algorithm 2 from Python dictionaries with the estimate of Sec. 2.2 built from the explicit nearest codeword
+    # o_p-bar = sign(o_p) / sqrt(D) in float64 -- no oracle call produces the expectation.  nprobe < K, so which tokens
+    # a query token retrieves (those of ITS OWN probed lists) decides the result.
+    ix, rq, raw, q = _rabitq_case(45, N=60, K=16, D=64, nq=6)
+    D = ix.dim
+    S = oracle.score_table(q, ix.centroids)
+    P64 = rq.rotation.astype(np.float64)
+    qp64 = q.astype(np.float64) @ P64.T
+    op = raw.astype(np.float64) @ P64.T
+    obar = np.sign(op) / np.sqrt(D)
+    est = (qp64 @ obar.T) / np.einsum("td,td->t", op, obar)[None, :]          # [nq, T]
+    qp = oracle.rotate(rq.rotation, q)
+    seen_partial = False
+    for P in (1, 2, 5):
+        pr = oracle.probes(S, P)
+        cand = oracle.candidates(pr, ix)
+        fp = oracle.rabitq_partial(qp, pr, cand, ix, rq)
+        score = {}
+        for i in range(len(q)):
+            mine = set(pr[i].tolist())
+            for d in range(ix.N):
+                for t in range(int(ix.doc_off[d]), int(ix.doc_off[d + 1])):
+                    if int(ix.cids[t]) in mine:
+                        score[(d, i)] = max(score.get((d, i), 0.0), est[i, t])
+        want = np.array([sum(score.get((int(d), i), 0.0) for i in range(len(q))) for d in cand])
+        assert np.allclose(fp, want, atol=2e-5)
+        # the case is selective: some candidate has a query token that retrieved none of its tokens
+        seen_partial |= any((int(d), i) not in score for d in cand for i in range(len(q)))
+        # and differs from probing every list for every query token (what a non-selective filter would compute)
+        every = np.array([sum(max(0.0, est[i, ix.doc_off[d]:ix.doc_off[d + 1]].max()) for i in range(len(q)))
+                          for d in cand])
+        assert np.abs(every - want).max() > 1e-2
+    assert seen_partial
