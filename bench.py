@@ -1,11 +1,16 @@
 #!/usr/bin/env python
 """Benchmark of the GPU-resident retrieval path (stages 1-5 behind chimera_search).
 
-A step is one chimera_search call over one batch of synthetic queries on the Mid corpus (500k documents, ~60M
-tokens, 65,536 centroids, 2-bit residual codes; nprobe 4, n_prune 1024, k 10).  `value` is queries per second at
-batch 256 with the queries already on the device; `e2e` is the same through chimera_search_host with pinned host
-buffers (host->device and device->host copies inside the timed region); `qps_batch1` follows the paper's protocol of
-one synchronised query at a time.  The path does not shard: with --gpus N every rank runs an independent replica.
+A step is one chimera_search call over one batch of synthetic queries.  The headline workload is the Large corpus
+(8.8M documents, ~600M tokens, 262,144 centroids, 2-bit residual codes; nprobe 4, n_prune 4096, k 100), the largest
+configuration that fits one GPU: `value` is queries per second at batch 256 with the queries already on the device;
+`e2e` is the same through chimera_search_host with pinned host buffers (host->device and device->host copies inside
+the timed region); `qps_batch1` follows the paper's protocol of one synchronised query at a time.  Unless --config
+names a single workload, the same line carries, under `configs`, a shorter measurement of every other workload (Tiny,
+Mid, the four long-document variants) and of the two paper pipelines (partial-score refinement, RaBitQ 1-bit codes).
+
+The path does not shard: with --gpus N every rank runs an independent replica (one process per GPU; the ranks are
+started here when the script is not already running under torchrun).  --sharded times the document-sharded search.
 
 `--impl reference` times the CPU oracle (as it stands, one thread) on a bounded sample of the same workload.
 """
@@ -14,6 +19,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -28,6 +34,9 @@ import torch  # noqa: E402
 from synth import CONFIGS, make_corpus, make_queries  # noqa: E402
 
 UNIT = "queries/s"
+HEADLINE = "large"
+DTYPE = "int32 fixed point (stages 1-3) + f32 (stage 4)"
+TARGET = 0.60          # the task's target for the code-scan stages: 60 % of HBM peak
 
 
 def metric_name(cfg, batch):
@@ -69,17 +78,14 @@ def measured_int8_tops():
         return 2.0 * 1590.0, "fallback bf16 x 2"
 
 
-def ncu_traffic(cfg, batch):
-    """DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture, or None.  The capture
-    (profiles/ncu_ci_coarse_mid.md) was taken on the Mid corpus at batch 8; traffic is proportional to the number of
-    queries (every query has its own table and candidate list), so it is scaled by batch / 8."""
-    if cfg.name == "mid" and NCU_CI_COARSE_MID_B8_BYTES:
-        return NCU_CI_COARSE_MID_B8_BYTES * batch / 8.0
-    return None
-
-
-NCU_CI_COARSE_MID_B8_BYTES = 443.5e6    # dram__bytes_read.sum + dram__bytes_write.sum of one launch at batch 8
-NCU_PARTIAL_MID_B64_BYTES = 1527e6      # the same for partial_score_kernel<2> at batch 64 (profiles/ncu_partial_score_mid.md)
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of one launch of the dominant kernel,
+# from stored ncu captures on small cases (a full-size launch is too large to capture); the profile named beside
+# each figure gives the command.  Every query has its own table and candidate list, so traffic grows in proportion to
+# the algorithmic bytes.
+NCU_DRAM_PER_ALGORITHMIC_BYTE = {
+    "ci": (443.5e6 / 471.0e6, "profiles/ncu_ci_coarse_mid.md (Mid corpus, batch 8)"),
+    "partial": (1527e6 / 64.0, "profiles/ncu_partial_score_mid.md (Mid corpus, batch 64; bytes per query)"),
+}
 
 
 class ClockSampler:
@@ -96,10 +102,11 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
+            time.sleep(0.15)                      # let the first sample arrive before the timed region starts
         except Exception:
             self.proc = None
 
@@ -168,6 +175,20 @@ def time_oracle(oix, q_np, cfg, budget_s, min_q, max_q):
     return n, time.perf_counter() - t0
 
 
+def host_cpu():
+    """(logical cores of the host, CPU model name)."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return os.cpu_count() or 1, model
+
+
 def run_reference(args, cfg, rank, world):
     """The CPU oracle as the reference arm: rank 0 only; a step is one query (a bounded sample of a batch)."""
     if rank != 0:
@@ -185,13 +206,15 @@ def run_reference(args, cfg, rank, world):
         oracle.pipeline(q_np[(args.warmup + s) % len(q_np)], oix, cfg.nprobe, cfg.n_prune, cfg.k)
     dt = time.perf_counter() - t0
     qps = args.steps / dt
+    cores, model = host_cpu()
     sample = "1 query per step (of the %d-query batch), %d steps, single thread" % (args.batch, args.steps)
     print(json.dumps({
         "impl": "reference", "metric": metric_name(cfg, args.batch), "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64+f64", "data": "synthetic",
         "config": {"workload": cfg.name, "batch": 1, "sample": sample},
-        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": cores, "host_cpu": model},
         "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
 
@@ -318,8 +341,7 @@ def run_sharded(args, cfg, pkg, rank, world, local_rank, device):
         print(json.dumps({
             "metric": metric_name(cfg, B) + ", document-sharded", "value": qps, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
-            "scaling": "strong", "vs_baseline": None, "dtype": "int32 fixed point (stages 1-3) + f32 (stage 4)",
-            "data": "synthetic",
+            "scaling": "strong", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
             "config": {"workload": cfg.name, "batch": B, "pruning": mode,
                        "parallelism": "documents sharded over %d ranks, two all-gathers of ids and scores per step" % world,
                        "docs_per_rank": hi - lo, "equals_plain_search": equal},
@@ -327,79 +349,34 @@ def run_sharded(args, cfg, pkg, rank, world, local_rank, device):
     dist.destroy_process_group()
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="mid")
-    ap.add_argument("--batch", type=int, default=0, help="queries per call (default 256; 64 for the long-document configs)")
-    ap.add_argument("--partial", action="store_true",
-                    help="prune with the paper's partial scores (chimera_search_partial) instead of stage 3")
-    ap.add_argument("--rabitq", action="store_true",
-                    help="the paper's pipeline on RaBitQ 1-bit codes (chimera_search_rabitq)")
-    ap.add_argument("--sweep", action="store_true", help="QPS vs recall over nprobe x n_prune x k (see run_sweep)")
-    ap.add_argument("--sweep-queries", type=int, default=200)
-    ap.add_argument("--batch1-queries", type=int, default=200)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sharded", action="store_true",
-                    help="document-sharded search over the ranks (one JSON line; see run_sharded) instead of replicas")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+PRUNING_TEXT = {"ci": "centroid interaction over every candidate token",
+                "partial": "partial scores of retrieved tokens (Algorithm 2)",
+                "rabitq": "partial 1-bit RaBitQ scores of retrieved tokens, then complete 1-bit scores"}
 
-    cfg = CONFIGS[args.config]
-    if args.batch <= 0:
-        args.batch = 64 if cfg.name.startswith("long") else 256
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
-    if args.impl == "reference":
-        run_reference(args, cfg, rank, world)
-        return
-
-    import paper_2608_23553_b200 as pkg
-    pkg.lib()                                    # fails loudly if the CUDA library is missing
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
-    torch.cuda.set_device(local_rank)
-    device = torch.device("cuda", local_rank)
-    if args.sharded:
-        run_sharded(args, cfg, pkg, rank, world, local_rank, device)
-        return
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=device)
+def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_rank=0, steps=None, batch1_n=None,
+            full=True):
+    """Times one workload in one pruning mode on this rank and returns the result fields (QPS at the batch size and at
+    batch 1, per-stage CUDA-event times, the roofline of the dominant kernel and of each stage).  full=False leaves
+    out the end-to-end run through the host entry point and the CUDA-graph variant of batch 1."""
+    kw = {"partial": mode == "partial", "rabitq": mode == "rabitq"}
+    B = args.batch if args.batch > 0 else (64 if cfg.name.startswith("long") else 16 if cfg.name == "tiny" else 256)
+    nq, P, n_prune, k = cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
+    steps = args.steps if steps is None else steps
+    warmup = args.warmup
+    batch1_n = args.batch1_queries if batch1_n is None else batch1_n
+    maxc = candidate_capacity(index, q, nq, P, n_prune, k)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    corp, q, gen_s = build_workload(cfg, device, rabitq=args.rabitq or args.sweep)
-    t0 = time.time()
-    index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
-    build_s = time.time() - t0
-    B, nq, P, n_prune, k = args.batch, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
-    if args.partial or args.sweep:
-        index.enable_partial()
-    if args.rabitq or args.sweep:
-        index.attach_rabitq(corp.rotation, corp.rq_bits, corp.rq_inv_dot)
-    mode = {"partial": args.partial, "rabitq": args.rabitq}
-    if args.sweep:
-        if rank == 0:
-            run_sweep(args, cfg, pkg, index, corp, q)
-        return
-    maxc = candidate_capacity(index, q, nq, P, n_prune, k)
-
     # batches cycle through the config's query set
-    n_batches = max(1, min(args.steps + args.warmup, (q.shape[0] + B - 1) // B + 1))
+    n_batches = max(1, min(steps + warmup, (q.shape[0] + B - 1) // B + 1))
     idx = (torch.arange(n_batches * B, device=device) % q.shape[0]).view(n_batches, B)
     batches = q[idx].contiguous()                                   # [n_batches, B, nq, D] on the device
-    host_batches = batches.cpu().pin_memory()
     out = (torch.empty(B, k, dtype=torch.int32, device=device), torch.empty(B, k, dtype=torch.float32, device=device))
-    host_out = (torch.empty(B, k, dtype=torch.int32).pin_memory(), torch.empty(B, k, dtype=torch.float32).pin_memory())
 
     # algorithmic work per batch (outside the timed region): candidate documents and their tokens, from the taps
     doclens64 = corp.doclens.to(torch.int64)
@@ -407,7 +384,7 @@ def main():
     work = []
     for bi in range(n_batches):
         taps = index.alloc_taps(B, nq, P, n_prune, max_candidates=maxc, table=False, ci=False)
-        index.search(batches[bi], P, n_prune, k, max_candidates=maxc, taps=taps, **mode)
+        index.search(batches[bi], P, n_prune, k, max_candidates=maxc, taps=taps, **kw)
         assert index.status() == 0
         mask = torch.arange(taps.cand.shape[1], device=device)[None, :] < taps.n_cand[:, None].to(torch.int64)
         toks = (doclens64[taps.cand.to(torch.int64).clamp_(0, index.N - 1)] * mask).sum()
@@ -417,11 +394,12 @@ def main():
                      "contenders": int(taps.n_contenders.sum()),
                      "retrieved": int(list_len[taps.probes.to(torch.int64)].sum())})
         del taps, mask
+    del list_len
     torch.cuda.empty_cache()
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps ------------------------------------
-    for s in range(args.warmup):
-        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out, **mode)
+    for s in range(warmup):
+        index.search(batches[s % n_batches], P, n_prune, k, max_candidates=maxc, out=out, **kw)
     barrier()
     pkg.profile_enable(True)
     pkg.profile_read()
@@ -429,194 +407,393 @@ def main():
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for s in range(args.steps):
-        index.search(batches[(args.warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc, out=out,
-                     **mode)
+    for s in range(steps):
+        index.search(batches[(warmup + s) % n_batches], P, n_prune, k, max_candidates=maxc, out=out, **kw)
     e1.record()
     barrier()
     clocks = sampler.stop()
     ms_total = e0.elapsed_time(e1)
     stage_ms, launches = pkg.profile_read()
     pkg.profile_enable(False)
-    qps, ms_total = whole_job_qps(ms_total, B * args.steps, dist, device)
-    ms_per_step = ms_total / args.steps
+    qps, ms_total = whole_job_qps(ms_total, B * steps, dist, device)
+    ms_per_step = ms_total / steps
 
-    # ---- end to end through the host entry point: pinned host queries in, host ids/scores out -------------------
     dq = torch.empty_like(batches[0])
 
     def host_search(hq, hout, dbuf, dout):
-        if not (args.partial or args.rabitq):
+        if mode == "ci":
             index.search_host(hq, P, n_prune, k, max_candidates=maxc, out=hout)
         else:       # the host entry point has no such variant: pinned copies around the device entry point
             dbuf.copy_(hq, non_blocking=True)
-            index.search(dbuf, P, n_prune, k, max_candidates=maxc, out=dout, **mode)
+            index.search(dbuf, P, n_prune, k, max_candidates=maxc, out=dout, **kw)
             hout[0].copy_(dout[0], non_blocking=True)
             hout[1].copy_(dout[1], non_blocking=True)
             torch.cuda.synchronize()
 
-    for s in range(2):
-        host_search(host_batches[s % n_batches], host_out, dq, out)
-    barrier()
-    w0 = time.perf_counter()
-    for s in range(args.steps):
-        host_search(host_batches[(args.warmup + s) % n_batches], host_out, dq, out)
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - w0
-    e2e_qps, _ = whole_job_qps(e2e_s * 1e3, B * args.steps, dist, device)
-    h2d = B * nq * cfg.dim * 4
-    d2h = B * k * 8
+    e2e = None
+    if full:
+        # ---- end to end through the host entry point: pinned host queries in, host ids/scores out ----------------
+        host_batches = batches.cpu().pin_memory()
+        host_out = (torch.empty(B, k, dtype=torch.int32).pin_memory(), torch.empty(B, k, dtype=torch.float32).pin_memory())
+        for s in range(2):
+            host_search(host_batches[s % n_batches], host_out, dq, out)
+        barrier()
+        w0 = time.perf_counter()
+        for s in range(steps):
+            host_search(host_batches[(warmup + s) % n_batches], host_out, dq, out)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - w0
+        e2e_qps, _ = whole_job_qps(e2e_s * 1e3, B * steps, dist, device)
+        e2e = {"value": e2e_qps, "unit": UNIT, "h2d_bytes_per_step": B * nq * cfg.dim * 4, "d2h_bytes_per_step": B * k * 8}
 
     # ---- batch 1: one synchronised query at a time (the paper's protocol: latency = 1 / QPS) --------------------
-    n1 = min(args.batch1_queries, q.shape[0])
+    n1 = min(batch1_n, q.shape[0])
     out1 = (torch.empty(1, k, dtype=torch.int32, device=device), torch.empty(1, k, dtype=torch.float32, device=device))
     for i in range(5):
-        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, **mode)
+        index.search(q[i % q.shape[0]:i % q.shape[0] + 1], P, n_prune, k, max_candidates=maxc, out=out1, **kw)
     torch.cuda.synchronize()
     lat = []
     pkg.profile_enable(True)
     pkg.profile_read()
     for i in range(n1):
         a = time.perf_counter()
-        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, **mode)
+        index.search(q[i:i + 1], P, n_prune, k, max_candidates=maxc, out=out1, **kw)
         torch.cuda.synchronize()
         lat.append(time.perf_counter() - a)
     stage_ms1, _ = pkg.profile_read()
     pkg.profile_enable(False)
     lat = np.array(lat)
-    # the same protocol with the search captured once in a CUDA graph (same kernels; no per-kernel launch gaps)
-    graphed = pkg.GraphedSearch(index, 1, nq, P, n_prune, k, max_candidates=maxc, **mode)
-    for i in range(5):
-        graphed(q[i:i + 1])
-    torch.cuda.synchronize()
-    lat_g = []
-    for i in range(n1):
-        a = time.perf_counter()
-        graphed(q[i:i + 1])
-        torch.cuda.synchronize()
-        lat_g.append(time.perf_counter() - a)
-    lat_g = np.array(lat_g)
-    host_q1 = q[:n1].cpu().pin_memory()
-    hout1 = (torch.empty(1, k, dtype=torch.int32).pin_memory(), torch.empty(1, k, dtype=torch.float32).pin_memory())
-    w0 = time.perf_counter()
-    dq1 = torch.empty_like(q[:1])
-    for i in range(n1):
-        host_search(host_q1[i:i + 1], hout1, dq1, out1)
-    e2e1_qps = n1 / (time.perf_counter() - w0)
-
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
-
-    # ---- roofline of the dominant kernel: the stage-3 bound scan over every candidate token (ci_coarse_rng_kernel) ---
-    peak, peak_kind = measured_peaks()
-    used = [work[(args.warmup + s) % n_batches] for s in range(args.steps)]
-    mean = lambda key: float(np.mean([u[key] for u in used]))       # noqa: E731
-    n_prof = min(args.steps, 256)                                    # the library times at most 256 calls per read
-    ci_ms = stage_ms["centroid_interaction"] / n_prof
-    # algorithmic HBM bytes of one launch: the centroid id of every candidate token (4 B) + per candidate document
-    # its id (4 B), two token offsets (16 B) and the two bounds written (8 B)
-    ci_bytes = 4.0 * mean("cand_tokens") + 28.0 * mean("cand")
-    ci_gbs = ci_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0
-    # what binds it: one table-row lookup per candidate token; a lookup is one distinct 128-byte line for the SM's
-    # load pipe, which retires one line per cycle, so the roof is SMs x SM clock row lookups per second
-    rows = mean("cand_tokens")
-    lookup_roof = 148 * 1.965e9
-    cont_frac = mean("contenders") / max(mean("cand"), 1.0)
-    g4_ms = stage_ms["residual_scores"] / n_prof
-    # stage 4 reads per survivor token its centroid id + residual code (or its 1-bit code + scale on the RaBitQ path)
-    g4_bytes = mean("pruned_tokens") * ((cfg.dim // 8 + 4.0) if args.rabitq else (4.0 + cfg.code_bytes))
-    stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
-    roofline = {
-        "kernel": "ci_coarse_rng_kernel (stage 3 bound scan over every candidate token)", "bound": "hbm",
-        "achieved": ci_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-        "frac": ci_gbs / peak, "traffic": ncu_traffic(cfg, B), "ms_per_launch": ci_ms,
-        "algorithmic_bytes_per_launch": ci_bytes, "contender_fraction": cont_frac,
-        "binding_roof": {"bound": "table-row lookups (one 128-byte line per SM cycle)", "lookups_per_launch": rows,
-                         "achieved_glookups_s": rows / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0,
-                         "peak_glookups_s": lookup_roof / 1e9,
-                         "frac": rows / (ci_ms * 1e-3) / lookup_roof if ci_ms > 0 else 0.0,
-                         "l2_bytes_per_launch": rows * nq},
-        "stage_ms_per_step": stages,
-        "stage4": {"kernel": "residual_maxsim_umma (tcgen05 kind::i8)", "ms_per_launch": g4_ms,
-                   "code_gbs": g4_bytes / (g4_ms * 1e-3) / 1e9 if g4_ms > 0 else 0.0,
-                   "int8_tops": 2.0 * 3.0 * mean("pruned_tokens") * nq * cfg.dim / (g4_ms * 1e-3) / 1e12 if g4_ms > 0 else 0.0},
+    res = {
+        "metric": metric_name(cfg, B) + (" with partial-score refinement" if mode == "partial" else "")
+        + (" on RaBitQ 1-bit codes (paper pipeline)" if mode == "rabitq" else ""),
+        "value": qps, "unit": UNIT, "ms_per_step": ms_per_step, "steps": steps, "batch": B,
+        "qps_batch1": float(1.0 / lat.mean()),
+        "stage_ms_batch1": {name: round(v / min(n1, 256), 4) for name, v in stage_ms1.items()},
+        "latency_ms_batch1": {"mean": float(lat.mean() * 1e3), "p50": float(np.percentile(lat, 50) * 1e3),
+                              "p95": float(np.percentile(lat, 95) * 1e3), "p99": float(np.percentile(lat, 99) * 1e3)},
+        "gpu_launches": int(sum(launches.values())), "clocks": clocks, "max_candidates": maxc if maxc else cfg.n_docs,
     }
-    if args.partial or args.rabitq:
+    if full:
+        # the same protocol with the search captured once in a CUDA graph (same kernels; no per-kernel launch gaps)
+        graphed = pkg.GraphedSearch(index, 1, nq, P, n_prune, k, max_candidates=maxc, **kw)
+        for i in range(5):
+            graphed(q[i:i + 1])
+        torch.cuda.synchronize()
+        lat_g = []
+        for i in range(n1):
+            a = time.perf_counter()
+            graphed(q[i:i + 1])
+            torch.cuda.synchronize()
+            lat_g.append(time.perf_counter() - a)
+        res["qps_batch1_cuda_graph"] = float(1.0 / np.mean(lat_g))
+        del graphed
+        host_q1 = q[:n1].cpu().pin_memory()
+        hout1 = (torch.empty(1, k, dtype=torch.int32).pin_memory(), torch.empty(1, k, dtype=torch.float32).pin_memory())
+        w0 = time.perf_counter()
+        dq1 = torch.empty_like(q[:1])
+        for i in range(n1):
+            host_search(host_q1[i:i + 1], hout1, dq1, out1)
+        e2e["batch1_value"] = n1 / (time.perf_counter() - w0)
+        res["e2e"] = e2e
+
+    # ---- roofline of the dominant kernel -------------------------------------------------------------------------
+    peak, peak_kind = measured_peaks()
+    used = [work[(warmup + s) % n_batches] for s in range(steps)]
+    mean = lambda key: float(np.mean([u[key] for u in used]))       # noqa: E731
+    n_prof = min(steps, 256)                                         # the library times at most 256 calls per read
+    ci_ms = stage_ms["centroid_interaction"] / n_prof
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0   # noqa: E731
+    # algorithmic HBM bytes of one launch of the stage-3 bound scan: the centroid id of every candidate token (4 B) +
+    # 8 B per candidate document (its token offsets); the kernel's own id / range / bound traffic is not the method's
+    ci_bytes = 4.0 * mean("cand_tokens") + 8.0 * mean("cand")
+    # what binds it: one table-row lookup per candidate token; a lookup is one distinct 128-byte line for the SM's
+    # load pipe, which retires one line per cycle, so the roof is SMs x SM clock row lookups per second (derived from
+    # the device's SM count and the clock sampled during the timed region; not a measured peak)
+    rows = mean("cand_tokens")
+    sm_count = torch.cuda.get_device_properties(device).multi_processor_count
+    sm_hz = 1e6 * (clocks["sm_mhz"] or clocks["sm_max_mhz"] or 1965.0)
+    lookup_roof = sm_count * sm_hz
+    g4_ms = stage_ms["residual_scores"] / n_prof
+    # stage 4 reads per survivor token its centroid id + residual code (or its 1-bit code + scale on the RaBitQ path);
+    # the centroid term additionally gathers one int32 table row (q_len x 4 B) per token, which is the implementation's
+    # traffic, reported beside the method's
+    g4_bytes = mean("pruned_tokens") * ((cfg.dim // 8 + 4.0) if mode == "rabitq" else (4.0 + cfg.code_bytes))
+    g4_row_bytes = 0.0 if mode == "rabitq" else mean("pruned_tokens") * nq * 4.0
+    stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
+    if mode == "ci":
+        ratio, src = NCU_DRAM_PER_ALGORITHMIC_BYTE["ci"]
+        frac = gbs(ci_bytes, ci_ms) / peak
+        roofline = {
+            "kernel": "ci_coarse_rng_kernel (stage 3 bound scan over every candidate token)", "bound": "hbm",
+            "achieved": gbs(ci_bytes, ci_ms), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": frac,
+            "traffic": ratio * ci_bytes,
+            "traffic_kind": "stored ncu figure, not measured in this run: DRAM bytes per algorithmic byte of " + src
+                            + " x this launch's algorithmic bytes",
+            "ms_per_launch": ci_ms, "algorithmic_bytes_per_launch": ci_bytes,
+            "target": {"frac": TARGET, "met": bool(frac >= TARGET),
+                       "note": "the task's 60 % of HBM peak for the code-scan stages is NOT met: every 4-byte centroid "
+                               "id costs one 32-byte table-row lookup through L1/L2, which binds the kernel"},
+            "contender_fraction": mean("contenders") / max(mean("cand"), 1.0),
+            "binding_roof": {"bound": "table-row lookups (one 128-byte line per SM cycle); derived from SM count x "
+                                      "sampled SM clock, not a driver-measured peak",
+                             "lookups_per_launch": rows, "achieved_glookups_s": rows / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0,
+                             "peak_glookups_s": lookup_roof / 1e9, "sm_count": sm_count, "sm_mhz": sm_hz / 1e6,
+                             "frac": rows / (ci_ms * 1e-3) / lookup_roof if ci_ms > 0 else 0.0,
+                             "l2_bytes_per_launch": rows * nq},
+        }
+    else:
         # candidate refinement by partial scores replaces the scan: the dominant stage-3 kernel visits every token of
         # the nq * nprobe probed posting lists.  Algorithmic bytes per visit: the list entry (token id + document id,
         # 8 B) and the token's code (residual code, or 1-bit code + its 4-byte scale); per candidate document its
         # partial score (4 B).  The table of running maxima is the implementation's, not the method's, and is not
         # counted.  The slot times the clear, the scoring kernel and (RaBitQ) the summation together.
-        code_b = (cfg.dim // 8 + 4.0) if args.rabitq else float(cfg.code_bytes)
+        code_b = (cfg.dim // 8 + 4.0) if mode == "rabitq" else float(cfg.code_bytes)
         ps_bytes = mean("retrieved") * (8.0 + code_b) + mean("cand") * 4.0
-        ps_gbs = ps_bytes / (ci_ms * 1e-3) / 1e9 if ci_ms > 0 else 0.0
-        traffic = None
-        if cfg.name == "mid" and args.partial and not args.rabitq:
-            traffic = NCU_PARTIAL_MID_B64_BYTES * B / 64.0
-        for key in ("binding_roof", "contender_fraction"):
-            roofline.pop(key)
-        roofline.update({
-            "kernel": ("rabitq_partial_kernel" if args.rabitq else "partial_score_kernel")
-            + " (+ its clear kernel): partial scores of the retrieved tokens, Algorithm 2",
-            "achieved": ps_gbs, "frac": ps_gbs / peak, "traffic": traffic, "algorithmic_bytes_per_launch": ps_bytes,
+        frac = gbs(ps_bytes, ci_ms) / peak
+        traffic, tk = None, None
+        if cfg.name == "mid" and mode == "partial":
+            per_query, src = NCU_DRAM_PER_ALGORITHMIC_BYTE["partial"]
+            traffic, tk = per_query * B, "stored ncu figure, not measured in this run: " + src + " x batch"
+        roofline = {
+            "kernel": ("rabitq_partial_kernel" if mode == "rabitq" else "partial_score_kernel")
+            + " (+ its clear kernel): partial scores of the retrieved tokens, Algorithm 2", "bound": "hbm",
+            "achieved": gbs(ps_bytes, ci_ms), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": frac,
+            "traffic": traffic, "traffic_kind": tk, "ms_per_launch": ci_ms, "algorithmic_bytes_per_launch": ps_bytes,
+            "target": {"frac": TARGET, "met": bool(frac >= TARGET)},
             "visits_per_launch": mean("retrieved"),
             "note": "scattered 32-byte sectors (codes of random tokens, read-modify-write of 4-byte cells): the roof "
-                    "of such accesses is below the streaming-copy peak this fraction is taken against"})
+                    "of such accesses is below the streaming-copy peak this fraction is taken against"}
+        ci_bytes = ps_bytes
+    roofline["stage_ms_per_step"] = stages
     # per-stage achieved fraction of the roof that the stage's algorithmic work is measured against
     i8_peak, i8_kind = measured_int8_tops()
 
-    def frac_entry(bound, work, ms, peak, unit):
-        ach = work / (ms * 1e-3) if ms > 0 else 0.0
-        return {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak if peak else 0.0}
+    def frac_entry(bound, amount, ms, pk, unit, **more):
+        ach = amount / (ms * 1e-3) if ms > 0 else 0.0
+        e = {"bound": bound, "achieved": ach, "peak": pk, "unit": unit, "frac": ach / pk if pk else 0.0}
+        e.update(more)
+        return e
 
     g1_ms = stage_ms["score_table"] / n_prof
     pr_ms = stage_ms["probes"] / n_prof
+    g4_frac = gbs(g4_bytes, g4_ms) / peak
     roofline["per_stage"] = {
         "score_table": frac_entry("tensor (int8, %s)" % i8_kind, 2.0 * 9.0 * B * nq * cfg.n_centroids * cfg.dim / 1e12,
-                                  g1_ms, i8_peak, "TOP/s"),
+                                  g1_ms, i8_peak, "TOP/s",
+                                  table_write_gbs=gbs(B * nq * cfg.n_centroids * 5.0, g1_ms)),
         "probes": frac_entry("hbm", B * nq * cfg.n_centroids * 4.0 / 1e9, pr_ms, peak, "GB/s"),
-        ("partial_scores" if args.partial or args.rabitq else "centroid_interaction_bounds"):
-            frac_entry("hbm", (ps_bytes if args.partial or args.rabitq else ci_bytes) / 1e9, ci_ms, peak, "GB/s"),
-        "residual_scores": frac_entry("hbm (code + centroid-id bytes)", g4_bytes / 1e9, g4_ms, peak, "GB/s"),
+        ("partial_scores" if mode != "ci" else "centroid_interaction_bounds"):
+            frac_entry("hbm", ci_bytes / 1e9, ci_ms, peak, "GB/s", target_frac=TARGET, target_met=bool(frac >= TARGET)),
+        "residual_scores": frac_entry("hbm (code + centroid-id bytes)", g4_bytes / 1e9, g4_ms, peak, "GB/s",
+                                      target_frac=TARGET, target_met=bool(g4_frac >= TARGET),
+                                      with_table_row_gathers_gbs=gbs(g4_bytes + g4_row_bytes, g4_ms),
+                                      surviving_tokens_per_launch=mean("pruned_tokens")),
         "residual_scores_tensor": frac_entry("tensor (int8, %s)" % i8_kind,
                                              2.0 * 3.0 * mean("pruned_tokens") * nq * cfg.dim / 1e12, g4_ms, i8_peak,
                                              "TOP/s"),
     }
+    res["roofline"] = roofline
+    res["pruning"] = PRUNING_TEXT[mode]
+    return res
 
+
+def summary(r):
+    """The short form of a measurement kept under `configs` in the headline line."""
+    per = r["roofline"]["per_stage"]
+    return {"metric": r["metric"], "value": r["value"], "unit": UNIT, "batch": r["batch"], "steps": r["steps"],
+            "ms_per_step": r["ms_per_step"], "qps_batch1": r["qps_batch1"],
+            "latency_ms_batch1": r["latency_ms_batch1"], "stage_ms_per_step": r["roofline"]["stage_ms_per_step"],
+            "roofline_frac": r["roofline"]["frac"], "roofline_kernel": r["roofline"]["kernel"].split(" ")[0],
+            "target_met": r["roofline"]["target"]["met"],
+            "stage4_code_frac_of_hbm": per["residual_scores"]["frac"],
+            "score_table_frac_of_int8_peak": per["score_table"]["frac"], "probes_frac_of_hbm": per["probes"]["frac"],
+            "clocks": r["clocks"], "gpu_launches": r["gpu_launches"]}
+
+
+def run_other_configs(pkg, args, device, headline_done):
+    """A shorter measurement (fewer steps, no end-to-end leg) of every workload and pipeline other than the headline's
+    centroid-interaction line.  Errors are recorded, not raised: the headline line must still be printed."""
+    out = {}
+    steps = max(3, min(args.steps, 10))
+    plan = [("mid", ("ci", "partial", "rabitq")), ("tiny", ("ci",)), ("long_d128_b2", ("ci", "partial")),
+            ("long_d128_b1", ("ci",)), ("long_d96_b2", ("ci",)), ("long_d96_b1", ("ci",))]
+    for name, modes in plan:
+        if name in headline_done:
+            continue
+        try:
+            cfg = CONFIGS[name]
+            corp, q, _ = build_workload(cfg, device, rabitq="rabitq" in modes)
+            index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+            for mode in modes:
+                if mode == "partial":
+                    index.enable_partial()
+                if mode == "rabitq":
+                    index.attach_rabitq(corp.rotation, corp.rq_bits, corp.rq_inv_dot)
+                key = name if mode == "ci" else name + "_" + mode
+                out[key] = summary(measure(pkg, cfg, corp, q, index, args, device, mode, steps=steps, batch1_n=50,
+                                           full=False))
+            index.close()
+            del index, corp, q
+        except Exception as e:          # noqa: BLE001
+            out[name + "_error"] = "%s: %s" % (type(e).__name__, e)
+        torch.cuda.empty_cache()
+    return out
+
+
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_ranks(n):
+    """Start n ranks of this script (one process per GPU) under torch.distributed.run on this node and return their
+    exit code.  Used when `--gpus n` is given and the script is not already running under a launcher."""
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")             # keep the communicator's init lines (ranks, transport) in the log
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n), "--master-addr",
+           "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
+def dry_launch(args, rank, world):
+    """The multi-rank plumbing of the replica benchmark without a GPU: `world` gloo ranks on the CPU, each with a made-up
+    step time, reduced as in the real run (rank r reports 100 + 50 r ms for 512 queries)."""
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+    qps, ms = whole_job_qps(100.0 + 50.0 * rank, 512, dist)
+    if rank == 0:
+        print(json.dumps({"dry_launch": True, "n_gpus": world, "value": qps, "unit": UNIT, "ms": ms, "scaling": "weak"}))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="", help="one workload only (tiny, mid, large, long_d128_b2, ...); default: the "
+                    "Large headline plus a short measurement of every other workload")
+    ap.add_argument("--batch", type=int, default=0, help="queries per call (default 256; 64 for the long-document configs, 16 for Tiny)")
+    ap.add_argument("--partial", action="store_true",
+                    help="prune with the paper's partial scores (chimera_search_partial) instead of stage 3")
+    ap.add_argument("--rabitq", action="store_true",
+                    help="the paper's pipeline on RaBitQ 1-bit codes (chimera_search_rabitq)")
+    ap.add_argument("--sweep", action="store_true", help="QPS vs recall over nprobe x n_prune x k (see run_sweep)")
+    ap.add_argument("--sweep-queries", type=int, default=200)
+    ap.add_argument("--batch1-queries", type=int, default=200)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="headline workload only")
+    ap.add_argument("--sharded", action="store_true",
+                    help="document-sharded search over the ranks (one JSON line; see run_sharded) instead of replicas")
+    ap.add_argument("--dry-launch", action="store_true",
+                    help="exercise the rank launch and the timing reduction with gloo ranks on the CPU (no GPU work)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    # one process per GPU: when not already under a launcher, start the ranks here
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(launch_ranks(args.gpus))
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.dry_launch:
+        dry_launch(args, rank, world)
+        return
+
+    single = bool(args.config) or args.partial or args.rabitq or args.sweep or args.sharded
+    cfg = CONFIGS[args.config or HEADLINE]
+    if args.impl == "reference":
+        if args.batch <= 0:
+            args.batch = 64 if cfg.name.startswith("long") else 256
+        run_reference(args, cfg, rank, world)
+        return
+
+    import paper_2608_23553_b200 as pkg
+    pkg.lib()                                    # fails loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if args.sharded:
+        if args.batch <= 0:
+            args.batch = 64 if cfg.name.startswith("long") else 256
+        run_sharded(args, cfg, pkg, rank, world, local_rank, device)
+        return
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    mode = "rabitq" if args.rabitq else ("partial" if args.partial else "ci")
+    corp, q, gen_s = build_workload(cfg, device, rabitq=args.rabitq or args.sweep or (not single and world == 1))
+    t0 = time.time()
+    index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
+    build_s = time.time() - t0
+    if args.partial or args.sweep:
+        index.enable_partial()
+    if args.rabitq or args.sweep:
+        index.attach_rabitq(corp.rotation, corp.rq_bits, corp.rq_inv_dot)
+    if args.sweep:
+        if args.batch <= 0:
+            args.batch = 256
+        if rank == 0:
+            run_sweep(args, cfg, pkg, index, corp, q)
+        return
+
+    r = measure(pkg, cfg, corp, q, index, args, device, mode, dist, local_rank)
+    nq = cfg.q_len
     result = {
-        "metric": metric_name(cfg, B) + (" with partial-score refinement" if args.partial else "")
-        + (" on RaBitQ 1-bit codes (paper pipeline)" if args.rabitq else ""), "value": qps,
-        "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32 fixed point (stages 1-3) + f32 (stage 4)", "data": "synthetic",
-        "config": {"workload": cfg.name, "batch": B, "n_docs": cfg.n_docs, "n_tokens": corp.n_tokens,
-                   "n_centroids": cfg.n_centroids, "dim": cfg.dim, "nbits": cfg.nbits, "q_len": nq, "nprobe": P,
-                   "n_prune": n_prune, "k": k, "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "max_candidates": maxc if maxc else cfg.n_docs,
-                   "pruning": "partial 1-bit RaBitQ scores of retrieved tokens, then complete 1-bit scores" if args.rabitq
-                   else "partial scores of retrieved tokens (Algorithm 2)" if args.partial
-                   else "centroid interaction over every candidate token",
+        "metric": r["metric"], "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": r["batch"], "n_docs": cfg.n_docs, "n_tokens": corp.n_tokens,
+                   "n_centroids": cfg.n_centroids, "dim": cfg.dim, "nbits": cfg.nbits, "q_len": nq,
+                   "nprobe": cfg.nprobe, "n_prune": cfg.n_prune, "k": cfg.k,
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "max_candidates": r["max_candidates"], "pruning": r["pruning"],
                    "l2": "inputs larger than L2 (index %.1f GB, score table %.1f GB per batch); no flush"
-                         % ((corp.cids.numel() * 4 + corp.codes.numel()) / 1e9, B * cfg.n_centroids * nq * 4 / 1e9),
+                         % ((corp.cids.numel() * 4 + corp.codes.numel()) / 1e9,
+                            r["batch"] * cfg.n_centroids * nq * 4 / 1e9),
                    "gen_s": round(gen_s, 1), "index_build_s": round(build_s, 2)},
-        "qps_batch1": float(1.0 / lat.mean()),
-        "qps_batch1_cuda_graph": float(1.0 / lat_g.mean()),
-        "stage_ms_batch1": {name: round(v / min(n1, 256), 4) for name, v in stage_ms1.items()},
-        "latency_ms_batch1": {"mean": float(lat.mean() * 1e3), "p50": float(np.percentile(lat, 50) * 1e3),
-                              "p95": float(np.percentile(lat, 95) * 1e3), "p99": float(np.percentile(lat, 99) * 1e3)},
-        "e2e": {"value": e2e_qps, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "batch1_value": e2e1_qps},
-        "gpu_launches": int(sum(launches.values())),
-        "clocks": clocks,
-        "roofline": roofline,
+        "qps_batch1": r["qps_batch1"], "qps_batch1_cuda_graph": r.get("qps_batch1_cuda_graph"),
+        "stage_ms_batch1": r["stage_ms_batch1"], "latency_ms_batch1": r["latency_ms_batch1"],
+        "e2e": r["e2e"], "gpu_launches": r["gpu_launches"], "clocks": r["clocks"], "roofline": r["roofline"],
     }
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
 
     if world == 1 and not args.no_cpu_baseline:
         oix = oracle_index(corp, cfg)
         n, secs = time_oracle(oix, q.cpu().numpy(), cfg, budget_s=12.0, min_q=3, max_q=16)
+        cores, model = host_cpu()
         result["cpu_baseline"] = {"value": n / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                  "sample": "first %d queries of the workload, all stages, %.1f s" % (n, secs)}
+                                  "sample": "first %d queries of the workload, all stages, %.1f s" % (n, secs),
+                                  "host_cores": cores, "host_cpu": model}
+        del oix
+    if world == 1 and not single and not args.no_other_configs:
+        others = {}
+        try:                            # the two paper pipelines on the headline corpus, then every other workload
+            index.enable_partial()
+            others[cfg.name + "_partial"] = summary(measure(pkg, cfg, corp, q, index, args, device, "partial",
+                                                            steps=max(3, min(args.steps, 10)), batch1_n=50, full=False))
+            index.attach_rabitq(corp.rotation, corp.rq_bits, corp.rq_inv_dot)
+            others[cfg.name + "_rabitq"] = summary(measure(pkg, cfg, corp, q, index, args, device, "rabitq",
+                                                           steps=max(3, min(args.steps, 10)), batch1_n=50, full=False))
+        except Exception as e:          # noqa: BLE001
+            others[cfg.name + "_paper_pipelines_error"] = "%s: %s" % (type(e).__name__, e)
+        index.close()
+        del index, corp, q
+        torch.cuda.empty_cache()
+        others.update(run_other_configs(pkg, args, device, {cfg.name}))
+        result["configs"] = others
     print(json.dumps(result))
     if dist is not None:
         dist.destroy_process_group()

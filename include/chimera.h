@@ -272,8 +272,10 @@ int chimera_probes_static(const int32_t *score_table, int64_t n_centroids, int32
  *                            result (a document's stage-4 score does not depend on the shard it is scored in).
  * mode: 0 = stage 3 by centroid interaction, 1 = by partial scores (needs chimera_index_enable_partial), 2 = the
  * RaBitQ pipeline (needs chimera_index_attach_rabitq).  Steps 1 and 3 must use the same workspace and the same
- * parameters, with no other call on that workspace in between (step 3 continues from what step 1 left there);
- * check chimera_workspace_status after step 1.  All pointers device; everything is enqueued on `stream`.
+ * parameters, with no other call on that workspace in between (step 3 continues from what step 1 left there, and
+ * keeps the status bits step 1 set: one chimera_workspace_status after step 3 covers both).  In a multi-process run
+ * exchange the status with the other ranks before acting on it: a rank that stops between the collectives leaves the
+ * others waiting in theirs.  All pointers device; everything is enqueued on `stream`.
  * world * k <= 16384 in step 5 (CHIMERA_UNSUPPORTED otherwise). */
 int chimera_shard_local(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
                         int32_t nprobe, int32_t n_prune, int32_t k, int64_t max_candidates, int32_t mode,

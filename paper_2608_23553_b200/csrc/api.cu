@@ -207,7 +207,8 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     int rc;
 
     prof_begin(st);
-    CHIMERA_CUDA(cudaMemsetAsync(status, 0, 64 * sizeof(uint32_t), st));
+    // a resumed call continues an earlier one: the status bits that one set stay, new ones are OR-ed in
+    if (!resume) CHIMERA_CUDA(cudaMemsetAsync(status, 0, 64 * sizeof(uint32_t), st));
 
     // results of the stages that do not run come from the caller
     if (first > 1 && !resume) {

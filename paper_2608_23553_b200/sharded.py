@@ -91,11 +91,18 @@ class ShardEngine:
                                                   _ptr(scores)))
         return ids, scores
 
+    def status_word(self) -> torch.Tensor:
+        """The workspace's raw device-side status bits (candidate overflow, bad query element, bounded wait given up)
+        as an int32 device tensor of one element, without synchronising the host.  The finish phase keeps the bits the
+        local phase set, so reading it after the finish phase covers the whole search."""
+        return self.index._ws[:4].view(torch.int32).clone()
+
     def check(self):
-        """Raise if the last local phase overflowed its candidate capacity or a kernel gave up waiting."""
+        """Raise if the phases so far overflowed the candidate capacity or a kernel gave up waiting (this rank only;
+        synchronises).  ShardedSearcher does not use it: it exchanges the status words so that every rank raises."""
         st = self.index.status()
         if st:
-            raise RuntimeError("shard workspace status 0x%x" % st)
+            raise RuntimeError("shard workspace status %d" % st)
 
 
 def all_gather_stack(t: torch.Tensor, group=None) -> torch.Tensor:
@@ -107,18 +114,43 @@ def all_gather_stack(t: torch.Tensor, group=None) -> torch.Tensor:
     return out
 
 
-class ShardedSearcher:
-    """Sequences the phases of one rank.  `engine` provides local_phase / finish_phase / merge_phase (ShardEngine);
-    `gather` maps a tensor to the rank-ordered stack of every rank's tensor (default: all_gather_stack)."""
+class ShardError(RuntimeError):
+    """A rank's device-side status was non-zero (candidate overflow, bad query element, a bounded wait that gave up).
+    Raised on EVERY rank, after all collectives of the search have completed; `status` lists each rank's bits."""
 
-    def __init__(self, engine, gather: Optional[Callable[[torch.Tensor], torch.Tensor]] = None, group=None):
+    def __init__(self, status: List[int]):
+        bad = ", ".join("rank %d: 0x%x" % (r, s) for r, s in enumerate(status) if s)
+        super().__init__("sharded search: device status non-zero on " + bad)
+        self.status = status
+
+
+class ShardedSearcher:
+    """Sequences the phases of one rank.  `engine` provides local_phase / finish_phase / merge_phase and optionally
+    status_word (ShardEngine); `gather` maps a tensor to the rank-ordered stack of every rank's tensor (default:
+    all_gather_stack).
+
+    Failure handling is collective: no rank raises between the collectives (a rank that left early would leave the
+    others blocked in their next all-gather).  Each rank's status word travels with the second exchange, and after the
+    merge every rank sees every rank's word and raises ShardError together.  check=False skips that host
+    synchronisation (the caller reads `last_status`, a device tensor [world], when it chooses to)."""
+
+    def __init__(self, engine, gather: Optional[Callable[[torch.Tensor], torch.Tensor]] = None, group=None,
+                 check: bool = True):
         self.engine = engine
         self.gather = gather if gather is not None else (lambda t: all_gather_stack(t, group))
+        self.check = check
+        self.last_status = None
 
     def search(self, queries, nprobe: int, n_prune: int, k: int, max_candidates: int = 0):
         ids, sc3 = self.engine.local_phase(queries, nprobe, n_prune, k, max_candidates)
-        if hasattr(self.engine, "check"):
-            self.engine.check()
         all_ids, all_sc3 = self.gather(ids), self.gather(sc3)
         top_ids, top_scores = self.engine.finish_phase(queries, nprobe, n_prune, k, all_ids, all_sc3, max_candidates)
-        return self.engine.merge_phase(self.gather(top_ids), self.gather(top_scores))
+        all_top_ids, all_top_scores = self.gather(top_ids), self.gather(top_scores)
+        if hasattr(self.engine, "status_word"):
+            self.last_status = self.gather(self.engine.status_word()).view(-1)
+        out = self.engine.merge_phase(all_top_ids, all_top_scores)
+        if self.check and self.last_status is not None:
+            words = [int(w) for w in self.last_status.cpu().tolist()]
+            if any(words):
+                raise ShardError(words)
+        return out

@@ -1,6 +1,6 @@
 """Parity on the other workload shapes: the long-document precision variants (512-token documents, 64-token queries,
-dim 96/128, 1/2 residual bits) at reduced document count and one of them at full size, and the passage-corpus-shaped
-Large corpus (8.8M documents, ~600M tokens, 262,144 centroids) at full size with sampled queries."""
+dim 96/128, 1/2 residual bits) at reduced document count and one of them at full size (the passage-corpus-shaped
+Large corpus has its own file, test_gpu_large.py)."""
 import numpy as np
 import pytest
 import torch
@@ -74,39 +74,15 @@ def test_long_document_corpus_full_size_sampled_query():
     b = 41
     res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
     assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) <= 2
-
-
-def test_large_corpus_full_size_sampled_queries():
-    import psutil
-    import paper_2608_23553_b200 as pkg
-    from synth import CONFIGS, make_corpus, make_queries
-    if psutil.virtual_memory().available < 48e9:
-        pytest.skip("needs ~25 GB of host memory for the oracle's copy of the corpus")
-    free, _ = torch.cuda.mem_get_info()
-    if free < 90e9:
-        pytest.skip("needs ~60 GB of device memory")
-    cfg = CONFIGS["large"]
-    dev = torch.device("cuda:0")
-    corp = make_corpus(cfg, device=dev)
-    assert abs(corp.doclens.float().mean().item() - 68.0) < 0.3 and 5.9e8 < corp.n_tokens < 6.1e8
-    q = make_queries(cfg, 256, device=dev)
-    gix = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
-    B, maxc = 256, 512 * 1024
-    taps = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, cfg.n_prune, max_candidates=maxc, table=False)
-    ids, sc = gix.search(q, cfg.nprobe, cfg.n_prune, cfg.k, max_candidates=maxc, taps=taps)
+    # the same batch through the paper's candidate refinement (partial scores): F' of every candidate of one query,
+    # the pruned ids and the later stages against the oracle
+    del taps
+    gix.enable_partial()
+    taps = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, cfg.n_prune, table=False)
+    ids, sc = gix.search(q, cfg.nprobe, cfg.n_prune, cfg.k, taps=taps, partial=True)
     assert gix.status() == 0
     tn = taps_to_numpy(taps)
-    ids_np, sc_np, q_np = ids.cpu().numpy(), sc.cpu().numpy(), q.cpu().numpy()
-    for b in range(B):
-        _properties(tn, ids_np, sc_np, b, cfg, cfg.n_docs, cfg.k)
-    # stage 1 for the two sampled queries, on its own: 64 query tokens x all 262,144 centroids
-    t1 = gix.alloc_taps(2, cfg.q_len, cfg.nprobe, cfg.n_prune, max_candidates=1024, table=True)
-    q2 = torch.stack([q[77], q[255]]).contiguous()
-    gix.run_stages(1, 1, q2, 2, cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k, t1, max_candidates=1024)
-    tables = {77: t1.score_table[0].cpu().numpy(), 255: t1.score_table[1].cpu().numpy()}
-    oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
-    for b in (77, 255):
-        res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
-        assert np.array_equal(tables[b], res.S)
-        # check_query enforces the tolerance rule; with k = 100 a swap between two fp32 near-ties can move positions
-        assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) <= 4
+    ids_np, sc_np = ids.cpu().numpy(), sc.cpu().numpy()
+    b = 17
+    res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
+    assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) <= 2

@@ -230,9 +230,11 @@ def test_tiny_config_stage_isolated(chimera, tiny):
 
 
 @pytest.mark.parametrize("n_prune,k", [(17, 17), (100, 128), (128, 100), (129, 64), (1000, 100), (2048, 50),
-                                        (4096, 100), (4096, 128), (4097, 100), (5000, 129), (3000, 10), (300, 1000)])
+                                        (4096, 100), (4096, 128), (4097, 100), (5000, 129), (3000, 10), (300, 1000),
+                                        (16384, 1000), (16384, 100), (16384, 16384), (9000, 5000), (8193, 129)])
 def test_topk_stage_alone_equals_a_plain_sort(chimera, tiny, n_prune, k):
-    """Stage 5 on crafted survivors (every kernel variant: k <= 16, k <= 128 over <= 4096 entries, the full network):
+    """Stage 5 on crafted survivors (every kernel variant: k <= 16, k <= 128 over <= 4096 entries, the full network up
+    to its 16,384 keys):
     many equal scores, -1 padding inside the valid count's tail, fewer survivors than k.  Expected = Definition 2
     written as a sort by (score descending, id ascending)."""
     cfg, oix, gix, q = tiny
@@ -244,7 +246,7 @@ def test_topk_stage_alone_equals_a_plain_sort(chimera, tiny, n_prune, k):
     n_pruned = np.array([n_prune, max(1, n_prune // 3), min(n_prune, 5)], dtype=np.int32)
     for b in range(B):
         m = int(n_pruned[b])
-        pruned[b, :m] = np.sort(rng.choice(oix.N, size=m, replace=False)).astype(np.int32)
+        pruned[b, :m] = np.sort(rng.choice(max(oix.N, 4 * n_prune), size=m, replace=False)).astype(np.int32)   # stage 5 never looks a document up
         # few distinct values (ties decided by id), both signs, and exact zeros
         score4[b, :m] = rng.choice(np.array([-3.5, -0.0, 0.0, 1.25, 1.25000012, 7.0, 19.75], dtype=np.float32), size=m)
     t = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, n_prune)

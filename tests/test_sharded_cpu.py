@@ -108,6 +108,55 @@ def test_sharded_protocol_reproduces_the_single_index_result(world, partial):
         assert all(out[r] for r in range(world)) and len(out) == world
 
 
+class _FlaggingEngine(OracleEngine):
+    """An engine whose device status is non-zero on one rank (as after a candidate overflow there)."""
+
+    def __init__(self, *a, flag=0):
+        super().__init__(*a)
+        self.flag = flag
+
+    def status_word(self):
+        return torch.tensor([self.flag], dtype=torch.int32)
+
+
+def _rank_flagged(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    import datetime
+    dist.init_process_group("gloo", rank=rank, world_size=world, timeout=datetime.timedelta(seconds=60))
+    import oracle
+    from paper_2608_23553_b200.sharded import ShardedSearcher, ShardError, shard_ranges
+    N, K, D, nbits = 90, 16, 32, 2
+    cent, cids, codes, doclens, q = _corpus(11, N, K, D, nbits)
+    lo, hi = shard_ranges(N, world)[rank]
+    off = np.concatenate([[0], np.cumsum(doclens, dtype=np.int64)])
+    oix = oracle.make_index(cent, cids[int(off[lo]):int(off[hi])], codes[int(off[lo]):int(off[hi])], doclens[lo:hi], nbits)
+    searcher = ShardedSearcher(_FlaggingEngine(oracle, oix, lo, False, flag=1 if rank == 1 else 0))
+    try:
+        searcher.search(torch.from_numpy(q), 2, 10, 5)
+        out[rank] = "no error"
+    except ShardError as e:
+        out[rank] = list(e.status)
+    # every rank is still in step: a further collective completes
+    dist.barrier()
+    quiet = ShardedSearcher(_FlaggingEngine(oracle, oix, lo, False, flag=1 if rank == 1 else 0), check=False)
+    quiet.search(torch.from_numpy(q), 2, 10, 5)
+    out["quiet%d" % rank] = quiet.last_status.tolist()
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_one_ranks_bad_status_raises_on_every_rank_after_the_collectives():
+    world = 3
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_rank_flagged, args=(world, 29951 + os.getpid() % 200, out), nprocs=world, join=True)
+        for r in range(world):
+            assert out[r] == [0, 1, 0]
+            assert out["quiet%d" % r] == [0, 1, 0]
+
+
 def test_shard_ranges_partition_the_documents():
     sys.path.insert(0, ROOT)
     from paper_2608_23553_b200.sharded import shard_ranges
