@@ -219,28 +219,75 @@ def run_reference(args, cfg, rank, world):
         "gpu_launches": 0}))
 
 
-def exhaustive_truth(index, q, cfg, k_max, chunk=16384):
-    """Ground truth for Recall@k: the stage-4 score (residual-decode MaxSim) of EVERY document for each query, through
-    the library's stage-isolated entry point in chunks of `chunk` documents, then the k_max best per query.  The
-    stage-4 kernel is itself parity-tested against the CPU oracle; here it only replaces candidate generation and
-    pruning by "all documents"."""
+def brute_force_maxsim(centroids, cids, codes, doclens, nbits, res_lo, res_hi, q, q_group=64, chunk_tokens=1 << 18):
+    """Exhaustive MaxSim (Definition 1) of EVERY document for every query, written out from the definition with
+    plain torch operations: the ground truth of the recall sweeps.  It shares nothing with the library (no call into
+    it, none of its kernels or layouts) and is itself compared with the CPU oracle's exhaustive scores in the GPU tests.
+
+    score(q, d) = sum_i max_{t in d} <q_i, c_cid(t) + r(code_t)>, computed per token as <q_i, c> + <q_i, r>:
+      * <q_i, c> for all centroids: one fp32 matmul (TF32 off);
+      * <q_i, r>: the decoded residual levels are exact in bfloat16 and q_i is split exactly into three bfloat16
+        terms (8 + 8 + 8 significant bits), so a bf16 matmul with fp32 accumulation over the three terms loses
+        nothing but fp32 summation rounding (~1e-7 relative);
+      * max over a document's tokens (segment maximum), then the sum over query tokens in fp32.
+    Returns scores [n_queries, n_docs] float32 on q's device."""
     dev = q.device
-    B, nq = q.shape[0], cfg.q_len
-    taps = index.alloc_taps(B, nq, cfg.nprobe, chunk, max_candidates=1024, table=True, ci=False)
-    index.run_stages(1, 1, q, B, nq, cfg.nprobe, chunk, 1, taps, max_candidates=1024)
-    scores = torch.empty(B, index.N, dtype=torch.float32, device=dev)
-    taps.n_pruned = torch.full((B,), chunk, dtype=torch.int32, device=dev)
-    for d0 in range(0, index.N, chunk):
-        ids = torch.arange(d0, d0 + chunk, device=dev, dtype=torch.int32)
-        ids[ids >= index.N] = -1
-        taps.pruned = ids[None, :].expand(B, chunk).contiguous()
-        index.run_stages(4, 4, q, B, nq, cfg.nprobe, chunk, 1, taps, max_candidates=1024)
-        n = min(chunk, index.N - d0)
-        scores[:, d0:d0 + n] = taps.score4[:, :n]
+    Bq, nq, D = q.shape
+    N = doclens.numel()
+    per, mask = 8 // nbits, (1 << nbits) - 1
+    delta = (res_hi - res_lo) / (1 << nbits)
+    levels = torch.tensor([res_lo + (u + 0.5) * delta for u in range(1 << nbits)], dtype=torch.float32, device=dev)
+    assert torch.equal(levels.bfloat16().float(), levels), "residual levels must be exact in bfloat16"
+    shifts = torch.arange(per, device=dev, dtype=torch.int32) * nbits
+    lens = doclens.to(torch.int64)
+    off = torch.cat([torch.zeros(1, dtype=torch.int64, device=dev), torch.cumsum(lens, 0)]).cpu().numpy()
+    # document chunks of at most chunk_tokens tokens (at least one document each)
+    bounds, d0 = [], 0
+    while d0 < N:
+        d1 = int(np.searchsorted(off, off[d0] + chunk_tokens, side="right")) - 1
+        d1 = min(max(d1, d0 + 1), N)
+        bounds.append((d0, d1))
+        d0 = d1
+    scores = torch.empty(Bq, N, dtype=torch.float32, device=dev)
+    tf32 = torch.backends.cuda.matmul.allow_tf32
+    red = torch.backends.cuda.matmul.allow_bf16_reduced_precision_reduction
+    torch.backends.cuda.matmul.allow_tf32 = False
+    torch.backends.cuda.matmul.allow_bf16_reduced_precision_reduction = False
+    try:
+        cent = centroids.to(torch.float32)
+        for g0 in range(0, Bq, q_group):
+            qg = q[g0:g0 + q_group].reshape(-1, D).to(torch.float32)            # [cols, D]
+            G = qg.shape[0] // nq
+            s_cent = cent @ qg.t()                                               # [K, cols]  <q_i, c>
+            hi = qg.bfloat16()
+            rem = qg - hi.float()
+            mid = rem.bfloat16()
+            low = (rem - mid.float()).bfloat16()
+            assert torch.equal(hi.float() + mid.float() + low.float(), qg)
+            qcat = torch.cat([hi, mid, low], dim=1).t().contiguous()              # [3 D, cols]
+            for a, b in bounds:
+                t0, t1 = int(off[a]), int(off[b])
+                u = ((codes[t0:t1].to(torch.int32)[:, :, None] >> shifts) & mask).reshape(t1 - t0, D)
+                r = levels[u.long()].bfloat16()
+                if dev.type == "cuda":
+                    val = torch.mm(r.repeat(1, 3), qcat, out_dtype=torch.float32)    # [tokens, cols]  <q_i, r>
+                else:                                  # CPU (tests of this function's logic): the same sum in fp32
+                    val = r.float().repeat(1, 3) @ qcat.float()
+                val += s_cent[cids[t0:t1].long()]
+                best = torch.segment_reduce(val, "max", lengths=lens[a:b], axis=0, unsafe=True)   # [docs, cols]
+                scores[g0:g0 + G, a:b] = best.view(b - a, G, nq).sum(dim=2).t()
+            del s_cent
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = tf32
+        torch.backends.cuda.matmul.allow_bf16_reduced_precision_reduction = red
+    return scores
+
+
+def exhaustive_truth(corp, cfg, q, k_max):
+    """Ground truth for Recall@k (Definition 3): the k_max best documents per query by exhaustive MaxSim over the
+    decoded corpus, from brute_force_maxsim (ties: smaller id)."""
+    scores = brute_force_maxsim(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi, q)
     top = torch.topk(scores, k_max, dim=1)
-    del scores, taps
-    index._ws = None
-    torch.cuda.empty_cache()
     return top.indices.to(torch.int32), top.values
 
 
@@ -252,12 +299,14 @@ def run_sweep(args, cfg, pkg, index, corp, q):
     nrec = min(args.sweep_queries, q.shape[0])
     qrec = q[:nrec].contiguous()
     t0 = time.time()
-    truth_ids, _ = exhaustive_truth(index, qrec, cfg, 1000)
+    truth_ids, _ = exhaustive_truth(corp, cfg, qrec, 1000)
+    torch.cuda.synchronize()
     truth_s = time.time() - t0
     n_batches = max(1, min(3, q.shape[0] // B))
     batches = q[:n_batches * B].view(n_batches, B, nq, cfg.dim).contiguous()
-    print(json.dumps({"sweep": cfg.name, "batch": B, "recall_queries": nrec, "ground_truth": "library stage 4 over "
-                      "every document (chunks of 16384), top-1000 per query", "ground_truth_s": round(truth_s, 1)}))
+    print(json.dumps({"sweep": cfg.name, "batch": B, "recall_queries": nrec, "ground_truth": "brute_force_maxsim "
+                      "(plain torch, independent of the library; checked against the CPU oracle in the GPU tests), "
+                      "top-1000 per query", "ground_truth_s": round(truth_s, 1)}))
     for P in (1, 2, 4, 8, 16, 32):
         if P > index.K:
             continue

@@ -93,6 +93,25 @@ def test_large_corpus_full_size_sampled_queries(large):
         assert check_query(tn, j, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) <= 4
 
 
+def test_sweep_ground_truth_scorer_on_a_10k_document_sample_matches_oracle(large):
+    """bench.brute_force_maxsim (the recall sweeps' ground truth, independent of the library) on 10,000 documents drawn
+    from the whole Large corpus against the oracle's exhaustive scores of the same documents, two queries."""
+    import bench
+    cfg, corp, gix, oix, q = large
+    dev = q.device
+    g = torch.Generator(device="cpu")
+    g.manual_seed(5)
+    docs = torch.sort(torch.randperm(cfg.n_docs, generator=g)[:10_000]).values
+    off = torch.from_numpy(oix.doc_off)
+    tok = torch.cat([torch.arange(int(off[d]), int(off[d + 1])) for d in docs.tolist()]).to(dev)
+    sc = bench.brute_force_maxsim(corp.centroids, corp.cids[tok], corp.codes[tok], corp.doclens[docs.to(dev)],
+                                  cfg.nbits, cfg.res_lo, cfg.res_hi, q[:2].contiguous()).cpu().numpy()
+    q_np = q[:2].cpu().numpy()
+    for b in range(2):
+        ref = oracle.score_docs(q_np[b], docs.numpy().astype(np.int32), oix)
+        assert np.abs(sc[b] - ref).max() <= 1e-5 * max(1.0, float(np.abs(ref).max()))
+
+
 def test_large_sweep_extreme_point_nprobe32_nprune16384_k1000(large):
     """The recall sweep's largest point in its launch shape: 256 queries per call, nprobe 32 (about two million
     candidates per query, capacity as the benchmark sizes it), n_prune 16384 (a real selection at the API's maximum),

@@ -110,3 +110,19 @@ def test_mid_batch256_four_document_shards_equal_the_single_index(mid):
     ids, sc = engines[0].merge_phase(torch.stack([t[0] for t in tops]).contiguous(),
                                      torch.stack([t[1] for t in tops]).contiguous())
     assert torch.equal(ids, ref_ids) and torch.equal(sc, ref_sc)
+
+
+def test_sweep_ground_truth_scorer_on_a_20k_document_slice_matches_oracle(mid):
+    """bench.brute_force_maxsim (the recall sweeps' ground truth, independent of the library) on the first 20,000
+    documents of the Mid corpus against the oracle's exhaustive scores, two queries."""
+    import bench
+    cfg, corp, gix, oix, q = mid
+    n = 20_000
+    T = int(corp.doclens[:n].to(torch.int64).sum())
+    sc = bench.brute_force_maxsim(corp.centroids, corp.cids[:T], corp.codes[:T], corp.doclens[:n], cfg.nbits,
+                                  cfg.res_lo, cfg.res_hi, q[:3].contiguous()).cpu().numpy()
+    q_np = q[:3].cpu().numpy()
+    docs = np.arange(n, dtype=np.int32)
+    for b in (0, 2):
+        ref = oracle.score_docs(q_np[b], docs, oix)
+        assert np.abs(sc[b] - ref).max() <= 1e-5 * max(1.0, float(np.abs(ref).max()))
