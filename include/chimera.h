@@ -44,7 +44,7 @@ typedef enum {
     CHIMERA_CUDA_ERROR = 2,         /* a CUDA runtime call failed; text in chimera_last_error() */
     CHIMERA_WORKSPACE_TOO_SMALL = 3,
     CHIMERA_CAPACITY_OVERFLOW = 4,  /* a query produced more candidates than max_candidates (reported by status) */
-    CHIMERA_TIMEOUT = 5,            /* a bounded device-side wait gave up (reported by status) */
+    CHIMERA_TIMEOUT = 5,            /* a bounded device-side wait gave up after ~50 ms (reported by status) */
     CHIMERA_UNSUPPORTED = 6         /* dim, nbits or a size outside the supported set */
 } chimera_status;
 
@@ -213,6 +213,16 @@ int chimera_search_rabitq(const chimera_index *index, const float *queries, int3
  * first max_candidates of them and are not the specified output), CHIMERA_INVALID_ARG (a query element outside
  * [-1, 1]) or CHIMERA_TIMEOUT to *status (host pointer). */
 int chimera_workspace_status(const void *workspace, void *stream, int32_t *status);
+
+/* Test hook for the give-up path of the bounded device-side waits (the paper has no counterpart).  The two tensor-core
+ * kernels (stage 1, stage 4) wait on mbarriers for their TMA loads and MMAs; each wait gives up after a limit (default
+ * 100,000,000 SM cycles, about 50 ms), sets the TIMEOUT status bit, and the block frees its tensor memory and returns.
+ * skip_loads != 0 makes every later search of this process issue NO TMA load in those kernels, so their waits run
+ * into the limit with nothing in flight; wait_cycles > 0 sets the limit (<= 0 restores the default).  The searches
+ * still return CHIMERA_OK (they only enqueue); chimera_workspace_status then reports CHIMERA_TIMEOUT and the results
+ * are undefined.  Call it again with (0, 0) to restore normal operation; the device context stays usable.
+ * Process-wide; not for production use. */
+int chimera_test_wait_fault(int32_t skip_loads, int64_t wait_cycles);
 
 /* Sizes held by an index (host pointers, each optional). */
 int chimera_index_info(const chimera_index *index, chimera_index_desc *desc, int64_t *posting_entries,

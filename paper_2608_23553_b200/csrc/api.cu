@@ -22,6 +22,12 @@ int fail(int code, const char *fmt, ...)
     return code;
 }
 
+// ------------------------------------------------------------------------------------------------ wait limit -----
+static std::atomic<long long> g_wait_cycles{100000000LL};      // = UMMA_WAIT_CYCLES (umma.cuh)
+static std::atomic<int> g_skip_tma{0};
+long long wait_limit_cycles() { return g_wait_cycles.load(std::memory_order_relaxed); }
+int fault_skip_tma_loads() { return g_skip_tma.load(std::memory_order_relaxed); }
+
 // ------------------------------------------------------------------------------------------------ profiling ------
 constexpr int PROF_MARKS = 16;
 struct ProfCall {
@@ -634,6 +640,13 @@ int chimera_workspace_status(const void *workspace, void *stream, int32_t *statu
     else if (bits & ST_BAD_QUERY) *status = CHIMERA_INVALID_ARG;
     else if (bits & ST_OVERFLOW) *status = CHIMERA_CAPACITY_OVERFLOW;
     else *status = CHIMERA_OK;
+    return CHIMERA_OK;
+}
+
+int chimera_test_wait_fault(int32_t skip_loads, int64_t wait_cycles)
+{
+    g_skip_tma.store(skip_loads ? 1 : 0, std::memory_order_relaxed);
+    g_wait_cycles.store(wait_cycles > 0 ? (long long)wait_cycles : 100000000LL, std::memory_order_relaxed);
     return CHIMERA_OK;
 }
 

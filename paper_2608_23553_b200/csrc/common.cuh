@@ -106,6 +106,10 @@ int fail(int code, const char *fmt, ...);
 // ---------------------------------------------------------------------------------------------------------------
 // Profiling hooks (api.cu).
 // ---------------------------------------------------------------------------------------------------------------
+// Limit of the bounded device-side waits and the test hook that makes them run out (api.cu; chimera_test_wait_fault).
+long long wait_limit_cycles();
+int fault_skip_tma_loads();
+
 enum Slot { SLOT_G1 = 0, SLOT_PROBE, SLOT_GATHER, SLOT_CI, SLOT_SELECT, SLOT_G4, SLOT_TOPK, SLOT_MISC, SLOT_CI_EXACT };
 void count_launch(int slot, int n = 1);
 

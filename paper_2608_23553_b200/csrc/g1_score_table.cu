@@ -48,7 +48,7 @@ __device__ __forceinline__ int32_t combine_digits(int32_t a0, int32_t a1, int32_
 __global__ void __launch_bounds__(G1_THREADS)
 score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_q, int64_t K,
                  int nq, int64_t q_rows, int k_steps, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
-                 uint8_t *__restrict__ table8, uint32_t *status)
+                 uint8_t *__restrict__ table8, uint32_t *status, long long wait_limit, int skip_loads)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t s_tmem_base;
@@ -88,7 +88,9 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
     constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(G1_N >> 3) << 17) |
                                ((uint32_t)(G1_M >> 4) << 24);
 
-    if (tid == 0 && t_begin < t_end) {
+    // skip_loads (test hook): no load is issued and no bytes are expected, so the waits below run into their limit
+    // with nothing in flight
+    if (tid == 0 && t_begin < t_end && !skip_loads) {
         mbar_expect_tx(bar_a, 3 * G1_A_PLANE);
         for (int p = 0; p < 3; ++p) tma_load_3d(sA + p * G1_A_PLANE, &map_c, 0, (int)c0, p, bar_a);
         mbar_expect_tx(bar_b0, 3 * G1_B_PLANE);
@@ -99,14 +101,14 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
         const int it = t - t_begin, stage = it & 1;
         if (tid == 0) {
             bool ok = true;
-            if (t + 1 < t_end) {           // the other stage was released by the previous tile's completed MMAs
+            if (t + 1 < t_end && !skip_loads) {   // the other stage was released by the previous tile's completed MMAs
                 const uint32_t nb = bar_b0 + 8 * (stage ^ 1);
                 mbar_expect_tx(nb, 3 * G1_B_PLANE);
                 for (int p = 0; p < 3; ++p)
                     tma_load_3d(sB + ((stage ^ 1) * 3 + p) * G1_B_PLANE, &map_q, 0, (t + 1) * G1_N, p, nb);
             }
-            if (it == 0) ok = mbar_wait(bar_a, 0);
-            if (ok) ok = mbar_wait(bar_b0 + 8 * stage, (it >> 1) & 1);
+            if (it == 0) ok = mbar_wait(bar_a, 0, wait_limit);
+            if (ok) ok = mbar_wait(bar_b0 + 8 * stage, (it >> 1) & 1, wait_limit);
             if (ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 for (int w = 0; w < 5; ++w) {              // accumulator = digit weight a + b
@@ -130,7 +132,7 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
         }
         __syncwarp();
         // everybody waits for the accumulators (bounded), then drains them
-        const bool ok = mbar_wait(bar_mma, it & 1);
+        const bool ok = mbar_wait(bar_mma, it & 1, wait_limit);
         if (!__syncthreads_and(ok && !*(volatile int *)&s_abort)) {      // uniform decision for the whole CTA
             if (tid == 0) atomicOr(status, ST_TIMEOUT);
             break;
@@ -287,7 +289,8 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
     dim3 grid((unsigned)c_tiles, (unsigned)((n_tiles + tiles_per_split - 1) / tiles_per_split));
     score_table_umma<<<grid, G1_THREADS, G1_SMEM, st>>>(map_c, map_q, ix.K, p.nq, rows, ix.D / 32, n_tiles,
-                                                        tiles_per_split, table, table8, status);
+                                                        tiles_per_split, table, table8, status, wait_limit_cycles(),
+                                                        fault_skip_tma_loads());
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_G1, 2);
     return CHIMERA_OK;

@@ -57,7 +57,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                      const int32_t *__restrict__ pruned, int n_prune, int docs_per_cta,
                      const int32_t *__restrict__ cids, const uint32_t *__restrict__ codes,
                      const float *__restrict__ factors, const int64_t *__restrict__ doc_off,
-                     float *__restrict__ score4, uint32_t *status)
+                     float *__restrict__ score4, uint32_t *status, long long wait_limit, int skip_loads)
 {
     constexpr int N = 3 * NQP;                               // MMA N: three digit planes side by side
     constexpr uint32_t TMEM_COLS = N <= 128 ? 128 : 256;
@@ -160,7 +160,8 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     const int total = s_off[nd];
     const int n_tiles = (total + G4U_TOK - 1) / G4U_TOK;
 
-    if (tid == 0) {          // the query's three digit planes, side by side: rows [p * NQP, (p + 1) * NQP)
+    // skip_loads (test hook): no load is issued, so the first wait below runs into its limit with nothing in flight
+    if (tid == 0 && !skip_loads) {   // the query's three digit planes, side by side: rows [p * NQP, (p + 1) * NQP)
         mbar_expect_tx(bar_b, B_BYTES);
         for (int p = 0; p < 3; ++p) tma_load_3d(sB + p * NQP * 128, &map_q, 0, b * nq, p, bar_b);
     }
@@ -258,7 +259,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         // ---- one thread issues the MMAs --------------------------------------------------------------------------
         if (tid == 0) {
             bool ok = true;
-            if (tile == 0) ok = mbar_wait(bar_b, 0);
+            if (tile == 0) ok = mbar_wait(bar_b, 0, wait_limit);
             if (ok) {
                 tc_fence_after();
                 const uint64_t da = umma_desc(sA), db = umma_desc(sB);
@@ -307,7 +308,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             }
         }
 
-        const bool ok = mbar_wait(bar_mma, tile & 1);
+        const bool ok = mbar_wait(bar_mma, tile & 1, wait_limit);
         if (!__syncthreads_and(ok && !*(volatile int *)&s_abort)) {
             if (tid == 0) atomicOr(status, ST_TIMEOUT);
             alive = false;
@@ -381,10 +382,13 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                 atomicMax(&docmax[doc * NQP + lane], f_order(m0));
                 if (NQP > 32) atomicMax(&docmax[doc * NQP + 32 + lane], f_order(m1));
             }
+            // the value rows of this warp (on the A tile when ON_A) are rewritten by the next tile's expansion, each
+            // lane its own row, while the fold above reads the rows of other lanes: all lanes finish reading first
+            __syncwarp();
         }
     }
 
-    if (n_tiles == 0 && tid == 0) mbar_wait(bar_b, 0);       // never leave with the TMA load in flight
+    if (n_tiles == 0 && tid == 0 && !skip_loads) mbar_wait(bar_b, 0, wait_limit);   // never leave with the TMA load in flight
     tc_fence_before();
     __syncthreads();
 
@@ -437,7 +441,7 @@ static int launch_g4_umma(const Index &ix, const Params &p, const float *queries
     const uint32_t *code_words = reinterpret_cast<const uint32_t *>(RQ ? ix.rq_bits : ix.codes);
     kern<<<grid, G4U_THREADS, smem, st>>>(map_q, queries, table, ix.K, p.nq, ix.D, RQ ? ix.D / 32 : ix.CB / 4, delta,
                                           kappa, pruned, p.n_prune, (int)dpc, ix.cids, code_words, ix.rq_inv, ix.doc_off,
-                                          score4, status);
+                                          score4, status, wait_limit_cycles(), fault_skip_tma_loads());
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_G4);
     return CHIMERA_OK;

@@ -8,7 +8,10 @@
 
 namespace chimera {
 
-constexpr long long UMMA_WAIT_CYCLES = 2000000000LL;       // ~1 s at 2 GHz: every mbarrier wait gives up after this
+// Every mbarrier wait gives up after this many SM clock cycles (~50 ms at 2 GHz; the operations waited for -- a TMA
+// tile load, a handful of MMAs -- take microseconds, so only a lost completion can make a wait this long).  The
+// kernels take the limit as an argument (wait_limit_cycles() on the host), so that a test can shorten it.
+constexpr long long UMMA_WAIT_CYCLES = 100000000LL;
 constexpr uint32_t UMMA_SUSPEND_HINT_NS = 20000u;          // one try_wait may sleep this long before re-checking
 
 // ------------------------------------------------------------------------------------------------ PTX wrappers ---
@@ -25,7 +28,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 // Bounded wait for the phase with the given parity to complete.  false = gave up.  Each try_wait may suspend the
 // thread in hardware for up to the hinted time (it returns early when the phase completes), so a waiting warp does not
 // burn issue slots; the loop around it enforces the overall limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit)
 {
     const long long t0 = clock64();
     for (;;) {
@@ -38,7 +41,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
             : "r"(bar), "r"(parity), "r"(UMMA_SUSPEND_HINT_NS)
             : "memory");
         if (done) return true;
-        if (clock64() - t0 > UMMA_WAIT_CYCLES) return false;
+        if (clock64() - t0 > limit) return false;
     }
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
