@@ -729,6 +729,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="", help="one workload only (tiny, mid, large, long_d128_b2, ...); default: the "
                     "Large headline plus a short measurement of every other workload")
+    ap.add_argument("--docs", type=int, default=0, help="keep only this many documents of the workload (same recipe; "
+                    "for profiler captures, which need a small case)")
     ap.add_argument("--batch", type=int, default=0, help="queries per call (default 256; 64 for the long-document configs, 16 for Tiny)")
     ap.add_argument("--partial", action="store_true",
                     help="prune with the paper's partial scores (chimera_search_partial) instead of stage 3")
@@ -758,6 +760,8 @@ def main():
 
     single = bool(args.config) or args.partial or args.rabitq or args.sweep or args.sharded
     cfg = CONFIGS[args.config or HEADLINE]
+    if args.docs > 0:
+        cfg = cfg.replace(n_docs=args.docs)
     if args.impl == "reference":
         if args.batch <= 0:
             args.batch = 64 if cfg.name.startswith("long") else 256

@@ -236,8 +236,8 @@ ci_wide_rng_kernel(const int32_t *__restrict__ table, int64_t K, const int2 *__r
 // spent on [0, 1) and a column whose best score is negative only loosens lo.)  A row of U8 is q_len bytes -- one
 // 32-byte sector for 32 query
 // tokens instead of four -- and a lane's 16-byte load covers 16 query tokens, so one warp load covers 32 / LPR tokens
-// (LPR = q_len / 16 lanes per row).  Bytes are widened to pairs of 16-bit integers with one byte-permute per pair and
-// the running maxima fold two rows per instruction with the three-input packed 16-bit integer maximum.
+// (LPR = q_len / 16 lanes per row).  The running maxima fold two rows per instruction with the three-input packed
+// 16-bit integer maximum (see coarse_accumulate2).
 // packed = sum | sat << 16 | zeros << 24 (see above)
 __device__ __forceinline__ int32_t coarse_lo(int packed)
 {
@@ -250,16 +250,23 @@ __device__ __forceinline__ int32_t coarse_hi(int packed, int nq)
 // The histogram key of a lower bound in the contender step: floor(lo / 2^16) clamped at 0 -- a valid, slightly smaller
 // lower bound (documents with an empty column fall to the bottom, which only lowers the threshold).
 __device__ __forceinline__ int coarse_key(int32_t lo) { return lo < 0 ? 0 : lo >> 16; }
+// Running maxima of a lane's 16 columns in eight registers of two 16-bit fields each, updated from two rows at a time
+// with the three-input packed 16-bit maximum.  A field compares as (column byte << 8 | whatever lies below it), so the
+// winner's HIGH byte is the column's maximum and no widening is needed: the odd bytes of a word already sit in the high
+// byte of a field (registers 4..7 take the raw words), the even bytes get there with one shift (registers 0..3).
+// coarse_field() extracts a field's maximum at the end.
 __device__ __forceinline__ void coarse_accumulate2(uint32_t (&m)[8], const int4 &va, const int4 &vb)
 {
     const uint32_t a[4] = {(uint32_t)va.x, (uint32_t)va.y, (uint32_t)va.z, (uint32_t)va.w};
     const uint32_t b[4] = {(uint32_t)vb.x, (uint32_t)vb.y, (uint32_t)vb.z, (uint32_t)vb.w};
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        m[2 * k] = __vimax3_u16x2(m[2 * k], __byte_perm(a[k], 0u, 0x4140), __byte_perm(b[k], 0u, 0x4140));
-        m[2 * k + 1] = __vimax3_u16x2(m[2 * k + 1], __byte_perm(a[k], 0u, 0x4342), __byte_perm(b[k], 0u, 0x4342));
+        m[k] = __vimax3_u16x2(m[k], a[k] << 8, b[k] << 8);
+        m[4 + k] = __vimax3_u16x2(m[4 + k], a[k], b[k]);
     }
 }
+__device__ __forceinline__ int coarse_field_lo(uint32_t m) { return (int)((m >> 8) & 0xffu); }
+__device__ __forceinline__ int coarse_field_hi(uint32_t m) { return (int)(m >> 24); }
 // SMEM = true: the query's whole 8-bit table (K * q_len bytes) is first staged in shared memory and the row lookups
 // are shared-memory loads (small K only); blocks are then larger (THREADS) because only one fits an SM.
 template <int LPR, bool SMEM, int THREADS>
@@ -367,7 +374,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
             }
         }
         // every lane now holds the maxima of two columns; sum over columns (skipping duplicate lanes)
-        const int u_lo = (int)(m[0] & 0xffffu), u_hi = (int)(m[0] >> 16);
+        const int u_lo = coarse_field_lo(m[0]), u_hi = coarse_field_hi(m[0]);
         int packed = 0;                                         // sum of maxima | saturated << 16 | zeros << 24
         if ((lane & dup_mask) == 0)
             packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 16) + (((u_lo == 0) + (u_hi == 0)) << 24);
@@ -511,7 +518,7 @@ ci_coarse_rng_body(const uint8_t *__restrict__ table8, int64_t K, const int2 *__
                     dup_mask |= (uint32_t)o;
                 }
             }
-            const int u_lo = (int)(m[0] & 0xffffu), u_hi = (int)(m[0] >> 16);
+            const int u_lo = coarse_field_lo(m[0]), u_hi = coarse_field_hi(m[0]);
             int packed = 0;                                         // sum of maxima | saturated << 16 | zeros << 24
             if ((lane & dup_mask) == 0)
                 packed = (u_lo + u_hi) + (((u_lo >= 255) + (u_hi >= 255)) << 16) + (((u_lo == 0) + (u_hi == 0)) << 24);
