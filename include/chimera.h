@@ -45,7 +45,9 @@ typedef enum {
     CHIMERA_WORKSPACE_TOO_SMALL = 3,
     CHIMERA_CAPACITY_OVERFLOW = 4,  /* a query produced more candidates than max_candidates (reported by status) */
     CHIMERA_TIMEOUT = 5,            /* a bounded device-side wait gave up after ~50 ms (reported by status) */
-    CHIMERA_UNSUPPORTED = 6         /* dim, nbits or a size outside the supported set */
+    CHIMERA_UNSUPPORTED = 6,        /* dim, nbits or a size outside the supported set */
+    CHIMERA_DEBUG_CHECK_FAILED = 7  /* debug build only: a kernel met an index out of range and skipped it (reported
+                                       by status) */
 } chimera_status;
 
 #define CHIMERA_MAX_NPROBE 64       /* nprobe per query token */
@@ -211,8 +213,22 @@ int chimera_search_rabitq(const chimera_index *index, const float *queries, int3
 /* Device-side status of the last search that used this workspace: synchronises the stream, then writes CHIMERA_OK,
  * CHIMERA_CAPACITY_OVERFLOW (some query had more than max_candidates candidates; its results are computed on the
  * first max_candidates of them and are not the specified output), CHIMERA_INVALID_ARG (a query element outside
- * [-1, 1]) or CHIMERA_TIMEOUT to *status (host pointer). */
+ * [-1, 1]), CHIMERA_TIMEOUT or (debug build) CHIMERA_DEBUG_CHECK_FAILED to *status (host pointer). */
 int chimera_workspace_status(const void *workspace, void *stream, int32_t *status);
+
+/* Debug build (the paper has no counterpart).  libchimera_debug.so is the same source compiled with -DCHIMERA_DEBUG:
+ * every kernel checks each centroid id, document id, token position and candidate rank before it gathers through it
+ * (an index out of range is not dereferenced; chimera_workspace_status then reports CHIMERA_DEBUG_CHECK_FAILED), and
+ * every workspace region is followed by a 256-byte guard pattern, so chimera_workspace_bytes is larger.  It stands in
+ * for a memory checker where none can be run; it is several times slower and serves one search at a time per process.
+ * chimera_is_debug_build: 1 in that library, 0 otherwise.
+ * chimera_workspace_check: after a search with the same parameters on `workspace`, verifies the guard patterns
+ * (synchronises the stream) and writes the index of the first damaged region to *damaged_region (host pointer), -1 if
+ * all are intact.  Returns CHIMERA_UNSUPPORTED in a release build. */
+int chimera_is_debug_build(void);
+int chimera_workspace_check(const chimera_index *index, int32_t n_queries, int32_t q_len, int32_t nprobe,
+                            int32_t n_prune, int32_t k, int64_t max_candidates, const void *workspace, void *stream,
+                            int32_t *damaged_region);
 
 /* Test hook for the give-up path of the bounded device-side waits (the paper has no counterpart).  The two tensor-core
  * kernels (stage 1, stage 4) wait on mbarriers for their TMA loads and MMAs; each wait gives up after a limit (default

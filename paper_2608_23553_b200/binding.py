@@ -14,14 +14,16 @@ from typing import Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_PKG, "libchimera.so")
+# CHIMERA_DEBUG_LIB=1 loads the debug build (index checks before every gather, guard regions in the workspace)
+_DEBUG = os.environ.get("CHIMERA_DEBUG_LIB", "0") == "1"
+_LIB_PATH = os.path.join(_PKG, "libchimera_debug.so" if _DEBUG else "libchimera.so")
 _lib = None
 
 PROFILE_SLOTS = ("score_table", "probes", "gather", "centroid_interaction", "select", "residual_scores", "topk",
                  "misc", "ci_exact")
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "CUDA_ERROR", 3: "WORKSPACE_TOO_SMALL", 4: "CAPACITY_OVERFLOW",
-                5: "TIMEOUT", 6: "UNSUPPORTED"}
+                5: "TIMEOUT", 6: "UNSUPPORTED", 7: "DEBUG_CHECK_FAILED"}
 
 
 class ChimeraError(RuntimeError):
@@ -50,8 +52,8 @@ def lib():
     global _lib
     if _lib is None:
         if not os.path.exists(_LIB_PATH):
-            raise ImportError("libchimera.so is not built: run `python -m paper_2608_23553_b200.build` "
-                              "(there is no CPU fallback)")
+            raise ImportError("%s is not built: run `python -m paper_2608_23553_b200.build%s` "
+                              "(there is no CPU fallback)" % (os.path.basename(_LIB_PATH), " --debug" if _DEBUG else ""))
         L = ctypes.CDLL(_LIB_PATH)
         L.chimera_last_error.restype = ctypes.c_char_p
         _lib = L
@@ -255,6 +257,16 @@ class Index:
                                         _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(), ctypes.byref(c),
                                         _ptr(ids), _ptr(scores)))
         return ids, scores
+
+    def workspace_check(self, n_queries, q_len, nprobe, n_prune, k, max_candidates=0) -> int:
+        """Debug build only: index of the first damaged guard region of the workspace after a search with these
+        parameters, -1 if all are intact (chimera_workspace_check)."""
+        bad = ctypes.c_int32()
+        _check(lib().chimera_workspace_check(self._h, ctypes.c_int32(n_queries), ctypes.c_int32(q_len),
+                                             ctypes.c_int32(nprobe), ctypes.c_int32(n_prune), ctypes.c_int32(k),
+                                             ctypes.c_int64(max_candidates), _ptr(self._ws), _stream(),
+                                             ctypes.byref(bad)))
+        return bad.value
 
     def status(self) -> int:
         """Device-side status of the last search (synchronises the current stream)."""

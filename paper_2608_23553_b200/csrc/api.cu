@@ -91,7 +91,18 @@ Layout make_layout(const Index &ix, const Params &p)
     L.n_chunks = (int32_t)((L.words + BITMAP_CHUNK_WORDS - 1) / BITMAP_CHUNK_WORDS);
 
     size_t o = 0;
+#ifdef CHIMERA_DEBUG
+    // a 256-byte guard region behind every region: a kernel that writes past its array damages the pattern there
+    auto take = [&](size_t bytes) {
+        size_t at = o;
+        o = align_up(o + bytes);
+        if (L.n_guards < MAX_GUARDS) L.guards[L.n_guards++] = o;
+        o += 256;
+        return at;
+    };
+#else
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+#endif
     const size_t B = (size_t)p.B, nq = (size_t)p.nq;
     L.status = take(64 * sizeof(uint32_t));
     L.q_stage = take(B * nq * ix.D * sizeof(float));
@@ -135,6 +146,41 @@ Layout make_layout(const Index &ix, const Params &p)
     L.total = o;
     return L;
 }
+
+// ------------------------------------------------------------------------------------------------ debug build ----
+#ifdef CHIMERA_DEBUG
+__device__ DbgLimits chimera_dbg;
+
+struct GuardList { size_t off[MAX_GUARDS]; int n; };
+constexpr uint32_t GUARD_PATTERN = 0xC0FFEE00u;
+// grid (n guards), 64 threads: guard g holds 64 words GUARD_PATTERN | g.
+__global__ void guard_fill_kernel(char *ws, GuardList g)
+{
+    reinterpret_cast<uint32_t *>(ws + g.off[blockIdx.x])[threadIdx.x] = GUARD_PATTERN | blockIdx.x;
+}
+// the lowest damaged guard goes to status[STATUS_WORD_CANARY] (preset to 0xffffffff)
+__global__ void guard_check_kernel(const char *ws, GuardList g, uint32_t *status)
+{
+    if (reinterpret_cast<const uint32_t *>(ws + g.off[blockIdx.x])[threadIdx.x] != (GUARD_PATTERN | blockIdx.x))
+        atomicMin(&status[STATUS_WORD_CANARY], (uint32_t)blockIdx.x);
+}
+
+int debug_begin_search(const Index &ix, const Params &p, const Layout &L, void *workspace, cudaStream_t st)
+{
+    DbgLimits lim;
+    lim.status = reinterpret_cast<uint32_t *>((char *)workspace + L.status);
+    lim.K = ix.K; lim.N = ix.N; lim.T = ix.T; lim.maxc = p.maxc;
+    CHIMERA_CUDA(cudaMemcpyToSymbolAsync(chimera_dbg, &lim, sizeof(lim), 0, cudaMemcpyHostToDevice, st));
+    GuardList g;
+    g.n = L.n_guards;
+    for (int i = 0; i < L.n_guards; ++i) g.off[i] = L.guards[i];
+    if (g.n > 0) guard_fill_kernel<<<g.n, 64, 0, st>>>((char *)workspace, g);
+    CHIMERA_CUDA(cudaGetLastError());
+    return CHIMERA_OK;
+}
+#else
+int debug_begin_search(const Index &, const Params &, const Layout &, void *, cudaStream_t) { return CHIMERA_OK; }
+#endif
 
 static int check_params(const Index *ix, int32_t B, int32_t nq, int32_t P, int32_t n_prune, int32_t k,
                         int64_t max_candidates, Params *out)
@@ -215,6 +261,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     prof_begin(st);
     // a resumed call continues an earlier one: the status bits that one set stay, new ones are OR-ed in
     if (!resume) CHIMERA_CUDA(cudaMemsetAsync(status, 0, 64 * sizeof(uint32_t), st));
+    if (!resume && (rc = debug_begin_search(ix, p, L, workspace, st))) return rc;      // debug builds only
 
     // results of the stages that do not run come from the caller
     if (first > 1 && !resume) {
@@ -636,11 +683,52 @@ int chimera_workspace_status(const void *workspace, void *stream, int32_t *statu
     uint32_t bits = 0;
     CHIMERA_CUDA(cudaMemcpyAsync(&bits, workspace, sizeof(bits), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     CHIMERA_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
-    if (bits & ST_TIMEOUT) *status = CHIMERA_TIMEOUT;
+    if (bits & ST_BAD_INDEX) *status = CHIMERA_DEBUG_CHECK_FAILED;
+    else if (bits & ST_TIMEOUT) *status = CHIMERA_TIMEOUT;
     else if (bits & ST_BAD_QUERY) *status = CHIMERA_INVALID_ARG;
     else if (bits & ST_OVERFLOW) *status = CHIMERA_CAPACITY_OVERFLOW;
     else *status = CHIMERA_OK;
     return CHIMERA_OK;
+}
+
+int chimera_is_debug_build(void)
+{
+#ifdef CHIMERA_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int chimera_workspace_check(const chimera_index *index, int32_t n_queries, int32_t q_len, int32_t nprobe,
+                            int32_t n_prune, int32_t k, int64_t max_candidates, const void *workspace, void *stream,
+                            int32_t *damaged_region)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, n_prune, k, max_candidates, &p);
+    if (rc) return rc;
+    if (!workspace || !damaged_region) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+#ifdef CHIMERA_DEBUG
+    const Layout L = make_layout(*ix, p);
+    cudaStream_t st = (cudaStream_t)stream;
+    uint32_t *status = reinterpret_cast<uint32_t *>((char *)workspace + L.status);
+    GuardList g;
+    g.n = L.n_guards;
+    for (int i = 0; i < L.n_guards; ++i) g.off[i] = L.guards[i];
+    CHIMERA_CUDA(cudaMemsetAsync(status + STATUS_WORD_CANARY, 0xff, sizeof(uint32_t), st));
+    if (g.n > 0) guard_check_kernel<<<g.n, 64, 0, st>>>((const char *)workspace, g, status);
+    CHIMERA_CUDA(cudaGetLastError());
+    uint32_t first = 0xffffffffu;
+    CHIMERA_CUDA(cudaMemcpyAsync(&first, status + STATUS_WORD_CANARY, sizeof(first), cudaMemcpyDeviceToHost, st));
+    CHIMERA_CUDA(cudaStreamSynchronize(st));
+    *damaged_region = first == 0xffffffffu ? -1 : (int32_t)first;
+    return CHIMERA_OK;
+#else
+    (void)stream;
+    *damaged_region = -1;
+    return fail(CHIMERA_UNSUPPORTED, "this library was built without CHIMERA_DEBUG: the workspace has no guard regions");
+#endif
 }
 
 int chimera_test_wait_fault(int32_t skip_loads, int64_t wait_cycles)

@@ -37,7 +37,8 @@ struct Index {
 };
 
 // Device status bits kept in the first word of a workspace.
-enum : uint32_t { ST_OVERFLOW = 1u, ST_BAD_QUERY = 2u, ST_TIMEOUT = 4u };
+enum : uint32_t { ST_OVERFLOW = 1u, ST_BAD_QUERY = 2u, ST_TIMEOUT = 4u, ST_BAD_INDEX = 8u };
+constexpr int STATUS_WORD_CANARY = 8;   // status[8]: first damaged guard region found by the debug build's check
 
 // ---------------------------------------------------------------------------------------------------------------
 // Workspace layout (all offsets 256-byte aligned).
@@ -47,7 +48,11 @@ struct Params {
     int64_t maxc;                     // candidate capacity per query
 };
 
+constexpr int MAX_GUARDS = 48;
 struct Layout {
+    // debug builds (CHIMERA_DEBUG) put a 256-byte guard region behind every region below; guards[i] is its offset
+    size_t guards[MAX_GUARDS];
+    int n_guards;
     size_t status;        // uint32[64]
     size_t q_stage;       // float  [B, nq, D]        (host-entry staging of the queries)
     size_t out_ids;       // int32  [B, k]            (host-entry staging)
@@ -185,6 +190,38 @@ int launch_rabitq_partial(const Index &ix, const Params &p, const Layout &L, con
                           const int32_t *n_cand, int32_t *partial_m, int32_t *fprime_bits, cudaStream_t st);
 int launch_topk(const Index &ix, const Params &p, const int32_t *pruned, const float *score4, int32_t *out_ids,
                 float *out_scores, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------------------
+// Debug build (-DCHIMERA_DEBUG, libchimera_debug.so): every index that a kernel is about to gather through (centroid
+// id, document id, token position, candidate rank) is checked first.  An index out of range sets ST_BAD_INDEX in the
+// status word of the running search and is replaced by 0 (DBG_*) or its access is skipped (DBG_*_OK), so the kernel
+// never touches memory outside its arrays.  The limits and the status pointer of the running search live in one
+// device variable, so a debug build serves one search at a time.  In release builds the macros vanish.
+// ---------------------------------------------------------------------------------------------------------------
+#ifdef CHIMERA_DEBUG
+struct DbgLimits { uint32_t *status; long long K, N, T, maxc; };
+extern __device__ DbgLimits chimera_dbg;
+__device__ __forceinline__ bool dbg_in_range(long long x, long long n)
+{
+    if (x >= 0 && x < n) return true;
+    if (chimera_dbg.status) atomicOr(chimera_dbg.status, ST_BAD_INDEX);
+    return false;
+}
+template <class I> __device__ __forceinline__ I dbg_index(I x, long long n) { return dbg_in_range((long long)x, n) ? x : (I)0; }
+#define DBG_CID(c) ::chimera::dbg_index((c), ::chimera::chimera_dbg.K)
+#define DBG_DOC(d) ::chimera::dbg_index((d), ::chimera::chimera_dbg.N)
+#define DBG_TOK(t) ::chimera::dbg_index((t), ::chimera::chimera_dbg.T)
+#define DBG_DOC_OK(d) ::chimera::dbg_in_range((long long)(d), ::chimera::chimera_dbg.N)
+#define DBG_RANK_OK(r) ::chimera::dbg_in_range((long long)(r), ::chimera::chimera_dbg.maxc)
+#else
+#define DBG_CID(c) (c)
+#define DBG_DOC(d) (d)
+#define DBG_TOK(t) (t)
+#define DBG_DOC_OK(d) true
+#define DBG_RANK_OK(r) true
+#endif
+// Host side (api.cu): publish the running search's limits / fill and check the guard regions (no-ops in release builds).
+int debug_begin_search(const Index &ix, const Params &p, const Layout &L, void *workspace, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------------------------
 // Device helpers.

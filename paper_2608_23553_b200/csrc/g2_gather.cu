@@ -14,7 +14,7 @@ mark_kernel(const int32_t *__restrict__ probes, int n_lists, const int64_t *__re
             const int32_t *__restrict__ ivf_doc, uint32_t *__restrict__ bitmap, int64_t words)
 {
     const int b = blockIdx.y;
-    const int32_t c = probes[(int64_t)b * n_lists + blockIdx.x];
+    const int32_t c = DBG_CID(probes[(int64_t)b * n_lists + blockIdx.x]);
     uint32_t *bm = bitmap + (int64_t)b * words;
     const int64_t lo = ivf_off[c], hi = ivf_off[c + 1];
     // four list entries per thread and iteration: their loads and the bitmap reads they lead to are in flight together
@@ -24,6 +24,7 @@ mark_kernel(const int32_t *__restrict__ probes, int n_lists, const int64_t *__re
         for (int u = 0; u < 4; ++u) {
             const int64_t e = e0 + u * (int64_t)blockDim.x;
             d[u] = e < hi ? (uint32_t)ivf_doc[e] : 0xffffffffu;
+            if (e < hi && !DBG_DOC_OK(d[u])) d[u] = 0xffffffffu;          // (debug build) skip a bad list entry
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) cur[u] = d[u] != 0xffffffffu ? bm[d[u] >> 5] : 0xffffffffu;

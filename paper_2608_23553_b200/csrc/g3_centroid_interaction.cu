@@ -43,7 +43,7 @@ ci_kernel(const int32_t *__restrict__ table, int64_t K, int nq, const int32_t *_
     int32_t *out = ci + (int64_t)b * maxc;
     const int warps_per_query = gridDim.x * CI_WARPS;
     for (int j = blockIdx.x * CI_WARPS + (threadIdx.x >> 5); j < n; j += warps_per_query) {
-        const int64_t d = cb[j];
+        const int64_t d = DBG_DOC(cb[j]);
         const int64_t t0 = doc_off[d], t1 = doc_off[d + 1];
         int m[NQW];
 #pragma unroll
@@ -59,7 +59,7 @@ ci_kernel(const int32_t *__restrict__ table, int64_t K, int nq, const int32_t *_
                 int32_t v[8][NQW];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    const int32_t *row = tb + (int64_t)c[u] * nq;
+                    const int32_t *row = tb + (int64_t)DBG_CID(c[u]) * nq;
 #pragma unroll
                     for (int w = 0; w < NQW; ++w) {
                         int col = lane + 32 * w;
@@ -102,7 +102,7 @@ ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__re
     int32_t *out = ci + (int64_t)b * maxc;
     const int warps_per_query = gridDim.x * CI_WARPS;
     for (int j = blockIdx.x * CI_WARPS + (threadIdx.x >> 5); j < n; j += warps_per_query) {
-        const int64_t d = cb[j];
+        const int64_t d = DBG_DOC(cb[j]);
         const int64_t t0 = doc_off[d], t1 = doc_off[d + 1];
         int4 m = make_int4(INT_MIN, INT_MIN, INT_MIN, INT_MIN);
         for (int64_t base = t0; base < t1; base += 32) {
@@ -116,7 +116,7 @@ ci_wide_kernel(const int32_t *__restrict__ table, int64_t K, const int32_t *__re
                     int src = (s + u) * TPL + grp;
                     src = src < 32 ? src : 31;    // lane 31 holds a valid (possibly repeated) token
                     const int32_t c = __shfl_sync(0xffffffffu, cidv, src);
-                    v[u] = __ldg(tb + (int64_t)c * LPR);
+                    v[u] = __ldg(tb + (int64_t)DBG_CID(c) * LPR);
                 }
 #pragma unroll
                 for (int u = 0; u < UNROLL; u += 2) {          // three-input integer maximum: two rows per instruction
@@ -175,20 +175,20 @@ ci_wide_rng_kernel(const int32_t *__restrict__ table, int64_t K, const int2 *__r
         int32_t nx_cid;
         {
             const int t0 = __shfl_sync(0xffffffffu, mine.x, 0), len = __shfl_sync(0xffffffffu, mine.y, 0);
-            nx_cid = cids[(int64_t)t0 + (lane < len - 1 ? lane : len - 1)];
+            nx_cid = cids[DBG_TOK((int64_t)t0 + (lane < len - 1 ? lane : len - 1))];
         }
         for (int di = 0; di < cnt_docs; ++di) {
             const int t0 = __shfl_sync(0xffffffffu, mine.x, di), len = __shfl_sync(0xffffffffu, mine.y, di);
             int32_t cidv = nx_cid;
             if (di + 1 < cnt_docs) {
                 const int n0 = __shfl_sync(0xffffffffu, mine.x, di + 1), nl = __shfl_sync(0xffffffffu, mine.y, di + 1);
-                nx_cid = cids[(int64_t)n0 + (lane < nl - 1 ? lane : nl - 1)];
+                nx_cid = cids[DBG_TOK((int64_t)n0 + (lane < nl - 1 ? lane : nl - 1))];
             }
             int4 m = make_int4(INT_MIN, INT_MIN, INT_MIN, INT_MIN);
             for (int base = 0; base < len; base += 32) {
                 const int cnt = len - base < 32 ? len - base : 32;
                 // lanes past the end repeat the last token: a duplicate cannot change a maximum
-                if (base != 0) cidv = cids[(int64_t)t0 + base + (lane < cnt ? lane : cnt - 1)];
+                if (base != 0) cidv = cids[DBG_TOK((int64_t)t0 + base + (lane < cnt ? lane : cnt - 1))];
                 for (int s = 0; s * TPL < cnt; s += UNROLL) {
                     int4 v[UNROLL];
 #pragma unroll
@@ -196,7 +196,7 @@ ci_wide_rng_kernel(const int32_t *__restrict__ table, int64_t K, const int2 *__r
                         int src = (s + u) * TPL + grp;
                         src = src < 32 ? src : 31;    // lane 31 holds a valid (possibly repeated) token
                         const int32_t c = __shfl_sync(0xffffffffu, cidv, src);
-                        v[u] = __ldg(tb + (int64_t)c * LPR);
+                        v[u] = __ldg(tb + (int64_t)DBG_CID(c) * LPR);
                     }
 #pragma unroll
                     for (int u = 0; u < UNROLL; u += 2) {
@@ -299,7 +299,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
     int64_t nx_t0 = 0, nx_t1 = 0;
     int32_t nx_cid[SLABS];
     auto prefetch = [&](int j) {
-        const int64_t d = cb[j];
+        const int64_t d = DBG_DOC(cb[j]);
         nx_t0 = doc_off[d];
         nx_t1 = doc_off[d + 1];
 #pragma unroll
@@ -337,7 +337,7 @@ ci_coarse_kernel(const uint8_t *__restrict__ table8, int64_t K, const int32_t *_
 #pragma unroll
                     for (int s = 0; s < STEPS; ++s) {
                         const int32_t c = __shfl_sync(0xffffffffu, cid[k], s * TPL + grp);
-                        v[k * STEPS + s] = SMEM ? ts[c * LPR] : __ldg(tb + (int64_t)c * LPR);
+                        v[k * STEPS + s] = SMEM ? ts[DBG_CID(c) * LPR] : __ldg(tb + (int64_t)DBG_CID(c) * LPR);
                     }
                 }
             }
@@ -395,7 +395,7 @@ cand_range_kernel(const int32_t *__restrict__ cand, const int32_t *__restrict__ 
     const int b = blockIdx.y;
     const int n = n_cand[b];
     for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
-        const int64_t d = cand[(int64_t)b * maxc + j];
+        const int64_t d = DBG_DOC(cand[(int64_t)b * maxc + j]);
         const int64_t t0 = doc_off[d];
         rng[(int64_t)b * maxc + j] = make_int2((int)t0, (int)(doc_off[d + 1] - t0));
     }
@@ -443,7 +443,7 @@ ci_coarse_rng_body(const uint8_t *__restrict__ table8, int64_t K, const int2 *__
 #pragma unroll
             for (int k = 0; k < SLABS; ++k) {
                 const int i = 32 * k + lane;
-                nx_cid[k] = cids[(int64_t)t0 + (i < len - 1 ? i : len - 1)];
+                nx_cid[k] = cids[DBG_TOK((int64_t)t0 + (i < len - 1 ? i : len - 1))];
             }
         }
         for (int di = 0; di < cnt; ++di) {
@@ -460,7 +460,7 @@ ci_coarse_rng_body(const uint8_t *__restrict__ table8, int64_t K, const int2 *__
 #pragma unroll
                 for (int k = 0; k < SLABS; ++k) {
                     const int i = 32 * k + lane;
-                    nx_cid[k] = cids[(int64_t)n0 + (i < nl - 1 ? i : nl - 1)];
+                    nx_cid[k] = cids[DBG_TOK((int64_t)n0 + (i < nl - 1 ? i : nl - 1))];
                 }
             }
             uint32_t m[8];
@@ -475,7 +475,7 @@ ci_coarse_rng_body(const uint8_t *__restrict__ table8, int64_t K, const int2 *__
 #pragma unroll
                         for (int s = 0; s < STEPS; ++s) {
                             const int32_t c = __shfl_sync(0xffffffffu, cid[k], s * TPL + grp);
-                            v[k * STEPS + s] = __ldg(tb + (int64_t)c * LPR);
+                            v[k * STEPS + s] = __ldg(tb + (int64_t)DBG_CID(c) * LPR);
                         }
                     }
                 }
@@ -484,7 +484,7 @@ ci_coarse_rng_body(const uint8_t *__restrict__ table8, int64_t K, const int2 *__
 #pragma unroll
                     for (int k = 0; k < SLABS; ++k) {
                         const int i = base + 32 * SLABS + 32 * k + lane;
-                        cid[k] = cids[(int64_t)t0 + (i < len - 1 ? i : len - 1)];
+                        cid[k] = cids[DBG_TOK((int64_t)t0 + (i < len - 1 ? i : len - 1))];
                     }
                 }
 #pragma unroll

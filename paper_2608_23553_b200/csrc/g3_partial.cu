@@ -86,7 +86,7 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
     __shared__ long long s_sq;
     const int b = blockIdx.y;
     const int i = blockIdx.x / P;
-    const int32_t c = probes[((int64_t)b * nq + i) * P + blockIdx.x % P];
+    const int32_t c = DBG_CID(probes[((int64_t)b * nq + i) * P + blockIdx.x % P]);
     const float *q = queries + ((int64_t)b * nq + i) * D;
     for (int x = threadIdx.x; x < D; x += PS_THREADS) {
         float v = fminf(fmaxf(q[x], -1.0f), 1.0f);
@@ -153,7 +153,7 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
         const long long dist = (long long)s_c + __double2ll_rn(r);
         if (dist > 0) {                                // the table starts at 0 (Algorithm 2)
             const int64_t rank = wr_word + __popc(bm_word & ((1u << (d & 31)) - 1u));
-            if (rank < maxc) {
+            if (rank < maxc && DBG_RANK_OK(rank)) {
                 // F' = sum_i M[., i] is kept up to date with the increments: M only grows, integer adds commute
                 int32_t old = 0;
                 if (HASH) {
@@ -187,8 +187,8 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
     const int64_t e1 = tok_off[c + 1];
     int64_t e = tok_off[c] + threadIdx.x;
     for (; e + PS_THREADS < e1; e += 2 * PS_THREADS) {
-        const int64_t ta = tok_id[e], tb2 = tok_id[e + PS_THREADS];
-        const uint32_t da = (uint32_t)tok_doc[e], db = (uint32_t)tok_doc[e + PS_THREADS];
+        const int64_t ta = DBG_TOK(tok_id[e]), tb2 = DBG_TOK(tok_id[e + PS_THREADS]);
+        const uint32_t da = (uint32_t)DBG_DOC(tok_doc[e]), db = (uint32_t)DBG_DOC(tok_doc[e + PS_THREADS]);
         const uint32_t bma = __ldg(bm + (da >> 5)), bmb = __ldg(bm + (db >> 5));
         const int32_t wra = __ldg(wr + (da >> 5)), wrb = __ldg(wr + (db >> 5));
         const int Ta = code_dot(ta), Tb = code_dot(tb2);
@@ -196,10 +196,10 @@ partial_score_kernel(const float *__restrict__ queries, const int32_t *__restric
         update(db, Tb, bmb, wrb);
     }
     if (e < e1) {
-        const uint32_t d = (uint32_t)tok_doc[e];
+        const uint32_t d = (uint32_t)DBG_DOC(tok_doc[e]);
         const uint32_t bmd = __ldg(bm + (d >> 5));
         const int32_t wrd = __ldg(wr + (d >> 5));
-        update(d, code_dot(tok_id[e]), bmd, wrd);
+        update(d, code_dot(DBG_TOK(tok_id[e])), bmd, wrd);
     }
 }
 

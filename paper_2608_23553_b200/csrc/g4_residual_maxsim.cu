@@ -65,7 +65,7 @@ residual_maxsim_kernel(const float *__restrict__ queries, const int32_t *__restr
             if (tid == 0) score4[(int64_t)b * n_prune + j] = -INFINITY;
             continue;
         }
-        const int64_t t0 = doc_off[d], t1 = doc_off[d + 1];
+        const int64_t t0 = doc_off[DBG_DOC(d)], t1 = doc_off[DBG_DOC(d) + 1];
         float best[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         for (int64_t base = t0; base < t1; base += TT) {
             const int cnt = (int)((t1 - base) < TT ? (t1 - base) : TT);
@@ -102,7 +102,7 @@ residual_maxsim_kernel(const float *__restrict__ queries, const int32_t *__restr
             for (int r = 0; r < 4; ++r) {
                 const int32_t c = tok_cid[4 * ty + r];
                 if (c < 0) continue;
-                const int32_t *row = tb + (int64_t)c * nq + 4 * tx;
+                const int32_t *row = tb + (int64_t)DBG_CID(c) * nq + 4 * tx;
                 int4 s;
                 if (vec_rows) {
                     s = __ldg(reinterpret_cast<const int4 *>(row));

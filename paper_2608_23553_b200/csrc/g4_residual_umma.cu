@@ -111,6 +111,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         long long t0 = 0;
         int len = 0;
         if (d >= 0) {
+            d = DBG_DOC(d);
             t0 = doc_off[d];
             len = (int)(doc_off[d + 1] - t0);
         }
@@ -183,7 +184,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         if (s < total) {
             while (dl_hint + 1 < nd && s_off[dl_hint + 1] <= s) ++dl_hint;    // positions only move forward
             dl = dl_hint;
-            const long long t = s_t0[dl] + (s - s_off[dl]);
+            const long long t = DBG_TOK(s_t0[dl] + (s - s_off[dl]));
             cid = RQ ? __float_as_int(factors[t]) : cids[t];     // RQ: the slot carries the token's factor bits (> 0)
             const uint32_t *src = codes + t * CW;
             if (NBITS == 2 && CW == 8) {                  // 32-byte codes (32-byte aligned): one load
@@ -274,7 +275,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
         // ---- while the tensor core works: this token's row of the score table, and the next tile's token -----------
         int4 sv[NQP / 4];
         if (!RQ && cid >= 0) {
-            const int32_t *srow = tb + (int64_t)cid * nq;
+            const int32_t *srow = tb + (int64_t)DBG_CID(cid) * nq;
 #pragma unroll
             for (int g = 0; g < NQP / 4; ++g) {
                 const int col = 4 * g;
@@ -303,7 +304,7 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             // are far larger): ask for it now so that HBM latency passes during this tile's epilogue
             // (measured: a gain for q_len <= 32, a loss for the two-line rows of longer queries)
             if (!RQ && NQP == 32 && cid_next >= 0) {
-                const char *row = reinterpret_cast<const char *>(tb + (int64_t)cid_next * nq);
+                const char *row = reinterpret_cast<const char *>(tb + (int64_t)DBG_CID(cid_next) * nq);
                 for (int off = 0; off < nq * 4; off += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + off));
             }
         }

@@ -91,7 +91,7 @@ rabitq_partial_kernel(const float *__restrict__ q_rot, int nq, int D, int P, flo
     __shared__ int s_sq;
     const int b = blockIdx.y;
     const int i = blockIdx.x / P;
-    const int32_t cen = probes[((int64_t)b * nq + i) * P + blockIdx.x % P];
+    const int32_t cen = DBG_CID(probes[((int64_t)b * nq + i) * P + blockIdx.x % P]);
     const float *q = q_rot + ((int64_t)b * nq + i) * D;
     for (int x = threadIdx.x; x < D; x += RP_THREADS)
         xq[x] = __float2int_rn(fminf(fmaxf(q[x], -1.0f), 1.0f) * 4194304.0f);
@@ -138,14 +138,14 @@ rabitq_partial_kernel(const float *__restrict__ q_rot, int nq, int D, int P, flo
         const float est = __fmul_rn(factor, __fmul_rn(c, (float)(2 * T - sq)));
         if (est > 0.0f) {                              // the table starts at 0 (Algorithm 2)
             const int64_t rank = wr_word + __popc(bm_word & ((1u << (d & 31)) - 1u));
-            if (rank < maxc) atomicMax(&Mb[rank * nq + i], __float_as_int(est));
+            if (rank < maxc && DBG_RANK_OK(rank)) atomicMax(&Mb[rank * nq + i], __float_as_int(est));
         }
     };
     const int64_t e1 = tok_off[cen + 1];
     int64_t e = tok_off[cen] + threadIdx.x;
     for (; e + RP_THREADS < e1; e += 2 * RP_THREADS) {         // two visits per iteration, their loads issued together
-        const int64_t ta = tok_id[e], tb = tok_id[e + RP_THREADS];
-        const uint32_t da = (uint32_t)tok_doc[e], db = (uint32_t)tok_doc[e + RP_THREADS];
+        const int64_t ta = DBG_TOK(tok_id[e]), tb = DBG_TOK(tok_id[e + RP_THREADS]);
+        const uint32_t da = (uint32_t)DBG_DOC(tok_doc[e]), db = (uint32_t)DBG_DOC(tok_doc[e + RP_THREADS]);
         const float fa = __ldg(inv_dot + ta), fb = __ldg(inv_dot + tb);
         const uint32_t bma = __ldg(bm + (da >> 5)), bmb = __ldg(bm + (db >> 5));
         const int32_t wra = __ldg(wr + (da >> 5)), wrb = __ldg(wr + (db >> 5));
@@ -154,8 +154,8 @@ rabitq_partial_kernel(const float *__restrict__ q_rot, int nq, int D, int P, flo
         update(db, fb, Tb, bmb, wrb);
     }
     if (e < e1) {
-        const int64_t t = tok_id[e];
-        const uint32_t d = (uint32_t)tok_doc[e];
+        const int64_t t = DBG_TOK(tok_id[e]);
+        const uint32_t d = (uint32_t)DBG_DOC(tok_doc[e]);
         const float f = __ldg(inv_dot + t);
         const uint32_t bmd = __ldg(bm + (d >> 5));
         const int32_t wrd = __ldg(wr + (d >> 5));
