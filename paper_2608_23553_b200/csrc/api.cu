@@ -111,7 +111,6 @@ Layout make_layout(const Index &ix, const Params &p)
     L.qdig = take(3 * B * nq * 128);
     L.table = take(B * (size_t)ix.K * nq * sizeof(int32_t));
     L.table8 = take(coarse_supported(p.nq) ? B * (size_t)ix.K * nq : 0);
-    L.table8g = take(coarse_group_table_bytes(ix, p));
     L.part = take(B * L.n_part * p.P * nq * sizeof(unsigned long long));
     L.probes = take(B * nq * p.P * sizeof(int32_t));
     L.bitmap = take(B * (size_t)L.words * sizeof(uint32_t));
@@ -324,12 +323,7 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
                 prof_mark(SLOT_MISC, st);
             }
             // bounds for every candidate, contenders for the top n_prune, exact CI and selection among those
-            // (the query-group form needs the candidate bitmap of stage 2: only when stage 2 ran in this call)
-            CoarseGroupArgs grouped{status + STATUS_WORD_DENSE, (uint8_t *)(ws + L.table8g), bitmap, word_rank, L.words};
-            const bool can_group = first <= 2 && coarse_group_table_bytes(ix, p) > 0;
-            if ((rc = launch_coarse_bounds(ix, p, table8, cand, n_cand, lo, hi, (int2 *)(ws + L.cand_rng),
-                                           can_group ? &grouped : nullptr, st)))
-                return rc;
+            if ((rc = launch_coarse_bounds(ix, p, table8, cand, n_cand, lo, hi, (int2 *)(ws + L.cand_rng), st))) return rc;
             prof_mark(SLOT_CI, st);
             if ((rc = launch_contenders(ix, p, cand, n_cand, lo, hi, cont, n_cont, ci, (const int2 *)(ws + L.cand_rng),
                                         (int2 *)(ws + L.cont_rng), st))) return rc;

@@ -39,7 +39,6 @@ struct Index {
 // Device status bits kept in the first word of a workspace.
 enum : uint32_t { ST_OVERFLOW = 1u, ST_BAD_QUERY = 2u, ST_TIMEOUT = 4u, ST_BAD_INDEX = 8u };
 constexpr int STATUS_WORD_CANARY = 8;   // status[8]: first damaged guard region found by the debug build's check
-constexpr int STATUS_WORD_DENSE = 9;    // status[9]: 1 when the stage-3 bound scan runs in its query-group form
 
 // ---------------------------------------------------------------------------------------------------------------
 // Workspace layout (all offsets 256-byte aligned).
@@ -60,9 +59,7 @@ struct Layout {
     size_t out_scores;    // float  [B, k]
     size_t qdig;          // int8   [3][B*nq][128]
     size_t table;         // int32  [B][K][nq]
-    size_t table8;        // uint8  [B][K][nq]        coarse copy: clamp(S >> 16, 0, 255)
-    size_t table8g;       // uint8  [groups][K][128]  the same with the rows of 128 / nq queries side by side (dense
-                          //                          candidate sets: one looked-up line serves the whole group)
+    size_t table8;        // uint8  [B][K][nq]        coarse copy: min((S + 2^24 + 64) >> 17, 255)
     size_t part;          // uint64 [B][n_part][P][nq] partial top-P keys
     size_t probes;        // int32  [B][nq][P]
     size_t bitmap;        // uint32 [B][words]
@@ -151,19 +148,8 @@ int launch_partial_scores(const Index &ix, const Params &p, const Layout &L, con
 bool coarse_supported(int nq);
 int launch_coarse_table(const Index &ix, const Params &p, const int32_t *table, uint8_t *table8, cudaStream_t st);
 // rng: int2 [B][maxc] scratch for the candidates' token ranges (may be NULL: per-document offset lookups instead).
-// grouped (may be NULL): the pieces of the query-group form of the scan, chosen on the device when most documents are
-// candidates of most queries -- flag word, grouped table, candidate bitmap and per-word candidate ranks of stage 2.
-struct CoarseGroupArgs {
-    uint32_t *flag;
-    uint8_t *table8g;
-    const uint32_t *bitmap;
-    const int32_t *word_rank;
-    int64_t words;
-};
-size_t coarse_group_table_bytes(const Index &ix, const Params &p);
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
-                         const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, const CoarseGroupArgs *grouped,
-                         cudaStream_t st);
+                         const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, cudaStream_t st);
 // scratch: an int32 [B][maxc] array that is free during this step.
 // rng / cont_rng (may be NULL): the candidates' token ranges and where to put those of the contenders.
 int launch_contenders(const Index &ix, const Params &p, const int32_t *cand, const int32_t *n_cand, const int32_t *lo,

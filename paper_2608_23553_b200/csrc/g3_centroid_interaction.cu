@@ -542,198 +542,23 @@ template <int LPR>
 __global__ void __launch_bounds__(CI_THREADS)
 ci_coarse_rng_kernel(const uint8_t *__restrict__ table8, int64_t K, const int2 *__restrict__ rng,
                      const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
-                     int32_t *__restrict__ lo, int32_t *__restrict__ hi, const uint32_t *__restrict__ skip_flag)
+                     int32_t *__restrict__ lo, int32_t *__restrict__ hi)
 {
-    if (skip_flag != nullptr && *skip_flag != 0u) return;      // the query-group form of the scan does this call's work
     ci_coarse_rng_body<LPR>(table8, K, rng, n_cand, maxc, cids, lo, hi);
 }
 template <int LPR>
 __global__ void __launch_bounds__(CI_THREADS, 4)
 ci_coarse_rng_kernel_b4(const uint8_t *__restrict__ table8, int64_t K, const int2 *__restrict__ rng,
                         const int32_t *__restrict__ n_cand, int64_t maxc, const int32_t *__restrict__ cids,
-                        int32_t *__restrict__ lo, int32_t *__restrict__ hi, const uint32_t *__restrict__ skip_flag)
+                        int32_t *__restrict__ lo, int32_t *__restrict__ hi)
 {
-    if (skip_flag != nullptr && *skip_flag != 0u) return;
     ci_coarse_rng_body<LPR>(table8, K, rng, n_cand, maxc, cids, lo, hi);
 }
 
 bool coarse_supported(int nq) { return nq == 32 || nq == 64; }
 
-// ------------------------------------------------------------------------------------------------ query groups ---
-// The bound scan for DENSE candidate sets (most documents are candidates of most queries, e.g. long documents with
-// many probes).  The per-query scan above looks up one table row per (query, candidate token); every lookup is a
-// distinct 128-byte line for the load pipe, which is what limits it, and a row of q_len bytes uses a quarter or half
-// of that line.  Here the rows of G = 128 / q_len queries lie side by side in one line (table8g), the documents are
-// scanned once per GROUP of queries, and one looked-up line serves all G queries: G times fewer lines and centroid-id
-// reads per (query, token).  Bounds are the same numbers as the per-query scan's (same bytes, same formula), so the
-// contenders and the pruned set do not depend on which form ran.
-//
-// Which form runs is decided on the device (the host never learns the candidate counts): dense_decide_kernel sets the
-// flag when the candidates are at least DENSE_MIN_SHARE of (queries x documents); the kernels of the form that is
-// not chosen return at once.
-constexpr int DENSE_MIN_PERCENT = 60;
-
-__global__ void dense_decide_kernel(const int32_t *__restrict__ n_cand, int B, int64_t N, uint32_t *flag)
-{
-    long long sum = 0;
-    for (int b = threadIdx.x; b < B; b += 32) sum += n_cand[b];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (threadIdx.x == 0) *flag = (sum * 100 >= (long long)DENSE_MIN_PERCENT * B * N) ? 1u : 0u;
-}
-
-// table8 [B][K][16 LPRQ] -> table8g [groups][K][128]: one thread per 16-byte piece of a grouped line.
-template <int LPRQ>
-__global__ void __launch_bounds__(256)
-group_table_kernel(const uint32_t *__restrict__ flag, const uint8_t *__restrict__ table8, int64_t K, int B,
-                   uint8_t *__restrict__ table8g)
-{
-    if (*flag == 0u) return;
-    constexpr int G = 8 / LPRQ, NQ = 16 * LPRQ;
-    const int groups = (B + G - 1) / G;
-    const int64_t total = (int64_t)groups * K * 8;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int piece = (int)(e & 7);
-        const int64_t c = (e >> 3) % K, g = (e >> 3) / K;
-        const int64_t b = g * G + piece / LPRQ;
-        int4 v = make_int4(0, 0, 0, 0);
-        if (b < B) v = __ldg(reinterpret_cast<const int4 *>(table8 + (b * K + c) * NQ) + piece % LPRQ);
-        reinterpret_cast<int4 *>(table8g)[e] = v;
-    }
-}
-
-// grid (blocks, groups).  A warp owns a run of 32-document words of the candidate bitmaps; lane i keeps the token range
-// and, at the end, the results of document 32 w + i.  Within a document lane = (token slot lane / 8, 16-byte piece
-// lane % 8 of the grouped line); pieces [LPRQ s, LPRQ (s + 1)) belong to query s of the group.
-template <int LPRQ>
-__global__ void __launch_bounds__(CI_THREADS)
-ci_coarse_group_kernel(const uint32_t *__restrict__ flag, const uint8_t *__restrict__ table8g, int64_t K, int B,
-                       int64_t N, const uint32_t *__restrict__ bitmap, const int32_t *__restrict__ word_rank,
-                       int64_t words, const int64_t *__restrict__ doc_off, const int32_t *__restrict__ cids,
-                       int64_t maxc, int32_t *__restrict__ lo, int32_t *__restrict__ hi)
-{
-    if (*flag == 0u) return;
-    constexpr int G = 8 / LPRQ, NQ = 16 * LPRQ;
-    const int group = blockIdx.y, b0 = group * G;
-    const int lane = threadIdx.x & 31;
-    const int piece = lane & 7, tslot = lane >> 3;
-    const int4 *tb = reinterpret_cast<const int4 *>(table8g + (int64_t)group * K * 128) + piece;
-    const int64_t warps = (int64_t)gridDim.x * CI_WARPS;
-    const int64_t per_warp = (words + warps - 1) / warps;
-    const int64_t wq = (int64_t)blockIdx.x * CI_WARPS + (threadIdx.x >> 5);
-    const int64_t w_begin = wq * per_warp < words ? wq * per_warp : words;
-    const int64_t w_end = w_begin + per_warp < words ? w_begin + per_warp : words;
-
-    for (int64_t w = w_begin; w < w_end; ++w) {
-        uint32_t mw[G];
-        int32_t rk[G];
-        uint32_t any = 0u;
-#pragma unroll
-        for (int s = 0; s < G; ++s) {
-            const bool live = b0 + s < B;
-            mw[s] = live ? bitmap[(int64_t)(b0 + s) * words + w] : 0u;
-            rk[s] = live ? word_rank[(int64_t)(b0 + s) * words + w] : 0;
-            any |= mw[s];
-        }
-        if (any == 0u) continue;
-        const int64_t d = w * 32 + lane;
-        int64_t my_t0 = 0;
-        int my_len = 1;
-        if (d < N) {
-            my_t0 = doc_off[d];
-            my_len = (int)(doc_off[d + 1] - my_t0);
-        }
-        int my_packed[G];
-#pragma unroll
-        for (int s = 0; s < G; ++s) my_packed[s] = 0;
-        for (uint32_t rest = any; rest != 0u; rest &= rest - 1u) {
-            const int di = __ffs(rest) - 1;
-            const int64_t t0 = __shfl_sync(0xffffffffu, my_t0, di);
-            const int len = __shfl_sync(0xffffffffu, my_len, di);
-            uint32_t m[8];
-#pragma unroll
-            for (int r = 0; r < 8; ++r) m[r] = 0u;
-            // lanes past the end repeat the last token (harmless for a maximum)
-            int32_t cid_next = cids[DBG_TOK(t0 + (lane < len - 1 ? lane : len - 1))];
-            for (int base = 0; base < len; base += 32) {
-                const int32_t cidv = cid_next;
-                if (base + 32 < len) {
-                    const int i = base + 32 + lane;
-                    cid_next = cids[DBG_TOK(t0 + (i < len - 1 ? i : len - 1))];
-                }
-                const int steps = len - base >= 32 ? 8 : (len - base + 3) >> 2;       // four tokens per load
-                int4 v[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (u < steps) {
-                        const int32_t c = __shfl_sync(0xffffffffu, cidv, u * 4 + tslot);
-                        v[u] = __ldg(tb + (int64_t)DBG_CID(c) * 8);
-                    } else {
-                        v[u] = v[0];                                               // a repeat: harmless
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 8; u += 2) coarse_accumulate2(m, v[u], v[u + 1]);
-            }
-            // merge the four token slots (same piece, different tokens), halving the registers with each exchange:
-            // afterwards every lane holds two registers = four columns, a different quarter of the piece per token slot
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const bool up = (lane & 16) != 0;
-                const uint32_t send = up ? m[r] : m[r + 4], keep = up ? m[r + 4] : m[r];
-                m[r] = __vmaxu2(keep, __shfl_xor_sync(0xffffffffu, send, 16));
-            }
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const bool up = (lane & 8) != 0;
-                const uint32_t send = up ? m[r] : m[r + 2], keep = up ? m[r + 2] : m[r];
-                m[r] = __vmaxu2(keep, __shfl_xor_sync(0xffffffffu, send, 8));
-            }
-            int packed = 0;                                     // sum of maxima | saturated << 16 | zeros << 24
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int f0 = coarse_field_lo(m[r]), f1 = coarse_field_hi(m[r]);
-                packed += (f0 + f1) + (((f0 >= 255) + (f1 >= 255)) << 16) + (((f0 == 0) + (f1 == 0)) << 24);
-            }
-            // sum over the lanes of one query: its LPRQ pieces x four token slots
-            packed += __shfl_xor_sync(0xffffffffu, packed, 16);
-            packed += __shfl_xor_sync(0xffffffffu, packed, 8);
-            packed += __shfl_xor_sync(0xffffffffu, packed, 1);
-            if (LPRQ == 4) packed += __shfl_xor_sync(0xffffffffu, packed, 2);
-#pragma unroll
-            for (int s = 0; s < G; ++s) {
-                const int val = __shfl_sync(0xffffffffu, packed, s * LPRQ);
-                if (lane == di) my_packed[s] = val;
-            }
-        }
-        // lane i writes document 32 w + i for every query of the group that has it as a candidate, at its rank
-#pragma unroll
-        for (int s = 0; s < G; ++s) {
-            if ((mw[s] >> lane) & 1u) {
-                const int64_t rank = rk[s] + __popc(mw[s] & ((1u << lane) - 1u));
-                if (rank < maxc && DBG_RANK_OK(rank)) {
-                    lo[(int64_t)(b0 + s) * maxc + rank] = coarse_lo(my_packed[s]);
-                    hi[(int64_t)(b0 + s) * maxc + rank] = coarse_hi(my_packed[s], NQ);
-                }
-            }
-        }
-    }
-}
-
-// Bytes of the grouped table, 0 when the group form is never used for these parameters (fewer than two full groups
-// of queries, tables that fit shared memory, corpora of 2^31 tokens or more).
-size_t coarse_group_table_bytes(const Index &ix, const Params &p)
-{
-    if (!coarse_supported(p.nq) || ix.T >= 0x7fffffffLL) return 0;
-    const int G = 128 / p.nq;
-    if (p.B < 2 * G || (size_t)ix.K * p.nq <= 160 * 1024) return 0;
-    return (size_t)((p.B + G - 1) / G) * (size_t)ix.K * 128;
-}
-
-
 int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8, const int32_t *cand,
-                         const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, const CoarseGroupArgs *grouped,
-                         cudaStream_t st)
+                         const int32_t *n_cand, int32_t *lo, int32_t *hi, int2 *rng, cudaStream_t st)
 {
     const size_t table_bytes = (size_t)ix.K * p.nq;
     // the candidates' token ranges, for this scan and for the exact scoring of the contenders afterwards
@@ -788,41 +613,10 @@ int launch_coarse_bounds(const Index &ix, const Params &p, const uint8_t *table8
     const unsigned gx = (unsigned)per_query;
     dim3 grid(gx, (unsigned)p.B);
     if (use_rng) {
-        // dense candidate sets: the query-group form (decided on the device; the form not chosen returns at once)
-        const bool group_form = grouped != nullptr && coarse_group_table_bytes(ix, p) > 0;
-        const uint32_t *skip = group_form ? grouped->flag : nullptr;
-        if (group_form) {
-            const int G = 128 / p.nq;
-            const int groups = (p.B + G - 1) / G;
-            dense_decide_kernel<<<1, 32, 0, st>>>(n_cand, p.B, ix.N, grouped->flag);
-            const unsigned tblocks = (unsigned)(8 * ix.sm_count);
-            // blocks per group: as for the per-query form, the grouped tables scanned at the same time stay in L2
-            int64_t per_group = (resident * (int64_t)ix.K * 128 + COARSE_L2_TABLES - 1) / COARSE_L2_TABLES;
-            const int64_t fill = (2 * resident + groups - 1) / groups;
-            if (per_group < fill) per_group = fill;
-            const int64_t most = (((ix.N + 31) / 32) + CI_WARPS - 1) / CI_WARPS;
-            if (per_group > most) per_group = most;
-            if (per_group < 1) per_group = 1;
-            dim3 ggrid((unsigned)per_group, (unsigned)groups);
-            if (p.nq == 32) {
-                group_table_kernel<2><<<tblocks, 256, 0, st>>>(grouped->flag, table8, ix.K, p.B, grouped->table8g);
-                ci_coarse_group_kernel<2><<<ggrid, CI_THREADS, 0, st>>>(grouped->flag, grouped->table8g, ix.K, p.B, ix.N,
-                                                                      grouped->bitmap, grouped->word_rank,
-                                                                      grouped->words, ix.doc_off, ix.cids, p.maxc, lo, hi);
-            } else {
-                group_table_kernel<4><<<tblocks, 256, 0, st>>>(grouped->flag, table8, ix.K, p.B, grouped->table8g);
-                ci_coarse_group_kernel<4><<<ggrid, CI_THREADS, 0, st>>>(grouped->flag, grouped->table8g, ix.K, p.B, ix.N,
-                                                                      grouped->bitmap, grouped->word_rank,
-                                                                      grouped->words, ix.doc_off, ix.cids, p.maxc, lo, hi);
-            }
-            CHIMERA_CUDA(cudaGetLastError());
-            count_launch(SLOT_CI, 3);
-        }
         if (p.nq == 32)
-            ci_coarse_rng_kernel<2><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi, skip);
+            ci_coarse_rng_kernel<2><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
         else
-            ci_coarse_rng_kernel_b4<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi,
-                                                                   skip);
+            ci_coarse_rng_kernel_b4<4><<<grid, CI_THREADS, 0, st>>>(table8, ix.K, rng, n_cand, p.maxc, ix.cids, lo, hi);
         CHIMERA_CUDA(cudaGetLastError());
         count_launch(SLOT_CI);
         return CHIMERA_OK;

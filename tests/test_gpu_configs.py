@@ -86,32 +86,3 @@ def test_long_document_corpus_full_size_sampled_query():
     b = 17
     res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k, partial=True)
     assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune, table=False) <= 2
-
-
-@pytest.mark.parametrize("q_len,n_queries", [(32, 9), (64, 5), (32, 8)])
-def test_dense_candidate_sets_take_the_query_group_scan_and_match_the_oracle(q_len, n_queries):
-    """When most documents are candidates of most queries the stage-3 bound scan runs once per GROUP of queries (the
-    8-bit rows of 4 or 2 queries side by side in one line).  Its results must be the per-query scan's: every stage of
-    every query against the oracle, with a ragged last group, and the same queries one at a time (per-query form)."""
-    import paper_2608_23553_b200 as pkg
-    from synth import CONFIGS, make_corpus, make_queries
-    cfg = CONFIGS["tiny"].replace(n_docs=6000, n_centroids=8192, n_queries=n_queries, q_len=q_len, nprobe=48,
-                                  n_prune=300, k=20, len_lo=20, len_hi=70)
-    corp = make_corpus(cfg)
-    q = make_queries(cfg)
-    oix = oracle.make_index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
-    gix = pkg.Index(corp.centroids.cuda(), corp.cids.cuda(), corp.codes.cuda(), corp.doclens.cuda(), cfg.nbits,
-                    cfg.res_lo, cfg.res_hi)
-    B = q.shape[0]
-    taps = gix.alloc_taps(B, cfg.q_len, cfg.nprobe, cfg.n_prune)
-    ids, sc = gix.search(q.cuda(), cfg.nprobe, cfg.n_prune, cfg.k, taps=taps)
-    assert gix.status() == 0
-    # dense: at least 60 % of (queries x documents) are candidates, so the group form ran
-    assert int(taps.n_cand.sum()) >= 0.6 * B * cfg.n_docs
-    tn = taps_to_numpy(taps)
-    ids_np, sc_np, q_np = ids.cpu().numpy(), sc.cpu().numpy(), q.numpy()
-    for b in range(B):
-        res = oracle.pipeline(q_np[b], oix, cfg.nprobe, cfg.n_prune, cfg.k)
-        assert check_query(tn, b, res, ids_np[b], sc_np[b], cfg.k, cfg.n_prune) == 0
-    one = gix.search(q[B - 1:].cuda(), cfg.nprobe, cfg.n_prune, cfg.k)
-    assert torch.equal(one[0][0], ids[B - 1]) and torch.equal(one[1][0], sc[B - 1])
