@@ -39,6 +39,7 @@ def lib():
         _lib.oracle_prune.restype = ctypes.c_int64
         _lib.oracle_chamfer.restype = ctypes.c_double
         _lib.oracle_recall.restype = ctypes.c_double
+        _lib.oracle_graph_probes.restype = ctypes.c_int64
     return _lib
 
 
@@ -189,12 +190,42 @@ def rabitq_partial(qp, pr, cand, ix: Index, rq: RabitqCodes) -> np.ndarray:
     return out
 
 
-def pipeline_rabitq(q, ix: Index, rq: RabitqCodes, nprobe: int, k_refine: int, k: int) -> "Result":
+def knn_graph(centroids, degree: int) -> np.ndarray:
+    """O-10: [K, degree] int32 nearest-neighbour graph over the centroids (best first, self excluded)."""
+    c = _arr(centroids, np.float32)
+    K, D = c.shape
+    assert 1 <= degree <= K - 1
+    g = np.empty((K, degree), dtype=np.int32)
+    lib().oracle_knn_graph(_p(c), ctypes.c_int64(K), ctypes.c_int32(D), ctypes.c_int32(degree), _p(g))
+    return g
+
+
+def graph_probes(q, centroids, graph: np.ndarray, nprobe: int, beam: int, n_entries: int, max_expansions: int = 1 << 40):
+    """O-10: best-first search of the centroid graph for every query token of q [nq, D].
+    Returns (probes [nq, nprobe] int32, scores [nq, nprobe] int32, visited [nq, K] bool)."""
+    q = _arr(q, np.float32)
+    c = _arr(centroids, np.float32)
+    g = _arr(graph, np.int32)
+    K, D = c.shape
+    assert nprobe <= beam and nprobe <= n_entries <= K and g.shape[0] == K
+    nq = q.shape[0]
+    pr = np.empty((nq, nprobe), dtype=np.int32)
+    sc = np.empty((nq, nprobe), dtype=np.int32)
+    vis = np.empty((nq, K), dtype=np.uint8)
+    for i in range(nq):
+        lib().oracle_graph_probes(_p(q[i]), _p(c), ctypes.c_int64(K), ctypes.c_int32(D), _p(g), ctypes.c_int32(g.shape[1]),
+                                  ctypes.c_int32(n_entries), ctypes.c_int32(beam), ctypes.c_int64(max_expansions),
+                                  ctypes.c_int32(nprobe), _p(pr[i]), _p(sc[i]), _p(vis[i]))
+    return pr, sc, vis.astype(bool)
+
+
+def pipeline_rabitq(q, ix: Index, rq: RabitqCodes, nprobe: int, k_refine: int, k: int, probes_override=None) -> "Result":
     """The paper's GPU pipeline on 1-bit codes (Algorithm 1 without its CPU half): centroid probes and candidates as
     usual, candidate refinement by partial 1-bit scores, complete 1-bit scores of the survivors, top-k.  `ci` holds
-    F' (float32); ordering floats >= 0 equals ordering their bit patterns, so O-4b selects on the int32 view."""
+    F' (float32); ordering floats >= 0 equals ordering their bit patterns, so O-4b selects on the int32 view.
+    probes_override: the probes of a graph search (O-10) in place of the exhaustive top-nprobe."""
     S = score_table(q, ix.centroids)
-    pr = probes(S, nprobe)
+    pr = probes(S, nprobe) if probes_override is None else _arr(probes_override, np.int32)
     cand = candidates(pr, ix)
     qp = rotate(rq.rotation, q)
     fp = rabitq_partial(qp, pr, cand, ix, rq)

@@ -20,6 +20,8 @@
  *   O-8 oracle_partial_scores  candidate refinement with partial scores F'(Q,V)  (Sec. 3.2 step 2, Algorithm 2)
  *   O-9 oracle_rotate, oracle_rabitq_score_docs, oracle_rabitq_partial   the same two steps on RaBitQ 1-bit codes
  *       (Sec. 2.2: rotation, 1-bit code, estimator <q_p, o_p-bar> / <o_p, o_p-bar>, code form of <q_p, o_p-bar>)
+ *   O-10 oracle_knn_graph, oracle_graph_probes   proximity graph over the centroids and the search that replaces the
+ *       exhaustive centroid scan (Sec. 2.3 "Proximity graph", Sec. 3.1, Algorithm 1 line searchCAGRA)
  *
  * Pins: every function above is pinned by tests that do not call it to produce their expectation
  * (closed forms, library routines on special cases, set identities, hand-worked values).  Unpinned:
@@ -304,6 +306,112 @@ void oracle_rabitq_partial(const float *qp, int32_t nq, int32_t D, const uint8_t
     free(score);
     free(xq);
     free(probed);
+}
+
+/* ---------------------------------------------------------------- O-10 ----------------------------------------- */
+/* Exact fixed-point score of one query token against one centroid (the O-1 formula for a single pair). */
+static int32_t fx_score(const int64_t *xq, const float *c, int32_t D)
+{
+    int64_t t = 0;
+    for (int d = 0; d < D; ++d) t += xq[d] * (int64_t)rint((double)c[d] * Q22);
+    int64_t u = t + (1LL << 19);
+    int64_t f = u / (1LL << 20);
+    if ((u % (1LL << 20)) < 0) f -= 1;
+    return (int32_t)f;
+}
+
+/* Sec. 2.3 / Sec. 3.1: a proximity graph over the IVF centroids, "constructed by linking each node to a limited number
+ * of nearest neighbors".  Here: node c is linked to the R other centroids with the largest fixed-point inner product
+ * S_fx(c, c') (all centroids are unit vectors, so this is nearest first), ties towards the smaller id, listed best
+ * first.  No pruning or diversification.  graph[c*R + r] = r-th neighbour of c.  Requires 1 <= R <= K - 1. */
+void oracle_knn_graph(const float *cent, int64_t K, int32_t D, int32_t R, int32_t *graph)
+{
+    si_pair *v = (si_pair *)malloc(sizeof(si_pair) * (size_t)K);
+    int64_t *xq = (int64_t *)malloc(sizeof(int64_t) * (size_t)D);
+    for (int64_t c = 0; c < K; ++c) {
+        for (int d = 0; d < D; ++d) xq[d] = (int64_t)rint((double)cent[c * D + d] * Q22);
+        int64_t n = 0;
+        for (int64_t o = 0; o < K; ++o) {
+            if (o == c) continue;
+            v[n].s = fx_score(xq, cent + o * D, D);
+            v[n].id = (int32_t)o;
+            ++n;
+        }
+        qsort(v, (size_t)n, sizeof(si_pair), cmp_si_desc);
+        for (int r = 0; r < R; ++r) graph[c * R + r] = v[r].id;
+    }
+    free(v);
+    free(xq);
+}
+
+/* Sec. 2.3: "the search starts from one or a few entry points and iteratively moves to neighboring nodes that are
+ * closer to the query until convergence"; Algorithm 1 uses it to get each query token's n_probe centroids.  Stated
+ * here as a best-first search with a bounded result list:
+ *   - entry points: the n_entries centroids floor(j K / n_entries), j = 0 .. n_entries - 1 (the same for every query);
+ *   - a list of at most `beam` visited centroids, ordered by (score descending, id ascending);
+ *   - every entry point is visited (scored, marked, offered to the list);
+ *   - repeat: take the first list member that has not been expanded, mark it expanded, and visit each of its graph
+ *     neighbours that has not been visited before; stop when every list member is expanded, or after
+ *     max_expansions expansions;
+ *   - a visited centroid enters the list if the list is not full or it ranks before the last member, which is then
+ *     dropped (a dropped centroid stays visited and is never scored again).
+ * The score is the exact fixed-point S_fx(q, c), so the outcome does not depend on evaluation order.
+ * Outputs: probes / scores = the first nprobe list members (requires nprobe <= beam and nprobe <= n_entries <= K);
+ * visited[c] = 1 for every scored centroid.  Returns the number of visited centroids. */
+int64_t oracle_graph_probes(const float *q, const float *cent, int64_t K, int32_t D, const int32_t *graph, int32_t R,
+                            int32_t n_entries, int32_t beam, int64_t max_expansions, int32_t nprobe, int32_t *probes,
+                            int32_t *scores, uint8_t *visited)
+{
+    int64_t *xq = (int64_t *)malloc(sizeof(int64_t) * (size_t)D);
+    for (int d = 0; d < D; ++d) xq[d] = (int64_t)rint((double)q[d] * Q22);
+    si_pair *list = (si_pair *)malloc(sizeof(si_pair) * (size_t)(beam + 1));
+    uint8_t *expanded = (uint8_t *)malloc((size_t)(beam + 1));
+    int32_t size = 0;
+    int64_t n_visited = 0, expansions = 0;
+    memset(visited, 0, (size_t)K);
+    for (int64_t step = -n_entries;; ++step) {
+        /* the centroids to visit in this step: one entry point, or the neighbours of the member to expand */
+        int32_t one, count;
+        const int32_t *todo;
+        if (step < 0) {
+            one = (int32_t)(((int64_t)(step + n_entries) * K) / n_entries);
+            todo = &one;
+            count = 1;
+        } else {
+            int32_t p = -1;
+            for (int32_t m = 0; m < size; ++m)
+                if (!expanded[m]) { p = m; break; }
+            if (p < 0 || expansions == max_expansions) break;
+            expanded[p] = 1;
+            ++expansions;
+            todo = graph + (int64_t)list[p].id * R;
+            count = R;
+        }
+        for (int32_t r = 0; r < count; ++r) {
+            const int32_t n = todo[r];
+            if (visited[n]) continue;
+            visited[n] = 1;
+            ++n_visited;
+            si_pair x;
+            x.s = fx_score(xq, cent + (int64_t)n * D, D);
+            x.id = n;
+            int32_t pos = size;                           /* position of x in the ordered list */
+            while (pos > 0 && cmp_si_desc(&x, &list[pos - 1]) < 0) --pos;
+            if (pos >= beam) continue;                    /* ranks behind a full list */
+            for (int32_t m = size; m > pos; --m) { list[m] = list[m - 1]; expanded[m] = expanded[m - 1]; }
+            list[pos] = x;
+            expanded[pos] = 0;
+            if (size < beam) ++size;                      /* else the former last member fell off */
+        }
+    }
+    for (int32_t r = 0; r < nprobe; ++r) {
+        probes[r] = r < size ? list[r].id : -1;
+        scores[r] = r < size ? list[r].s : INT32_MIN;
+    }
+    free(xq);
+    free(list);
+    free(expanded);
+    return n_visited;
 }
 
 /* ---------------------------------------------------------------- O-5 ------------------------------------------ */
