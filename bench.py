@@ -398,7 +398,70 @@ def run_sharded(args, cfg, pkg, rank, world, local_rank, device):
     dist.destroy_process_group()
 
 
-PRUNING_TEXT = {"ci": "centroid interaction over every candidate token",
+def run_graph_eval(args, cfg, pkg, index, corp, q):
+    """The centroid-graph search against the exhaustive scan it replaces (stage 1 + stage 2a), probe stage alone:
+    time per batch and recall of the exhaustive top-nprobe / of the best centroid, for several (entry points, list
+    size), on the workload's own centroids and on a structured centroid set of the same size (unit vectors of an
+    8-dimensional subspace, where a nearest-neighbour graph has local structure to navigate by; the workloads'
+    centroids are near-orthogonal random directions).  One JSON line per point."""
+    dev = q.device
+    B, nq, P, R = args.batch, cfg.q_len, cfg.nprobe, args.graph_degree
+    qb = q[:B].contiguous()
+
+    def timed(fn, reps=5):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    def evaluate(name, ix, queries):
+        taps = ix.alloc_taps(B, nq, P, 16, max_candidates=1024, table=False, ci=False)
+        ix.run_stages(1, 2, queries, B, nq, P, 16, 1, taps, max_candidates=1024)
+        exact = taps.probes.clone()
+        pkg.profile_enable(True)
+        pkg.profile_read()
+        for _ in range(3):
+            ix.run_stages(1, 2, queries, B, nq, P, 16, 1, taps, max_candidates=1024)
+        ms, _ = pkg.profile_read()
+        pkg.profile_enable(False)
+        exact_ms = (ms["score_table"] + ms["probes"]) / 3
+        t0 = time.time()
+        ix.build_graph(R)
+        build_s = time.time() - t0
+        for E, beam in ((64, 32), (256, 32), (1024, 32), (4096, 32), (4096, 64), (16384, 64)):
+            if E > ix.K:
+                continue
+            pr, sc, nvis, _ = ix.graph_probes(queries, P, beam, E)
+            ms_g = timed(lambda: ix.graph_probes(queries, P, beam, E))
+            hit = (pr[:, :, :, None] == exact[:, :, None, :]).any(dim=3).float().mean().item()
+            first = (pr[:, :, 0] == exact[:, :, 0]).float().mean().item()
+            print(json.dumps({"graph_eval": name, "n_centroids": ix.K, "degree": R, "n_entries": E, "beam": beam,
+                              "batch": B, "graph_probe_ms": ms_g, "exhaustive_ms": exact_ms,
+                              "probe_recall": hit, "best_centroid_recall": first,
+                              "visited_per_token": float(nvis.float().mean()), "graph_build_s": round(build_s, 2)}))
+
+    evaluate(cfg.name + " centroids (random directions)", index, qb)
+    # structured centroids: unit vectors of a random 8-dimensional subspace; query tokens = a centroid plus noise
+    g = torch.Generator(device=dev)
+    g.manual_seed(1234)
+    basis = torch.linalg.qr(torch.randn(cfg.dim, 8, generator=g, device=dev)).Q            # [D, 8] orthonormal
+    z = torch.randn(cfg.n_centroids, 8, generator=g, device=dev)
+    cent = (z / z.norm(dim=1, keepdim=True)) @ basis.t()
+    qi = torch.randint(0, cfg.n_centroids, (B * nq,), generator=g, device=dev)
+    qs = cent[qi] + 0.02 * torch.randn(B * nq, cfg.dim, generator=g, device=dev)
+    qs = (qs / qs.norm(dim=1, keepdim=True)).view(B, nq, cfg.dim).contiguous()
+    ix2 = pkg.Index(cent.contiguous(), corp.cids[:1024].contiguous(), corp.codes[:1024].contiguous(),
+                    torch.full((16,), 64, dtype=torch.int32, device=dev), cfg.nbits, cfg.res_lo, cfg.res_hi)
+    evaluate("structured centroids (8-dimensional subspace)", ix2, qs)
+
+
+PRUNING_TEXT = {"rabitq_graph": "probes from the centroid graph, then the RaBitQ pipeline",
+                "ci": "centroid interaction over every candidate token",
                 "partial": "partial scores of retrieved tokens (Algorithm 2)",
                 "rabitq": "partial 1-bit RaBitQ scores of retrieved tokens, then complete 1-bit scores"}
 
@@ -408,7 +471,9 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     """Times one workload in one pruning mode on this rank and returns the result fields (QPS at the batch size and at
     batch 1, per-stage CUDA-event times, the roofline of the dominant kernel and of each stage).  full=False leaves
     out the end-to-end run through the host entry point and the CUDA-graph variant of batch 1."""
-    kw = {"partial": mode == "partial", "rabitq": mode == "rabitq"}
+    kw = {"partial": mode == "partial", "rabitq": mode in ("rabitq", "rabitq_graph")}
+    if mode == "rabitq_graph":
+        kw["graph"] = (args.graph_beam, args.graph_entries, 1 << 30)
     B = args.batch if args.batch > 0 else (64 if cfg.name.startswith("long") else 16 if cfg.name == "tiny" else 256)
     nq, P, n_prune, k = cfg.q_len, cfg.nprobe, cfg.n_prune, cfg.k
     steps = args.steps if steps is None else steps
@@ -514,7 +579,9 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     lat = np.array(lat)
     res = {
         "metric": metric_name(cfg, B) + (" with partial-score refinement" if mode == "partial" else "")
-        + (" on RaBitQ 1-bit codes (paper pipeline)" if mode == "rabitq" else ""),
+        + (" on RaBitQ 1-bit codes (paper pipeline)" if mode == "rabitq" else "")
+        + (" on RaBitQ 1-bit codes with probes from the centroid graph (degree %d, %d entry points, list of %d)"
+           % (args.graph_degree, args.graph_entries, args.graph_beam) if mode == "rabitq_graph" else ""),
         "value": qps, "unit": UNIT, "ms_per_step": ms_per_step, "steps": steps, "batch": B,
         "qps_batch1": float(1.0 / lat.mean()),
         "stage_ms_batch1": {name: round(v / min(n1, 256), 4) for name, v in stage_ms1.items()},
@@ -566,8 +633,9 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     # stage 4 reads per survivor token its centroid id + residual code (or its 1-bit code + scale on the RaBitQ path);
     # the centroid term additionally gathers one int32 table row (q_len x 4 B) per token, which is the implementation's
     # traffic, reported beside the method's
-    g4_bytes = mean("pruned_tokens") * ((cfg.dim // 8 + 4.0) if mode == "rabitq" else (4.0 + cfg.code_bytes))
-    g4_row_bytes = 0.0 if mode == "rabitq" else mean("pruned_tokens") * nq * 4.0
+    rq_mode = mode in ("rabitq", "rabitq_graph")
+    g4_bytes = mean("pruned_tokens") * ((cfg.dim // 8 + 4.0) if rq_mode else (4.0 + cfg.code_bytes))
+    g4_row_bytes = 0.0 if rq_mode else mean("pruned_tokens") * nq * 4.0
     stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
     if mode == "ci":
         ratio, src = NCU_DRAM_PER_ALGORITHMIC_BYTE["ci"]
@@ -596,7 +664,7 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
         # 8 B) and the token's code (residual code, or 1-bit code + its 4-byte scale); per candidate document its
         # partial score (4 B).  The table of running maxima is the implementation's, not the method's, and is not
         # counted.  The slot times the clear, the scoring kernel and (RaBitQ) the summation together.
-        code_b = (cfg.dim // 8 + 4.0) if mode == "rabitq" else float(cfg.code_bytes)
+        code_b = (cfg.dim // 8 + 4.0) if rq_mode else float(cfg.code_bytes)
         ps_bytes = mean("retrieved") * (8.0 + code_b) + mean("cand") * 4.0
         frac = gbs(ps_bytes, ci_ms) / peak
         traffic, tk = None, None
@@ -604,7 +672,7 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
             per_query, src = NCU_DRAM_PER_ALGORITHMIC_BYTE["partial"]
             traffic, tk = per_query * B, "stored ncu figure, not measured in this run: " + src + " x batch"
         roofline = {
-            "kernel": ("rabitq_partial_kernel" if mode == "rabitq" else "partial_score_kernel")
+            "kernel": ("rabitq_partial_kernel" if rq_mode else "partial_score_kernel")
             + " (+ its clear kernel): partial scores of the retrieved tokens, Algorithm 2", "bound": "hbm",
             "achieved": gbs(ps_bytes, ci_ms), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": frac,
             "traffic": traffic, "traffic_kind": tk, "ms_per_launch": ci_ms, "algorithmic_bytes_per_launch": ps_bytes,
@@ -643,6 +711,16 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     }
     res["roofline"] = roofline
     res["pruning"] = PRUNING_TEXT[mode]
+    if mode == "rabitq_graph":
+        # how many of the exhaustive top-nprobe centroids (and of the best ones) the graph search found, first batch
+        t = index.alloc_taps(B, nq, P, 16, max_candidates=1024, table=False, ci=False)
+        index.run_stages(1, 2, batches[0], B, nq, P, 16, 1, t, max_candidates=1024)
+        pr, _, nvis, _ = index.graph_probes(batches[0], P, args.graph_beam, args.graph_entries)
+        res["graph"] = {"degree": args.graph_degree, "n_entries": args.graph_entries, "beam": args.graph_beam,
+                        "probe_recall": (pr[:, :, :, None] == t.probes[:, :, None, :]).any(dim=3).float().mean().item(),
+                        "best_centroid_recall": (pr[:, :, 0] == t.probes[:, :, 0]).float().mean().item(),
+                        "visited_per_query_token": float(nvis.float().mean()), "n_centroids": cfg.n_centroids}
+        del t
     return res
 
 
@@ -656,7 +734,7 @@ def summary(r):
             "target_met": r["roofline"]["target"]["met"],
             "stage4_code_frac_of_hbm": per["residual_scores"]["frac"],
             "score_table_frac_of_int8_peak": per["score_table"]["frac"], "probes_frac_of_hbm": per["probes"]["frac"],
-            "clocks": r["clocks"], "gpu_launches": r["gpu_launches"]}
+            "clocks": r["clocks"], "gpu_launches": r["gpu_launches"], **({"graph": r["graph"]} if "graph" in r else {})}
 
 
 def run_other_configs(pkg, args, device, headline_done):
@@ -736,6 +814,13 @@ def main():
                     help="prune with the paper's partial scores (chimera_search_partial) instead of stage 3")
     ap.add_argument("--rabitq", action="store_true",
                     help="the paper's pipeline on RaBitQ 1-bit codes (chimera_search_rabitq)")
+    ap.add_argument("--graph", action="store_true",
+                    help="with --rabitq: probes from the proximity graph over the centroids (chimera_search_rabitq_graph)")
+    ap.add_argument("--graph-eval", action="store_true",
+                    help="graph search vs exhaustive centroid scan: time and probe recall (see run_graph_eval)")
+    ap.add_argument("--graph-degree", type=int, default=32)
+    ap.add_argument("--graph-beam", type=int, default=32)
+    ap.add_argument("--graph-entries", type=int, default=256)
     ap.add_argument("--sweep", action="store_true", help="QPS vs recall over nprobe x n_prune x k (see run_sweep)")
     ap.add_argument("--sweep-queries", type=int, default=200)
     ap.add_argument("--batch1-queries", type=int, default=200)
@@ -758,7 +843,7 @@ def main():
         dry_launch(args, rank, world)
         return
 
-    single = bool(args.config) or args.partial or args.rabitq or args.sweep or args.sharded
+    single = bool(args.config) or args.partial or args.rabitq or args.sweep or args.sharded or args.graph_eval
     cfg = CONFIGS[args.config or HEADLINE]
     if args.docs > 0:
         cfg = cfg.replace(n_docs=args.docs)
@@ -783,7 +868,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    mode = "rabitq" if args.rabitq else ("partial" if args.partial else "ci")
+    mode = ("rabitq_graph" if args.graph else "rabitq") if args.rabitq else ("partial" if args.partial else "ci")
     corp, q, gen_s = build_workload(cfg, device, rabitq=args.rabitq or args.sweep or (not single and world == 1))
     t0 = time.time()
     index = pkg.Index(corp.centroids, corp.cids, corp.codes, corp.doclens, cfg.nbits, cfg.res_lo, cfg.res_hi)
@@ -798,6 +883,14 @@ def main():
         if rank == 0:
             run_sweep(args, cfg, pkg, index, corp, q)
         return
+    if args.graph_eval:
+        if args.batch <= 0:
+            args.batch = 256
+        if rank == 0:
+            run_graph_eval(args, cfg, pkg, index, corp, q)
+        return
+    if args.graph:
+        index.build_graph(args.graph_degree)
 
     r = measure(pkg, cfg, corp, q, index, args, device, mode, dist, local_rank)
     nq = cfg.q_len
@@ -840,6 +933,10 @@ def main():
             index.attach_rabitq(corp.rotation, corp.rq_bits, corp.rq_inv_dot)
             others[cfg.name + "_rabitq"] = summary(measure(pkg, cfg, corp, q, index, args, device, "rabitq",
                                                            steps=max(3, min(args.steps, 10)), batch1_n=50, full=False))
+            index.build_graph(args.graph_degree)
+            others[cfg.name + "_rabitq_graph"] = summary(measure(pkg, cfg, corp, q, index, args, device, "rabitq_graph",
+                                                                 steps=max(3, min(args.steps, 10)), batch1_n=20,
+                                                                 full=False))
         except Exception as e:          # noqa: BLE001
             others[cfg.name + "_paper_pipelines_error"] = "%s: %s" % (type(e).__name__, e)
         index.close()

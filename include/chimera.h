@@ -210,6 +210,44 @@ int chimera_search_rabitq(const chimera_index *index, const float *queries, int3
                           size_t workspace_bytes, void *stream, int32_t *out_ids, float *out_scores,
                           const chimera_taps *taps);
 
+/* ---- Proximity graph over the centroids (Sec. 3.1; Algorithm 1, line searchCAGRA; Sec. 2.3) -----------------------
+ * The paper finds each query token's n_probe centroids by searching a proximity graph built over the IVF centroids
+ * instead of scoring all of them.  Here:
+ *   graph   node c is linked to the `degree` other centroids with the largest fixed-point inner product S_fx(c, c')
+ *           (ties: smaller id), best first;
+ *   search  per query token a best-first search with a bounded list: the entry points floor(j K / n_entries),
+ *           j < n_entries, are visited (scored, marked, offered to the list); then, repeatedly, the first list member not
+ *           yet expanded is expanded -- each of its neighbours that was never visited is visited -- until every member
+ *           is expanded or max_expansions expansions are done; the list keeps the best `beam` visited centroids by
+ *           (S_fx descending, id ascending); the probes are its first nprobe members.
+ * Scores are the exact S_fx of stage 1, so probes, their scores and the set of visited centroids are reproducible bit
+ * for bit; whether the probes are the exhaustive top nprobe depends on the data and on (degree, n_entries, beam).
+ *
+ * chimera_index_build_graph: builds the graph inside the index (cudaMalloc of K * degree * 4 + K * dim * 4 bytes, plus
+ *   about 0.7 GB of temporary memory freed before returning); synchronises the stream.  centroids: device, the same
+ *   [K, dim] float32 array the index was built from.  1 <= degree <= min(63, K - 1).  Query chimera_workspace_bytes
+ *   again afterwards.  Errors: INVALID_ARG, CUDA_ERROR (nothing stays allocated).
+ * chimera_graph_probes: the search alone.  queries: device [n_queries, q_len, dim].  scratch: device,
+ *   chimera_graph_scratch_bytes(...) bytes (one bit per centroid and query token: afterwards the visited sets, row
+ *   t = query * q_len + token, bit c & 31 of word c / 32).  out_probes: device [n_queries, q_len, nprobe] int32 (-1 if
+ *   fewer were visited); out_scores (optional): their S_fx; out_n_visited (optional): [n_queries, q_len] counts.
+ *   nprobe <= beam <= 64, nprobe <= n_entries <= K, max_expansions >= 0.
+ * chimera_search_rabitq_graph: chimera_search_rabitq with these probes in place of stage 1 and stage 2a -- the
+ *   paper's GPU pipeline as Algorithm 1 states it (no score table is built; taps->score_table is not written). */
+int chimera_index_build_graph(chimera_index *index, const float *centroids, int32_t degree, void *stream);
+/* Degree of the index's graph (0 = none) to *out_degree (host); with out_graph non-NULL also a copy of the graph,
+ * [K, degree] int32 row-major, to that device buffer (enqueued on `stream`). */
+int chimera_index_copy_graph(const chimera_index *index, int32_t *out_graph, int32_t *out_degree, void *stream);
+int chimera_graph_scratch_bytes(const chimera_index *index, int32_t n_queries, int32_t q_len, size_t *out);
+int chimera_graph_probes(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                         int32_t nprobe, int32_t beam, int32_t n_entries, int32_t max_expansions, void *scratch,
+                         size_t scratch_bytes, void *stream, int32_t *out_probes, int32_t *out_scores,
+                         int32_t *out_n_visited);
+int chimera_search_rabitq_graph(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                                int32_t nprobe, int32_t k_refine, int32_t k, int64_t max_candidates, int32_t beam,
+                                int32_t n_entries, int32_t max_expansions, void *workspace, size_t workspace_bytes,
+                                void *stream, int32_t *out_ids, float *out_scores, const chimera_taps *taps);
+
 /* Device-side status of the last search that used this workspace: synchronises the stream, then writes CHIMERA_OK,
  * CHIMERA_CAPACITY_OVERFLOW (some query had more than max_candidates candidates; its results are computed on the
  * first max_candidates of them and are not the specified output), CHIMERA_INVALID_ARG (a query element outside

@@ -195,10 +195,50 @@ class Index:
                                                      _stream()))
         self._ws = None
 
+    def build_graph(self, degree: int):
+        """Build the proximity graph over the centroids (chimera_index_build_graph) for graph_probes() and
+        search(..., rabitq=True, graph=...)."""
+        with torch.cuda.device(self.device):
+            _check(lib().chimera_index_build_graph(self._h, _ptr(self.centroids), ctypes.c_int32(degree), _stream()))
+        self._ws = None
+
+    def graph(self) -> Optional[torch.Tensor]:
+        """A copy of the centroid graph, [K, degree] int32 (None before build_graph)."""
+        deg = ctypes.c_int32()
+        _check(lib().chimera_index_copy_graph(self._h, None, ctypes.byref(deg), _stream()))
+        if deg.value == 0:
+            return None
+        out = torch.empty(self.K, deg.value, dtype=torch.int32, device=self.device)
+        with torch.cuda.device(self.device):
+            _check(lib().chimera_index_copy_graph(self._h, _ptr(out), ctypes.byref(deg), _stream()))
+        return out
+
+    def graph_probes(self, queries: torch.Tensor, nprobe: int, beam: int, n_entries: int, max_expansions: int = 1 << 30):
+        """The graph search alone (chimera_graph_probes).  Returns (probes [B, q_len, nprobe] int32, their fixed-point
+        scores, visited counts [B, q_len] int32, visited bitmaps [B * q_len, ceil(K / 32)] int32)."""
+        assert queries.is_cuda and queries.dtype == torch.float32 and queries.is_contiguous()
+        B, q_len, dim = queries.shape
+        assert dim == self.dim
+        need = ctypes.c_size_t()
+        _check(lib().chimera_graph_scratch_bytes(self._h, ctypes.c_int32(B), ctypes.c_int32(q_len), ctypes.byref(need)))
+        vis = torch.empty(need.value // 4, dtype=torch.int32, device=self.device)
+        probes = torch.empty(B, q_len, nprobe, dtype=torch.int32, device=self.device)
+        scores = torch.empty(B, q_len, nprobe, dtype=torch.int32, device=self.device)
+        n_vis = torch.empty(B, q_len, dtype=torch.int32, device=self.device)
+        with torch.cuda.device(self.device):
+            _check(lib().chimera_graph_probes(self._h, _ptr(queries), ctypes.c_int32(B), ctypes.c_int32(q_len),
+                                              ctypes.c_int32(nprobe), ctypes.c_int32(beam), ctypes.c_int32(n_entries),
+                                              ctypes.c_int32(min(max_expansions, (1 << 31) - 1)), _ptr(vis),
+                                              ctypes.c_size_t(need.value), _stream(), _ptr(probes), _ptr(scores),
+                                              _ptr(n_vis)))
+        return probes, scores, n_vis, vis.view(B * q_len, -1)
+
     def search(self, queries: torch.Tensor, nprobe: int, n_prune: int, k: int, max_candidates: int = 0,
-               taps: Optional[Taps] = None, out=None, partial: bool = False, rabitq: bool = False):
+               taps: Optional[Taps] = None, out=None, partial: bool = False, rabitq: bool = False, graph=None):
         """queries: [B, q_len, dim] float32 CUDA tensor.  Returns (ids [B,k] int32, scores [B,k] float32).
-        partial=True prunes with the paper's partial scores (chimera_search_partial)."""
+        partial=True prunes with the paper's partial scores (chimera_search_partial); rabitq=True runs the paper's
+        pipeline on 1-bit codes, with graph=(beam, n_entries, max_expansions) taking its probes from the centroid graph
+        (chimera_search_rabitq_graph)."""
         assert queries.is_cuda and queries.dtype == torch.float32 and queries.is_contiguous()
         B, q_len, dim = queries.shape
         assert dim == self.dim
@@ -212,7 +252,14 @@ class Index:
         args = (self._h, _ptr(queries), ctypes.c_int32(B), ctypes.c_int32(q_len), ctypes.c_int32(nprobe),
                 ctypes.c_int32(n_prune), ctypes.c_int32(k), ctypes.c_int64(max_candidates), _ptr(ws),
                 ctypes.c_size_t(ws.numel()), _stream(), _ptr(ids), _ptr(scores))
-        if partial or rabitq:
+        if graph is not None:
+            assert rabitq, "graph probes belong to the RaBitQ pipeline"
+            c = taps._c() if taps is not None else None
+            beam, n_entries, max_exp = graph
+            _check(lib().chimera_search_rabitq_graph(*args[:8], ctypes.c_int32(beam), ctypes.c_int32(n_entries),
+                                                     ctypes.c_int32(min(max_exp, (1 << 31) - 1)), *args[8:],
+                                                     ctypes.byref(c) if c is not None else None))
+        elif partial or rabitq:
             c = taps._c() if taps is not None else None
             fn = lib().chimera_search_rabitq if rabitq else lib().chimera_search_partial
             _check(fn(*args, ctypes.byref(c) if c is not None else None))

@@ -137,6 +137,7 @@ Layout make_layout(const Index &ix, const Params &p)
         if (ix.rot_t && bytes < dense) bytes = dense;
         L.partial_m = take(bytes);
     }
+    L.graph_vis = take(ix.graph ? graph_scratch_bytes(ix, (int64_t)p.B * p.nq) : 0);
     L.q_rot = take(ix.rot_t ? B * nq * ix.D * sizeof(float) : 0);
     L.qdig_rot = take(ix.rot_t ? 3 * B * nq * 128 : 0);
     L.n_pruned = take(B * sizeof(int32_t));
@@ -209,8 +210,15 @@ static int copy_d2d(void *dst, const void *src, size_t bytes, cudaStream_t st)
 
 static int run(const Index &ix, const Params &p, int first, int last, const float *queries, void *workspace,
                size_t workspace_bytes, cudaStream_t st, const chimera_taps *taps, int32_t *out_ids, float *out_scores,
-               bool partial = false, bool rabitq = false, bool resume = false)
+               bool partial = false, bool rabitq = false, bool resume = false, const GraphSearch *graph = nullptr)
 {
+    // graph: the probes come from a search of the centroid graph; stage 1 and stage 2a do not run (only the RaBitQ
+    // pipeline can do without the score table)
+    if (graph && (!rabitq || first > 1)) return fail(CHIMERA_INVALID_ARG, "graph probes are for the RaBitQ pipeline");
+    if (graph) {
+        const int grc = check_graph_params(ix, *graph, p.P);
+        if (grc) return grc;
+    }
     // resume: stages before `first` ran in an earlier call on this workspace with the same parameters and their
     // results are still there (document-sharded search: the exchange happens between the two calls)
     if (partial && !ix.tok_id)
@@ -287,12 +295,18 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     }
     prof_mark(SLOT_MISC, st);
 
-    if (first <= 1 && last >= 1) {
+    if (first <= 1 && last >= 1 && !graph) {
         if ((rc = launch_score_table(ix, p, queries, qdig, table, table8, status, st))) return rc;
         prof_mark(SLOT_G1, st);
     }
     if (first <= 2 && last >= 2) {
-        if ((rc = launch_probes(ix, p, L, table, part, probes, st))) return rc;
+        if (graph) {
+            if ((rc = launch_graph_probes(ix, queries, (int64_t)p.B * p.nq, p.P, *graph, (uint32_t *)(ws + L.graph_vis),
+                                          probes, nullptr, nullptr, st)))
+                return rc;
+        } else if ((rc = launch_probes(ix, p, L, table, part, probes, st))) {
+            return rc;
+        }
         prof_mark(SLOT_PROBE, st);
         if ((rc = launch_gather(ix, p, L, probes, bitmap, chunk_cnt, cand, n_cand, word_rank, status, st))) return rc;
         prof_mark(SLOT_GATHER, st);
@@ -368,7 +382,9 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     }
 
     if (taps) {
-        if (taps->score_table && first <= 1 && last >= 1 && (rc = copy_d2d(taps->score_table, table, table_bytes, st))) return rc;
+        if (taps->score_table && first <= 1 && last >= 1 && !graph &&
+            (rc = copy_d2d(taps->score_table, table, table_bytes, st)))
+            return rc;
         if (first <= 2 && last >= 2) {
             if (taps->probes && (rc = copy_d2d(taps->probes, probes, B * p.nq * p.P * sizeof(int32_t), st))) return rc;
             if (taps->cand && (rc = copy_d2d(taps->cand, cand, cand_bytes, st))) return rc;
@@ -503,6 +519,71 @@ int chimera_search_rabitq(const chimera_index *index, const float *queries, int3
                false, true);
 }
 
+// ---- centroid graph ---------------------------------------------------------------------------------------------
+int chimera_index_build_graph(chimera_index *index, const float *centroids, int32_t degree, void *stream)
+{
+    Index *ix = reinterpret_cast<Index *>(index);
+    if (!ix || !centroids) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if ((uintptr_t)centroids & 15) return fail(CHIMERA_INVALID_ARG, "centroids must be 16-byte aligned");
+    return build_graph(*ix, centroids, degree, (cudaStream_t)stream);
+}
+
+int chimera_index_copy_graph(const chimera_index *index, int32_t *out_graph, int32_t *out_degree, void *stream)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    if (!ix || !out_degree) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    *out_degree = ix->graph_deg;
+    if (out_graph && ix->graph)
+        CHIMERA_CUDA(cudaMemcpyAsync(out_graph, ix->graph, sizeof(int32_t) * (size_t)ix->K * ix->graph_deg,
+                                     cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return CHIMERA_OK;
+}
+
+int chimera_graph_scratch_bytes(const chimera_index *index, int32_t n_queries, int32_t q_len, size_t *out)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    if (!ix || !out) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if (n_queries < 1 || q_len < 1 || q_len > CHIMERA_MAX_QLEN) return fail(CHIMERA_INVALID_ARG, "n_queries or q_len out of range");
+    *out = graph_scratch_bytes(*ix, (int64_t)n_queries * q_len);
+    return CHIMERA_OK;
+}
+
+int chimera_graph_probes(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                         int32_t nprobe, int32_t beam, int32_t n_entries, int32_t max_expansions, void *scratch,
+                         size_t scratch_bytes, void *stream, int32_t *out_probes, int32_t *out_scores,
+                         int32_t *out_n_visited)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    if (!ix || !queries || !scratch || !out_probes) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    if ((uintptr_t)queries & 15) return fail(CHIMERA_INVALID_ARG, "queries must be 16-byte aligned");
+    if (n_queries < 1 || q_len < 1 || q_len > CHIMERA_MAX_QLEN || nprobe < 1 || nprobe > CHIMERA_MAX_NPROBE)
+        return fail(CHIMERA_INVALID_ARG, "n_queries, q_len or nprobe out of range");
+    GraphSearch g;
+    g.beam = beam; g.n_entries = n_entries; g.max_expansions = max_expansions;
+    int rc = check_graph_params(*ix, g, nprobe);
+    if (rc) return rc;
+    const int64_t tokens = (int64_t)n_queries * q_len;
+    if (scratch_bytes < graph_scratch_bytes(*ix, tokens))
+        return fail(CHIMERA_WORKSPACE_TOO_SMALL, "scratch has %zu bytes, %zu needed", scratch_bytes, graph_scratch_bytes(*ix, tokens));
+    return launch_graph_probes(*ix, queries, tokens, nprobe, g, (uint32_t *)scratch, out_probes, out_scores, out_n_visited,
+                               (cudaStream_t)stream);
+}
+
+int chimera_search_rabitq_graph(const chimera_index *index, const float *queries, int32_t n_queries, int32_t q_len,
+                                int32_t nprobe, int32_t k_refine, int32_t k, int64_t max_candidates, int32_t beam,
+                                int32_t n_entries, int32_t max_expansions, void *workspace, size_t workspace_bytes,
+                                void *stream, int32_t *out_ids, float *out_scores, const chimera_taps *taps)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, k_refine, k, max_candidates, &p);
+    if (rc) return rc;
+    GraphSearch g;
+    g.beam = beam; g.n_entries = n_entries; g.max_expansions = max_expansions;
+    return run(*ix, p, 1, 5, queries, workspace, workspace_bytes, (cudaStream_t)stream, taps, out_ids, out_scores,
+               false, true, false, &g);
+}
+
 // ---- document-sharded search ------------------------------------------------------------------------------------
 static int shard_mode(int32_t mode, bool *partial, bool *rabitq)
 {
@@ -576,6 +657,8 @@ int chimera_destroy_index(chimera_index *index)
 {
     Index *ix = reinterpret_cast<Index *>(index);
     if (!ix) return CHIMERA_OK;
+    cudaFree(ix->graph);
+    cudaFree(ix->xc);
     cudaFree(ix->rot_t);
     cudaFree(ix->tok_off);
     cudaFree(ix->tok_id);

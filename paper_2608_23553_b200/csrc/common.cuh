@@ -34,6 +34,15 @@ struct Index {
     const uint8_t *rq_bits = nullptr; // [T, D/8]   borrowed: sign bits of the rotated tokens
     const float *rq_inv = nullptr;    // [T]        borrowed: 1 / <o_p, o_p-bar>
     float *rot_t = nullptr;           // [D][D]     owned: transposed rotation, rot_t[x * D + r] = P[r][x]
+    // proximity graph over the centroids (only after chimera_index_build_graph)
+    int32_t *graph = nullptr;         // [K][graph_deg] owned: nearest other centroids of each centroid, best first
+    int32_t *xc = nullptr;            // [K][D]     owned: rint(centroid * 2^22)
+    int graph_deg = 0;
+};
+
+// Parameters of the graph search that can stand in for stage 1 + stage 2a (g7_graph.cu).
+struct GraphSearch {
+    int32_t beam = 0, n_entries = 0, max_expansions = 0;
 };
 
 // Device status bits kept in the first word of a workspace.
@@ -78,6 +87,7 @@ struct Layout {
     size_t partial_m;     // int32  [B][maxc][nq]     per (candidate, query token) best retrieved-token score, or
                           // uint64 [B][hash_slots]   the same as an open-addressing table (see partial_hash_slots)
     int64_t hash_slots;   // slots per query of that table; 0 = the dense form
+    size_t graph_vis;     // uint32 [B*nq][K/32]      visited centroids of the graph search (only with a centroid graph)
     size_t q_rot;         // float  [B, nq, D]        rotated queries (RaBitQ pipeline)
     size_t qdig_rot;      // int8   [3][B*nq][128]    their digit planes
     size_t n_pruned;      // int32  [B]
@@ -182,6 +192,13 @@ int launch_residual_scores_umma(const Index &ix, const Params &p, const float *q
                                 cudaStream_t st);
 int launch_rabitq_scores_umma(const Index &ix, const Params &p, const float *q_rot, const int8_t *qdig_rot,
                               const int32_t *pruned, float *score4, uint32_t *status, cudaStream_t st);
+// g7_graph.cu
+int build_graph(Index &ix, const float *centroids, int degree, cudaStream_t st);
+size_t graph_scratch_bytes(const Index &ix, int64_t n_tokens);
+int check_graph_params(const Index &ix, const GraphSearch &g, int nprobe);
+// visited: graph_scratch_bytes(ix, n_tokens) bytes; out_scores / out_nvis may be NULL.
+int launch_graph_probes(const Index &ix, const float *queries, int64_t n_tokens, int nprobe, const GraphSearch &g,
+                        uint32_t *visited, int32_t *out_probes, int32_t *out_scores, int32_t *out_nvis, cudaStream_t st);
 // rabitq.cu
 int attach_rabitq(Index &ix, const float *rotation, cudaStream_t st);
 int launch_rotate(const Index &ix, const Params &p, const float *queries, float *q_rot, cudaStream_t st);
