@@ -80,7 +80,8 @@ const char *chimera_last_error(void);
 
 /* Build the device-resident index (offline step; Sec. 3.1: centroids, posting lists, per-token codes).
  *   desc       host pointer.
- *   centroids  device, 16-byte aligned, [K, dim] float32 row-major, unit-norm rows (every |element| <= 1).  Copied (as fixed-point
+ *   centroids  device, 16-byte aligned, [K, dim] float32 row-major, unit-norm rows (every |element| <= 1 and norm <= 1 + 2^-10:
+ *              checked, INVALID_ARG otherwise).  Copied (as fixed-point
  *              digits); may be freed after the call returns.
  *   cids       device, [T] int32 in [0, K), document-major (document 0's tokens first).  REFERENCED, not copied:
  *              must outlive the index.
@@ -109,7 +110,8 @@ int chimera_workspace_bytes(const chimera_index *index, int32_t n_queries, int32
 
 /* Stages 1-5 for a batch of queries (Algorithm 1 with the stage list at the top of this file).
  *   queries     device, 16-byte aligned, [n_queries, q_len, dim] float32, unit-norm rows (the library does not
- *               normalise).
+ *               normalise; an element outside [-1, 1] or a row longer than 1 + 2^-10 is reported by
+ *               chimera_workspace_status as CHIMERA_INVALID_ARG and the results are then unspecified).
  *   workspace   device, 256-byte aligned, at least chimera_workspace_bytes(...) bytes; contents are scratch.  Two
  *               calls that may overlap on the device need distinct workspaces.
  *   out_ids     device, [n_queries, k] int32: best first; -1 where fewer than k documents survive.
@@ -313,8 +315,9 @@ int chimera_profile_read(float *ms, int64_t *launches);
  * enqueue nothing (use chimera_search with a workspace).  Other argument limits are those of chimera_search.
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device current)
- * and caches it; make that first call before starting any stream capture.  The call itself allocates and frees
- * nothing.  All calls share the one array per device and it keeps the previous call's contents: the kernels overwrite
+ * and caches it; under lazy module loading that first call may also make the CUDA runtime load the library's kernels
+ * and place the array, so make it once at start-up, before any stream capture and before memory is frozen.  After
+ * that a call allocates and frees nothing.  A cached address does not survive cudaDeviceReset.  All calls share the one array per device and it keeps the previous call's contents: the kernels overwrite
  * every entry they later read, so no clearing is needed, but two calls whose kernels may overlap on the same device
  * (different streams, or concurrent host threads) race on it -- serialise them. */
 int chimera_probes_static(const int32_t *score_table, int64_t n_centroids, int32_t n_queries, int32_t q_len,

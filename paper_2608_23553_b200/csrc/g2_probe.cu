@@ -5,6 +5,8 @@
 // thread keeps a sorted list of its best P keys in shared memory (column layout list[j][thread], conflict-free); a
 // key is a 64-bit integer whose order is (score desc, id asc).  Pass 1 turns slices of the table into partial lists,
 // pass 2 folds the partial lists of a query into the final P per token.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace chimera {
@@ -205,7 +207,9 @@ constexpr int STATIC_MAX_DEVICES = 64;
 // Device address of g_probe_scratch on each device (0 = not looked up yet).  In host code the symbol's name is only a
 // handle for the runtime, not a device address: it must be translated with cudaGetSymbolAddress, with the device in
 // question current, before a kernel can be given it.
-static unsigned long long *g_probe_scratch_ptr[STATIC_MAX_DEVICES] = {nullptr};
+// Host threads may make their first calls at the same time: the entries are atomics (every writer stores the same
+// address, so relaxed ordering is enough).  A cached address does not survive cudaDeviceReset.
+static std::atomic<unsigned long long *> g_probe_scratch_ptr[STATIC_MAX_DEVICES];
 
 }  // namespace chimera
 
@@ -224,12 +228,13 @@ extern "C" int chimera_probes_static(const int32_t *score_table, int64_t n_centr
     CHIMERA_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= STATIC_MAX_DEVICES) return fail(CHIMERA_UNSUPPORTED, "device ordinal %d is not supported", dev);
     CHIMERA_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    if (!g_probe_scratch_ptr[dev]) {          // first call on this device (it is the current one)
+    unsigned long long *part = g_probe_scratch_ptr[dev].load(std::memory_order_relaxed);
+    if (!part) {                              // first call on this device (it is the current one)
         void *p = nullptr;
         CHIMERA_CUDA(cudaGetSymbolAddress(&p, g_probe_scratch));
-        g_probe_scratch_ptr[dev] = static_cast<unsigned long long *>(p);
+        part = static_cast<unsigned long long *>(p);
+        g_probe_scratch_ptr[dev].store(part, std::memory_order_relaxed);
     }
-    unsigned long long *part = g_probe_scratch_ptr[dev];
 
     // same slicing rule as the workspace-based stage: about four blocks per SM over the batch, at most 512 per query,
     // at least ~256 rows per block; one partial list per block

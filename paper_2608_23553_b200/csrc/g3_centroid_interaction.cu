@@ -227,11 +227,13 @@ ci_wide_rng_kernel(const int32_t *__restrict__ table, int64_t K, const int2 *__r
 // ------------------------------------------------------------------------------------------------ coarse bounds --
 // Bounds on CI from the 8-bit table U8[c, i] = clamp(S[c, i] >> 16, 0, 255) (stage 1 writes it next to the exact
 // table): 256 buckets of width 2^16 over [0, 2^24), everything negative in bucket 0, everything from 255 * 2^16 up in
-// bucket 255 (|S| <= 2^24 + 64).  The map is monotone, so m_i = max_t U8[cid_t, i] is the bucket of the exact maximum:
+// bucket 255.  |S| <= 2^24 + 2^16 = SMAX: queries and centroids are at most unit-norm up to 2^-10 (checked where their
+// fixed-point digits are made; a longer row is reported through the status word).  The map is monotone, so
+// m_i = max_t U8[cid_t, i] is the bucket of the exact maximum:
 //     2^16 m_i <= max_t S <= 2^16 m_i + 2^16 - 1        for 0 < m_i < 255,
-// the lower end drops to -(2^24 + 64) for m_i = 0 and the upper end rises to 2^24 + 64 for m_i = 255.  With
+// the lower end drops to -SMAX for m_i = 0 and the upper end rises to SMAX = 2^16 * 255 + 2^17 for m_i = 255.  With
 // sum = sum_i m_i, zeros = #{i : m_i = 0}, sat = #{i : m_i = 255}:
-//     lo(d) = 2^16 sum - zeros (2^24 + 64)  <=  CI(d)  <=  2^16 sum + nq (2^16 - 1) + 65 sat = hi(d).
+//     lo(d) = 2^16 sum - zeros SMAX  <=  CI(d)  <=  2^16 sum + nq (2^16 - 1) + (2^16 + 1) sat = hi(d).
 // (The scores that decide a maximum are positive -- a document token close to the query token -- so the buckets are
 // spent on [0, 1) and a column whose best score is negative only loosens lo.)  A row of U8 is q_len bytes -- one
 // 32-byte sector for 32 query
@@ -241,11 +243,11 @@ ci_wide_rng_kernel(const int32_t *__restrict__ table, int64_t K, const int2 *__r
 // packed = sum | sat << 16 | zeros << 24 (see above)
 __device__ __forceinline__ int32_t coarse_lo(int packed)
 {
-    return ((packed & 0xffff) << 16) - (packed >> 24) * ((1 << 24) + 64);
+    return ((packed & 0xffff) << 16) - (packed >> 24) * ((1 << 24) + (1 << 16));
 }
 __device__ __forceinline__ int32_t coarse_hi(int packed, int nq)
 {
-    return ((packed & 0xffff) << 16) + nq * ((1 << 16) - 1) + ((packed >> 16) & 0xff) * 65;
+    return ((packed & 0xffff) << 16) + nq * ((1 << 16) - 1) + ((packed >> 16) & 0xff) * ((1 << 16) + 1);
 }
 // The histogram key of a lower bound in the contender step: floor(lo / 2^16) clamped at 0 -- a valid, slightly smaller
 // lower bound (documents with an empty column fall to the bottom, which only lowers the threshold).

@@ -111,18 +111,25 @@ static int exclusive_scan(const int32_t *in, int64_t n, int64_t *out, int64_t *t
 // X = rint(x * 2^22) split into balanced base-256 digits X = d0 + 256 d1 + 65536 d2, d0, d1 in [-128, 127],
 // |d2| <= 64.  Planes have a fixed row pitch of DIGIT_PITCH (128) bytes, dimensions >= D are zero:
 // plane p of row r, dimension d sits at dig[(p * rows + r) * 128 + d].
+// Rows must also be (at most) unit-norm: later stages rely on |S_fx| <= 2^24 + 2^16, which holds when both factors
+// have sum_d X[d]^2 <= 2^44 + 2^35 (norm <= 1 + 2^-10).  A longer row sets the same status bit as an element out of
+// range.  A block of 256 threads holds two rows (one thread per padded dimension).
 constexpr int DIGIT_PITCH = 128;
+constexpr long long MAX_ROW_SQUARE_SUM = (1LL << 44) + (1LL << 35);
 
 __global__ void digits_kernel(const float *__restrict__ x, int64_t rows, int D, int8_t *__restrict__ dig,
                               uint32_t *status)
 {
+    __shared__ unsigned long long row_sq[2];
     const int64_t n = rows * DIGIT_PITCH;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
+    if (threadIdx.x < 2) row_sq[threadIdx.x] = 0ull;
+    __syncthreads();
     const int64_t r = i / DIGIT_PITCH;
     const int d = (int)(i % DIGIT_PITCH);
     int d0 = 0, d1 = 0, d2 = 0;
-    if (d < D) {
+    unsigned long long sq = 0ull;
+    if (i < n && d < D) {
         float v = x[r * D + d];
         if (!(fabsf(v) <= 1.0f)) {
             if (status) atomicOr(status, ST_BAD_QUERY);
@@ -130,14 +137,23 @@ __global__ void digits_kernel(const float *__restrict__ x, int64_t rows, int D, 
             if (v != v) v = 0.f;
         }
         const int X = __float2int_rn(v * 4194304.0f);
+        sq = (unsigned long long)((long long)X * X);
         d0 = ((X + 128) & 255) - 128;
         const int X1 = (X - d0) >> 8;
         d1 = ((X1 + 128) & 255) - 128;
         d2 = (X1 - d1) >> 8;
     }
-    dig[i] = (int8_t)d0;
-    dig[n + i] = (int8_t)d1;
-    dig[2 * n + i] = (int8_t)d2;
+    if (i < n) {
+        dig[i] = (int8_t)d0;
+        dig[n + i] = (int8_t)d1;
+        dig[2 * n + i] = (int8_t)d2;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if ((threadIdx.x & 31) == 0 && sq) atomicAdd(&row_sq[threadIdx.x / DIGIT_PITCH], sq);
+    __syncthreads();
+    if (threadIdx.x < 2 && row_sq[threadIdx.x] > (unsigned long long)MAX_ROW_SQUARE_SUM && status)
+        atomicOr(status, ST_BAD_QUERY);
 }
 
 int launch_digits(const float *x, int64_t rows, int D, int8_t *dig, uint32_t *status, cudaStream_t st)
@@ -332,7 +348,7 @@ int build_index_device(Index &ix, const float *centroids, const int32_t *doclens
     BUILD_CUDA(cudaMemcpyAsync(&ix.ivf_len, ix.ivf_off + ix.K, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
     BUILD_CUDA(cudaMemcpyAsync(h_flags, flags, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     BUILD_CUDA(cudaStreamSynchronize(st));
-    if (h_flags[0] & ST_BAD_QUERY) { cleanup(); return fail(CHIMERA_INVALID_ARG, "a centroid element lies outside [-1, 1]"); }
+    if (h_flags[0] & ST_BAD_QUERY) { cleanup(); return fail(CHIMERA_INVALID_ARG, "a centroid element lies outside [-1, 1] or a centroid is longer than a unit vector"); }
     BUILD_CUDA(cudaMalloc(&ix.ivf_doc, sizeof(int32_t) * (size_t)(ix.ivf_len > 0 ? ix.ivf_len : 1)));
     BUILD_CUDA(cudaMemsetAsync(count, 0, sizeof(int32_t) * ix.K, st));
     ivf_kernel<1><<<ivf_blocks, 256, 0, st>>>(ix.cids, ix.doc_off, ix.N, count, ix.ivf_off, ix.ivf_doc);

@@ -126,6 +126,22 @@ def test_candidate_overflow_is_reported(chimera):
     bad[0, 0, 0] = 1.5
     gix.search(bad, 8, 10, 5)
     assert gix.status() == 1
+    # a query token twice as long as a unit vector (every element inside [-1, 1]): the stage-3 bounds assume unit
+    # norms, so it is reported as well
+    long_q = q.clone()
+    long_q[0, 2] *= 2.0
+    assert float(long_q.abs().max()) <= 1.0
+    gix.search(long_q, 8, 10, 5)
+    assert gix.status() == 1
+    gix.search(q, 8, 10, 5)
+    assert gix.status() == 0
+    # and a centroid that is not unit-norm is rejected when the index is built
+    cent2 = cent.copy()
+    cent2[5] *= 1.5
+    assert np.abs(cent2).max() <= 1.0
+    with pytest.raises(chimera.ChimeraError) as e:
+        _gpu_index(chimera, cent2, cids, codes, doclens, nbits)
+    assert e.value.code == 1
 
 
 def test_bad_index_arrays_are_rejected(chimera):

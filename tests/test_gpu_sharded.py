@@ -33,7 +33,8 @@ def _emulate(engines, q, nprobe, n_prune, k):
     for m in merged[1:]:                                  # every rank ends with the same answer
         assert torch.equal(m[0], merged[0][0]) and torch.equal(m[1], merged[0][1])
     # the searcher's own sequencing on rank 0, fed by the other ranks' tensors
-    feeds = iter([all_ids, all_sc3, top_ids, top_sc])
+    # (the fifth exchange carries every rank's device status word, so that a failure is raised on all ranks together)
+    feeds = iter([all_ids, all_sc3, top_ids, top_sc, torch.stack([e.status_word() for e in engines])])
     s = ShardedSearcher(engines[0], gather=lambda t: next(feeds))
     ids0, sc0 = s.search(q, nprobe, n_prune, k)
     assert torch.equal(ids0, merged[0][0]) and torch.equal(sc0, merged[0][1])

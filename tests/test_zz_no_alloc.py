@@ -43,6 +43,30 @@ def test_static_probes_match_workspace_probes_on_two_calls_in_a_row():
     assert torch.equal(got_a2, probes_a)
 
 
+def test_static_probes_allocate_no_device_memory():
+    """What the entry point exists for: after one warm-up call (which may load the library's kernels and look the
+    built-in array up), a call straight through the C ABI with a caller-owned output buffer leaves the device's free
+    memory and torch's own allocation count exactly where they were."""
+    import ctypes
+    import paper_2608_23553_b200 as pkg
+    table, probes = _case(pkg, 33, K=1500, N=100, D=32, nq=32, B=2, nprobe=4)
+    out = torch.empty_like(probes)
+    L = pkg.lib()
+    args = (ctypes.c_void_p(table.data_ptr()), ctypes.c_int64(table.shape[1]), ctypes.c_int32(table.shape[0]),
+            ctypes.c_int32(table.shape[2]), ctypes.c_int32(4), ctypes.c_void_p(torch.cuda.current_stream().cuda_stream),
+            ctypes.c_void_p(out.data_ptr()))
+    assert L.chimera_probes_static(*args) == 0                   # warm-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    torch0 = torch.cuda.memory_allocated()
+    for _ in range(3):
+        assert L.chimera_probes_static(*args) == 0
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and torch.cuda.memory_allocated() == torch0
+    assert torch.equal(out, probes)
+
+
 def test_static_probes_reject_sizes_beyond_the_built_in_array():
     import paper_2608_23553_b200 as pkg
     # 64 queries x 10 lists x nprobe 64 x q_len 120 x 8 B is far beyond 4 MiB
