@@ -78,14 +78,16 @@ def measured_int8_tops():
         return 2.0 * 1590.0, "fallback bf16 x 2"
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of one launch of the dominant kernel,
-# from stored ncu captures on small cases (a full-size launch is too large to capture); the profile named beside
-# each figure gives the command.  Every query has its own table and candidate list, so traffic grows in proportion to
-# the algorithmic bytes.
-NCU_DRAM_PER_ALGORITHMIC_BYTE = {
-    "ci": (443.5e6 / 471.0e6, "profiles/ncu_ci_coarse_mid.md (Mid corpus, batch 8)"),
-    "partial": (1527e6 / 64.0, "profiles/ncu_partial_score_mid.md (Mid corpus, batch 64; bytes per query)"),
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from stored ncu
+# captures on small cases (a full-size launch is too large to capture; the profile named beside each figure gives the
+# command).  The stage-3 bound scan reads each query's 8-bit table once (batch x K x q_len bytes) and otherwise moves
+# a fixed number of bytes per algorithmic byte (centroid ids, ranges, ids, bounds), so a full-size launch is
+# ratio x algorithmic bytes + batch x K x q_len.
+NCU_CI_DRAM_PER_ALGORITHMIC_BYTE = {
+    "large": (1.243, "profiles/ncu_ci_coarse_large_slice.md (Large recipe, 1M documents, batch 16)"),
+    None: (0.939, "profiles/ncu_ci_coarse_mid.md (Mid corpus, batch 8)"),
 }
+NCU_PARTIAL_DRAM_PER_QUERY = (1527e6 / 64.0, "profiles/ncu_partial_score_mid.md (Mid corpus, batch 64; bytes per query)")
 
 
 class ClockSampler:
@@ -638,14 +640,14 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     g4_row_bytes = 0.0 if rq_mode else mean("pruned_tokens") * nq * 4.0
     stages = {name: round(v / n_prof, 4) for name, v in stage_ms.items()}
     if mode == "ci":
-        ratio, src = NCU_DRAM_PER_ALGORITHMIC_BYTE["ci"]
+        ratio, src = NCU_CI_DRAM_PER_ALGORITHMIC_BYTE.get(cfg.name, NCU_CI_DRAM_PER_ALGORITHMIC_BYTE[None])
         frac = gbs(ci_bytes, ci_ms) / peak
         roofline = {
             "kernel": "ci_coarse_rng_kernel (stage 3 bound scan over every candidate token)", "bound": "hbm",
             "achieved": gbs(ci_bytes, ci_ms), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": frac,
-            "traffic": ratio * ci_bytes,
-            "traffic_kind": "stored ncu figure, not measured in this run: DRAM bytes per algorithmic byte of " + src
-                            + " x this launch's algorithmic bytes",
+            "traffic": ratio * ci_bytes + float(B) * cfg.n_centroids * nq,
+            "traffic_kind": "stored ncu figure, not measured in this run: %.3f DRAM bytes per algorithmic byte from %s, "
+                            "x this launch's algorithmic bytes, + each query's 8-bit table once" % (ratio, src),
             "ms_per_launch": ci_ms, "algorithmic_bytes_per_launch": ci_bytes,
             "target": {"frac": TARGET, "met": bool(frac >= TARGET),
                        "note": "the task's 60 % of HBM peak for the code-scan stages is NOT met: every 4-byte centroid "
@@ -669,7 +671,7 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
         frac = gbs(ps_bytes, ci_ms) / peak
         traffic, tk = None, None
         if cfg.name == "mid" and mode == "partial":
-            per_query, src = NCU_DRAM_PER_ALGORITHMIC_BYTE["partial"]
+            per_query, src = NCU_PARTIAL_DRAM_PER_QUERY
             traffic, tk = per_query * B, "stored ncu figure, not measured in this run: " + src + " x batch"
         roofline = {
             "kernel": ("rabitq_partial_kernel" if rq_mode else "partial_score_kernel")
@@ -712,6 +714,10 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     res["roofline"] = roofline
     res["pruning"] = PRUNING_TEXT[mode]
     if mode == "rabitq_graph":
+        # stage 1 does not run and the probes slot times the graph search, which streams no table
+        roofline["per_stage"]["score_table"] = {"bound": "not run (probes come from the centroid graph)", "frac": None}
+        roofline["per_stage"]["probes"] = {"bound": "latency of dependent expansions (graph search)", "frac": None,
+                                           "ms_per_launch": pr_ms}
         # how many of the exhaustive top-nprobe centroids (and of the best ones) the graph search found, first batch
         t = index.alloc_taps(B, nq, P, 16, max_candidates=1024, table=False, ci=False)
         index.run_stages(1, 2, batches[0], B, nq, P, 16, 1, t, max_candidates=1024)
