@@ -63,7 +63,8 @@ def test_static_probes_allocate_no_device_memory():
         assert L.chimera_probes_static(*args) == 0
     torch.cuda.synchronize()
     free1, _ = torch.cuda.mem_get_info()
-    assert free1 == free0 and torch.cuda.memory_allocated() == torch0
+    # (free memory is device-wide: it must not have gone down; torch's own count must not have moved at all)
+    assert free1 >= free0 and torch.cuda.memory_allocated() == torch0
     assert torch.equal(out, probes)
 
 
