@@ -770,6 +770,14 @@ def run_other_configs(pkg, args, device, headline_done):
                 out[key] = summary(measure(pkg, cfg, corp, q, index, args, device, mode, steps=steps, batch1_n=50,
                                            full=False))
             index.close()
+            if name in ("tiny", "mid") and not args.no_cpu_baseline:
+                # the oracle on one host core: Tiny all 16 queries, Mid ten queries
+                n_o = 16 if name == "tiny" else 10
+                oix = oracle_index(corp, cfg)
+                n, secs = time_oracle(oix, q.cpu().numpy(), cfg, budget_s=0.0, min_q=n_o, max_q=n_o)
+                out[name]["cpu_baseline"] = {"value": n / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                             "sample": "first %d queries, all stages, %.1f s" % (n, secs)}
+                del oix
             del index, corp, q
         except Exception as e:          # noqa: BLE001
             out[name + "_error"] = "%s: %s" % (type(e).__name__, e)
