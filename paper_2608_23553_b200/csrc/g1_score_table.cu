@@ -33,21 +33,24 @@ constexpr uint32_t G1_A_PLANE = G1_M * G1_ROW_BYTES;      // 16 KB
 constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;      // 6 KB
 constexpr uint32_t G1_SMEM = 3 * G1_A_PLANE + 2 * 3 * G1_B_PLANE + 1024 /* alignment slack */ + 64 /* barriers */;
 
-// floor((a0 + 2^8 a1 + 2^16 a2 + 2^24 a3 + 2^32 a4 + 2^19) / 2^20) in 32-bit arithmetic.  The two high terms are
-// multiples of 2^20 and contribute 2^4 a3 + 2^12 a4.  With a1 = 2^12 h1 + l1 (0 <= l1 < 2^12) and a2 = 2^4 h2 + l2
-// (0 <= l2 < 2^4) -- arithmetic shifts, so this also holds for negative values -- the middle terms are
-// 2^20 (h1 + h2) + 2^8 l1 + 2^16 l2, and what is left under the floor, a0 + 2^8 l1 + 2^16 l2 + 2^19, is below 2^24
-// in magnitude (|a0| < 2^23).  32-bit wrap-around of the sum is harmless: the result fits int32.
+// floor((T + 2^19) / 2^20) with T = a0 + 2^8 a1 + 2^16 a2 + 2^24 a3 + 2^32 a4, in 32-bit arithmetic.  Split T as
+// u + 2^16 v with u = a0 + 2^8 a1 (|a0| < 2^23, |a1| < 2^23: no overflow together with the rounding constant) and
+// v = a2 + 2^8 a3 + 2^16 a4.  v is about T / 2^16, which fits 32 bits whenever the result does (|S| < 2^31 means
+// |T| < 2^51; here |T| < 2^45), so computing it modulo 2^32 loses nothing.  Nested floor divisions compose:
+// floor((x + 2^16 v) / 2^20) = floor((floor(x / 2^16) + v) / 2^4) for any integers x, v; arithmetic right shifts are
+// floor divisions.
 __device__ __forceinline__ int32_t combine_digits(int32_t a0, int32_t a1, int32_t a2, int32_t a3, int32_t a4)
 {
-    const int32_t inner = a0 + ((a1 & 4095) << 8) + ((a2 & 15) << 16) + (1 << 19);
-    return (inner >> 20) + (a1 >> 12) + (a2 >> 4) + a3 * 16 + a4 * 4096;
+    const int32_t u = a0 + (a1 << 8) + (1 << 19);
+    const int32_t v = a2 + (int32_t)((uint32_t)a3 << 8) + (int32_t)((uint32_t)a4 << 16);
+    return ((u >> 16) + v) >> 4;
 }
 
 // grid (ceil(K / 128), n_splits).  Each CTA: centroid tile blockIdx.x, query-row tiles [blockIdx.y * tiles_per_split, ...).
+template <int KS>
 __global__ void __launch_bounds__(G1_THREADS)
 score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_q, int64_t K,
-                 int nq, int64_t q_rows, int k_steps, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
+                 int nq, int64_t q_rows, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
                  uint8_t *__restrict__ table8, uint32_t *status, long long wait_limit, int skip_loads)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -111,17 +114,19 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
             if (ok) ok = mbar_wait(bar_b0 + 8 * stage, (it >> 1) & 1, wait_limit);
             if (ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                for (int w = 0; w < 5; ++w) {              // accumulator = digit weight a + b
-                    bool first = true;
+                // accumulator w = digit weight a + b; fully unrolled, so every descriptor is a base plus a constant
+                const uint64_t da0 = umma_desc(sA), db0 = umma_desc(sB + stage * 3 * G1_B_PLANE);
+#pragma unroll
+                for (int w = 0; w < 5; ++w) {
+#pragma unroll
                     for (int a = 0; a < 3; ++a) {          // query digit
                         const int bdig = w - a;            // centroid digit
                         if (bdig < 0 || bdig > 2) continue;
-                        const uint64_t da = umma_desc(sA + bdig * G1_A_PLANE);
-                        const uint64_t db = umma_desc(sB + (stage * 3 + a) * G1_B_PLANE);
-                        for (int k = 0; k < k_steps; ++k) {
-                            umma_i8(tmem + w * G1_N, da + 2 * k, db + 2 * k, IDESC, first ? 0u : 1u);
-                            first = false;
-                        }
+                        const bool first = (a == (w > 2 ? w - 2 : 0));
+#pragma unroll
+                        for (int k = 0; k < KS; ++k)
+                            umma_i8(tmem + w * G1_N, da0 + (uint64_t)(bdig * (G1_A_PLANE >> 4) + 2 * k),
+                                    db0 + (uint64_t)(a * (G1_B_PLANE >> 4) + 2 * k), IDESC, (first && k == 0) ? 0u : 1u);
                     }
                 }
                 umma_commit(bar_mma);
@@ -168,7 +173,7 @@ score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constan
                     for (int g = 0; g < 2; ++g) {
                         uint32_t v[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) v[e] = (uint32_t)min(max(out[4 * g + e] >> 16, 0), 255);
+                        for (int e = 0; e < 4; ++e) v[e] = (uint32_t)__vimin_s32_relu(out[4 * g + e] >> 16, 255);
                         w[g] = __byte_perm(__byte_perm(v[0], v[1], 0x0040), __byte_perm(v[2], v[3], 0x0040), 0x5410);
                     }
                     // a warp's two chunks are adjacent (16 query tokens of one query): one 16-byte store for the pair
@@ -278,8 +283,6 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     CUtensorMap map_c, map_q;
     if ((rc = make_plane_map(&map_c, ix.cdig, ix.K, G1_M))) return rc;
     if ((rc = make_plane_map(&map_q, qdig, rows, G1_N))) return rc;
-    // per device, so set on every launch (it is a cheap host-side call)
-    CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G1_SMEM));
     const int c_tiles = (int)((ix.K + G1_M - 1) / G1_M);
     const int n_tiles = (int)((rows + G1_N - 1) / G1_N);
     // about eight waves of two CTAs per SM, so the last wave is mostly full
@@ -288,9 +291,22 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     if (splits < 1) splits = 1;
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
     dim3 grid((unsigned)c_tiles, (unsigned)((n_tiles + tiles_per_split - 1) / tiles_per_split));
-    score_table_umma<<<grid, G1_THREADS, G1_SMEM, st>>>(map_c, map_q, ix.K, p.nq, rows, ix.D / 32, n_tiles,
-                                                        tiles_per_split, table, table8, status, wait_limit_cycles(),
-                                                        fault_skip_tma_loads());
+    const long long limit = wait_limit_cycles();
+    const int skip = fault_skip_tma_loads();
+#define CHIMERA_G1_LAUNCH(KS)                                                                                          \
+    do {                                                                                                               \
+        CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
+                                          (int)G1_SMEM));                                                              \
+        score_table_umma<KS><<<grid, G1_THREADS, G1_SMEM, st>>>(map_c, map_q, ix.K, p.nq, rows, n_tiles,               \
+                                                                tiles_per_split, table, table8, status, limit, skip);  \
+    } while (0)
+    switch (ix.D / 32) {                       // MMA steps of 32 dimensions
+    case 1: CHIMERA_G1_LAUNCH(1); break;
+    case 2: CHIMERA_G1_LAUNCH(2); break;
+    case 3: CHIMERA_G1_LAUNCH(3); break;
+    default: CHIMERA_G1_LAUNCH(4); break;
+    }
+#undef CHIMERA_G1_LAUNCH
     CHIMERA_CUDA(cudaGetLastError());
     count_launch(SLOT_G1, 2);
     return CHIMERA_OK;
