@@ -7,14 +7,19 @@
 // them with shifts (in 32-bit arithmetic, see combine_digits) and rounds.
 //
 // The contraction runs on the 5th-generation tensor cores: tcgen05.mma kind::i8 (int8 operands, int32 accumulators in
-// tensor memory), M = 128 centroids x N = 48 query tokens x K = 32 dimensions per instruction.  Both operands are
-// K-major digit planes with a 128-byte row pitch (dimensions beyond D are zero), brought into 128-byte-swizzled shared
-// memory by TMA (plain per-CTA cp.async.bulk.tensor loads, no multicast).  One CTA owns a tile of 128 centroids (its
-// three digit planes stay in shared memory) and walks over tiles of 48 query-token rows, double-buffering the query
-// planes.  The five accumulators take 240 of the 256 tensor-memory columns a CTA allocates, so two CTAs share an SM and
-// one's epilogue overlaps the other's MMAs.  Twelve warps drain the accumulators (three per tensor-memory lane quarter,
-// chunks of eight columns, the next chunk's tcgen05.ld issued ahead) and store 32 bytes of the table per chunk.  Every wait on an mbarrier is bounded; a wait that gives up sets the
-// workspace's TIMEOUT status bit and the CTA frees its tensor memory and returns.
+// tensor memory), M = 128 centroids x N = 32 query tokens x K = 32 dimensions per instruction.  One CTA owns a tile of
+// 128 centroids for its whole life and keeps their three digit planes IN TENSOR MEMORY (the A operand of the
+// instruction is read from there: lane = centroid, 32 bytes per K step), so an instruction fetches only its 1 KB of
+// query digits from shared memory; with the A tile in shared memory every instruction re-read 4 KB of it and the
+// operand fetch, not the arithmetic, set the pace (measured: 51 cycles per instruction at N = 48).  The query planes
+// are K-major rows with a 128-byte pitch (dimensions beyond D are zero), brought into 128-byte-swizzled shared memory
+// by TMA (one plain per-CTA cp.async.bulk.tensor load of all three planes per tile, no multicast), four tiles deep.
+// Tensor memory per CTA: 5 accumulators x 32 columns + 96 columns of centroid digits = 256 columns, so two CTAs share
+// an SM.  A producer warp issues the loads and the MMAs; eight warps drain the accumulators (two per tensor-memory
+// lane quarter, a pair of eight-column chunks each).  A draining warp hands the accumulators back as soon as its
+// tcgen05.ld's have landed in registers, so the next tile's MMAs run while it recombines and stores.  Every wait on
+// an mbarrier is bounded; a wait that gives up sets the workspace's TIMEOUT status bit, and the CTA waits (bounded)
+// for its loads in flight, frees its tensor memory and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -23,15 +28,19 @@
 namespace chimera {
 
 constexpr int G1_M = 128;            // centroids per tile (MMA M)
-constexpr int G1_N = 48;             // query-token rows per tile (MMA N)
+constexpr int G1_N = 32;             // query-token rows per tile (MMA N)
 constexpr int G1_ROW_BYTES = 128;    // digit-plane row pitch = padded dimension count
-constexpr int G1_WPQ = 3;              // warps per tensor-memory lane quarter that drain the accumulators (2: 1.53 ms,
-                                       // 3: 1.43 ms, 6: 1.76 ms on the Mid corpus at batch 256)
-constexpr int G1_THREADS = 128 * G1_WPQ;
+constexpr int G1_WPQ = 2;            // draining warps per tensor-memory lane quarter
+constexpr int G1_DRAIN_WARPS = 4 * G1_WPQ;
+constexpr int G1_THREADS = 32 * (G1_DRAIN_WARPS + 1);      // + the producer warp
+constexpr int G1_STAGES = 4;         // query tiles in flight
 constexpr int G1_TMEM_COLS = 256;
-constexpr uint32_t G1_A_PLANE = G1_M * G1_ROW_BYTES;      // 16 KB
-constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;      // 6 KB
-constexpr uint32_t G1_SMEM = 3 * G1_A_PLANE + 2 * 3 * G1_B_PLANE + 1024 /* alignment slack */ + 64 /* barriers */;
+constexpr int G1_ACC_COLS = 5 * G1_N;                      // accumulators in columns [0, 160)
+constexpr int G1_A_COL = G1_ACC_COLS;                      // centroid digits in columns [160, 256): 32 per plane
+constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;       // 4 KB
+constexpr uint32_t G1_B_STAGE = 3 * G1_B_PLANE;            // 12 KB
+constexpr uint32_t G1_SMEM = G1_STAGES * G1_B_STAGE + 1024 /* alignment slack */ + 64 /* barriers */;
+static_assert(G1_ACC_COLS + 96 <= G1_TMEM_COLS, "accumulators and centroid digits share the allocation");
 
 // floor((T + 2^19) / 2^20) with T = a0 + 2^8 a1 + 2^16 a2 + 2^24 a3 + 2^32 a4, in 32-bit arithmetic.  Split T as
 // u + 2^16 v with u = a0 + 2^8 a1 (|a0| < 2^23, |a1| < 2^23: no overflow together with the rounding constant) and
@@ -46,196 +55,253 @@ __device__ __forceinline__ int32_t combine_digits(int32_t a0, int32_t a1, int32_
     return ((u >> 16) + v) >> 4;
 }
 
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (128 rows = lanes, 32 bytes = 8 columns per K step) from tensor memory
+__device__ __forceinline__ void umma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 // grid (ceil(K / 128), n_splits).  Each CTA: centroid tile blockIdx.x, query-row tiles [blockIdx.y * tiles_per_split, ...).
+// KS = D / 32 MMA steps per digit-plane product.
 template <int KS>
 __global__ void __launch_bounds__(G1_THREADS)
-score_table_umma(const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_q, int64_t K,
-                 int nq, int64_t q_rows, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
+score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtensorMap map_q, int64_t K, int nq,
+                 int64_t q_rows, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
                  uint8_t *__restrict__ table8, uint32_t *status, long long wait_limit, int skip_loads)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sA = base;                                  // 3 planes x 16 KB
-    const uint32_t sB = base + 3 * G1_A_PLANE;                 // 2 stages x 3 planes x 6 KB
-    const uint32_t bars = sB + 2 * 3 * G1_B_PLANE;             // full_a, full_b[2], mma_done
-    const uint32_t bar_a = bars, bar_b0 = bars + 8, bar_mma = bars + 24;
+    const uint32_t sB = base;                                  // G1_STAGES x 3 planes x 4 KB
+    const uint32_t bars = sB + G1_STAGES * G1_B_STAGE;
+    const uint32_t bar_full = bars;                            // [G1_STAGES]: a query tile has landed
+    const uint32_t bar_mma = bars + 8 * G1_STAGES;             // a tile's accumulators are complete
+    const uint32_t bar_empty = bar_mma + 8;                    // every draining warp has the accumulators in registers
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t c0 = (int64_t)blockIdx.x * G1_M;
     const int t_begin = blockIdx.y * tiles_per_split;
     int t_end = t_begin + tiles_per_split;
     if (t_end > n_tiles) t_end = n_tiles;
+    const int my_tiles = t_end > t_begin ? t_end - t_begin : 0;
 
     if (tid == 0) {
-        mbar_init(bar_a, 1);
-        mbar_init(bar_b0, 1);
-        mbar_init(bar_b0 + 8, 1);
+        for (int s = 0; s < G1_STAGES; ++s) mbar_init(bar_full + 8 * s, 1);
         mbar_init(bar_mma, 1);
-        s_abort = 0;
+        mbar_init(bar_empty, G1_DRAIN_WARPS);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
         __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                     "r"(G1_TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc(&s_tmem_base, G1_TMEM_COLS);
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    tc_fence_before();
     __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    tc_fence_after();
     const uint32_t tmem = s_tmem_base;
 
-    // instruction descriptor: D = S32, A and B signed 8-bit, both K-major, N = 48, M = 128
+    // ---- the centroid tile's digit planes into tensor memory: one warp per lane quarter, lane = centroid ------------
+    if (warp < 4) {
+        const int64_t c = c0 + warp * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16) + G1_A_COL;
+        for (int p = 0; p < 3; ++p) {
+            uint32_t r[32];
+            if (c < K) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(cdig + ((int64_t)p * K + c) * G1_ROW_BYTES);
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    const uint4 v = __ldg(src + x);
+                    r[4 * x] = v.x; r[4 * x + 1] = v.y; r[4 * x + 2] = v.z; r[4 * x + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int x = 0; x < 32; ++x) r[x] = 0u;
+            }
+            tmem_st32(lane_addr + p * 32, r);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    // instruction descriptor: D = S32, A and B signed 8-bit, both K-major, N = 32, M = 128
     constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(G1_N >> 3) << 17) |
                                ((uint32_t)(G1_M >> 4) << 24);
 
-    // skip_loads (test hook): no load is issued and no bytes are expected, so the waits below run into their limit
-    // with nothing in flight
-    if (tid == 0 && t_begin < t_end && !skip_loads) {
-        mbar_expect_tx(bar_a, 3 * G1_A_PLANE);
-        for (int p = 0; p < 3; ++p) tma_load_3d(sA + p * G1_A_PLANE, &map_c, 0, (int)c0, p, bar_a);
-        mbar_expect_tx(bar_b0, 3 * G1_B_PLANE);
-        for (int p = 0; p < 3; ++p) tma_load_3d(sB + p * G1_B_PLANE, &map_q, 0, t_begin * G1_N, p, bar_b0);
-    }
-
-    for (int t = t_begin; t < t_end; ++t) {
-        const int it = t - t_begin, stage = it & 1;
-        if (tid == 0) {
+    if (warp == G1_DRAIN_WARPS) {
+        // ================================================================================= producer (one thread) ===
+        if (lane == 0) {
+            // skip_loads (test hook): no load is issued and no bytes are expected, so the first wait below runs into
+            // its limit with nothing in flight
+            int issued = 0;                                    // tiles whose load has been issued
+            auto load_tile = [&](int it) {
+                const uint32_t bar = bar_full + 8 * (it % G1_STAGES);
+                mbar_expect_tx(bar, G1_B_STAGE);
+                tma_load_3d(sB + (it % G1_STAGES) * G1_B_STAGE, &map_q, 0, (t_begin + it) * G1_N, 0, bar);
+            };
+            if (!skip_loads)
+                for (; issued < my_tiles && issued < G1_STAGES; ++issued) load_tile(issued);
             bool ok = true;
-            if (t + 1 < t_end && !skip_loads) {   // the other stage was released by the previous tile's completed MMAs
-                const uint32_t nb = bar_b0 + 8 * (stage ^ 1);
-                mbar_expect_tx(nb, 3 * G1_B_PLANE);
-                for (int p = 0; p < 3; ++p)
-                    tma_load_3d(sB + ((stage ^ 1) * 3 + p) * G1_B_PLANE, &map_q, 0, (t + 1) * G1_N, p, nb);
-            }
-            if (it == 0) ok = mbar_wait(bar_a, 0, wait_limit);
-            if (ok) ok = mbar_wait(bar_b0 + 8 * stage, (it >> 1) & 1, wait_limit);
-            if (ok) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // accumulator w = digit weight a + b; fully unrolled, so every descriptor is a base plus a constant
-                const uint64_t da0 = umma_desc(sA), db0 = umma_desc(sB + stage * 3 * G1_B_PLANE);
+            int it = 0;
+            for (; it < my_tiles; ++it) {
+                const int stage = it % G1_STAGES;
+                ok = mbar_wait(bar_full + 8 * stage, (it / G1_STAGES) & 1, wait_limit);
+                // the previous tile's accumulators are in the draining warps' registers: its MMAs are complete (so
+                // its stage of query digits is free) and tensor memory may be overwritten
+                if (ok && it > 0) ok = mbar_wait(bar_empty, (it - 1) & 1, wait_limit);
+                if (!ok) break;
+                tc_fence_after();
+                // accumulator w = digit weight a + b; fully unrolled, so every operand address is a base plus a constant
+                const uint64_t db0 = umma_desc(sB + stage * G1_B_STAGE);
 #pragma unroll
                 for (int w = 0; w < 5; ++w) {
 #pragma unroll
-                    for (int a = 0; a < 3; ++a) {          // query digit
-                        const int bdig = w - a;            // centroid digit
+                    for (int a = 0; a < 3; ++a) {              // query digit
+                        const int bdig = w - a;                // centroid digit
                         if (bdig < 0 || bdig > 2) continue;
                         const bool first = (a == (w > 2 ? w - 2 : 0));
 #pragma unroll
                         for (int k = 0; k < KS; ++k)
-                            umma_i8(tmem + w * G1_N, da0 + (uint64_t)(bdig * (G1_A_PLANE >> 4) + 2 * k),
-                                    db0 + (uint64_t)(a * (G1_B_PLANE >> 4) + 2 * k), IDESC, (first && k == 0) ? 0u : 1u);
+                            umma_i8_ts(tmem + w * G1_N, tmem + G1_A_COL + bdig * 32 + 8 * k,
+                                       db0 + (uint64_t)(a * (G1_B_PLANE >> 4) + 2 * k), IDESC,
+                                       (first && k == 0) ? 0u : 1u);
                     }
                 }
                 umma_commit(bar_mma);
-            } else {
-                s_abort = 1;
+                // refill the stage that the previous tile used
+                if (it > 0 && issued < my_tiles && !skip_loads) {
+                    load_tile(issued);                         // issued == it - 1 + G1_STAGES: the same stage
+                    ++issued;
+                }
+            }
+            if (!ok) {
                 atomicOr(status, ST_TIMEOUT);
+                // loads in flight write this CTA's shared memory: wait for them (bounded) before leaving
+                if (!skip_loads)
+                    for (int j = it; j < issued; ++j)
+                        mbar_wait(bar_full + 8 * (j % G1_STAGES), (j / G1_STAGES) & 1, wait_limit);
+            } else if (my_tiles > 0) {
+                // the last tile's MMAs read shared memory and tensor memory: complete before the CTA leaves
+                if (!mbar_wait(bar_mma, (my_tiles - 1) & 1, wait_limit)) atomicOr(status, ST_TIMEOUT);
             }
         }
-        __syncwarp();
-        // everybody waits for the accumulators (bounded), then drains them
-        const bool ok = mbar_wait(bar_mma, it & 1, wait_limit);
-        if (!__syncthreads_and(ok && !*(volatile int *)&s_abort)) {      // uniform decision for the whole CTA
-            if (tid == 0) atomicOr(status, ST_TIMEOUT);
-            break;
-        }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        __syncwarp();
+    } else {
+        // ============================================================================================ draining warps ===
         // warp w reads tensor-memory lanes 32 (w % 4) ... + 31 (its centroids); the G1_WPQ warps of a lane quarter
-        // take the chunks of eight query-token columns in turn
+        // take one pair of adjacent eight-column chunks each
         const int quad = warp & 3;
         const int64_t c = c0 + quad * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
         const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
-        // (query, token) coordinates of the tile's first row: one 32-bit division per tile
-        const uint32_t tile_qb = ((uint32_t)t * G1_N) / unq, tile_qi = (uint32_t)t * G1_N - tile_qb * unq;
-        // Each warp takes one pair of adjacent chunks.  The tensor-memory loads of the next
-        // chunk are issued before the current one is recombined and stored, so their latency hides behind that work.
-        uint32_t w8_carry[2] = {0u, 0u};                  // 8-bit words of the even chunk of a pair
-        auto emit = [&](const int32_t (&acc)[5][8], const int chunk) {
-            int32_t out[8];
+        const int first_chunk = 2 * (warp >> 2);
+        for (int it = 0; it < my_tiles; ++it) {
+            const int t = t_begin + it;
+            // (the vote makes the decision uniform: the tensor-memory loads below need the whole warp)
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_mma, it & 1, wait_limit))) {
+                if (lane == 0) atomicOr(status, ST_TIMEOUT);
+                break;
+            }
+            tc_fence_after();
+            int32_t accs[2][5][8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) out[e] = combine_digits(acc[0][e], acc[1][e], acc[2][e], acc[3][e], acc[4][e]);
-            // first query-token row of this chunk and its (query, token) coordinates (rows fit 32 bits:
-            // n_queries * q_len < 2^23)
-            const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)chunk * 8;
-            uint32_t qb = tile_qb, qi = tile_qi + (uint32_t)chunk * 8;      // chunk * 8 < 48: few subtractions
-            while (qi >= unq) { qi -= unq; ++qb; }
-            if (c < K && r0 < rows32) {
-                if (table8 != nullptr) {
-                    // coarse copy for the bound phase of stage 3: clamp(S >> 16, 0, 255); q_len is a multiple
-                    // of 16 here, so the 8 rows of a chunk belong to one query and the store is 8-byte aligned
-                    uint32_t w[2];
+            for (int ch = 0; ch < 2; ++ch)
 #pragma unroll
-                    for (int g = 0; g < 2; ++g) {
-                        uint32_t v[4];
+                for (int w = 0; w < 5; ++w) tmem_ld8(lane_addr + w * G1_N + (first_chunk + ch) * 8, accs[ch][w]);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty);             // the accumulators may be overwritten from here on
+
+            // (query, token) coordinates of the tile's first row: one 32-bit division per tile
+            const uint32_t tile_qb = ((uint32_t)t * G1_N) / unq, tile_qi = (uint32_t)t * G1_N - tile_qb * unq;
+            uint32_t w8_carry[2] = {0u, 0u};                  // 8-bit words of the even chunk of the pair
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) v[e] = (uint32_t)__vimin_s32_relu(out[4 * g + e] >> 16, 255);
-                        w[g] = __byte_perm(__byte_perm(v[0], v[1], 0x0040), __byte_perm(v[2], v[3], 0x0040), 0x5410);
+            for (int ch = 0; ch < 2; ++ch) {
+                const int chunk = first_chunk + ch;
+                int32_t out[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    out[e] = combine_digits(accs[ch][0][e], accs[ch][1][e], accs[ch][2][e], accs[ch][3][e], accs[ch][4][e]);
+                // first query-token row of this chunk and its (query, token) coordinates (rows fit 32 bits:
+                // n_queries * q_len < 2^23)
+                const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)chunk * 8;
+                uint32_t qb = tile_qb, qi = tile_qi + (uint32_t)chunk * 8;      // chunk * 8 < 32: few subtractions
+                while (qi >= unq) { qi -= unq; ++qb; }
+                if (c < K && r0 < rows32) {
+                    if (table8 != nullptr) {
+                        // coarse copy for the bound phase of stage 3: clamp(S >> 16, 0, 255); q_len is a multiple
+                        // of 16 here, so the 8 rows of a chunk belong to one query and the store is 8-byte aligned
+                        uint32_t w[2];
+#pragma unroll
+                        for (int g = 0; g < 2; ++g) {
+                            uint32_t v[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) v[e] = (uint32_t)__vimin_s32_relu(out[4 * g + e] >> 16, 255);
+                            w[g] = __byte_perm(__byte_perm(v[0], v[1], 0x0040), __byte_perm(v[2], v[3], 0x0040), 0x5410);
+                        }
+                        // a warp's two chunks are adjacent (16 query tokens of one query): one 16-byte store for the pair
+                        if (ch == 0) {
+                            w8_carry[0] = w[0];
+                            w8_carry[1] = w[1];
+                        } else {
+                            *reinterpret_cast<uint4 *>(table8 + ((int64_t)qb * K + c) * nq + qi - 8) =
+                                make_uint4(w8_carry[0], w8_carry[1], w[0], w[1]);
+                        }
                     }
-                    // a warp's two chunks are adjacent (16 query tokens of one query): one 16-byte store for the pair
-                    if ((chunk & 1) == 0) {
-                        w8_carry[0] = w[0];
-                        w8_carry[1] = w[1];
-                    } else {
-                        *reinterpret_cast<uint4 *>(table8 + ((int64_t)qb * K + c) * nq + qi - 8) =
-                            make_uint4(w8_carry[0], w8_carry[1], w[0], w[1]);
-                    }
-                }
-                if ((nq & 7) == 0) {
-                    // the chunk's eight values are consecutive tokens of one query, 32-byte aligned: one store
-                    if (r0 < rows32)                                  // q_rows is a multiple of 8 here
+                    if ((nq & 7) == 0) {
+                        // the chunk's eight values are consecutive tokens of one query, 32-byte aligned: one store
                         asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(
                                          table + ((int64_t)qb * K + c) * nq + qi),
                                      "r"(out[0]), "r"(out[1]), "r"(out[2]), "r"(out[3]), "r"(out[4]), "r"(out[5]),
                                      "r"(out[6]), "r"(out[7])
                                      : "memory");
-                } else if ((nq & 3) == 0) {
+                    } else if ((nq & 3) == 0) {
 #pragma unroll
-                    for (int e = 0; e < 8; e += 4) {
-                        if (r0 + e < rows32)                          // q_rows is a multiple of 4 here
-                            *reinterpret_cast<int4 *>(table + ((int64_t)qb * K + c) * nq + qi) =
-                                make_int4(out[e], out[e + 1], out[e + 2], out[e + 3]);
-                        qi += 4;
-                        if (qi >= unq) { qi -= unq; ++qb; }           // groups of four never straddle two queries
-                    }
-                } else {
+                        for (int e = 0; e < 8; e += 4) {
+                            if (r0 + e < rows32)                          // q_rows is a multiple of 4 here
+                                *reinterpret_cast<int4 *>(table + ((int64_t)qb * K + c) * nq + qi) =
+                                    make_int4(out[e], out[e + 1], out[e + 2], out[e + 3]);
+                            qi += 4;
+                            if (qi >= unq) { qi -= unq; ++qb; }           // groups of four never straddle two queries
+                        }
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        if (r0 + e < rows32) table[((int64_t)qb * K + c) * nq + qi] = out[e];
-                        if (++qi == unq) { qi = 0; ++qb; }
+                        for (int e = 0; e < 8; ++e) {
+                            if (r0 + e < rows32) table[((int64_t)qb * K + c) * nq + qi] = out[e];
+                            if (++qi == unq) { qi = 0; ++qb; }
+                        }
                     }
                 }
             }
-        };
-        constexpr int CHUNKS_PER_WARP = (G1_N / 8) / G1_WPQ;
-        static_assert(CHUNKS_PER_WARP == 2, "a warp drains one pair of adjacent chunks");
-        const int first_chunk = 2 * (warp >> 2);
-        int32_t accs[2][5][8];
-#pragma unroll
-        for (int w = 0; w < 5; ++w) tmem_ld8(lane_addr + w * G1_N + first_chunk * 8, accs[0][w]);
-#pragma unroll
-        for (int it = 0; it < CHUNKS_PER_WARP; ++it) {
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (it + 1 < CHUNKS_PER_WARP) {
-#pragma unroll
-                for (int w = 0; w < 5; ++w)
-                    tmem_ld8(lane_addr + w * G1_N + (first_chunk + (it + 1)) * 8, accs[(it + 1) & 1][w]);
-            }
-            emit(accs[it & 1], first_chunk + it);
         }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();                   // accumulators drained before the next tile overwrites them
     }
 
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    tc_fence_before();
     __syncthreads();
     if (warp == 0) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(G1_TMEM_COLS) : "memory");
+        tc_fence_after();
+        tmem_dealloc(tmem, G1_TMEM_COLS);
     }
 }
 
@@ -257,15 +323,15 @@ static EncodeTiledFn encode_fn()
     return fn;
 }
 
-// Digit planes [3][rows][128] int8 as a 3-D tensor (128 bytes, rows, 3 planes); box = (128, box_rows, 1); rows past
-// the end read as zeros.
-int make_plane_map(CUtensorMap *map, const int8_t *planes, int64_t rows, int box_rows)
+// Digit planes [3][rows][128] int8 as a 3-D tensor (128 bytes, rows, 3 planes); box = (128, box_rows, box_planes);
+// rows past the end read as zeros.
+int make_plane_map(CUtensorMap *map, const int8_t *planes, int64_t rows, int box_rows, int box_planes)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return fail(CHIMERA_CUDA_ERROR, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t dims[3] = {(cuuint64_t)G1_ROW_BYTES, (cuuint64_t)rows, 3};
     cuuint64_t strides[2] = {(cuuint64_t)G1_ROW_BYTES, (cuuint64_t)rows * G1_ROW_BYTES};
-    cuuint32_t box[3] = {(cuuint32_t)G1_ROW_BYTES, (cuuint32_t)box_rows, 1};
+    cuuint32_t box[3] = {(cuuint32_t)G1_ROW_BYTES, (cuuint32_t)box_rows, (cuuint32_t)box_planes};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, (void *)planes, dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -280,9 +346,8 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     const int64_t rows = (int64_t)p.B * p.nq;
     int rc = launch_digits(queries, rows, ix.D, qdig, status, st);
     if (rc) return rc;
-    CUtensorMap map_c, map_q;
-    if ((rc = make_plane_map(&map_c, ix.cdig, ix.K, G1_M))) return rc;
-    if ((rc = make_plane_map(&map_q, qdig, rows, G1_N))) return rc;
+    CUtensorMap map_q;
+    if ((rc = make_plane_map(&map_q, qdig, rows, G1_N, 3))) return rc;        // one load brings a tile's three planes
     const int c_tiles = (int)((ix.K + G1_M - 1) / G1_M);
     const int n_tiles = (int)((rows + G1_N - 1) / G1_N);
     // about eight waves of two CTAs per SM, so the last wave is mostly full
@@ -297,7 +362,7 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     do {                                                                                                               \
         CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
                                           (int)G1_SMEM));                                                              \
-        score_table_umma<KS><<<grid, G1_THREADS, G1_SMEM, st>>>(map_c, map_q, ix.K, p.nq, rows, n_tiles,               \
+        score_table_umma<KS><<<grid, G1_THREADS, G1_SMEM, st>>>(ix.cdig, map_q, ix.K, p.nq, rows, n_tiles,                \
                                                                 tiles_per_split, table, table8, status, limit, skip);  \
     } while (0)
     switch (ix.D / 32) {                       // MMA steps of 32 dimensions

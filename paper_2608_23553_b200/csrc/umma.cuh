@@ -102,8 +102,8 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Digit planes [3][rows][128] int8 as a 3-D tensor map (128 bytes, rows, 3 planes); box = (128, box_rows, 1); rows
-// past the end read as zeros.  Host side; defined in g1_score_table.cu.
-int make_plane_map(CUtensorMap *map, const int8_t *planes, int64_t rows, int box_rows);
+// Digit planes [3][rows][128] int8 as a 3-D tensor map (128 bytes, rows, 3 planes); box = (128, box_rows, box_planes);
+// rows past the end read as zeros.  Host side; defined in g1_score_table.cu.
+int make_plane_map(CUtensorMap *map, const int8_t *planes, int64_t rows, int box_rows, int box_planes = 1);
 
 }  // namespace chimera
