@@ -120,6 +120,18 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
 
+    // the first query tiles are requested before the centroid tile is fetched, so the two latencies overlap.
+    // skip_loads (test hook): no load is issued and no bytes are expected, so the producer's first wait runs into its
+    // limit with nothing in flight
+    int issued = 0;                                            // producer thread: tiles whose load has been issued
+    auto load_tile = [&](int it) {
+        const uint32_t bar = bar_full + 8 * (it % G1_STAGES);
+        mbar_expect_tx(bar, G1_B_STAGE);
+        tma_load_3d(sB + (it % G1_STAGES) * G1_B_STAGE, &map_q, 0, (t_begin + it) * G1_N, 0, bar);
+    };
+    if (warp == G1_DRAIN_WARPS && lane == 0 && !skip_loads)
+        for (; issued < my_tiles && issued < G1_STAGES; ++issued) load_tile(issued);
+
     // ---- the centroid tile's digit planes into tensor memory: one warp per lane quarter, lane = centroid ------------
     if (warp < 4) {
         const int64_t c = c0 + warp * 32 + lane;
@@ -152,16 +164,6 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
     if (warp == G1_DRAIN_WARPS) {
         // ================================================================================= producer (one thread) ===
         if (lane == 0) {
-            // skip_loads (test hook): no load is issued and no bytes are expected, so the first wait below runs into
-            // its limit with nothing in flight
-            int issued = 0;                                    // tiles whose load has been issued
-            auto load_tile = [&](int it) {
-                const uint32_t bar = bar_full + 8 * (it % G1_STAGES);
-                mbar_expect_tx(bar, G1_B_STAGE);
-                tma_load_3d(sB + (it % G1_STAGES) * G1_B_STAGE, &map_q, 0, (t_begin + it) * G1_N, 0, bar);
-            };
-            if (!skip_loads)
-                for (; issued < my_tiles && issued < G1_STAGES; ++issued) load_tile(issued);
             bool ok = true;
             int it = 0;
             for (; it < my_tiles; ++it) {
