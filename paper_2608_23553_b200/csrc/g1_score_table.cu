@@ -38,7 +38,8 @@ constexpr int G1_TMEM_COLS = 256;
 constexpr int G1_ACC_COLS = 5 * G1_N;                      // accumulators in columns [0, 160)
 constexpr int G1_A_COL = G1_ACC_COLS;                      // centroid digits in columns [160, 256): 32 per plane
 constexpr uint32_t G1_B_PLANE = G1_N * G1_ROW_BYTES;       // 4 KB
-constexpr uint32_t G1_B_STAGE = 3 * G1_B_PLANE;            // 12 KB
+constexpr uint32_t G1_B_LOAD = 3 * G1_B_PLANE;             // 12 KB: the three digit planes of a tile, one after the other
+constexpr uint32_t G1_B_STAGE = 5 * G1_B_PLANE;            // 20 KB: + 64 rows of zeros (see the MMA schedule)
 constexpr uint32_t G1_SMEM = G1_STAGES * G1_B_STAGE + 1024 /* alignment slack */ + 64 /* barriers */;
 static_assert(G1_ACC_COLS + 96 <= G1_TMEM_COLS, "accumulators and centroid digits share the allocation");
 
@@ -93,7 +94,7 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t s_tmem_base;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sB = base;                                  // G1_STAGES x 3 planes x 4 KB
+    const uint32_t sB = base;                                  // G1_STAGES x (3 planes x 4 KB + 8 KB of zeros)
     const uint32_t bars = sB + G1_STAGES * G1_B_STAGE;
     const uint32_t bar_full = bars;                            // [G1_STAGES]: a query tile has landed
     const uint32_t bar_mma = bars + 8 * G1_STAGES;             // a tile's accumulators are complete
@@ -115,6 +116,13 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
         __syncwarp();
         tmem_alloc(&s_tmem_base, G1_TMEM_COLS);
     }
+    // the 64 zero rows behind each stage's planes (the loads never touch them)
+    for (uint32_t e = tid; e < G1_STAGES * (G1_B_STAGE - G1_B_LOAD) / 16; e += G1_THREADS) {
+        const uint32_t per = (G1_B_STAGE - G1_B_LOAD) / 16;
+        const uint32_t addr = sB + (e / per) * G1_B_STAGE + G1_B_LOAD + (e % per) * 16;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // visible to the tensor core's reads
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -126,7 +134,7 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
     int issued = 0;                                            // producer thread: tiles whose load has been issued
     auto load_tile = [&](int it) {
         const uint32_t bar = bar_full + 8 * (it % G1_STAGES);
-        mbar_expect_tx(bar, G1_B_STAGE);
+        mbar_expect_tx(bar, G1_B_LOAD);
         tma_load_3d(sB + (it % G1_STAGES) * G1_B_STAGE, &map_q, 0, (t_begin + it) * G1_N, 0, bar);
     };
     if (warp == G1_DRAIN_WARPS && lane == 0 && !skip_loads)
@@ -157,9 +165,10 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
     __syncthreads();
     tc_fence_after();
 
-    // instruction descriptor: D = S32, A and B signed 8-bit, both K-major, N = 32, M = 128
-    constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(G1_N >> 3) << 17) |
-                               ((uint32_t)(G1_M >> 4) << 24);
+    // instruction descriptors: D = S32, A and B signed 8-bit, both K-major, M = 128, N = 96 or 160
+    constexpr uint32_t IDESC_BASE = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(G1_M >> 4) << 24);
+    constexpr uint32_t IDESC_3 = IDESC_BASE | ((uint32_t)((3 * G1_N) >> 3) << 17);
+    constexpr uint32_t IDESC_5 = IDESC_BASE | ((uint32_t)((5 * G1_N) >> 3) << 17);
 
     if (warp == G1_DRAIN_WARPS) {
         // ================================================================================= producer (one thread) ===
@@ -174,20 +183,22 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
                 if (ok && it > 0) ok = mbar_wait(bar_empty, (it - 1) & 1, wait_limit);
                 if (!ok) break;
                 tc_fence_after();
-                // accumulator w = digit weight a + b; fully unrolled, so every operand address is a base plus a constant
+                // The stage holds the query's digit planes a = 0, 1, 2 as 96 consecutive B rows, and the accumulators
+                // of weight w = 0..4 are consecutive groups of 32 columns.  One instruction with the centroids' digit
+                // plane b as A and all 96 rows as B therefore adds the products of weight b, b + 1, b + 2 to the
+                // accumulators starting at column 32 b: three instructions per K step instead of nine, which matters
+                // because a single thread issues an instruction only every ~50 cycles.  The very first instruction
+                // runs over 160 rows (the last 64 are zeros) without accumulating, which clears weights 3 and 4.
                 const uint64_t db0 = umma_desc(sB + stage * G1_B_STAGE);
 #pragma unroll
-                for (int w = 0; w < 5; ++w) {
+                for (int k = 0; k < KS; ++k) {
 #pragma unroll
-                    for (int a = 0; a < 3; ++a) {              // query digit
-                        const int bdig = w - a;                // centroid digit
-                        if (bdig < 0 || bdig > 2) continue;
-                        const bool first = (a == (w > 2 ? w - 2 : 0));
-#pragma unroll
-                        for (int k = 0; k < KS; ++k)
-                            umma_i8_ts(tmem + w * G1_N, tmem + G1_A_COL + bdig * 32 + 8 * k,
-                                       db0 + (uint64_t)(a * (G1_B_PLANE >> 4) + 2 * k), IDESC,
-                                       (first && k == 0) ? 0u : 1u);
+                    for (int bdig = 0; bdig < 3; ++bdig) {     // centroid digit
+                        if (k == 0 && bdig == 0)
+                            umma_i8_ts(tmem, tmem + G1_A_COL, db0, IDESC_5, 0u);
+                        else
+                            umma_i8_ts(tmem + bdig * G1_N, tmem + G1_A_COL + bdig * 32 + 8 * k, db0 + (uint64_t)(2 * k),
+                                       IDESC_3, 1u);
                     }
                 }
                 umma_commit(bar_mma);
