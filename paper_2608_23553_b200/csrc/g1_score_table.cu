@@ -7,19 +7,21 @@
 // them with shifts (in 32-bit arithmetic, see combine_digits) and rounds.
 //
 // The contraction runs on the 5th-generation tensor cores: tcgen05.mma kind::i8 (int8 operands, int32 accumulators in
-// tensor memory), M = 128 centroids x N = 32 query tokens x K = 32 dimensions per instruction.  One CTA owns a tile of
-// 128 centroids for its whole life and keeps their three digit planes IN TENSOR MEMORY (the A operand of the
-// instruction is read from there: lane = centroid, 32 bytes per K step), so an instruction fetches only its 1 KB of
-// query digits from shared memory; with the A tile in shared memory every instruction re-read 4 KB of it and the
-// operand fetch, not the arithmetic, set the pace (measured: 51 cycles per instruction at N = 48).  The query planes
+// tensor memory), M = 128 centroids, K = 32 dimensions per instruction.  One CTA owns a tile of 128 centroids for its
+// whole life and keeps their three digit planes IN TENSOR MEMORY (the A operand of the instruction is read from there:
+// lane = centroid, 32 bytes per K step), so only the query digits come from shared memory and the 48 KB that the tile
+// would take there go to a deeper pipeline of query tiles.  A query tile is 32 query-token rows; its three digit planes
 // are K-major rows with a 128-byte pitch (dimensions beyond D are zero), brought into 128-byte-swizzled shared memory
-// by TMA (one plain per-CTA cp.async.bulk.tensor load of all three planes per tile, no multicast), four tiles deep.
-// Tensor memory per CTA: 5 accumulators x 32 columns + 96 columns of centroid digits = 256 columns, so two CTAs share
-// an SM.  A producer warp issues the loads and the MMAs; eight warps drain the accumulators (two per tensor-memory
-// lane quarter, a pair of eight-column chunks each).  A draining warp hands the accumulators back as soon as its
-// tcgen05.ld's have landed in registers, so the next tile's MMAs run while it recombines and stores.  Every wait on
-// an mbarrier is bounded; a wait that gives up sets the workspace's TIMEOUT status bit, and the CTA waits (bounded)
-// for its loads in flight, frees its tensor memory and returns.
+// one after the other by TMA (one plain per-CTA cp.async.bulk.tensor load per tile, no multicast), four tiles deep, so
+// that one instruction with N = 96 multiplies a centroid digit plane with all three query planes (see the schedule at
+// the MMA loop).  Tensor memory per CTA: 5 accumulators x 32 columns + 96 columns of centroid digits = 256 columns, so
+// two CTAs share an SM.  A producer warp issues the loads and the MMAs; eight warps drain the accumulators (two per
+// tensor-memory lane quarter, a pair of eight-column chunks each).  A draining warp hands the accumulators back as soon
+// as its tcgen05.ld's have landed in registers, so the next tile's MMAs run while it recombines and stores.  Measured
+// with clock64 stamps: the tensor pipe is busy about 90 % of a CTA's steady state, at one column of a 128 x N x 32
+// instruction per cycle (4,096 multiply-adds per SM cycle, the 16-bit rate).  Every wait on an mbarrier is bounded; a
+// wait that gives up sets the workspace's TIMEOUT status bit, and the CTA waits (bounded) for its loads in flight,
+// frees its tensor memory and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -186,9 +188,10 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
                 // The stage holds the query's digit planes a = 0, 1, 2 as 96 consecutive B rows, and the accumulators
                 // of weight w = 0..4 are consecutive groups of 32 columns.  One instruction with the centroids' digit
                 // plane b as A and all 96 rows as B therefore adds the products of weight b, b + 1, b + 2 to the
-                // accumulators starting at column 32 b: three instructions per K step instead of nine, which matters
-                // because a single thread issues an instruction only every ~50 cycles.  The very first instruction
-                // runs over 160 rows (the last 64 are zeros) without accumulating, which clears weights 3 and 4.
+                // accumulators starting at column 32 b: three instructions of N = 96 per K step instead of nine of
+                // N = 32 (fewer, larger instructions keep the tensor pipe fuller: -8 % on the whole kernel).  The very
+                // first instruction runs over 160 rows (the last 64 are zeros) without accumulating, which clears
+                // weights 3 and 4.
                 const uint64_t db0 = umma_desc(sB + stage * G1_B_STAGE);
 #pragma unroll
                 for (int k = 0; k < KS; ++k) {
