@@ -717,6 +717,14 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     }
     res["roofline"] = roofline
     res["pruning"] = PRUNING_TEXT[mode]
+    joint = index.probe_plan(B, nq, P) if mode != "rabitq_graph" else 0
+    if joint:
+        # stages 1 and 2a run together: the stage-1 slot also times the scans of the sampled rows, and the probes
+        # slot only the selection from the queues; the finished table is not read again
+        roofline["per_stage"]["score_table"]["includes"] = "bounds and queues of the probe stage (sample stride %d)" % joint
+        roofline["per_stage"]["probes"] = {"bound": "selection from the queues filled by the score table's epilogue "
+                                                    "(the table is not read again)", "frac": None,
+                                           "ms_per_launch": pr_ms}
     if mode == "rabitq_graph":
         # stage 1 does not run and the probes slot times the graph search, which streams no table
         roofline["per_stage"]["score_table"] = {"bound": "not run (probes come from the centroid graph)", "frac": None}

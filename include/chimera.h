@@ -256,6 +256,16 @@ int chimera_search_rabitq_graph(const chimera_index *index, const float *queries
  * [-1, 1]), CHIMERA_TIMEOUT or (debug build) CHIMERA_DEBUG_CHECK_FAILED to *status (host pointer). */
 int chimera_workspace_status(const void *workspace, void *stream, int32_t *status);
 
+/* How a search with these parameters finds its probes (Sec. 3.2 step 1, the top-n_probe centroids of each query
+ * token).  Writes to *sample_stride (host pointer) 0 when stage 2a is a scan of the finished score table, or s > 1
+ * when stages 1 and 2a run together in calls that cover both: every s-th tile of 128 centroids is scored first, a
+ * lower bound on each query token's nprobe-th best score is taken from that sample, and the score-table kernel queues
+ * every score at or above the bound while it writes the rest of the table, so the table is not read again (a query
+ * whose queue overflows is redone by the scan; the result is the same exact top n_probe either way).  The joint form
+ * needs nprobe <= 32, q_len a multiple of 4 and at least 8 sample tiles. */
+int chimera_probe_plan(const chimera_index *index, int32_t n_queries, int32_t q_len, int32_t nprobe,
+                       int32_t *sample_stride);
+
 /* Debug build (the paper has no counterpart).  libchimera_debug.so is the same source compiled with -DCHIMERA_DEBUG:
  * every kernel checks each centroid id, document id, token position and candidate rank before it gathers through it
  * (an index out of range is not dereferenced; chimera_workspace_status then reports CHIMERA_DEBUG_CHECK_FAILED), and

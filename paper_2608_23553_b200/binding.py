@@ -305,6 +305,14 @@ class Index:
                                         _ptr(ids), _ptr(scores)))
         return ids, scores
 
+    def probe_plan(self, n_queries, q_len, nprobe) -> int:
+        """0 when the probes come from a scan of the finished score table; otherwise the sampling stride of the joint
+        form of stages 1 and 2a (chimera_probe_plan)."""
+        s = ctypes.c_int32()
+        _check(lib().chimera_probe_plan(self._h, ctypes.c_int32(n_queries), ctypes.c_int32(q_len),
+                                        ctypes.c_int32(nprobe), ctypes.byref(s)))
+        return s.value
+
     def workspace_check(self, n_queries, q_len, nprobe, n_prune, k, max_candidates=0) -> int:
         """Debug build only: index of the first damaged guard region of the workspace after a search with these
         parameters, -1 if all are intact (chimera_workspace_check)."""

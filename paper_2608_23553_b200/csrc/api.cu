@@ -111,8 +111,16 @@ Layout make_layout(const Index &ix, const Params &p)
     L.qdig = take(3 * B * nq * 128);
     L.table = take(B * (size_t)ix.K * nq * sizeof(int32_t));
     L.table8 = take(coarse_supported(p.nq) ? B * (size_t)ix.K * nq : 0);
+    L.pq_stride = probe_queue_stride(ix, p);
+    L.pq_groups = L.pq_stride ? probe_sample_groups(ix, L.pq_stride) : 0;
     L.part = take(B * L.n_part * p.P * nq * sizeof(unsigned long long));
     L.probes = take(B * nq * p.P * sizeof(int32_t));
+    L.pq_cap = L.pq_stride ? probe_queue_cap() : 0;
+    L.pq_gmax = take(L.pq_stride ? B * (size_t)L.pq_groups * nq * sizeof(int32_t) : 0);
+    L.pq_thr = take(L.pq_stride ? B * nq * sizeof(int32_t) : 0);
+    L.pq_cnt = take(L.pq_stride ? B * nq * sizeof(int32_t) : 0);
+    L.pq_keys = take(L.pq_stride ? B * nq * (size_t)L.pq_cap * sizeof(unsigned long long) : 0);
+    L.pq_ovf = take(L.pq_stride ? B * sizeof(int32_t) : 0);
     L.bitmap = take(B * (size_t)L.words * sizeof(uint32_t));
     L.chunk_cnt = take(B * (size_t)(L.n_chunks + 1) * sizeof(int32_t));
     L.cand = take(B * (size_t)p.maxc * sizeof(int32_t));
@@ -295,8 +303,15 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
     }
     prof_mark(SLOT_MISC, st);
 
+    // stages 1 and 2a of one call run together when the layout provides for it: the probes come out of the score
+    // table's epilogue and the table is not read again
+    const bool together = first <= 1 && last >= 2 && !graph && L.pq_stride > 0;
     if (first <= 1 && last >= 1 && !graph) {
-        if ((rc = launch_score_table(ix, p, queries, qdig, table, table8, status, st))) return rc;
+        if (together)
+            rc = launch_score_table_probes(ix, p, L, queries, qdig, table, table8, ws, status, st);
+        else
+            rc = launch_score_table(ix, p, queries, qdig, table, table8, status, st);
+        if (rc) return rc;
         prof_mark(SLOT_G1, st);
     }
     if (first <= 2 && last >= 2) {
@@ -304,6 +319,8 @@ static int run(const Index &ix, const Params &p, int first, int last, const floa
             if ((rc = launch_graph_probes(ix, queries, (int64_t)p.B * p.nq, p.P, *graph, (uint32_t *)(ws + L.graph_vis),
                                           probes, nullptr, nullptr, st)))
                 return rc;
+        } else if (together) {
+            if ((rc = launch_probe_merge(ix, p, L, table, ws, st))) return rc;
         } else if ((rc = launch_probes(ix, p, L, table, part, probes, st))) {
             return rc;
         }
@@ -771,6 +788,18 @@ int chimera_workspace_status(const void *workspace, void *stream, int32_t *statu
     else if (bits & ST_BAD_QUERY) *status = CHIMERA_INVALID_ARG;
     else if (bits & ST_OVERFLOW) *status = CHIMERA_CAPACITY_OVERFLOW;
     else *status = CHIMERA_OK;
+    return CHIMERA_OK;
+}
+
+int chimera_probe_plan(const chimera_index *index, int32_t n_queries, int32_t q_len, int32_t nprobe,
+                       int32_t *sample_stride)
+{
+    const Index *ix = reinterpret_cast<const Index *>(index);
+    Params p;
+    int rc = check_params(ix, n_queries, q_len, nprobe, 1, 1, 0, &p);
+    if (rc) return rc;
+    if (!sample_stride) return fail(CHIMERA_INVALID_ARG, "NULL argument");
+    *sample_stride = probe_queue_stride(*ix, p);
     return CHIMERA_OK;
 }
 

@@ -71,6 +71,11 @@ struct Layout {
     size_t table8;        // uint8  [B][K][nq]        coarse copy: min((S + 2^24 + 64) >> 17, 255)
     size_t part;          // uint64 [B][n_part][P][nq] partial top-P keys
     size_t probes;        // int32  [B][nq][P]
+    size_t pq_gmax;       // int32  [B][pq_groups][nq] stages 1 + 2a together: largest score of each group of sample rows,
+    size_t pq_thr;        // int32  [B*nq]            score bound per query-token row,
+    size_t pq_cnt;        // int32  [B*nq]            keys queued for the row,
+    size_t pq_keys;       // uint64 [B*nq][pq_cap]    the keys,
+    size_t pq_ovf;        // int32  [B]               1 = a queue of this query overflowed (redo by the table scan)
     size_t bitmap;        // uint32 [B][words]
     size_t chunk_cnt;     // int32  [B][n_chunks + 1]
     size_t cand;          // int32  [B][maxc]
@@ -96,6 +101,9 @@ struct Layout {
     size_t score4;        // float  [B][n_prune]
     size_t total;
     // derived sizes
+    int32_t pq_stride;    // every pq_stride-th centroid tile is a sample tile; 0 = stages 1 and 2a run separately
+    int32_t pq_cap;       // keys per queue
+    int32_t pq_groups;    // groups of sample rows per query (one maximum each)
     int32_t n_part;       // partial lists per query in the probe stage
     int32_t probe_blocks; // blocks per query in the probe stage
     int64_t words;        // bitmap words per query
@@ -141,6 +149,17 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
                        uint8_t *table8, uint32_t *status, cudaStream_t st);
 int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32_t *table, unsigned long long *part,
                   int32_t *probes, cudaStream_t st);
+// Stages 1 and 2a together (g1_score_table.cu), used when the layout has pq_stride > 0, and its probe-side pieces
+// (g2_probe.cu): the sample's top nprobe and bounds; the final top nprobe from sample list and queues, with the table
+// scan as the fallback for queries whose queue overflowed.
+int probe_queue_stride(const Index &ix, const Params &p);
+int probe_queue_cap();
+int probe_sample_groups(const Index &ix, int stride);
+int launch_score_table_probes(const Index &ix, const Params &p, const Layout &L, const float *queries, int8_t *qdig,
+                              int32_t *table, uint8_t *table8, char *ws, uint32_t *status, cudaStream_t st);
+int launch_probe_sample(const Index &ix, const Params &p, const Layout &L, const int32_t *table, char *ws,
+                        int n_sample_tiles, cudaStream_t st);
+int launch_probe_merge(const Index &ix, const Params &p, const Layout &L, const int32_t *table, char *ws, cudaStream_t st);
 int launch_gather(const Index &ix, const Params &p, const Layout &L, const int32_t *probes, uint32_t *bitmap,
                   int32_t *chunk_cnt, int32_t *cand, int32_t *n_cand, int32_t *word_rank, uint32_t *status,
                   cudaStream_t st);

@@ -85,13 +85,29 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// grid (ceil(K / 128), n_splits).  Each CTA: centroid tile blockIdx.x, query-row tiles [blockIdx.y * tiles_per_split, ...).
-// KS = D / 32 MMA steps per digit-plane product.
-template <int KS>
+// Which centroid tiles a launch covers, and whether it feeds the probe stage (FILTER).
+//   tile_stride == 0: every tile (tile = blockIdx.x).
+//   tile_stride  > 1, sample != 0: the sample tiles 0, s, 2s, ... (tile = blockIdx.x * s).
+//   tile_stride  > 1, sample == 0: all the others (the j-th tile that is not a multiple of s).
+// FILTER (only with the "others"): thr[row] holds, for every query-token row, a lower bound on the score of the row's
+// nprobe-th best centroid (found on the sample); every score >= thr[row] goes, as a (score, centroid) key, into that
+// row's queue (keys[row][cap], counted in cnt[row]; entries past cap are dropped and the count tells).  The top nprobe
+// of a row are then in its queue, so the probe stage never reads the table again.
+struct G1Tiles {
+    int tile_stride, sample;
+    const int32_t *thr;
+    int32_t *cnt;
+    unsigned long long *keys;
+    int cap;
+};
+
+// grid (centroid tiles of the launch, n_splits).  Each CTA: one centroid tile, query-row tiles
+// [blockIdx.y * tiles_per_split, ...).  KS = D / 32 MMA steps per digit-plane product.
+template <int KS, bool FILTER>
 __global__ void __launch_bounds__(G1_THREADS)
 score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtensorMap map_q, int64_t K, int nq,
                  int64_t q_rows, int n_tiles, int tiles_per_split, int32_t *__restrict__ table,
-                 uint8_t *__restrict__ table8, uint32_t *status, long long wait_limit, int skip_loads)
+                 uint8_t *__restrict__ table8, uint32_t *status, long long wait_limit, int skip_loads, G1Tiles tiles)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t s_tmem_base;
@@ -102,7 +118,10 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
     const uint32_t bar_mma = bars + 8 * G1_STAGES;             // a tile's accumulators are complete
     const uint32_t bar_empty = bar_mma + 8;                    // every draining warp has the accumulators in registers
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t c0 = (int64_t)blockIdx.x * G1_M;
+    int c_tile = (int)blockIdx.x;
+    if (tiles.tile_stride > 1)
+        c_tile = tiles.sample ? c_tile * tiles.tile_stride : c_tile + c_tile / (tiles.tile_stride - 1) + 1;
+    const int64_t c0 = (int64_t)c_tile * G1_M;
     const int t_begin = blockIdx.y * tiles_per_split;
     int t_end = t_begin + tiles_per_split;
     if (t_end > n_tiles) t_end = n_tiles;
@@ -231,8 +250,22 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
         const uint32_t unq = (uint32_t)nq, rows32 = (uint32_t)q_rows;
         const int first_chunk = 2 * (warp >> 2);
+        unsigned long long pend_key = 0ull, *pend_dst = nullptr;   // FILTER: this thread's last key, not stored yet
+        int pend_slot = 0;
         for (int it = 0; it < my_tiles; ++it) {
             const int t = t_begin + it;
+            // FILTER: the thresholds of this warp's 16 query-token rows (the same for every lane), asked for before
+            // the wait
+            int32_t thr_v[16];
+            if (FILTER) {
+                const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)first_chunk * 8;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    int4 v = make_int4(0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff);     // rows past the end
+                    if (r0 + 4 * g < rows32) v = __ldg(reinterpret_cast<const int4 *>(tiles.thr + r0) + g);
+                    thr_v[4 * g] = v.x; thr_v[4 * g + 1] = v.y; thr_v[4 * g + 2] = v.z; thr_v[4 * g + 3] = v.w;
+                }
+            }
             // (the vote makes the decision uniform: the tensor-memory loads below need the whole warp)
             if (!__all_sync(0xffffffffu, mbar_wait(bar_mma, it & 1, wait_limit))) {
                 if (lane == 0) atomicOr(status, ST_TIMEOUT);
@@ -264,6 +297,27 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
                 const uint32_t r0 = (uint32_t)t * G1_N + (uint32_t)chunk * 8;
                 uint32_t qb = tile_qb, qi = tile_qi + (uint32_t)chunk * 8;      // chunk * 8 < 32: few subtractions
                 while (qi >= unq) { qi -= unq; ++qb; }
+                if (FILTER && c < K) {
+                    bool any = false;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) any |= out[e] >= thr_v[ch * 8 + e];
+                    if (any) {                  // about nprobe x tile_stride keys per row in all: one lane of a warp
+                                                // every few chunks
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            if (out[e] >= thr_v[ch * 8 + e]) {  // (rows past the end have the largest threshold and
+                                                                //  zero digits: they never pass)
+                                // The slot comes back from the atomic hundreds of cycles later; the key is stored
+                                // only when this thread's next key turns up (or at the end), so nobody waits for it.
+                                if (pend_key && pend_slot < tiles.cap) pend_dst[pend_slot] = pend_key;
+                                const uint32_t row = r0 + e;
+                                pend_key = key_int(out[e], (int32_t)c);
+                                pend_dst = tiles.keys + (int64_t)row * tiles.cap;
+                                pend_slot = atomicAdd(tiles.cnt + row, 1);
+                            }
+                        }
+                    }
+                }
                 if (c < K && r0 < rows32) {
                     if (table8 != nullptr) {
                         // coarse copy for the bound phase of stage 3: clamp(S >> 16, 0, 255); q_len is a multiple
@@ -311,6 +365,7 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
                 }
             }
         }
+        if (FILTER && pend_key && pend_slot < tiles.cap) pend_dst[pend_slot] = pend_key;
     }
 
     tc_fence_before();
@@ -356,18 +411,16 @@ int make_plane_map(CUtensorMap *map, const int8_t *planes, int64_t rows, int box
     return CHIMERA_OK;
 }
 
-int launch_score_table(const Index &ix, const Params &p, const float *queries, int8_t *qdig, int32_t *table,
-                       uint8_t *table8, uint32_t *status, cudaStream_t st)
+// One launch of the kernel over `c_tiles` centroid tiles (see G1Tiles for which).
+template <bool FILTER>
+static int launch_g1_tiles(const Index &ix, const Params &p, const CUtensorMap &map_q, int c_tiles, int32_t *table,
+                           uint8_t *table8, uint32_t *status, const G1Tiles &tiles, cudaStream_t st)
 {
     const int64_t rows = (int64_t)p.B * p.nq;
-    int rc = launch_digits(queries, rows, ix.D, qdig, status, st);
-    if (rc) return rc;
-    CUtensorMap map_q;
-    if ((rc = make_plane_map(&map_q, qdig, rows, G1_N, 3))) return rc;        // one load brings a tile's three planes
-    const int c_tiles = (int)((ix.K + G1_M - 1) / G1_M);
     const int n_tiles = (int)((rows + G1_N - 1) / G1_N);
-    // about eight waves of two CTAs per SM, so the last wave is mostly full
-    int splits = (16 * ix.sm_count + c_tiles - 1) / c_tiles;
+    // about eight waves of two CTAs per SM, so the last wave is mostly full; a launch over few centroid tiles (the
+    // sample) fills one wave instead, because a CTA's start-up costs as much as three tiles
+    int splits = c_tiles < 2 * ix.sm_count ? (2 * ix.sm_count) / c_tiles : (16 * ix.sm_count + c_tiles - 1) / c_tiles;
     if (splits > n_tiles) splits = n_tiles;
     if (splits < 1) splits = 1;
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
@@ -376,10 +429,11 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     const int skip = fault_skip_tma_loads();
 #define CHIMERA_G1_LAUNCH(KS)                                                                                          \
     do {                                                                                                               \
-        CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
+        CHIMERA_CUDA(cudaFuncSetAttribute(score_table_umma<KS, FILTER>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
                                           (int)G1_SMEM));                                                              \
-        score_table_umma<KS><<<grid, G1_THREADS, G1_SMEM, st>>>(ix.cdig, map_q, ix.K, p.nq, rows, n_tiles,                \
-                                                                tiles_per_split, table, table8, status, limit, skip);  \
+        score_table_umma<KS, FILTER><<<grid, G1_THREADS, G1_SMEM, st>>>(ix.cdig, map_q, ix.K, p.nq, rows, n_tiles,     \
+                                                                        tiles_per_split, table, table8, status, limit, \
+                                                                        skip, tiles);                                  \
     } while (0)
     switch (ix.D / 32) {                       // MMA steps of 32 dimensions
     case 1: CHIMERA_G1_LAUNCH(1); break;
@@ -389,7 +443,50 @@ int launch_score_table(const Index &ix, const Params &p, const float *queries, i
     }
 #undef CHIMERA_G1_LAUNCH
     CHIMERA_CUDA(cudaGetLastError());
+    return CHIMERA_OK;
+}
+
+int launch_score_table(const Index &ix, const Params &p, const float *queries, int8_t *qdig, int32_t *table,
+                       uint8_t *table8, uint32_t *status, cudaStream_t st)
+{
+    const int64_t rows = (int64_t)p.B * p.nq;
+    int rc = launch_digits(queries, rows, ix.D, qdig, status, st);
+    if (rc) return rc;
+    CUtensorMap map_q;
+    if ((rc = make_plane_map(&map_q, qdig, rows, G1_N, 3))) return rc;        // one load brings a tile's three planes
+    const G1Tiles all = {0, 0, nullptr, nullptr, nullptr, 0};
+    if ((rc = launch_g1_tiles<false>(ix, p, map_q, (int)((ix.K + G1_M - 1) / G1_M), table, table8, status, all, st)))
+        return rc;
     count_launch(SLOT_G1, 2);
+    return CHIMERA_OK;
+}
+
+// Stages 1 and 2a together (Sec. 3.2 step 1 on top of Definition 1's products): the table of a sample of the centroid
+// tiles first, from it a lower bound per query token on the score of the token's true nprobe-th best centroid, then
+// the rest of the table with every score at or above that bound queued beside it (the sample's own scores are queued
+// by a scan of their rows), and the nprobe best keys of each queue.  The result is the exact top nprobe by (score
+// descending, centroid id ascending): a centroid that belongs to it has a score >= the bound, so it is queued.
+// A query with a token whose queue overflowed is redone by the table scan of the separate probe stage.
+int launch_score_table_probes(const Index &ix, const Params &p, const Layout &L, const float *queries, int8_t *qdig,
+                              int32_t *table, uint8_t *table8, char *ws, uint32_t *status, cudaStream_t st)
+{
+    const int64_t rows = (int64_t)p.B * p.nq;
+    int rc = launch_digits(queries, rows, ix.D, qdig, status, st);
+    if (rc) return rc;
+    CUtensorMap map_q;
+    if ((rc = make_plane_map(&map_q, qdig, rows, G1_N, 3))) return rc;
+    const int c_tiles = (int)((ix.K + G1_M - 1) / G1_M);
+    const int stride = L.pq_stride;
+    const int n_sample = (c_tiles + stride - 1) / stride;
+    int32_t *thr = (int32_t *)(ws + L.pq_thr), *cnt = (int32_t *)(ws + L.pq_cnt);
+    unsigned long long *keys = (unsigned long long *)(ws + L.pq_keys);
+
+    const G1Tiles sample = {stride, 1, nullptr, nullptr, nullptr, 0};
+    if ((rc = launch_g1_tiles<false>(ix, p, map_q, n_sample, table, table8, status, sample, st))) return rc;
+    if ((rc = launch_probe_sample(ix, p, L, table, ws, n_sample, st))) return rc;
+    const G1Tiles rest = {stride, 0, thr, cnt, keys, L.pq_cap};
+    if ((rc = launch_g1_tiles<true>(ix, p, map_q, c_tiles - n_sample, table, table8, status, rest, st))) return rc;
+    count_launch(SLOT_G1, 3);
     return CHIMERA_OK;
 }
 

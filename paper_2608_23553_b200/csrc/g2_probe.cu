@@ -6,6 +6,7 @@
 // key is a 64-bit integer whose order is (score desc, id asc).  Pass 1 turns slices of the table into partial lists,
 // pass 2 folds the partial lists of a query into the final P per token.
 #include <atomic>
+#include <stdint.h>
 
 #include "common.cuh"
 
@@ -29,11 +30,13 @@ __device__ __forceinline__ void list_insert(unsigned long long *list, int P, uns
 }
 
 // grid (probe_blocks, B, ceil(nq / 32)).  part: [B][n_part][P][nq], n_part = probe_blocks (one list per block).
+// only_flagged: NULL, or int32[B]: blocks of queries whose entry is 0 return at once.
 __global__ void __launch_bounds__(PROBE_THREADS)
 probe_partial(const int32_t *__restrict__ table, int64_t K, int nq, int P, int rows_per_block, int n_part,
-              unsigned long long *__restrict__ part)
+              unsigned long long *__restrict__ part, const int32_t *__restrict__ only_flagged)
 {
     extern __shared__ unsigned long long lists[];    // [P][PROBE_THREADS]
+    if (only_flagged && !only_flagged[blockIdx.y]) return;      // (fallback use: only the flagged queries)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int col = blockIdx.z * 32 + lane;
     const int b = blockIdx.y;
@@ -78,9 +81,11 @@ probe_partial(const int32_t *__restrict__ table, int64_t K, int nq, int P, int r
 // shared-memory lists of 1024 threads.
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS)
-probe_final(const unsigned long long *__restrict__ part, int nq, int P, int n_part, int32_t *__restrict__ probes)
+probe_final(const unsigned long long *__restrict__ part, int nq, int P, int n_part, int32_t *__restrict__ probes,
+            const int32_t *__restrict__ only_flagged)
 {
     extern __shared__ unsigned long long lists[];      // [P][THREADS]
+    if (only_flagged && !only_flagged[blockIdx.y]) return;
     constexpr int W = THREADS / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int col = blockIdx.z * 32 + lane;
@@ -151,20 +156,20 @@ probe_final(const unsigned long long *__restrict__ part, int nq, int P, int n_pa
 // The widest block whose lists (nprobe keys of 8 bytes per thread) fit the default 48 KB of shared memory, at least
 // PROBE_THREADS (whose lists may need the opt-in limit: 128 KB at nprobe = 64).
 static int launch_probe_final(const unsigned long long *part, int B, int nq, int P, int n_part, int32_t *probes,
-                              cudaStream_t st)
+                              cudaStream_t st, const int32_t *only_flagged = nullptr)
 {
     const dim3 grid(1, (unsigned)B, (unsigned)((nq + 31) / 32));
     const size_t per_thread = sizeof(unsigned long long) * (size_t)P;
     if (per_thread * 1024 <= 48 * 1024) {
-        probe_final<1024><<<grid, 1024, per_thread * 1024, st>>>(part, nq, P, n_part, probes);
+        probe_final<1024><<<grid, 1024, per_thread * 1024, st>>>(part, nq, P, n_part, probes, only_flagged);
     } else if (per_thread * 512 <= 48 * 1024) {
-        probe_final<512><<<grid, 512, per_thread * 512, st>>>(part, nq, P, n_part, probes);
+        probe_final<512><<<grid, 512, per_thread * 512, st>>>(part, nq, P, n_part, probes, only_flagged);
     } else {
         const size_t smem = per_thread * PROBE_THREADS;
         if (smem > 48 * 1024)
             CHIMERA_CUDA(cudaFuncSetAttribute(probe_final<PROBE_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)smem));
-        probe_final<PROBE_THREADS><<<grid, PROBE_THREADS, smem, st>>>(part, nq, P, n_part, probes);
+        probe_final<PROBE_THREADS><<<grid, PROBE_THREADS, smem, st>>>(part, nq, P, n_part, probes, only_flagged);
     }
     CHIMERA_CUDA(cudaGetLastError());
     return CHIMERA_OK;
@@ -179,11 +184,238 @@ int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32
     const int rows_per_block = (int)((ix.K + L.probe_blocks - 1) / L.probe_blocks);
     const unsigned col_groups = (unsigned)((p.nq + 31) / 32);
     dim3 g1((unsigned)L.probe_blocks, (unsigned)p.B, col_groups);
-    probe_partial<<<g1, PROBE_THREADS, smem, st>>>(table, ix.K, p.nq, p.P, rows_per_block, L.n_part, part);
+    probe_partial<<<g1, PROBE_THREADS, smem, st>>>(table, ix.K, p.nq, p.P, rows_per_block, L.n_part, part, nullptr);
     CHIMERA_CUDA(cudaGetLastError());
     const int rc = launch_probe_final(part, p.B, p.nq, p.P, L.n_part, probes, st);
     if (rc) return rc;
     count_launch(SLOT_PROBE, 2);
+    return CHIMERA_OK;
+}
+
+// =====================================================================================================================
+// Probe side of stages 1 and 2a run together (launch_score_table_probes in g1_score_table.cu).
+// =====================================================================================================================
+constexpr int PQ_CAP = 1024;            // keys per queue: several times the expected number (see below)
+constexpr int PQ_WARPS = 8;             // warps per block of the kernels below
+constexpr int PQ_MAX_GROUPS = 256;      // groups of sample rows per query
+
+int probe_queue_cap() { return PQ_CAP; }
+
+// Every how-many-th centroid tile (128 centroids) is a sample tile, or 0 when the stages run separately.  The bound of
+// a query-token row is (a little below) its nprobe-th best score among the sample, a fraction 1 / stride of the
+// centroids, so about nprobe x stride centroids in all reach it (for exchangeable scores the count is
+// negative-binomial with that mean); stride = 128 / max(nprobe, 4) keeps the mean near 128 keys, an eighth of PQ_CAP
+// (for nprobe = 4 the chance of 1024 or more is below 1e-9 per row).  Strided tiles rather than the first ones, so
+// that centroids stored in some spatial order still give a representative sample.
+int probe_queue_stride(const Index &ix, const Params &p)
+{
+    if (p.P > 32 || (p.nq & 3) != 0) return 0;
+    const int stride = 128 / (p.P > 4 ? p.P : 4);          // 32, ..., 4
+    const int64_t c_tiles = (ix.K + 127) / 128;
+    if (stride < 2 || c_tiles < 8 * (int64_t)stride) return 0;      // at least 8 sample tiles (1024 centroids)
+    return stride;
+}
+
+// The sample rows of a query are cut into groups (16 rows or more, at most PQ_MAX_GROUPS groups, at least 64).
+int probe_sample_groups(const Index &ix, int stride)
+{
+    const int64_t c_tiles = (ix.K + 127) / 128;
+    const int64_t sample_rows = (c_tiles + stride - 1) / stride * 128;
+    int64_t groups = sample_rows / 16;
+    if (groups > PQ_MAX_GROUPS) groups = PQ_MAX_GROUPS;
+    return (int)groups;
+}
+
+// Sample row r -> centroid: tile (r / 128) * stride, row r % 128 of it.
+__device__ __forceinline__ int64_t sample_centroid(int64_t r, int stride) { return ((r >> 7) * stride << 7) + (r & 127); }
+
+// grid (ceil(G / PQ_WARPS), B, ceil(nq / 32)): warp = one group of sample rows, lane = query token; the largest score
+// of the group per token.  gmax: [B][G][nq].
+__global__ void __launch_bounds__(32 * PQ_WARPS)
+sample_max_kernel(const int32_t *__restrict__ table, int64_t K, int nq, int64_t sample_rows, int stride, int G,
+                  int rows_per_group, int32_t *__restrict__ gmax)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int col = blockIdx.z * 32 + lane;
+    const int b = blockIdx.y;
+    const int g = blockIdx.x * PQ_WARPS + warp;
+    if (g >= G || col >= nq) return;
+    const int32_t *tb = table + (int64_t)b * K * nq + col;
+    const int64_t r0 = (int64_t)g * rows_per_group;
+    int64_t r1 = r0 + rows_per_group;
+    if (r1 > sample_rows) r1 = sample_rows;
+    int32_t best = INT32_MIN;
+    for (int64_t r = r0; r < r1; r += 8) {
+        int32_t v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int64_t c = sample_centroid(r + u, stride);
+            v[u] = (r + u < r1 && c < K) ? tb[c * nq] : INT32_MIN;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) best = max(best, v[u]);
+    }
+    gmax[((int64_t)b * G + g) * nq + col] = best;
+}
+
+// One warp per query-token row: the nprobe-th largest of the row's G group maxima.  The nprobe largest maxima are
+// nprobe different centroids, so the true nprobe-th best score is at least that: a bound.  Also empties the row's
+// queue and clears the query's flag.
+__global__ void __launch_bounds__(32 * PQ_WARPS)
+sample_bound_kernel(const int32_t *__restrict__ gmax, int G, int nq, int P, int64_t rows, int32_t *__restrict__ thr,
+                    int32_t *__restrict__ cnt, int32_t *__restrict__ ovf)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * PQ_WARPS + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int64_t b = row / nq;
+    const int col = (int)(row - b * nq);
+    // (value, group) keys are distinct, so "the largest key below the previous one" walks down the order
+    unsigned long long mine[PQ_MAX_GROUPS / 32];
+#pragma unroll
+    for (int i = 0; i < PQ_MAX_GROUPS / 32; ++i) {
+        const int g = lane + 32 * i;
+        mine[i] = g < G ? key_int(gmax[(b * G + g) * nq + col], g) : 0ull;
+    }
+    unsigned long long prev = ~0ull;
+    for (int j = 0; j < P; ++j) {
+        unsigned long long best = 0ull;
+#pragma unroll
+        for (int i = 0; i < PQ_MAX_GROUPS / 32; ++i)
+            if (mine[i] < prev && mine[i] > best) best = mine[i];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+            if (other > best) best = other;
+        }
+        prev = best;
+    }
+    if (lane == 0) {
+        thr[row] = (int32_t)((uint32_t)(prev >> 32) ^ 0x80000000u);
+        cnt[row] = 0;
+        if (col == 0) ovf[b] = 0;
+    }
+}
+
+// Same grid as sample_max_kernel: the sample rows once more, every score at or above the row's bound into its queue
+// (the rest of the table does this in the score-table kernel's epilogue).
+__global__ void __launch_bounds__(32 * PQ_WARPS)
+sample_push_kernel(const int32_t *__restrict__ table, int64_t K, int nq, int64_t sample_rows, int stride, int G,
+                   int rows_per_group, const int32_t *__restrict__ thr, int32_t *__restrict__ cnt,
+                   unsigned long long *__restrict__ keys, int cap)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int col = blockIdx.z * 32 + lane;
+    const int b = blockIdx.y;
+    const int g = blockIdx.x * PQ_WARPS + warp;
+    if (g >= G || col >= nq) return;
+    const int32_t *tb = table + (int64_t)b * K * nq + col;
+    const int64_t row = (int64_t)b * nq + col;
+    const int32_t bound = thr[row];
+    const int64_t r0 = (int64_t)g * rows_per_group;
+    int64_t r1 = r0 + rows_per_group;
+    if (r1 > sample_rows) r1 = sample_rows;
+    for (int64_t r = r0; r < r1; r += 8) {
+        int32_t v[8];
+        int64_t c[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            c[u] = sample_centroid(r + u, stride);
+            v[u] = (r + u < r1 && c[u] < K) ? tb[c[u] * nq] : INT32_MIN;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (v[u] >= bound && r + u < r1 && c[u] < K) {
+                const int slot = atomicAdd(cnt + row, 1);
+                if (slot < cap) keys[row * cap + slot] = key_int(v[u], (int32_t)c[u]);
+            }
+        }
+    }
+}
+
+// One warp per query-token row: the nprobe best keys of the row's queue -> probes[row].  A row whose queue
+// overflowed flags its query instead.
+__global__ void __launch_bounds__(32 * PQ_WARPS)
+probe_merge_kernel(int nq, int P, int64_t rows, const int32_t *__restrict__ cnt,
+                   const unsigned long long *__restrict__ keys, int cap, int32_t *__restrict__ probes,
+                   int32_t *__restrict__ ovf)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * PQ_WARPS + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int n = cnt[row];
+    if (n > cap) {
+        if (lane == 0) ovf[row / nq] = 1;
+        return;
+    }
+    const unsigned long long *mine = keys + row * cap;
+    unsigned long long prev = ~0ull;
+    int32_t my_id = 0;
+    for (int j = 0; j < P; ++j) {                            // keys are distinct (they contain the centroid id)
+        unsigned long long best = 0ull;
+        for (int i = lane; i < n; i += 32) {
+            const unsigned long long k = __ldg(mine + i);
+            if (k < prev && k > best) best = k;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+            if (other > best) best = other;
+        }
+        prev = best;
+        if (lane == j) my_id = key_id(best);
+    }
+    if (lane < P) probes[row * P + lane] = my_id;            // (the queue holds at least nprobe keys: the group maxima)
+}
+
+int launch_probe_sample(const Index &ix, const Params &p, const Layout &L, const int32_t *table, char *ws,
+                        int n_sample_tiles, cudaStream_t st)
+{
+    const int64_t sample_rows = (int64_t)n_sample_tiles * 128;
+    const int G = L.pq_groups;
+    const int rows_per_group = (int)((sample_rows + G - 1) / G);
+    const int64_t rows = (int64_t)p.B * p.nq;
+    int32_t *gmax = (int32_t *)(ws + L.pq_gmax), *thr = (int32_t *)(ws + L.pq_thr), *cnt = (int32_t *)(ws + L.pq_cnt);
+    int32_t *ovf = (int32_t *)(ws + L.pq_ovf);
+    unsigned long long *keys = (unsigned long long *)(ws + L.pq_keys);
+    const dim3 grid((unsigned)((G + PQ_WARPS - 1) / PQ_WARPS), (unsigned)p.B, (unsigned)((p.nq + 31) / 32));
+    sample_max_kernel<<<grid, 32 * PQ_WARPS, 0, st>>>(table, ix.K, p.nq, sample_rows, L.pq_stride, G, rows_per_group,
+                                                      gmax);
+    CHIMERA_CUDA(cudaGetLastError());
+    sample_bound_kernel<<<(unsigned)((rows + PQ_WARPS - 1) / PQ_WARPS), 32 * PQ_WARPS, 0, st>>>(gmax, G, p.nq, p.P, rows,
+                                                                                                thr, cnt, ovf);
+    CHIMERA_CUDA(cudaGetLastError());
+    sample_push_kernel<<<grid, 32 * PQ_WARPS, 0, st>>>(table, ix.K, p.nq, sample_rows, L.pq_stride, G, rows_per_group,
+                                                       thr, cnt, keys, L.pq_cap);
+    CHIMERA_CUDA(cudaGetLastError());
+    count_launch(SLOT_PROBE, 3);
+    return CHIMERA_OK;
+}
+
+int launch_probe_merge(const Index &ix, const Params &p, const Layout &L, const int32_t *table, char *ws, cudaStream_t st)
+{
+    const int64_t rows = (int64_t)p.B * p.nq;
+    const int32_t *cnt = (const int32_t *)(ws + L.pq_cnt);
+    const unsigned long long *keys = (const unsigned long long *)(ws + L.pq_keys);
+    int32_t *ovf = (int32_t *)(ws + L.pq_ovf);
+    unsigned long long *part = (unsigned long long *)(ws + L.part);
+    int32_t *probes = (int32_t *)(ws + L.probes);
+    probe_merge_kernel<<<(unsigned)((rows + PQ_WARPS - 1) / PQ_WARPS), 32 * PQ_WARPS, 0, st>>>(p.nq, p.P, rows, cnt, keys,
+                                                                                               L.pq_cap, probes, ovf);
+    CHIMERA_CUDA(cudaGetLastError());
+    // queries with an overflowed queue (none, except for inputs with masses of equal scores): the table scan, whose
+    // blocks return at once for every other query
+    const size_t smem = sizeof(unsigned long long) * (size_t)p.P * PROBE_THREADS;
+    if (smem > 48 * 1024)
+        CHIMERA_CUDA(cudaFuncSetAttribute(probe_partial, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int rows_per_block = (int)((ix.K + L.probe_blocks - 1) / L.probe_blocks);
+    const unsigned col_groups = (unsigned)((p.nq + 31) / 32);
+    probe_partial<<<dim3((unsigned)L.probe_blocks, (unsigned)p.B, col_groups), PROBE_THREADS, smem, st>>>(
+        table, ix.K, p.nq, p.P, rows_per_block, L.n_part, part, ovf);
+    CHIMERA_CUDA(cudaGetLastError());
+    const int rc = launch_probe_final(part, p.B, p.nq, p.P, L.n_part, probes, st, ovf);
+    if (rc) return rc;
+    count_launch(SLOT_PROBE, 3);
     return CHIMERA_OK;
 }
 
@@ -259,7 +491,7 @@ extern "C" int chimera_probes_static(const int32_t *score_table, int64_t n_centr
     // probe_partial writes every entry probe_final reads (all n_part lists x nprobe keys x q_len columns), so nothing
     // of the previous call's contents survives into this call's result and nothing needs clearing.
     probe_partial<<<dim3((unsigned)blocks, (unsigned)n_queries, col_groups), PROBE_THREADS, smem, st>>>(
-        score_table, n_centroids, q_len, nprobe, rows_per_block, n_part, part);
+        score_table, n_centroids, q_len, nprobe, rows_per_block, n_part, part, nullptr);
     CHIMERA_CUDA(cudaGetLastError());
     return launch_probe_final(part, n_queries, q_len, nprobe, n_part, out_probes, st);
 }
