@@ -17,11 +17,11 @@
 // the MMA loop).  Tensor memory per CTA: 5 accumulators x 32 columns + 96 columns of centroid digits = 256 columns, so
 // two CTAs share an SM.  A producer warp issues the loads and the MMAs; eight warps drain the accumulators (two per
 // tensor-memory lane quarter, a pair of eight-column chunks each).  A draining warp hands the accumulators back as soon
-// as its tcgen05.ld's have landed in registers, so the next tile's MMAs run while it recombines and stores.  Measured
-// with clock64 stamps: the tensor pipe is busy about 90 % of a CTA's steady state, at one column of a 128 x N x 32
-// instruction per cycle (4,096 multiply-adds per SM cycle, the 16-bit rate).  Every wait on an mbarrier is bounded; a
-// wait that gives up sets the workspace's TIMEOUT status bit, and the CTA waits (bounded) for its loads in flight,
-// frees its tensor memory and returns.
+// as its tcgen05.ld's have landed in registers, so the next tile's MMAs run while it recombines and stores.  An
+// isolated loop of these instructions runs at half a cycle per column of N (8,192 multiply-adds per SM cycle) but
+// never faster than ~45 cycles per instruction, which is why the instructions here are N = 96 wide (48 cycles).
+// Every wait on an mbarrier is bounded; a wait that gives up sets the workspace's TIMEOUT status bit, and the CTA
+// waits (bounded) for its loads in flight, frees its tensor memory and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -208,7 +208,7 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
                 // of weight w = 0..4 are consecutive groups of 32 columns.  One instruction with the centroids' digit
                 // plane b as A and all 96 rows as B therefore adds the products of weight b, b + 1, b + 2 to the
                 // accumulators starting at column 32 b: three instructions of N = 96 per K step instead of nine of
-                // N = 32 (fewer, larger instructions keep the tensor pipe fuller: -8 % on the whole kernel).  The very
+                // N = 32 (an instruction takes N / 2 cycles but at least ~45: -8 % on the whole kernel).  The very
                 // first instruction runs over 160 rows (the last 64 are zeros) without accumulating, which clears
                 // weights 3 and 4.
                 const uint64_t db0 = umma_desc(sB + stage * G1_B_STAGE);
