@@ -60,7 +60,19 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     return lib
 
 
+def build_microbench(force: bool = False) -> str:
+    """The stand-alone tensor-core instruction-rate microbenchmark (microbench/mma_rate.cu) -> build/mma_rate."""
+    src = os.path.join(ROOT, "paper_2608_23553_b200", "microbench", "mma_rate.cu")
+    exe = os.path.join(OBJ, "mma_rate")
+    os.makedirs(OBJ, exist_ok=True)
+    if force or not _newer(exe, [src, os.path.join(CSRC, "umma.cuh")]):
+        subprocess.check_call([NVCC] + FLAGS + ["-o", exe, src])
+    return exe
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--microbench" in sys.argv:
+        print(build_microbench(force="--force" in sys.argv))
     if "--debug" in sys.argv:
         print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug=True))
