@@ -359,6 +359,32 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             const uint32_t valid = __ballot_sync(0xffffffffu, dl >= 0);
             uint32_t starts = __ballot_sync(0xffffffffu, dl >= 0 && (lane == 0 || dl != prev));
             const int n_rows = __popc(valid);                 // valid rows are a prefix of the warp's rows
+            if (ON_A && starts == 1u && valid == 0xffffffffu) {
+                // The warp's 32 tokens belong to one document (most tiles of a long document): lane = (four columns,
+                // a quarter of the rows), eight 16-byte loads per lane instead of 32 scalar ones, then two exchange
+                // steps among the four lanes of a column group.
+                const int grp = lane & 7, sub = lane >> 3;
+                const float *vb = vals + warp * 32 * VP;
+                float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int r = sub + 4 * j;
+                    const float4 v = *reinterpret_cast<const float4 *>(vb + r * VP + ((grp ^ (r & 7)) << 2));
+                    m.x = fmaxf(m.x, v.x); m.y = fmaxf(m.y, v.y); m.z = fmaxf(m.z, v.z); m.w = fmaxf(m.w, v.w);
+                }
+#pragma unroll
+                for (int o = 8; o <= 16; o <<= 1) {
+                    m.x = fmaxf(m.x, __shfl_xor_sync(0xffffffffu, m.x, o));
+                    m.y = fmaxf(m.y, __shfl_xor_sync(0xffffffffu, m.y, o));
+                    m.z = fmaxf(m.z, __shfl_xor_sync(0xffffffffu, m.z, o));
+                    m.w = fmaxf(m.w, __shfl_xor_sync(0xffffffffu, m.w, o));
+                }
+                const int doc = __shfl_sync(0xffffffffu, dl, 0);
+                // lane (grp, sub) publishes column 4 grp + sub
+                const float mine = sub == 0 ? m.x : sub == 1 ? m.y : sub == 2 ? m.z : m.w;
+                atomicMax(&docmax[doc * NQP + 4 * grp + sub], f_order(mine));
+                starts = 0u;
+            }
             while (starts) {
                 const int a = __ffs(starts) - 1;
                 starts &= starts - 1;
