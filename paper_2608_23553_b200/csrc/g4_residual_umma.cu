@@ -8,12 +8,15 @@
 // int32; the three planes are recombined in fp32 (relative error 2^-24).
 //
 // A CTA owns one query and a run of its surviving documents, whose tokens form one stream cut into tiles of 128
-// (MMA M).  Per tile: every thread expands the packed code of one token into a 128-byte int8 row (two integer
-// multiplications and two masks per four dimensions) and stores it, 128-byte swizzled, into the A tile; one thread issues D/32 MMAs (N = 3 * padded q_len: the
-// three digit planes side by side, loaded once per CTA by TMA); the accumulators come back with tcgen05.ld, get the
-// centroid term from the stage-1 table, and go to shared memory, where each warp folds its 32 tokens into per-document
-// maxima.  Tensor memory: 128 or 256 columns per CTA, so several CTAs share an SM and overlap each other's phases.
-// All mbarrier waits are bounded.
+// (MMA M).  Per tile: every thread expands the packed code of one token into 128 int8 values (two integer
+// multiplications and two masks per four dimensions) and writes them with one tcgen05.st into its lane of the A
+// operand IN TENSOR MEMORY (32 columns behind the accumulators; through shared memory the same row cost eight
+// 16-byte stores per thread, and the load/store pipe is what this kernel is short of); one thread issues D/32 MMAs
+// (N = 3 * padded q_len: the three digit planes side by side, loaded once per CTA by TMA); the accumulators come back
+// with tcgen05.ld, get the centroid term from the stage-1 table, and go to shared memory, where each warp folds its
+// 32 tokens into per-document maxima (a warp whose tokens are all of one document reads 16 bytes per lane and row
+// quarter instead of a word per row).  Tensor memory: 128 or 256 columns per CTA, so several CTAs share an SM and
+// overlap each other's phases.  All mbarrier waits are bounded.
 #include <math.h>
 
 #include "common.cuh"
@@ -60,18 +63,21 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                      float *__restrict__ score4, uint32_t *status, long long wait_limit, int skip_loads)
 {
     constexpr int N = 3 * NQP;                               // MMA N: three digit planes side by side
-    constexpr uint32_t TMEM_COLS = N <= 128 ? 128 : 256;
-    constexpr uint32_t A_BYTES = G4U_TOK * 128;              // 16 KB
+    constexpr uint32_t TMEM_COLS = N <= 96 ? 128 : 256;
+    constexpr uint32_t A_COL = N;                            // the expanded codes: 32 columns behind the accumulators
+    static_assert(N + 32 <= TMEM_COLS, "accumulators and the A operand share the allocation");
     constexpr uint32_t B_BYTES = N * 128;
-    // Value rows (one per token, floats).  ON_A (q_len <= 32, residual codes): a row is 128 bytes and lies on the
-    // token's own row of the A tile, which is free between the MMAs' completion and the next expansion; its 16-byte
-    // groups are XOR-swizzled like the A rows, so the row-per-thread writes and the lane = column reads are both
-    // conflict-free.  18 KB less shared memory per CTA lets the SM run with a smaller shared-memory carve-out, i.e.
-    // more L1 for the scattered score-table rows (Mid, batch 256: 2.72 -> 2.41 ms; forcing the largest carve-out
-    // brings 2.71 ms back).  The RaBitQ variant gathers no rows and is slower that way (1.45 -> 1.56 ms).  Otherwise
-    // the rows have their own buffer with pitch NQP + 4 (read with lane = column: conflict-free).
+    // Value rows (one per token, floats) in shared memory.  PACKED (q_len <= 32, residual codes): a row is exactly 128
+    // bytes and its 16-byte groups are XOR-swizzled with the row number, so the row-per-thread writes and the
+    // lane = column reads are both conflict-free without padding: 16 KB, which with the query planes and the
+    // per-document maxima keeps the CTA at 32 KB and lets the SM run with a small shared-memory carve-out, i.e. more L1
+    // for the scattered score-table rows (Mid, batch 256: 2.72 -> 2.41 ms against padded rows; forcing the largest
+    // carve-out brings 2.71 ms back).  The RaBitQ variant gathers no rows and is faster with padded rows (pitch
+    // NQP + 4, read with lane = column: conflict-free), as are 64-token queries.
     constexpr bool ON_A = NQP == 32 && !RQ;
     constexpr int VP = ON_A ? 32 : NQP + 4;
+    constexpr uint32_t V_BYTES = sizeof(float) * G4U_TOK * VP;       // a multiple of 1024 for every variant
+    static_assert(V_BYTES % 1024 == 0, "the query planes behind the value rows stay 1024-byte aligned");
     constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) |
                                ((uint32_t)(G4U_TOK >> 4) << 24);
 
@@ -84,10 +90,9 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
     __shared__ int s_sq[NQP];                                // RQ: sum_x rint(q_p[x] * 2^22) per query token
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to the aligned area
-    const uint32_t sA = base, sB = base + A_BYTES;
-    float *vals = reinterpret_cast<float *>(ON_A ? gen : gen + A_BYTES + B_BYTES);          // [128][VP]
-    uint32_t *docmax = reinterpret_cast<uint32_t *>(
-        gen + A_BYTES + B_BYTES + (ON_A ? 0 : sizeof(float) * G4U_TOK * VP));              // [MAX_DOCS][NQP]
+    float *vals = reinterpret_cast<float *>(gen);                                            // [128][VP]
+    const uint32_t sB = base + V_BYTES;                                                      // [3][NQP][128] int8
+    uint32_t *docmax = reinterpret_cast<uint32_t *>(gen + V_BYTES + B_BYTES);                // [MAX_DOCS][NQP]
     const uint32_t bars = smem_u32(docmax + G4U_MAX_DOCS * NQP);
     const uint32_t bar_b = (bars + 7u) & ~7u, bar_mma = bar_b + 8;
 
@@ -225,35 +230,31 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
 #pragma unroll
         for (int w = 0; w < MAXCW; ++w) cw[w] = cw_next[w];
 
-        // ---- expand this thread's token into row `tid` of the A tile -------------------------------------------
-        if (dl >= 0) {
-            const uint32_t row = sA + ((uint32_t)(tid >> 3) << 10) + ((uint32_t)(tid & 7) << 7);
-            const uint32_t sw = (uint32_t)(tid & 7);
+        // ---- expand this thread's token into lane `tid` of the A operand in tensor memory (128 int8 = 32 columns) ----
+        {
+            uint32_t row[32];
 #pragma unroll
-            for (int w = 0; w < MAXCW; ++w) {
-                if (w < CW) {
-                    const uint32_t word = cw[w];
-                    if (NBITS == 2) {
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((uint32_t)w ^ sw) << 4)),
-                                     "r"(spread2(word & 255u)), "r"(spread2((word >> 8) & 255u)),
-                                     "r"(spread2((word >> 16) & 255u)), "r"(spread2(word >> 24))
-                                     : "memory");
-                    } else {
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(
-                                         row + (((uint32_t)(2 * w) ^ sw) << 4)),
-                                     "r"(spread1(word & 15u)), "r"(spread1((word >> 4) & 15u)),
-                                     "r"(spread1((word >> 8) & 15u)), "r"(spread1((word >> 12) & 15u))
-                                     : "memory");
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(
-                                         row + (((uint32_t)(2 * w + 1) ^ sw) << 4)),
-                                     "r"(spread1((word >> 16) & 15u)), "r"(spread1((word >> 20) & 15u)),
-                                     "r"(spread1((word >> 24) & 15u)), "r"(spread1(word >> 28))
-                                     : "memory");
+            for (int x = 0; x < 32; ++x) row[x] = 0u;
+            if (dl >= 0) {
+#pragma unroll
+                for (int w = 0; w < MAXCW; ++w) {
+                    if (w < CW) {
+                        const uint32_t word = cw[w];
+                        if (NBITS == 2) {
+                            row[4 * w + 0] = spread2(word & 255u);
+                            row[4 * w + 1] = spread2((word >> 8) & 255u);
+                            row[4 * w + 2] = spread2((word >> 16) & 255u);
+                            row[4 * w + 3] = spread2(word >> 24);
+                        } else if (w < 4) {                  // 1 bit per dimension: at most four words
+#pragma unroll
+                            for (int h = 0; h < 8; ++h) row[8 * w + h] = spread1((word >> (4 * h)) & 15u);
+                        }
                     }
                 }
             }
+            tmem_st32(tmem + ((uint32_t)(warp * 32) << 16) + A_COL, row);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // rows visible to the tensor core's reads
         tc_fence_before();
         __syncthreads();
 
@@ -263,8 +264,8 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
             if (tile == 0) ok = mbar_wait(bar_b, 0, wait_limit);
             if (ok) {
                 tc_fence_after();
-                const uint64_t da = umma_desc(sA), db = umma_desc(sB);
-                for (int k = 0; k < k_steps; ++k) umma_i8(tmem, da + 2 * k, db + 2 * k, IDESC, k > 0 ? 1u : 0u);
+                const uint64_t db = umma_desc(sB);
+                for (int k = 0; k < k_steps; ++k) umma_i8_ts(tmem, tmem + A_COL + 8 * k, db + 2 * k, IDESC, k > 0 ? 1u : 0u);
                 umma_commit(bar_mma);
             } else {
                 s_abort = 1;
@@ -409,8 +410,8 @@ residual_maxsim_umma(const __grid_constant__ CUtensorMap map_q, const float *__r
                 atomicMax(&docmax[doc * NQP + lane], f_order(m0));
                 if (NQP > 32) atomicMax(&docmax[doc * NQP + 32 + lane], f_order(m1));
             }
-            // the value rows of this warp (on the A tile when ON_A) are rewritten by the next tile's expansion, each
-            // lane its own row, while the fold above reads the rows of other lanes: all lanes finish reading first
+            // the value rows of this warp are rewritten by the next tile's epilogue, each lane its own row, while the
+            // fold above reads the rows of other lanes: all lanes finish reading first
             __syncwarp();
         }
     }
@@ -452,10 +453,15 @@ static int launch_g4_umma(const Index &ix, const Params &p, const float *queries
     CUtensorMap map_q;
     int rc = make_plane_map(&map_q, qdig, (int64_t)p.B * p.nq, NQP);
     if (rc) return rc;
-    // (q_len <= 32 with residual codes: the value rows lie on the A tile)
-    const size_t smem = 1024 + (size_t)G4U_TOK * 128 + (size_t)N * 128 +
-                        (NQP == 32 && !RQ ? 0 : sizeof(float) * G4U_TOK * (NQP + 4)) +
-                        sizeof(uint32_t) * G4U_MAX_DOCS * NQP + 32;
+    // value rows (128-byte rows for q_len <= 32 with residual codes, padded rows otherwise), query planes, maxima
+    size_t smem = 1024 + sizeof(float) * G4U_TOK * (NQP == 32 && !RQ ? 32 : NQP + 4) + (size_t)N * 128 +
+                  sizeof(uint32_t) * G4U_MAX_DOCS * NQP + 32;
+    // No more CTAs may become resident on an SM than its 512 tensor-memory columns serve: one more would sit in
+    // tcgen05.alloc with its registers and shared memory until another leaves (64-token queries: three CTAs of 66 KB
+    // fit an SM, two get tensor memory; measured 5.97 -> 8.92 ms).  Registers cap the 128-column residual variants at
+    // four; the 256-column variants ask for a third of an SM's shared memory plus one byte.  (The 128-column RaBitQ
+    // variant, whose tiles are short, measured the same with and without such a cap and has none.)
+    if (N > 96 && smem < 227 * 1024 / 3 + 1) smem = 227 * 1024 / 3 + 1;
     auto kern = residual_maxsim_umma<NQP, NBITS, RQ>;
     CHIMERA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // documents per CTA: about four CTAs per SM in total, at most 32 documents each (with few queries per call a CTA
