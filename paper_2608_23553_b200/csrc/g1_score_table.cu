@@ -115,8 +115,9 @@ score_table_umma(const int8_t *__restrict__ cdig, const __grid_constant__ CUtens
         __syncwarp();
         tmem_alloc(&s_tmem_base, G1_TMEM_COLS);
     }
-    // the 64 zero rows behind each stage's planes (the loads never touch them)
-    for (uint32_t e = tid; e < G1_STAGES * (G1_B_STAGE - G1_B_LOAD) / 16; e += G1_THREADS) {
+    // the 64 zero rows behind each stage's planes (the loads never touch them); only the stages this CTA will use
+    const uint32_t used_stages = my_tiles < G1_STAGES ? (uint32_t)my_tiles : (uint32_t)G1_STAGES;
+    for (uint32_t e = tid; e < used_stages * (G1_B_STAGE - G1_B_LOAD) / 16; e += G1_THREADS) {
         const uint32_t per = (G1_B_STAGE - G1_B_LOAD) / 16;
         const uint32_t addr = sB + (e / per) * G1_B_STAGE + G1_B_LOAD + (e % per) * 16;
         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
