@@ -112,3 +112,44 @@ def test_full_search_uses_the_joint_stages_and_matches_oracle():
         res = oracle.pipeline(q[b], oix, 4, 64, 10)
         check_query(tn, b, res, ids[b].cpu().numpy(), sc[b].cpu().numpy(), 10, 64)
     gix.close()
+
+
+def test_random_shapes_of_both_forms_match_oracle():
+    """Random (dimension, centroid count, nprobe, q_len, batch) draws, a third of them with masses of duplicated
+    centroids (ties; sometimes overflowing queues): whichever form of stage 2a the library chooses, the table and the
+    probes are the oracle's."""
+    import paper_2608_23553_b200 as pkg
+    rng = np.random.default_rng(2024)
+    dev = torch.device("cuda:0")
+    forms = set()
+    for case in range(14):
+        D = int(rng.choice([32, 64, 96, 128]))
+        K = int(rng.integers(1100, 50000))
+        P = int(rng.integers(1, 40))
+        nq = int(rng.choice([4, 8, 12, 16, 20, 32, 36, 48, 64, 100]))
+        B = int(rng.integers(1, 5))
+        dup = case % 3 == 2
+        cent = unit_rows(rng, K, D)
+        if dup:
+            dst = rng.permutation(K)[:K // 2]
+            cent[dst] = cent[int(rng.integers(0, K))] if case % 2 == 0 else cent[rng.integers(0, K, size=K // 2)]
+        doclens = rng.integers(1, 6, size=32).astype(np.int32)
+        T = int(doclens.sum())
+        cids = rng.integers(0, K, size=T).astype(np.int32)
+        codes = rng.integers(0, 256, size=(T, D // 4)).astype(np.uint8)
+        gix = pkg.Index(torch.from_numpy(cent).to(dev), torch.from_numpy(cids).to(dev),
+                        torch.from_numpy(codes).to(dev), torch.from_numpy(doclens).to(dev), 2)
+        q = np.stack([unit_rows(rng, nq, D) for _ in range(B)])
+        if dup:
+            q[0, 0] = cent[dst[0]]                      # a query token equal to a duplicated centroid
+        forms.add(gix.probe_plan(B, nq, P) > 1)
+        taps = gix.alloc_taps(B, nq, P, 4)
+        gix.run_stages(1, 2, torch.from_numpy(q).to(dev), B, nq, P, 4, 2, taps)
+        assert gix.status() == 0
+        got, tab = taps.probes.cpu().numpy(), taps.score_table.cpu().numpy()
+        for b in range(B):
+            S = oracle.score_table(q[b], cent)
+            assert np.array_equal(tab[b], S), (case, D, K, P, nq, B)
+            assert np.array_equal(got[b], oracle.probes(S, P)), (case, D, K, P, nq, B)
+        gix.close()
+    assert forms == {True, False}                       # the draw covers both forms
