@@ -78,6 +78,23 @@ def measured_int8_tops():
         return 2.0 * 1590.0, "fallback bf16 x 2"
 
 
+def isolated_int8_mma_tops():
+    """TOP/s of a back-to-back loop of tcgen05.mma kind::i8 instructions (M 128, N 256, K 32) on all SMs, from the
+    library's own microbenchmark when its binary has been built (build.build_microbench); None otherwise.  Reported
+    beside the stage-1 roofline entry as context: the entry's peak stays the measured bf16 rate x 2."""
+    exe = os.path.join(ROOT, "paper_2608_23553_b200", "build", "mma_rate")
+    if not os.path.exists(exe):
+        return None
+    try:
+        out = subprocess.run([exe], capture_output=True, text=True, timeout=60).stdout
+        for line in out.splitlines():
+            if line.startswith("N=256 A in TMEM") and "TOP/s" in line:
+                return float(line.split("ms,")[1].split("TOP/s")[0])
+    except Exception:
+        pass
+    return None
+
+
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from stored ncu
 # captures on small cases (a full-size launch is too large to capture; the profile named beside each figure gives the
 # command).  The stage-3 bound scan reads each query's 8-bit table once (batch x K x q_len bytes) and otherwise moves
@@ -717,6 +734,10 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     }
     res["roofline"] = roofline
     res["pruning"] = PRUNING_TEXT[mode]
+    if full:
+        iso = isolated_int8_mma_tops()
+        if iso:
+            roofline["per_stage"]["score_table"]["isolated_mma_loop_tops"] = iso
     joint = index.probe_plan(B, nq, P) if mode != "rabitq_graph" else 0
     if joint:
         # stages 1 and 2a run together: the stage-1 slot also times the scans of the sampled rows, and the probes
