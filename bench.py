@@ -734,7 +734,7 @@ def measure(pkg, cfg, corp, q, index, args, device, mode="ci", dist=None, local_
     }
     res["roofline"] = roofline
     res["pruning"] = PRUNING_TEXT[mode]
-    if full:
+    if full and dist is None:                  # (one process: the microbenchmark runs on device 0)
         iso = isolated_int8_mma_tops()
         if iso:
             roofline["per_stage"]["score_table"]["isolated_mma_loop_tops"] = iso
