@@ -265,6 +265,9 @@ int chimera_workspace_status(const void *workspace, void *stream, int32_t *statu
  * needs nprobe <= 32, q_len a multiple of 4 and at least 8 sample tiles. */
 int chimera_probe_plan(const chimera_index *index, int32_t n_queries, int32_t q_len, int32_t nprobe,
                        int32_t *sample_stride);
+/* The same rule as plain arithmetic on the sizes (no index, no device): the sampling stride for n_centroids centroids,
+ * queries of q_len tokens and nprobe probes per token, or 0 for the table scan. */
+int32_t chimera_probe_sample_stride(int64_t n_centroids, int32_t q_len, int32_t nprobe);
 
 /* Debug build (the paper has no counterpart).  libchimera_debug.so is the same source compiled with -DCHIMERA_DEBUG:
  * every kernel checks each centroid id, document id, token position and candidate rank before it gathers through it

@@ -152,6 +152,7 @@ int launch_probes(const Index &ix, const Params &p, const Layout &L, const int32
 // Stages 1 and 2a together (g1_score_table.cu), used when the layout has pq_stride > 0, and its probe-side pieces
 // (g2_probe.cu): the sample's top nprobe and bounds; the final top nprobe from sample list and queues, with the table
 // scan as the fallback for queries whose queue overflowed.
+int probe_sample_stride(int64_t K, int nq, int P);       // host arithmetic only
 int probe_queue_stride(const Index &ix, const Params &p);
 int probe_queue_cap();
 int probe_sample_groups(const Index &ix, int stride);

@@ -207,14 +207,16 @@ int probe_queue_cap() { return PQ_CAP; }
 // negative-binomial with that mean); stride = 128 / max(nprobe, 4) keeps the mean near 128 keys, an eighth of PQ_CAP
 // (for nprobe = 4 the chance of 1024 or more is below 1e-9 per row).  Strided tiles rather than the first ones, so
 // that centroids stored in some spatial order still give a representative sample.
-int probe_queue_stride(const Index &ix, const Params &p)
+int probe_sample_stride(int64_t K, int nq, int P)
 {
-    if (p.P > 32 || (p.nq & 3) != 0) return 0;
-    const int stride = 128 / (p.P > 4 ? p.P : 4);          // 32, ..., 4
-    const int64_t c_tiles = (ix.K + 127) / 128;
+    if (P < 1 || P > 32 || nq < 1 || (nq & 3) != 0) return 0;
+    const int stride = 128 / (P > 4 ? P : 4);              // 32, ..., 4
+    const int64_t c_tiles = (K + 127) / 128;
     if (stride < 2 || c_tiles < 8 * (int64_t)stride) return 0;      // at least 8 sample tiles (1024 centroids)
     return stride;
 }
+
+int probe_queue_stride(const Index &ix, const Params &p) { return probe_sample_stride(ix.K, p.nq, p.P); }
 
 // The sample rows of a query are cut into groups (16 rows or more, at most PQ_MAX_GROUPS groups, at least 64).
 int probe_sample_groups(const Index &ix, int stride)
@@ -444,6 +446,11 @@ constexpr int STATIC_MAX_DEVICES = 64;
 static std::atomic<unsigned long long *> g_probe_scratch_ptr[STATIC_MAX_DEVICES];
 
 }  // namespace chimera
+
+extern "C" int32_t chimera_probe_sample_stride(int64_t n_centroids, int32_t q_len, int32_t nprobe)
+{
+    return chimera::probe_sample_stride(n_centroids, q_len, nprobe);
+}
 
 extern "C" int chimera_probes_static(const int32_t *score_table, int64_t n_centroids, int32_t n_queries, int32_t q_len,
                                      int32_t nprobe, void *stream, int32_t *out_probes)

@@ -69,3 +69,21 @@ def test_binding_refuses_to_run_without_the_library(monkeypatch):
     monkeypatch.setattr(binding, "_LIB_PATH", "/nonexistent/libchimera.so")
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_probe_sampling_rule_on_the_configurations_sizes(lib):
+    """chimera_probe_sample_stride is plain arithmetic (no device): every 128 / max(nprobe, 4)-th tile of 128 centroids
+    is a sample tile when there are at least 8 of them, nprobe <= 32 and q_len is a multiple of 4; 0 = table scan."""
+    f = lib.chimera_probe_sample_stride
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32]
+    assert f(262144, 32, 4) == 32 and f(65536, 32, 4) == 32          # Large, Mid
+    assert f(32768, 64, 8) == 16                                     # long documents
+    assert f(1024, 32, 4) == 0                                       # Tiny: 8 tiles in all
+    assert f(262144, 32, 1) == 32 and f(262144, 32, 16) == 8 and f(262144, 32, 32) == 4
+    assert f(262144, 32, 33) == 0 and f(262144, 30, 4) == 0 and f(262144, 32, 0) == 0
+    for nprobe in range(1, 33):
+        s = f(1 << 20, 32, nprobe)
+        assert s == 128 // max(nprobe, 4)
+        k_min = 8 * s * 128 - 127                                    # fewest centroids with 8 * s tiles
+        assert f(k_min, 32, nprobe) == s and f(k_min - 1, 32, nprobe) == 0
